@@ -1,0 +1,535 @@
+/*
+ * CPU oracle for the CacheCard create / inject path.       *** TEST INFRASTRUCTURE ***
+ *
+ * This file is a plain, slow, scalar restatement of what the path computes, written to be
+ * checked against the method's definition by eye.  It is not part of the product: only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg may call it.  It shares no
+ * code, header, table or constant generator with the CUDA library; every constant below is
+ * typed out here on its own.
+ *
+ * What the paper fixes (Sections 3.1, 3.3, 4.2.1, 4.2.2): a card holds the keys and values
+ * as quantised groups, the per-token bit-width vector b(t) in {2,4,8,16} (16 = FP16 kept
+ * as is), the sequence length, model and sender identifiers, a position-offset placeholder
+ * and the achieved average bit-width; injection rebuilds FP16 keys and values in the
+ * [heads, tokens, head_dim] layout of a HuggingFace cache.  The paper gives no formula,
+ * group size, rounding rule or byte layout; the readings taken here are:
+ *   - groups of 32 consecutive channels along head_dim, for K and V alike;
+ *   - asymmetric min/max: zero = group minimum (fp32), scale = (max-min)/(2^b-1) (fp32);
+ *   - codes q = clamp(rint((x-zero) * inv), 0, 2^b-1), inv = (2^b-1)/(max-min), one IEEE
+ *     binary32 operation per step, round-to-nearest-even everywhere, nothing fused;
+ *   - a constant group has scale = inv = 0 and all-zero codes; a zero minimum is stored +0;
+ *   - reconstruction x^ = fp16_rne( fl32(fl32(q) * scale) + zero );
+ *   - the byte layout described at write_prefix() / encode_record() below.
+ * NaN or infinity inside a quantised (b < 16) token is outside the definition (codes are
+ * then unspecified); inside an FP16 token the bit patterns are preserved.
+ *
+ * Pins (see tests): closed-form size, uniform offsets, brute-force scan, FP16 round trip,
+ * |x - x^| <= scale/2 (+ rounding slack), min -> code 0 / max -> code 2^b-1, monotone codes,
+ * hand-worked 2-bit and 4-bit groups with exact ties, exact-rational recomputation of codes,
+ * the 8-bit case against the textbook affine uint8 quantiser, all-FP16 card == memcpy.
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* status values (same numbering as the library's public header, typed here separately) */
+enum { ORC_OK = 0, ORC_INVALID_ARG = 1, ORC_UNSUPPORTED_SHAPE = 2, ORC_BAD_BITS = 3,
+       ORC_BUFFER_TOO_SMALL = 4, ORC_BAD_CARD = 5 };
+
+typedef struct {
+    int32_t n_layers, n_kv_heads, head_dim, n_tokens;
+    int32_t group_size; /* 32 */
+    int32_t bits_mode;  /* 0: one bits[T] for the whole model; 1: bits[L*H][T] */
+    int64_t head_stride;  /* elements between heads  */
+    int64_t token_stride; /* elements between tokens */
+} orc_layout;
+
+/* ------------------------------------------------------------------ FP16 <-> FP32 */
+
+/* Exact: every FP16 value is an FP32 value. */
+float orc_half_to_float(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h >> 15) & 1u;
+    uint32_t e = (uint32_t)(h >> 10) & 31u;
+    uint32_t m = (uint32_t)h & 1023u;
+    float v;
+    if (e == 31u) { /* infinity / NaN: keep the payload */
+        uint32_t b = (sign << 31) | 0x7f800000u | (m << 13);
+        memcpy(&v, &b, 4);
+        return v;
+    }
+    if (e == 0u)
+        v = (float)ldexp((double)m, -24);            /* subnormal: m * 2^-24 */
+    else
+        v = (float)ldexp((double)(1024u + m), (int)e - 25); /* 1.m * 2^(e-15) */
+    return sign ? -v : v;
+}
+
+/* Round-to-nearest-even conversion of a binary32 value to FP16. */
+uint16_t orc_float_to_half(float f)
+{
+    uint32_t b;
+    memcpy(&b, &f, 4);
+    uint16_t sign = (uint16_t)((b >> 31) << 15);
+    uint32_t mag = b & 0x7fffffffu;
+    if (mag > 0x7f800000u) return (uint16_t)(sign | 0x7e00u | ((mag >> 13) & 0x3ffu)); /* NaN */
+    double v = fabs((double)f);
+    if (v >= 65520.0) return (uint16_t)(sign | 0x7c00u); /* halfway to 65536 rounds to inf */
+    if (v < 6.103515625e-05) {                           /* below 2^-14: multiples of 2^-24 */
+        double r = nearbyint(v * 16777216.0);            /* ties to even; 1024 -> smallest normal */
+        return (uint16_t)(sign | (uint16_t)r);
+    }
+    int e2;
+    (void)frexp(v, &e2);      /* v = frac * 2^e2, frac in [0.5, 1) -> v = 1.x * 2^(e2-1) */
+    int E = e2 - 1;
+    double r = nearbyint(ldexp(v, 10 - E)); /* in [1024, 2048], ties to even */
+    if (r == 2048.0) { r = 1024.0; E += 1; }
+    return (uint16_t)(sign | (uint16_t)((E + 15) << 10) | (uint16_t)((int)r - 1024));
+}
+
+/* ------------------------------------------------------------------ sizes and offsets */
+
+static uint64_t round_up_256(uint64_t x) { return (x + 255u) / 256u * 256u; }
+
+/* Bytes of one token row inside one stream: G (scale, zero) fp32 pairs then the packed
+ * codes; an FP16 token is the row itself.  Code bytes alone are d*b/8 (Section 3.1's
+ * bytes-per-element law). */
+int64_t orc_record_bytes(int head_dim, int b)
+{
+    if (b == 16) return 2 * (int64_t)head_dim;
+    if (b == 2 || b == 4 || b == 8) return (int64_t)head_dim * b / 8 + 8 * (int64_t)(head_dim / 32);
+    return -1;
+}
+
+static int layout_ok(const orc_layout *L)
+{
+    if (!L) return ORC_INVALID_ARG;
+    if (L->n_layers < 1 || L->n_kv_heads < 1 || L->n_tokens < 0) return ORC_INVALID_ARG;
+    if (L->bits_mode != 0 && L->bits_mode != 1) return ORC_INVALID_ARG;
+    if (L->group_size != 32) return ORC_UNSUPPORTED_SHAPE;
+    if (L->head_dim < 64 || L->head_dim % 64 != 0) return ORC_UNSUPPORTED_SHAPE;
+    return ORC_OK;
+}
+
+static int64_t n_segments(const orc_layout *L)
+{
+    return L->bits_mode == 0 ? 1 : (int64_t)L->n_layers * L->n_kv_heads;
+}
+
+/* stream index of (layer, kv, head); kv 0 = K, 1 = V */
+static int64_t stream_index(const orc_layout *L, int l, int kv, int h)
+{
+    return ((int64_t)l * 2 + kv) * L->n_kv_heads + h;
+}
+
+static int64_t segment_of(const orc_layout *L, int l, int h)
+{
+    return L->bits_mode == 0 ? 0 : (int64_t)l * L->n_kv_heads + h;
+}
+
+/* Exclusive prefix sum of record sizes over one segment: off[0] = 0,
+ * off[t+1] = off[t] + rec(b_t).  Returns ORC_BAD_BITS on a value outside {2,4,8,16}. */
+int orc_scan_offsets(int head_dim, const uint8_t *bits, int64_t n_tokens, uint32_t *off,
+                     uint64_t *sum_bits)
+{
+    uint64_t run = 0, sb = 0;
+    off[0] = 0;
+    for (int64_t t = 0; t < n_tokens; ++t) {
+        int64_t r = orc_record_bytes(head_dim, bits[t]);
+        if (r < 0) return ORC_BAD_BITS;
+        run += (uint64_t)r;
+        sb += bits[t];
+        off[t + 1] = (uint32_t)run;
+    }
+    if (sum_bits) *sum_bits = sb;
+    return ORC_OK;
+}
+
+/* Section sizes.  Card = header (256) | bits | offsets | [stream bases, mode 1] | payload. */
+static void section_offsets(const orc_layout *L, uint64_t *bits_off, uint64_t *offs_off,
+                            uint64_t *sbase_off, uint64_t *payload_off)
+{
+    uint64_t nseg = (uint64_t)n_segments(L), T = (uint64_t)L->n_tokens;
+    uint64_t S = 2u * (uint64_t)L->n_layers * (uint64_t)L->n_kv_heads;
+    *bits_off = 256;
+    *offs_off = *bits_off + round_up_256(nseg * T);
+    uint64_t after = *offs_off + round_up_256(4u * nseg * (T + 1u));
+    if (L->bits_mode == 1) {
+        *sbase_off = after;
+        after += round_up_256(8u * (S + 1u));
+    } else {
+        *sbase_off = 0;
+    }
+    *payload_off = after;
+}
+
+/* Exact card size for a bit-width vector (host memory); bits == NULL gives the worst case
+ * (every token FP16). */
+int orc_card_size(const orc_layout *L, const uint8_t *bits, uint64_t *out_bytes)
+{
+    int st = layout_ok(L);
+    if (st) return st;
+    uint64_t bo, oo, so, po;
+    section_offsets(L, &bo, &oo, &so, &po);
+    uint64_t payload = 0;
+    int64_t nseg = n_segments(L);
+    for (int64_t seg = 0; seg < nseg; ++seg) {
+        uint64_t seg_bytes = 0;
+        for (int64_t t = 0; t < L->n_tokens; ++t) {
+            int64_t r = orc_record_bytes(L->head_dim, bits ? bits[seg * L->n_tokens + t] : 16);
+            if (r < 0) return ORC_BAD_BITS;
+            seg_bytes += (uint64_t)r;
+        }
+        /* mode 0: the one segment serves all 2*L*H streams; mode 1: K and V of (l,h) */
+        payload += seg_bytes * (L->bits_mode == 0 ? 2u * (uint64_t)L->n_layers * L->n_kv_heads : 2u);
+    }
+    *out_bytes = po + payload;
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ little-endian stores */
+
+static void put_u32(uint8_t *p, uint32_t v)
+{
+    for (int i = 0; i < 4; ++i) p[i] = (uint8_t)(v >> (8 * i));
+}
+static void put_u64(uint8_t *p, uint64_t v)
+{
+    for (int i = 0; i < 8; ++i) p[i] = (uint8_t)(v >> (8 * i));
+}
+static void put_f32(uint8_t *p, float f)
+{
+    uint32_t b;
+    memcpy(&b, &f, 4);
+    put_u32(p, b);
+}
+static uint32_t get_u32(const uint8_t *p)
+{
+    uint32_t v = 0;
+    for (int i = 0; i < 4; ++i) v |= (uint32_t)p[i] << (8 * i);
+    return v;
+}
+static uint64_t get_u64(const uint8_t *p)
+{
+    uint64_t v = 0;
+    for (int i = 0; i < 8; ++i) v |= (uint64_t)p[i] << (8 * i);
+    return v;
+}
+static float get_f32(const uint8_t *p)
+{
+    uint32_t b = get_u32(p);
+    float f;
+    memcpy(&f, &b, 4);
+    return f;
+}
+
+/* ------------------------------------------------------------------ one group of 32 */
+
+/* Quantise 32 FP16 values at b in {2,4,8} bits. */
+void orc_quantize_group(const uint16_t *x, int b, float *scale_out, float *zero_out, uint8_t *q)
+{
+    float xf[32];
+    for (int i = 0; i < 32; ++i) xf[i] = orc_half_to_float(x[i]);
+    float mn = xf[0], mx = xf[0];
+    for (int i = 1; i < 32; ++i) {
+        if (xf[i] < mn) mn = xf[i];
+        if (xf[i] > mx) mx = xf[i];
+    }
+    if (mn == 0.0f) { /* a zero minimum is stored as +0 whatever sign it carried */
+        uint32_t z = 0;
+        memcpy(&mn, &z, 4);
+    }
+    int qmax = (1 << b) - 1;
+    float qmaxf = (float)qmax;
+    float range = mx - mn;
+    float scale = 0.0f, inv = 0.0f;
+    if (range > 0.0f) {
+        scale = range / qmaxf;
+        inv = qmaxf / range;
+    }
+    for (int i = 0; i < 32; ++i) {
+        float t = xf[i] - mn;
+        float u = t * inv;
+        float r = nearbyintf(u); /* ties to even (default rounding mode) */
+        int qi;
+        if (!(r >= 0.0f)) qi = 0;
+        else if (r > qmaxf) qi = qmax;
+        else qi = (int)r;
+        q[i] = (uint8_t)qi;
+    }
+    *scale_out = scale;
+    *zero_out = mn;
+}
+
+/* Reconstruct 32 FP16 values: multiply, then add, each rounded to binary32, then to FP16. */
+void orc_dequantize_group(const uint8_t *q, float scale, float zero, uint16_t *out)
+{
+    for (int i = 0; i < 32; ++i) {
+        float p = (float)q[i] * scale;
+        float r = p + zero;
+        out[i] = orc_float_to_half(r);
+    }
+}
+
+/* Codes as a little-endian bit string: code i occupies bits [i*b, i*b+b). */
+void orc_pack_codes(const uint8_t *q, int n, int b, uint8_t *out)
+{
+    memset(out, 0, (size_t)n * b / 8);
+    for (int i = 0; i < n; ++i) {
+        int bit = i * b;
+        out[bit / 8] |= (uint8_t)(q[i] << (bit % 8));
+    }
+}
+
+void orc_unpack_codes(const uint8_t *in, int n, int b, uint8_t *q)
+{
+    for (int i = 0; i < n; ++i) {
+        int bit = i * b;
+        q[i] = (uint8_t)((in[bit / 8] >> (bit % 8)) & ((1 << b) - 1));
+    }
+}
+
+/* ------------------------------------------------------------------ one token row */
+
+/* Record of a b<16 token: G pairs {scale_g, zero_g} (fp32, little-endian), group g covering
+ * channels 32g..32g+31, then the d*b/8 code bytes of the whole row.  b == 16: the row's
+ * FP16 bit patterns verbatim. */
+static void encode_record(const uint16_t *row, int d, int b, uint8_t *rec)
+{
+    if (b == 16) {
+        for (int i = 0; i < d; ++i) {
+            rec[2 * i] = (uint8_t)(row[i] & 0xff);
+            rec[2 * i + 1] = (uint8_t)(row[i] >> 8);
+        }
+        return;
+    }
+    int G = d / 32;
+    uint8_t q[32];
+    for (int g = 0; g < G; ++g) {
+        float scale, zero;
+        orc_quantize_group(row + 32 * g, b, &scale, &zero, q);
+        put_f32(rec + 8 * g, scale);
+        put_f32(rec + 8 * g + 4, zero);
+        orc_pack_codes(q, 32, b, rec + 8 * G + (size_t)g * 32 * b / 8);
+    }
+}
+
+static void decode_record(const uint8_t *rec, int d, int b, uint16_t *row)
+{
+    if (b == 16) {
+        for (int i = 0; i < d; ++i) row[i] = (uint16_t)(rec[2 * i] | (rec[2 * i + 1] << 8));
+        return;
+    }
+    int G = d / 32;
+    uint8_t q[32];
+    for (int g = 0; g < G; ++g) {
+        float scale = get_f32(rec + 8 * g);
+        float zero = get_f32(rec + 8 * g + 4);
+        orc_unpack_codes(rec + 8 * G + (size_t)g * 32 * b / 8, 32, b, q);
+        orc_dequantize_group(q, scale, zero, row + 32 * g);
+    }
+}
+
+/* One stream (a [T, d] matrix with a row stride) -> its payload bytes. */
+void orc_encode_stream(const uint16_t *x, int64_t token_stride, int64_t n_tokens, int d,
+                       const uint8_t *bits, const uint32_t *off, uint8_t *out)
+{
+    for (int64_t t = 0; t < n_tokens; ++t)
+        encode_record(x + t * token_stride, d, bits[t], out + off[t]);
+}
+
+void orc_decode_stream(const uint8_t *in, const uint8_t *bits, const uint32_t *off,
+                       int64_t n_tokens, int d, uint16_t *x, int64_t token_stride)
+{
+    for (int64_t t = 0; t < n_tokens; ++t)
+        decode_record(in + off[t], d, bits[t], x + t * token_stride);
+}
+
+/* ------------------------------------------------------------------ whole card */
+
+/* Header (256 bytes, little-endian, fields at these byte offsets, everything else zero):
+ *   0 magic "QKVS" = 0x53564B51   4 version = 1     8 status        12 bits_mode
+ *  16 n_layers  20 n_kv_heads  24 head_dim  28 n_tokens  32 group_size
+ *  36 meta_bytes_per_group = 8    40 model_id u64   48 sender_id u64
+ *  56 position_offset i64 (placeholder)  64 sum_bits u64   72 avg_code_bits f32
+ *  80 bits_off u64   88 offs_off u64   96 payload_off u64
+ * 104 stream_bytes u64 (mode 0: bytes of one stream; mode 1: 0)   112 total_bytes u64
+ * 120 sbase_off u64 (mode 1: offset of the u64 stream-base table; mode 0: 0)
+ * Then bits[seg][t] u8, then off[seg][0..T] u32, then (mode 1) sbase[0..S] u64, each
+ * section zero-padded to a multiple of 256, then the payload, stream after stream with
+ * stream (l, kv, h) at index (l*2 + kv)*H + h. */
+int orc_write_prefix(const orc_layout *L, const uint8_t *bits, uint64_t model_id,
+                     uint64_t sender_id, int64_t position_offset, uint8_t *card,
+                     uint64_t capacity)
+{
+    int st = layout_ok(L);
+    if (st) return st;
+    uint64_t bo, oo, so, po;
+    section_offsets(L, &bo, &oo, &so, &po);
+    if (capacity < po) return ORC_BUFFER_TOO_SMALL;
+    memset(card, 0, (size_t)po);
+
+    int64_t nseg = n_segments(L), T = L->n_tokens;
+    uint64_t S = 2u * (uint64_t)L->n_layers * (uint64_t)L->n_kv_heads;
+    uint64_t sum_bits = 0;
+    int status = ORC_OK;
+    for (int64_t seg = 0; seg < nseg && status == ORC_OK; ++seg) {
+        uint32_t *off_tmp = (uint32_t *)(void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1));
+        /* the host is little-endian, so writing uint32_t in place equals put_u32 */
+        uint64_t sb = 0;
+        status = orc_scan_offsets(L->head_dim, bits + seg * T, T, off_tmp, &sb);
+        sum_bits += sb;
+        memcpy(card + bo + (uint64_t)seg * (uint64_t)T, bits + seg * T, (size_t)T);
+    }
+    uint64_t payload = 0, stream_bytes = 0;
+    if (status == ORC_OK) {
+        if (L->bits_mode == 0) {
+            stream_bytes = get_u32(card + oo + 4u * (uint64_t)T);
+            payload = S * stream_bytes;
+        } else {
+            for (int l = 0; l < L->n_layers; ++l)
+                for (int kv = 0; kv < 2; ++kv)
+                    for (int h = 0; h < L->n_kv_heads; ++h) {
+                        int64_t s = stream_index(L, l, kv, h), seg = segment_of(L, l, h);
+                        put_u64(card + so + 8u * (uint64_t)s, payload);
+                        payload += get_u32(card + oo + 4u * ((uint64_t)seg * (uint64_t)(T + 1) + (uint64_t)T));
+                    }
+            put_u64(card + so + 8u * S, payload);
+        }
+        if (po + payload > capacity) status = ORC_BUFFER_TOO_SMALL;
+    }
+    put_u32(card + 0, 0x53564B51u);
+    put_u32(card + 4, 1u);
+    put_u32(card + 8, (uint32_t)status);
+    put_u32(card + 12, (uint32_t)L->bits_mode);
+    put_u32(card + 16, (uint32_t)L->n_layers);
+    put_u32(card + 20, (uint32_t)L->n_kv_heads);
+    put_u32(card + 24, (uint32_t)L->head_dim);
+    put_u32(card + 28, (uint32_t)L->n_tokens);
+    put_u32(card + 32, (uint32_t)L->group_size);
+    put_u32(card + 36, 8u);
+    put_u64(card + 40, model_id);
+    put_u64(card + 48, sender_id);
+    put_u64(card + 56, (uint64_t)position_offset);
+    if (status == ORC_OK) {
+        put_u64(card + 64, sum_bits);
+        float avg = (nseg * T) > 0 ? (float)sum_bits / (float)((uint64_t)nseg * (uint64_t)T) : 0.0f;
+        put_f32(card + 72, avg);
+    }
+    put_u64(card + 80, bo);
+    put_u64(card + 88, oo);
+    put_u64(card + 96, po);
+    if (status == ORC_OK) {
+        put_u64(card + 104, stream_bytes);
+        put_u64(card + 112, po + payload);
+    }
+    put_u64(card + 120, so);
+    return status;
+}
+
+/* Location of stream s inside a card whose prefix is already written. */
+static uint64_t stream_base(const uint8_t *card, const orc_layout *L, int64_t s)
+{
+    uint64_t po = get_u64(card + 96);
+    if (L->bits_mode == 0) return po + (uint64_t)s * get_u64(card + 104);
+    return po + get_u64(card + get_u64(card + 120) + 8u * (uint64_t)s);
+}
+
+/* FP16 cache + bit-widths -> card.  K_layers[l], V_layers[l] point at [H, *, d] FP16 blocks
+ * addressed with the layout's strides.  Streams in [s_begin, s_end) are encoded (use 0 and
+ * 2*L*H for the whole card); the prefix is always written. */
+int orc_card_create_range(const orc_layout *L, const uint16_t *const *K_layers,
+                          const uint16_t *const *V_layers, const uint8_t *bits,
+                          uint64_t model_id, uint64_t sender_id, int64_t position_offset,
+                          uint8_t *card, uint64_t capacity, int64_t s_begin, int64_t s_end)
+{
+    int st = orc_write_prefix(L, bits, model_id, sender_id, position_offset, card, capacity);
+    if (st) return st;
+    uint64_t bo = get_u64(card + 80), oo = get_u64(card + 88);
+    int64_t T = L->n_tokens, S = 2 * (int64_t)L->n_layers * L->n_kv_heads;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int64_t s = s_begin; s < (s_end < S ? s_end : S); ++s) {
+        int h = (int)(s % L->n_kv_heads);
+        int kv = (int)((s / L->n_kv_heads) % 2);
+        int l = (int)(s / (2 * L->n_kv_heads));
+        int64_t seg = segment_of(L, l, h);
+        const uint16_t *x = (kv == 0 ? K_layers[l] : V_layers[l]) + (int64_t)h * L->head_stride;
+        orc_encode_stream(x, L->token_stride, T, L->head_dim, card + bo + (uint64_t)seg * (uint64_t)T,
+                          (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1)),
+                          card + stream_base(card, L, s));
+    }
+    return ORC_OK;
+}
+
+int orc_card_create(const orc_layout *L, const uint16_t *const *K_layers,
+                    const uint16_t *const *V_layers, const uint8_t *bits, uint64_t model_id,
+                    uint64_t sender_id, int64_t position_offset, uint8_t *card, uint64_t capacity)
+{
+    return orc_card_create_range(L, K_layers, V_layers, bits, model_id, sender_id,
+                                 position_offset, card, capacity, 0,
+                                 L ? 2 * (int64_t)L->n_layers * L->n_kv_heads : 0);
+}
+
+/* Card -> FP16 keys and values.  `dst` gives the destination's strides and its capacity in
+ * tokens (dst->n_tokens); token t of the card lands on row dst_token_offset + t. */
+int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *dst,
+                    uint16_t *const *K_out, uint16_t *const *V_out, int64_t dst_token_offset)
+{
+    int st = layout_ok(dst);
+    if (st) return st;
+    if (card_bytes < 256) return ORC_BAD_CARD;
+    if (get_u32(card + 0) != 0x53564B51u || get_u32(card + 4) != 1u) return ORC_BAD_CARD;
+    if (get_u32(card + 8) != 0u) return ORC_BAD_CARD;
+    orc_layout C = *dst;
+    C.bits_mode = (int32_t)get_u32(card + 12);
+    C.n_tokens = (int32_t)get_u32(card + 28);
+    if ((int32_t)get_u32(card + 16) != dst->n_layers || (int32_t)get_u32(card + 20) != dst->n_kv_heads ||
+        (int32_t)get_u32(card + 24) != dst->head_dim || get_u32(card + 32) != 32u ||
+        get_u32(card + 36) != 8u || (C.bits_mode != 0 && C.bits_mode != 1) || C.n_tokens < 0)
+        return ORC_BAD_CARD;
+    if (get_u64(card + 112) > card_bytes) return ORC_BAD_CARD;
+    if (dst_token_offset < 0 || dst_token_offset + C.n_tokens > dst->n_tokens) return ORC_INVALID_ARG;
+    uint64_t bo = get_u64(card + 80), oo = get_u64(card + 88);
+    int64_t T = C.n_tokens, S = 2 * (int64_t)C.n_layers * C.n_kv_heads;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int64_t s = 0; s < S; ++s) {
+        int h = (int)(s % C.n_kv_heads);
+        int kv = (int)((s / C.n_kv_heads) % 2);
+        int l = (int)(s / (2 * C.n_kv_heads));
+        int64_t seg = segment_of(&C, l, h);
+        uint16_t *x = (kv == 0 ? K_out[l] : V_out[l]) + (int64_t)h * dst->head_stride +
+                      dst_token_offset * dst->token_stride;
+        orc_decode_stream(card + stream_base(card, &C, s), card + bo + (uint64_t)seg * (uint64_t)T,
+                          (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1)),
+                          T, C.head_dim, x, dst->token_stride);
+    }
+    return ORC_OK;
+}
+
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void orc_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
