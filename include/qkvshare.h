@@ -1,0 +1,169 @@
+/*
+ * qkvshare.h -- C interface of the CacheCard create / inject library (CUDA, sm_100a).
+ *
+ * A CacheCard is the artifact one agent hands to the next in place of re-prefilling a shared
+ * context (Section 4.2 of the QKVShare paper): the sender's FP16 key/value cache, quantised
+ * token by token at a bit-width b(t) in {2, 4, 8, 16} (Section 3.3; 16 keeps the token in
+ * FP16), packed together with the bit-width vector, the sequence length, model and sender
+ * identifiers, a position-offset placeholder and the achieved average bit-width
+ * (Section 4.2.1).  The receiver rebuilds FP16 keys and values in the [heads, tokens,
+ * head_dim] layout of a HuggingFace cache (Section 4.2.2).
+ *
+ * The paper fixes no arithmetic or byte layout; this library uses:
+ *   groups of 32 consecutive channels of one token row, for K and V alike;
+ *   zero = group minimum, scale = (max - min) / (2^b - 1), both fp32;
+ *   code = round-to-nearest-even((x - zero) * ((2^b - 1) / (max - min))), clamped to [0, 2^b - 1];
+ *   reconstruction = fp16_rne(fl32(code * scale) + zero);  every step one IEEE binary32
+ *   operation, never fused; a constant group has scale 0 and all-zero codes.
+ *
+ * Card bytes (little-endian; every section padded with zeros to a multiple of 256):
+ *   [0, 256)        qkvs_card_header_t
+ *   bits_off        bits[seg][t]  u8           seg = 0 (bits_mode 0) or layer*H + head (mode 1)
+ *   offs_off        off[seg][0..T] u32         exclusive prefix sum of record sizes
+ *   sbase_off       sbase[0..S] u64            (bits_mode 1 only) start of each stream in the payload
+ *   payload_off     streams one after another, stream index s = (layer*2 + kv)*H + head,
+ *                   kv 0 = K, 1 = V; token t's record sits at off[seg][t] inside its stream.
+ *   record, b < 16: d/32 pairs {fp32 scale, fp32 zero}, then d*b/8 code bytes; the code of
+ *                   channel i occupies bits [i*b, i*b + b) of the code bytes read as a
+ *                   little-endian bit string.  record, b = 16: the d FP16 values verbatim.
+ *   record size:    d*b/8 + 8*(d/32) bytes for b in {2,4,8};  2*d bytes for b = 16.
+ *
+ * All entry points return a qkvs_status_t.  Unless stated otherwise a pointer named *_dev is a
+ * device pointer, anything else is a host pointer.  The library allocates no device memory and
+ * keeps no state between calls; every buffer belongs to the caller.  Launches are asynchronous
+ * on the given CUDA stream (a cudaStream_t passed as void*; NULL is the default stream).
+ */
+#ifndef QKVSHARE_H_
+#define QKVSHARE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define QKVS_API __attribute__((visibility("default")))
+#else
+#define QKVS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QKVS_OK = 0,
+    QKVS_ERR_INVALID_ARG = 1,      /* null pointer, negative size, misaligned pointer or stride */
+    QKVS_ERR_UNSUPPORTED_SHAPE = 2,/* head_dim not in {64,128,192,256}, group_size != 32 */
+    QKVS_ERR_BAD_BITS = 3,         /* a bit-width outside {2,4,8,16} */
+    QKVS_ERR_BUFFER_TOO_SMALL = 4, /* card capacity below what the bit-widths need */
+    QKVS_ERR_BAD_CARD = 5,         /* header magic/version/shape/status/size does not check out */
+    QKVS_ERR_CUDA = 6,             /* a CUDA runtime call or launch failed */
+    QKVS_ERR_TIMEOUT = 7           /* a bounded wait inside a kernel gave up */
+} qkvs_status_t;
+
+/* One agent's KV cache: per layer one K and one V block of FP16, HuggingFace layout
+ * [1, n_kv_heads, tokens, head_dim] (Section 4.2.2), addressed as
+ * base + head*head_stride + token*token_stride + channel (strides in elements). */
+typedef struct {
+    int32_t n_layers;
+    int32_t n_kv_heads;
+    int32_t head_dim;     /* 64, 128, 192 or 256 */
+    int32_t n_tokens;     /* tokens in the card (sequence length, Section 4.2.1) */
+    int32_t group_size;   /* must be 32 */
+    int32_t bits_mode;    /* 0: one bits[n_tokens] for the whole model (the paper's token-level
+                             vector); 1: bits[n_layers*n_kv_heads][n_tokens] */
+    int64_t head_stride;  /* elements between heads; multiple of 8 */
+    int64_t token_stride; /* elements between tokens; >= head_dim, multiple of 8 */
+} qkvs_layout_t;
+
+/* Identifiers carried in the card (Section 4.2.1).  position_offset is the placeholder the
+ * paper reserves for cross-prefix alignment; it is stored and returned, never interpreted. */
+typedef struct {
+    uint64_t model_id;
+    uint64_t sender_id;
+    int64_t position_offset;
+} qkvs_card_meta_t;
+
+/* The first 256 bytes of every card. */
+typedef struct {
+    uint32_t magic;                /* 0x53564B51, "QKVS" */
+    uint32_t version;              /* 1 */
+    uint32_t status;               /* qkvs_status_t recorded on the device; 0 = usable card */
+    uint32_t bits_mode;
+    int32_t n_layers, n_kv_heads, head_dim, n_tokens, group_size;
+    uint32_t meta_bytes_per_group; /* 8 */
+    uint64_t model_id;
+    uint64_t sender_id;
+    int64_t position_offset;
+    uint64_t sum_bits;             /* sum of b(t) over all segments and tokens */
+    float avg_code_bits;           /* (float)sum_bits / (float)(segments * n_tokens) (Section 4.2.1) */
+    uint32_t pad0_;
+    uint64_t bits_off, offs_off, payload_off;
+    uint64_t stream_bytes;         /* bits_mode 0: bytes of one stream; bits_mode 1: 0 */
+    uint64_t total_bytes;          /* header + tables + payload */
+    uint64_t sbase_off;            /* bits_mode 1: offset of the stream-base table; else 0 */
+    uint8_t reserved_[128];
+} qkvs_card_header_t;
+
+/* Record size in bytes of one token row of `head_dim` channels at bit-width b, or 0 if b is
+ * not one of {2,4,8,16}.  Host only.  (Closed form above; Section 3.1 for the code bytes.) */
+QKVS_API size_t qkvs_record_bytes(int32_t head_dim, int32_t b);
+
+/* Exact size of the card for a bit-width vector (Section 4.2.1: the card is variable-length,
+ * its size follows from b(t)).  Host only, no GPU work.
+ *   bits_host  host array, n_tokens entries (mode 0) or n_layers*n_kv_heads*n_tokens (mode 1);
+ *              NULL gives the worst case (every token FP16).
+ *   out_bytes  receives header + tables + payload.
+ * Strides of `layout` are not looked at.  Errors: INVALID_ARG, UNSUPPORTED_SHAPE, BAD_BITS. */
+QKVS_API qkvs_status_t qkvs_card_size(const qkvs_layout_t *layout, const uint8_t *bits_host,
+                             size_t *out_bytes);
+
+/* Bytes in front of the payload (header + bits + offsets [+ stream bases]); a card buffer must
+ * hold at least this much for qkvs_card_create to start.  Host only. */
+QKVS_API qkvs_status_t qkvs_card_prefix_size(const qkvs_layout_t *layout, size_t *out_bytes);
+
+/* Card creation (Section 4.2.1): offset scan over the bit-widths, then fused
+ * min/max -> scale/zero -> quantise -> bit-pack of every (layer, K|V, head) stream.
+ *   K_layers, V_layers  HOST arrays of n_layers DEVICE pointers to FP16 blocks (16-byte aligned)
+ *   bits_dev            device array of bit-widths (see qkvs_card_size for its length)
+ *   meta                identifiers to store; NULL stores zeros
+ *   card_dev            device buffer, 16-byte aligned, written from byte 0
+ *   card_capacity       its size in bytes; must cover at least the prefix
+ * Returns after enqueueing on `stream`.  Problems visible on the host (arguments, shape,
+ * alignment, capacity below the prefix) are returned at once and nothing is launched.
+ * Problems only the device can see -- a bit-width outside {2,4,8,16}, or a payload that does
+ * not fit card_capacity -- are recorded in the card header's `status` (BAD_BITS,
+ * BUFFER_TOO_SMALL); the payload is then not written and nothing outside the buffer is touched.
+ * Read the outcome with qkvs_card_info.  The card's bytes are fully determined by the inputs. */
+QKVS_API qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K_layers,
+                               const void *const *V_layers, const uint8_t *bits_dev,
+                               const qkvs_card_meta_t *meta, void *card_dev,
+                               size_t card_capacity, void *stream);
+
+/* Receiver-side injection (Section 4.2.2): unpack, dequantise and write FP16 rows so that
+ * token t of the card lands on row dst_token_offset + t of every head of every layer.
+ *   card_dev, card_bytes   the card and the number of valid bytes behind the pointer
+ *   dst                    shape and strides of the destination; n_layers, n_kv_heads, head_dim
+ *                          and n_tokens must equal the card's (checked on the device), and
+ *                          (dst_token_offset + n_tokens - 1)*token_stride + head_dim <= head_stride
+ *   K_layers_out, V_layers_out   HOST arrays of n_layers DEVICE pointers (16-byte aligned)
+ *   status_dev             optional device int32, set to 0 by this call and raised to
+ *                          BAD_CARD by the kernel if the header or its tables do not check out
+ *                          (then no row is written); may be NULL
+ * Bytes of the destination outside the injected rows and channels are left untouched. */
+QKVS_API qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qkvs_layout_t *dst,
+                               void *const *K_layers_out, void *const *V_layers_out,
+                               int64_t dst_token_offset, int32_t *status_dev, void *stream);
+
+/* Synchronises `stream`, copies the card's header to the host and returns its recorded status
+ * (or BAD_CARD if magic/version are wrong, or CUDA on a runtime error). */
+QKVS_API qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_card_header_t *out_host);
+
+QKVS_API const char *qkvs_status_string(qkvs_status_t status);
+
+/* Library version, major*100 + minor. */
+QKVS_API int32_t qkvs_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QKVSHARE_H_ */

@@ -478,8 +478,9 @@ int orc_card_create(const orc_layout *L, const uint16_t *const *K_layers,
                                  L ? 2 * (int64_t)L->n_layers * L->n_kv_heads : 0);
 }
 
-/* Card -> FP16 keys and values.  `dst` gives the destination's strides and its capacity in
- * tokens (dst->n_tokens); token t of the card lands on row dst_token_offset + t. */
+/* Card -> FP16 keys and values.  `dst` gives the destination's shape (which must be the
+ * card's, n_tokens included) and strides; token t of the card lands on row
+ * dst_token_offset + t, and those rows must fit inside one head's slab. */
 int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *dst,
                     uint16_t *const *K_out, uint16_t *const *V_out, int64_t dst_token_offset)
 {
@@ -493,10 +494,14 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
     C.n_tokens = (int32_t)get_u32(card + 28);
     if ((int32_t)get_u32(card + 16) != dst->n_layers || (int32_t)get_u32(card + 20) != dst->n_kv_heads ||
         (int32_t)get_u32(card + 24) != dst->head_dim || get_u32(card + 32) != 32u ||
-        get_u32(card + 36) != 8u || (C.bits_mode != 0 && C.bits_mode != 1) || C.n_tokens < 0)
+        get_u32(card + 36) != 8u || (C.bits_mode != 0 && C.bits_mode != 1) ||
+        C.n_tokens != dst->n_tokens)
         return ORC_BAD_CARD;
     if (get_u64(card + 112) > card_bytes) return ORC_BAD_CARD;
-    if (dst_token_offset < 0 || dst_token_offset + C.n_tokens > dst->n_tokens) return ORC_INVALID_ARG;
+    if (dst_token_offset < 0 || dst->token_stride < dst->head_dim) return ORC_INVALID_ARG;
+    if (C.n_tokens > 0 &&
+        (dst_token_offset + C.n_tokens - 1) * dst->token_stride + dst->head_dim > dst->head_stride)
+        return ORC_INVALID_ARG;
     uint64_t bo = get_u64(card + 80), oo = get_u64(card + 88);
     int64_t T = C.n_tokens, S = 2 * (int64_t)C.n_layers * C.n_kv_heads;
 #ifdef _OPENMP

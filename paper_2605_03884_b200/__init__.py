@@ -1,0 +1,9 @@
+"""QKVShare CacheCard create / inject for B200: thin Python face of the CUDA library.
+
+`binding` marshals arguments into the C entry points of libqkvshare.so; `workloads` generates
+the seeded synthetic caches and bit-width vectors; `build` compiles the library in-tree.
+"""
+from . import binding, workloads  # noqa: F401
+from .binding import (CardHeader, CardMeta, Layout, QkvsError, card_create, card_info,  # noqa: F401
+                      card_inject, card_prefix_size, card_size, layout_of, load_library,
+                      make_layout, record_bytes, status_string, version)

@@ -1,0 +1,195 @@
+"""ctypes binding of libqkvshare.so: argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels.  PyTorch tensors are used as
+device buffers and for the current stream; nothing here computes.  If the shared library is
+missing the functions raise: there is no fallback implementation.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG_DIR, "libqkvshare.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_BAD_BITS, ERR_BUFFER_TOO_SMALL, ERR_BAD_CARD, \
+    ERR_CUDA, ERR_TIMEOUT = range(8)
+
+
+class QkvsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class Layout(C.Structure):
+    """qkvs_layout_t"""
+    _fields_ = [("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("n_tokens", C.c_int32), ("group_size", C.c_int32), ("bits_mode", C.c_int32),
+                ("head_stride", C.c_int64), ("token_stride", C.c_int64)]
+
+
+class CardMeta(C.Structure):
+    """qkvs_card_meta_t"""
+    _fields_ = [("model_id", C.c_uint64), ("sender_id", C.c_uint64), ("position_offset", C.c_int64)]
+
+
+class CardHeader(C.Structure):
+    """qkvs_card_header_t"""
+    _fields_ = [("magic", C.c_uint32), ("version", C.c_uint32), ("status", C.c_uint32),
+                ("bits_mode", C.c_uint32), ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("n_tokens", C.c_int32), ("group_size", C.c_int32),
+                ("meta_bytes_per_group", C.c_uint32), ("model_id", C.c_uint64),
+                ("sender_id", C.c_uint64), ("position_offset", C.c_int64), ("sum_bits", C.c_uint64),
+                ("avg_code_bits", C.c_float), ("pad0_", C.c_uint32), ("bits_off", C.c_uint64),
+                ("offs_off", C.c_uint64), ("payload_off", C.c_uint64), ("stream_bytes", C.c_uint64),
+                ("total_bytes", C.c_uint64), ("sbase_off", C.c_uint64), ("reserved_", C.c_uint8 * 128)]
+
+
+assert C.sizeof(CardHeader) == 256
+
+EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
+           "qkvs_card_inject", "qkvs_card_info", "qkvs_status_string", "qkvs_version")
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None):
+    """Load libqkvshare.so (built in-tree by paper_2605_03884_b200/build.py)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise RuntimeError(
+            f"{p} not found: build it with `python -m paper_2605_03884_b200.build` "
+            "(there is no CPU fallback)")
+    lib = C.CDLL(p)
+    vp = C.c_void_p
+    lib.qkvs_record_bytes.restype = C.c_size_t
+    lib.qkvs_record_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.qkvs_card_size.restype = C.c_int
+    lib.qkvs_card_size.argtypes = [C.POINTER(Layout), vp, C.POINTER(C.c_size_t)]
+    lib.qkvs_card_prefix_size.restype = C.c_int
+    lib.qkvs_card_prefix_size.argtypes = [C.POINTER(Layout), C.POINTER(C.c_size_t)]
+    lib.qkvs_card_create.restype = C.c_int
+    lib.qkvs_card_create.argtypes = [C.POINTER(Layout), vp, vp, vp, C.POINTER(CardMeta), vp, C.c_size_t, vp]
+    lib.qkvs_card_inject.restype = C.c_int
+    lib.qkvs_card_inject.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
+    lib.qkvs_card_info.restype = C.c_int
+    lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
+    lib.qkvs_status_string.restype = C.c_char_p
+    lib.qkvs_status_string.argtypes = [C.c_int]
+    lib.qkvs_version.restype = C.c_int32
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().qkvs_status_string(int(status)).decode()
+
+
+def make_layout(n_layers: int, n_kv_heads: int, head_dim: int, n_tokens: int, bits_mode: int = 0,
+                head_stride: Optional[int] = None, token_stride: Optional[int] = None) -> Layout:
+    ts = head_dim if token_stride is None else token_stride
+    hs = n_tokens * ts if head_stride is None else head_stride
+    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, 32, bits_mode, hs, ts)
+
+
+def layout_of(tensors: Sequence, n_tokens: Optional[int] = None, bits_mode: int = 0) -> Layout:
+    """Layout of a list of per-layer torch tensors shaped [H, T_cap, d] or [1, H, T_cap, d]."""
+    t = tensors[0]
+    if t.dim() == 4:
+        if t.shape[0] != 1:
+            raise ValueError("batch size must be 1")
+        t = t[0]
+    if t.dim() != 3 or t.stride(2) != 1:
+        raise ValueError("expected [H, T, d] with unit channel stride")
+    h, tcap, d = t.shape
+    return Layout(len(tensors), h, d, tcap if n_tokens is None else n_tokens, 32, bits_mode,
+                  t.stride(0), t.stride(1))
+
+
+def _ptr_array(tensors: Sequence):
+    return (C.c_void_p * len(tensors))(*[int(t.data_ptr()) for t in tensors])
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)
+
+
+def record_bytes(head_dim: int, b: int) -> int:
+    return int(load_library().qkvs_record_bytes(head_dim, b))
+
+
+def card_size(layout: Layout, bits_host=None) -> int:
+    """qkvs_card_size.  bits_host: numpy uint8 array / bytes on the host, or None (worst case)."""
+    out = C.c_size_t(0)
+    ptr = None
+    keep = None
+    if bits_host is not None:
+        import numpy as np
+        keep = np.ascontiguousarray(bits_host, dtype=np.uint8)
+        ptr = keep.ctypes.data
+    st = load_library().qkvs_card_size(C.byref(layout), ptr, C.byref(out))
+    if st != OK:
+        raise QkvsError(st, "qkvs_card_size")
+    return int(out.value)
+
+
+def card_prefix_size(layout: Layout) -> int:
+    out = C.c_size_t(0)
+    st = load_library().qkvs_card_prefix_size(C.byref(layout), C.byref(out))
+    if st != OK:
+        raise QkvsError(st, "qkvs_card_prefix_size")
+    return int(out.value)
+
+
+def card_create(layout: Layout, K_layers: Sequence, V_layers: Sequence, bits_dev, card_dev,
+                meta: Optional[CardMeta] = None, card_capacity: Optional[int] = None,
+                stream=None, check: bool = True) -> int:
+    """qkvs_card_create.  K_layers / V_layers: per-layer CUDA tensors (FP16); bits_dev: CUDA uint8
+    tensor; card_dev: CUDA uint8 tensor that receives the card.  Returns the status."""
+    lib = load_library()
+    kp, vp = _ptr_array(K_layers), _ptr_array(V_layers)
+    cap = int(card_dev.numel() * card_dev.element_size()) if card_capacity is None else int(card_capacity)
+    st = lib.qkvs_card_create(C.byref(layout), kp, vp, int(bits_dev.data_ptr()) if bits_dev is not None else None,
+                              C.byref(meta) if meta is not None else None, int(card_dev.data_ptr()), cap,
+                              _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_card_create")
+    return st
+
+
+def card_inject(card_dev, dst_layout: Layout, K_out: Sequence, V_out: Sequence,
+                dst_token_offset: int = 0, card_bytes: Optional[int] = None, status_dev=None,
+                stream=None, check: bool = True) -> int:
+    """qkvs_card_inject.  status_dev: optional CUDA int32 tensor of one element."""
+    lib = load_library()
+    kp, vp = _ptr_array(K_out), _ptr_array(V_out)
+    nbytes = int(card_dev.numel() * card_dev.element_size()) if card_bytes is None else int(card_bytes)
+    st = lib.qkvs_card_inject(int(card_dev.data_ptr()), nbytes, C.byref(dst_layout), kp, vp,
+                              int(dst_token_offset),
+                              int(status_dev.data_ptr()) if status_dev is not None else None,
+                              _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_card_inject")
+    return st
+
+
+def card_info(card_dev, stream=None):
+    """qkvs_card_info -> (status, CardHeader).  Synchronises the stream."""
+    hdr = CardHeader()
+    st = load_library().qkvs_card_info(int(card_dev.data_ptr()), _stream_handle(stream), C.byref(hdr))
+    return st, hdr
+
+
+def version() -> int:
+    return int(load_library().qkvs_version())

@@ -1,0 +1,751 @@
+// CacheCard create / inject: kernels and the C entry points declared in qkvshare.h.
+//
+// Three kernels make up the path:
+//   scan_offsets_kernel   per-segment exclusive prefix sum of record sizes over the bit-width
+//                         vector; writes the card's header, bits and offset tables
+//   create_kernel         fused group min/max -> scale/zero -> quantise -> bit-pack; one CTA
+//                         turns a tile of consecutive tokens of one stream into one contiguous
+//                         span of the card, staged in shared memory and stored 16 bytes a lane
+//   inject_kernel         reads records, unpacks, dequantises and writes FP16 rows into the
+//                         destination cache layout
+// A stream is one (layer, K|V, head) matrix [tokens, head_dim].
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+
+#include "qkvs_common.cuh"
+
+namespace qkvs {
+
+// ---------------------------------------------------------------------------------------------
+// Offset scan
+
+constexpr int kScanThreads = 1024;
+constexpr int kScanItems = 8;
+
+struct ScanParams {
+    const uint8_t *bits;  // device, [nseg][T]
+    uint8_t *card;
+    uint64_t capacity;
+    int32_t n_layers, n_kv_heads, head_dim, n_tokens, bits_mode;
+    uint64_t model_id, sender_id;
+    int64_t position_offset;
+};
+
+// Exclusive scan of one value per thread over the block; returns the block total through
+// `total`.  `warp_sums` is shared scratch of 32 entries.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t *warp_sums, uint32_t &total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, inc, s);
+        if (lane >= s) inc += n;
+    }
+    __syncthreads();  // warp_sums may still be read from the previous call
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < (int)(blockDim.x >> 5) ? warp_sums[lane] : 0u;
+        uint32_t winc = w;
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) {
+            const uint32_t n = __shfl_up_sync(0xffffffffu, winc, s);
+            if (lane >= s) winc += n;
+        }
+        warp_sums[lane] = winc - w;  // exclusive warp prefix
+        if (lane == 31) warp_sums[32] = winc;
+    }
+    __syncthreads();
+    total = warp_sums[32];
+    return warp_sums[warp] + inc - v;
+}
+
+__device__ __forceinline__ void write_header_static(qkvs_card_header_t *h, const ScanParams &p, const Sections &sec)
+{
+    h->magic = kMagic;
+    h->version = kVersion;
+    h->bits_mode = (uint32_t)p.bits_mode;
+    h->n_layers = p.n_layers;
+    h->n_kv_heads = p.n_kv_heads;
+    h->head_dim = p.head_dim;
+    h->n_tokens = p.n_tokens;
+    h->group_size = kGroup;
+    h->meta_bytes_per_group = kMetaBytesPerGroup;
+    h->model_id = p.model_id;
+    h->sender_id = p.sender_id;
+    h->position_offset = p.position_offset;
+    h->pad0_ = 0;
+    h->bits_off = sec.bits_off;
+    h->offs_off = sec.offs_off;
+    h->payload_off = sec.payload_off;
+    h->sbase_off = sec.sbase_off;
+}
+
+__device__ __forceinline__ void zero_fill(uint8_t *p, uint64_t begin, uint64_t end)
+{
+    for (uint64_t i = begin + threadIdx.x; i < end; i += blockDim.x) p[i] = 0;
+}
+
+// One CTA per segment.  bits_mode 0 has a single segment, and its CTA also finishes the
+// header; in bits_mode 1 the per-segment results are combined by finalize_kernel.
+__global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p)
+{
+    __shared__ uint32_t warp_sums[33];
+    __shared__ int s_bad;
+    const int seg = blockIdx.x;
+    const int64_t T = p.n_tokens;
+    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
+    const uint8_t *bits = p.bits + (int64_t)seg * T;
+    uint8_t *bits_out = p.card + sec.bits_off + (uint64_t)seg * (uint64_t)T;
+    uint32_t *off_out = reinterpret_cast<uint32_t *>(p.card + sec.offs_off) + (uint64_t)seg * (uint64_t)(T + 1);
+    const int d = p.head_dim;
+
+    if (threadIdx.x == 0) s_bad = 0;
+    uint32_t carry = 0;
+    uint64_t sum_bits = 0;
+    bool bad = false;
+    for (int64_t tile = 0; tile < T; tile += (int64_t)kScanThreads * kScanItems) {
+        const int64_t t0 = tile + (int64_t)threadIdx.x * kScanItems;
+        uint32_t rec[kScanItems];
+        uint8_t bv[kScanItems];
+        uint32_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < kScanItems; ++i) {
+            rec[i] = 0;
+            bv[i] = 0;
+            if (t0 + i < T) {
+                bv[i] = bits[t0 + i];
+                rec[i] = record_bytes(d, bv[i]);
+                bad |= rec[i] == 0u;
+                sum_bits += bv[i];
+                mine += rec[i];
+            }
+        }
+        uint32_t total;
+        uint32_t run = carry + block_exclusive_scan(mine, warp_sums, total);
+#pragma unroll
+        for (int i = 0; i < kScanItems; ++i) {
+            if (t0 + i < T) {
+                off_out[t0 + i] = run;
+                bits_out[t0 + i] = bv[i];
+                run += rec[i];
+            }
+        }
+        carry += total;
+    }
+    if (threadIdx.x == 0) off_out[T] = carry;
+    if (bad) s_bad = 1;
+
+    // total of sum_bits over the block
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) sum_bits += __shfl_xor_sync(0xffffffffu, sum_bits, s);
+    __shared__ unsigned long long s_sum;
+    __syncthreads();
+    if (threadIdx.x == 0) s_sum = 0;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) atomicAdd(&s_sum, (unsigned long long)sum_bits);
+    __syncthreads();
+
+    qkvs_card_header_t *h = reinterpret_cast<qkvs_card_header_t *>(p.card);
+    if (p.bits_mode == 0) {
+        // zero padding of the tables and the header's reserved tail
+        zero_fill(p.card, sec.bits_off + (uint64_t)T, sec.offs_off);
+        zero_fill(p.card, sec.offs_off + 4u * (uint64_t)(T + 1), sec.payload_off);
+        zero_fill(p.card, offsetof(qkvs_card_header_t, reserved_), kHeaderBytes);
+        if (threadIdx.x == 0) {
+            const uint64_t S = 2u * (uint64_t)p.n_layers * (uint64_t)p.n_kv_heads;
+            const uint64_t total = sec.payload_off + S * (uint64_t)carry;
+            uint32_t status = QKVS_OK;
+            if (s_bad) status = QKVS_ERR_BAD_BITS;
+            else if (total > p.capacity) status = QKVS_ERR_BUFFER_TOO_SMALL;
+            write_header_static(h, p, sec);
+            h->status = status;
+            const bool ok = status == QKVS_OK;
+            h->sum_bits = ok ? s_sum : 0;
+            h->avg_code_bits = (ok && T > 0) ? __fdiv_rn((float)s_sum, (float)(uint64_t)T) : 0.0f;
+            h->stream_bytes = ok ? carry : 0;
+            h->total_bytes = ok ? total : 0;
+        }
+    } else if (threadIdx.x == 0) {
+        // header was cleared before this launch; combine across segments
+        atomicAdd(reinterpret_cast<unsigned long long *>(&h->sum_bits), s_sum);
+        if (s_bad) atomicMax(&h->status, (uint32_t)QKVS_ERR_BAD_BITS);
+    }
+}
+
+// bits_mode 1 only: one CTA turns the per-segment totals into the stream-base table, pads the
+// tables with zeros and completes the header.
+__global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
+{
+    __shared__ uint64_t s_carry;
+    __shared__ uint64_t s_warp[33];
+    const int64_t T = p.n_tokens;
+    const int H = p.n_kv_heads;
+    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
+    const int64_t nseg = (int64_t)p.n_layers * H;
+    const int64_t S = 2 * nseg;
+    qkvs_card_header_t *h = reinterpret_cast<qkvs_card_header_t *>(p.card);
+    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off);
+    uint64_t *sbase = reinterpret_cast<uint64_t *>(p.card + sec.sbase_off);
+    const bool bad = h->status != QKVS_OK;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < S; base += kScanThreads) {
+        const int64_t s = base + threadIdx.x;
+        uint64_t v = 0;
+        if (s < S && !bad) {
+            const int64_t l = s / (2 * H), hh = s % H;
+            v = offs[(l * H + hh) * (T + 1) + T];
+        }
+        uint64_t inc = v;
+#pragma unroll
+        for (int k = 1; k < 32; k <<= 1) {
+            const uint64_t n = __shfl_up_sync(0xffffffffu, inc, k);
+            if (lane >= k) inc += n;
+        }
+        if (lane == 31) s_warp[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            const uint64_t w = s_warp[lane];
+            uint64_t winc = w;
+#pragma unroll
+            for (int k = 1; k < 32; k <<= 1) {
+                const uint64_t n = __shfl_up_sync(0xffffffffu, winc, k);
+                if (lane >= k) winc += n;
+            }
+            s_warp[lane] = winc - w;
+            if (lane == 31) s_warp[32] = winc;
+        }
+        __syncthreads();
+        if (s < S) sbase[s] = bad ? 0 : s_carry + s_warp[warp] + inc - v;
+        __syncthreads();
+        if (threadIdx.x == 0) s_carry += s_warp[32];
+        __syncthreads();
+    }
+    zero_fill(p.card, sec.bits_off + (uint64_t)nseg * (uint64_t)T, sec.offs_off);
+    zero_fill(p.card, sec.offs_off + 4u * (uint64_t)nseg * (uint64_t)(T + 1), sec.sbase_off);
+    zero_fill(p.card, sec.sbase_off + 8u * (uint64_t)(S + 1), sec.payload_off);
+    if (threadIdx.x == 0) {
+        const uint64_t payload = s_carry;
+        sbase[S] = bad ? 0 : payload;
+        uint32_t status = h->status;
+        const uint64_t total = sec.payload_off + payload;
+        if (status == QKVS_OK && total > p.capacity) status = QKVS_ERR_BUFFER_TOO_SMALL;
+        write_header_static(h, p, sec);
+        h->status = status;
+        const bool ok = status == QKVS_OK;
+        const uint64_t sb = h->sum_bits;
+        h->sum_bits = ok ? sb : 0;
+        h->avg_code_bits = (ok && nseg * T > 0) ? __fdiv_rn((float)sb, (float)(uint64_t)(nseg * T)) : 0.0f;
+        h->stream_bytes = 0;
+        h->total_bytes = ok ? total : 0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Stream bookkeeping shared by create and inject
+
+struct StreamInfo {
+    int layer_local;   // layer index inside this launch's pointer block
+    int kv, head;
+    int64_t seg;       // segment whose bits / offsets the stream uses
+    uint64_t base;     // byte offset of the stream inside the card
+};
+
+__device__ __forceinline__ StreamInfo locate_stream(const PathParams &p, const Sections &sec, int64_t s_local,
+                                                    uint64_t stream_bytes)
+{
+    StreamInfo si;
+    const int H = p.n_kv_heads;
+    si.head = (int)(s_local % H);
+    si.kv = (int)((s_local / H) & 1);
+    si.layer_local = (int)(s_local / (2 * H));
+    const int64_t layer = p.layer_begin + si.layer_local;
+    const int64_t s = (layer * 2 + si.kv) * H + si.head;
+    if (p.bits_mode == 0) {
+        si.seg = 0;
+        si.base = sec.payload_off + (uint64_t)s * stream_bytes;
+    } else {
+        si.seg = layer * H + si.head;
+        si.base = sec.payload_off + reinterpret_cast<const uint64_t *>(p.card + sec.sbase_off)[s];
+    }
+    return si;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Card creation: fused min/max -> scale/zero -> quantise -> pack
+
+template <int D, int TB, int THREADS>
+__global__ void __launch_bounds__(THREADS) create_kernel(PathParams p, LayerPtrs ptrs)
+{
+    constexpr int CPR = D / 8;  // chunks (threads) per token row
+    constexpr int G = D / kGroup;
+    constexpr int ITER = (TB * CPR + THREADS - 1) / THREADS;
+    static_assert((TB * CPR) % THREADS == 0, "tile must be a whole number of passes");
+    __shared__ __align__(16) uint8_t s_out[TB * 2 * D];
+    __shared__ uint32_t s_off[TB + 1];
+    __shared__ uint8_t s_bits[TB];
+
+    const qkvs_card_header_t *hdr = reinterpret_cast<const qkvs_card_header_t *>(p.card);
+    if (hdr->status != QKVS_OK) return;  // bad bits or short buffer: no payload is written
+    const uint64_t stream_bytes = hdr->stream_bytes;
+    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
+
+    const int64_t s_local = blockIdx.x / p.tiles_per_stream;
+    const int64_t t0 = (int64_t)(blockIdx.x % p.tiles_per_stream) * TB;
+    const int rows = (int)min((int64_t)TB, (int64_t)p.n_tokens - t0);
+    const StreamInfo si = locate_stream(p, sec, s_local, stream_bytes);
+    const int64_t T = p.n_tokens;
+    const uint8_t *bits = p.card + sec.bits_off + (uint64_t)si.seg * (uint64_t)T + t0;
+    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) + (uint64_t)si.seg * (uint64_t)(T + 1) + t0;
+    for (int i = threadIdx.x; i <= rows; i += THREADS) {
+        s_off[i] = offs[i];
+        if (i < rows) s_bits[i] = bits[i];
+    }
+    __syncthreads();
+    const uint32_t off0 = s_off[0];
+
+    const __half *src = reinterpret_cast<const __half *>(si.kv == 0 ? ptrs.k[si.layer_local] : ptrs.v[si.layer_local]) +
+                        (int64_t)si.head * p.head_stride + t0 * p.token_stride;
+
+    uint4 v[ITER];
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int c = it * THREADS + threadIdx.x;
+        const int row = c / CPR, pos = c % CPR;
+        v[it] = make_uint4(0, 0, 0, 0);
+        if (row < rows) v[it] = __ldg(reinterpret_cast<const uint4 *>(src + (int64_t)row * p.token_stride + pos * 8));
+    }
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int c = it * THREADS + threadIdx.x;
+        const int row = c / CPR, pos = c % CPR;
+        const bool valid = row < rows;
+        const int b = valid ? s_bits[row] : 16;
+        float mn, mx;
+        group_min_max(v[it], mn, mx);
+        if (!valid) continue;
+        uint8_t *rec = s_out + (s_off[row] - off0);
+        if (b == 16) {
+            *reinterpret_cast<uint4 *>(rec + pos * 16) = v[it];
+            continue;
+        }
+        const int qmax = (1 << b) - 1;
+        const GroupParams g = group_params(mn, mx, (float)qmax);
+        if ((pos & 3) == 0) *reinterpret_cast<float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup) = make_float2(g.scale, g.zero);
+        uint32_t q[8];
+        quantize_chunk(v[it], g, qmax, q);
+        uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * b;  // 8 codes of b bits = b bytes
+        if (b == 4) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w |= q[i] << (4 * i);
+            *reinterpret_cast<uint32_t *>(codes) = w;
+        } else if (b == 2) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w |= q[i] << (2 * i);
+            *reinterpret_cast<uint16_t *>(codes) = (uint16_t)w;
+        } else {
+            const uint32_t w0 = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
+            const uint32_t w1 = q[4] | (q[5] << 8) | (q[6] << 16) | (q[7] << 24);
+            *reinterpret_cast<uint2 *>(codes) = make_uint2(w0, w1);
+        }
+    }
+    __syncthreads();
+    const uint32_t n16 = (s_off[rows] - off0) >> 4;
+    uint4 *dst = reinterpret_cast<uint4 *>(p.card + si.base + off0);
+    const uint4 *so = reinterpret_cast<const uint4 *>(s_out);
+    for (uint32_t i = threadIdx.x; i < n16; i += THREADS) dst[i] = so[i];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Injection: unpack -> dequantise -> scatter
+
+__device__ __forceinline__ bool header_matches(const qkvs_card_header_t *h, const PathParams &p, const Sections &sec)
+{
+    bool ok = h->magic == kMagic && h->version == kVersion && h->status == QKVS_OK;
+    ok = ok && h->bits_mode == (uint32_t)p.bits_mode;
+    ok = ok && h->n_layers == p.n_layers && h->n_kv_heads == p.n_kv_heads && h->head_dim == p.head_dim;
+    ok = ok && h->n_tokens == p.n_tokens && h->group_size == kGroup && h->meta_bytes_per_group == kMetaBytesPerGroup;
+    ok = ok && h->bits_off == sec.bits_off && h->offs_off == sec.offs_off && h->payload_off == sec.payload_off;
+    ok = ok && h->sbase_off == sec.sbase_off;
+    ok = ok && h->total_bytes <= p.card_bytes && h->total_bytes >= sec.payload_off;
+    return ok;
+}
+
+template <int D, int TB, int THREADS>
+__global__ void __launch_bounds__(THREADS) inject_kernel(PathParams p, LayerPtrs ptrs)
+{
+    constexpr int CPR = D / 8;
+    constexpr int G = D / kGroup;
+    constexpr int ITER = (TB * CPR + THREADS - 1) / THREADS;
+    static_assert((TB * CPR) % THREADS == 0, "tile must be a whole number of passes");
+    __shared__ uint32_t s_off[TB + 1];
+    __shared__ uint8_t s_bits[TB];
+    __shared__ int s_ok;
+    __shared__ uint64_t s_base;
+
+    const qkvs_card_header_t *hdr = reinterpret_cast<const qkvs_card_header_t *>(p.card);
+    const int64_t s_local = blockIdx.x / p.tiles_per_stream;
+    const int64_t t0 = (int64_t)(blockIdx.x % p.tiles_per_stream) * TB;
+    const int rows = (int)min((int64_t)TB, (int64_t)p.n_tokens - t0);
+    const int64_t T = p.n_tokens;
+
+    // The card is untrusted input: nothing is read beyond card_bytes and no row is written
+    // unless the header and this tile's table entries are consistent.
+    if (threadIdx.x == 0) {
+        int ok = 0;
+        uint64_t base = 0;
+        const uint32_t mode = hdr->bits_mode;
+        if (mode <= 1u) {
+            PathParams q = p;
+            q.bits_mode = (int32_t)mode;
+            const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, (int)mode);
+            if (sec.payload_off <= p.card_bytes && header_matches(hdr, q, sec)) {
+                const uint64_t total = hdr->total_bytes;
+                const StreamInfo si = locate_stream(q, sec, s_local, hdr->stream_bytes);
+                base = si.base;
+                ok = base >= sec.payload_off && base <= total && (base & 15u) == 0;
+            }
+        }
+        s_ok = ok;
+        s_base = base;
+    }
+    __syncthreads();
+    if (!s_ok) {
+        if (threadIdx.x == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
+        return;
+    }
+    const int mode = (int)hdr->bits_mode;
+    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, mode);
+    const int H = p.n_kv_heads;
+    const int head = (int)(s_local % H), kv = (int)((s_local / H) & 1), layer_local = (int)(s_local / (2 * H));
+    const int64_t seg = mode == 0 ? 0 : (int64_t)(p.layer_begin + layer_local) * H + head;
+    const uint8_t *bits = p.card + sec.bits_off + (uint64_t)seg * (uint64_t)T + t0;
+    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) + (uint64_t)seg * (uint64_t)(T + 1) + t0;
+    for (int i = threadIdx.x; i <= rows; i += THREADS) {
+        s_off[i] = offs[i];
+        if (i < rows) s_bits[i] = bits[i];
+    }
+    __syncthreads();
+    int bad = 0;
+    for (int i = threadIdx.x; i < rows; i += THREADS) {
+        const uint32_t r = record_bytes(D, s_bits[i]);
+        bad |= (r == 0u) || (s_off[i + 1] - s_off[i] != r) || (s_off[i + 1] < s_off[i]);
+    }
+    if (threadIdx.x == 0) bad |= (s_base + (uint64_t)s_off[rows] > hdr->total_bytes) || (s_off[0] & 15u);
+    if (__syncthreads_or(bad)) {
+        if (threadIdx.x == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
+        return;
+    }
+
+    const uint8_t *stream = p.card + s_base;
+    __half *dst = reinterpret_cast<__half *>(kv == 0 ? ptrs.k[layer_local] : ptrs.v[layer_local]) +
+                  (int64_t)head * p.head_stride + (p.dst_token_offset + t0) * p.token_stride;
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+        const int c = it * THREADS + threadIdx.x;
+        const int row = c / CPR, pos = c % CPR;
+        if (row >= rows) continue;
+        const int b = s_bits[row];
+        const uint8_t *rec = stream + s_off[row];
+        uint4 out;
+        if (b == 16) {
+            out = __ldg(reinterpret_cast<const uint4 *>(rec + pos * 16));
+        } else {
+            const float2 m = __ldg(reinterpret_cast<const float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup));
+            const uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * b;
+            uint32_t q[8];
+            if (b == 4) {
+                const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(codes));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) q[i] = (w >> (4 * i)) & 15u;
+            } else if (b == 2) {
+                const uint32_t w = __ldg(reinterpret_cast<const uint16_t *>(codes));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) q[i] = (w >> (2 * i)) & 3u;
+            } else {
+                const uint2 w = __ldg(reinterpret_cast<const uint2 *>(codes));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    q[i] = (w.x >> (8 * i)) & 255u;
+                    q[4 + i] = (w.y >> (8 * i)) & 255u;
+                }
+            }
+            out.x = pack_half2(dequantize_one(q[0], m.x, m.y), dequantize_one(q[1], m.x, m.y));
+            out.y = pack_half2(dequantize_one(q[2], m.x, m.y), dequantize_one(q[3], m.x, m.y));
+            out.z = pack_half2(dequantize_one(q[4], m.x, m.y), dequantize_one(q[5], m.x, m.y));
+            out.w = pack_half2(dequantize_one(q[6], m.x, m.y), dequantize_one(q[7], m.x, m.y));
+        }
+        *reinterpret_cast<uint4 *>(dst + (int64_t)row * p.token_stride + pos * 8) = out;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+
+static qkvs_status_t check_shape(const qkvs_layout_t *l)
+{
+    if (!l) return QKVS_ERR_INVALID_ARG;
+    if (l->n_layers < 1 || l->n_kv_heads < 1 || l->n_tokens < 0) return QKVS_ERR_INVALID_ARG;
+    if (l->bits_mode != 0 && l->bits_mode != 1) return QKVS_ERR_INVALID_ARG;
+    if (l->group_size != kGroup) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (l->head_dim != 64 && l->head_dim != 128 && l->head_dim != 192 && l->head_dim != 256)
+        return QKVS_ERR_UNSUPPORTED_SHAPE;
+    // offsets inside a stream are 32-bit
+    if ((uint64_t)l->n_tokens * 2u * (uint64_t)l->head_dim > 0xffffffffull) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if ((uint64_t)l->n_layers * (uint64_t)l->n_kv_heads > (1u << 24)) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    return QKVS_OK;
+}
+
+static qkvs_status_t check_strides(const qkvs_layout_t *l, int64_t first_row)
+{
+    if (l->token_stride < l->head_dim || (l->token_stride & 7) || (l->head_stride & 7) || l->head_stride < 0)
+        return QKVS_ERR_INVALID_ARG;
+    if (first_row < 0) return QKVS_ERR_INVALID_ARG;
+    if (l->n_tokens > 0 && (first_row + l->n_tokens - 1) * l->token_stride + l->head_dim > l->head_stride &&
+        l->n_kv_heads > 1)
+        return QKVS_ERR_INVALID_ARG;
+    return QKVS_OK;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Tile of consecutive tokens handled by one CTA: 1024 chunks (4 passes of 256 threads), except
+// head_dim 192 where 32 tokens give 768 chunks (3 passes).
+template <int D>
+struct TileCfg {
+    static constexpr int THREADS = 256;
+    static constexpr int TB = D == 192 ? 32 : 8192 / D;
+};
+
+template <int D>
+static cudaError_t launch_create(const PathParams &pp, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+{
+    using C = TileCfg<D>;
+    PathParams p = pp;
+    p.tiles_per_stream = (uint32_t)((p.n_tokens + C::TB - 1) / C::TB);
+    const int64_t blocks = streams * p.tiles_per_stream;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7fffffffll) return cudaErrorInvalidConfiguration;
+    create_kernel<D, C::TB, C::THREADS><<<(unsigned)blocks, C::THREADS, 0, st>>>(p, ptrs);
+    return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t launch_inject(const PathParams &pp, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+{
+    using C = TileCfg<D>;
+    PathParams p = pp;
+    p.tiles_per_stream = (uint32_t)((p.n_tokens + C::TB - 1) / C::TB);
+    const int64_t blocks = streams * p.tiles_per_stream;
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7fffffffll) return cudaErrorInvalidConfiguration;
+    inject_kernel<D, C::TB, C::THREADS><<<(unsigned)blocks, C::THREADS, 0, st>>>(p, ptrs);
+    return cudaGetLastError();
+}
+
+}  // namespace qkvs
+
+using namespace qkvs;
+
+extern "C" {
+
+size_t qkvs_record_bytes(int32_t head_dim, int32_t b)
+{
+    if (head_dim <= 0 || head_dim % 64 != 0) return 0;
+    return record_bytes(head_dim, b);
+}
+
+qkvs_status_t qkvs_card_prefix_size(const qkvs_layout_t *layout, size_t *out_bytes)
+{
+    const qkvs_status_t st = check_shape(layout);
+    if (st != QKVS_OK) return st;
+    if (!out_bytes) return QKVS_ERR_INVALID_ARG;
+    *out_bytes = (size_t)card_sections(layout->n_layers, layout->n_kv_heads, layout->n_tokens, layout->bits_mode).payload_off;
+    return QKVS_OK;
+}
+
+qkvs_status_t qkvs_card_size(const qkvs_layout_t *layout, const uint8_t *bits_host, size_t *out_bytes)
+{
+    const qkvs_status_t st = check_shape(layout);
+    if (st != QKVS_OK) return st;
+    if (!out_bytes) return QKVS_ERR_INVALID_ARG;
+    const Sections sec = card_sections(layout->n_layers, layout->n_kv_heads, layout->n_tokens, layout->bits_mode);
+    const int64_t nseg = layout->bits_mode == 0 ? 1 : (int64_t)layout->n_layers * layout->n_kv_heads;
+    const uint64_t streams_per_seg = layout->bits_mode == 0 ? 2u * (uint64_t)layout->n_layers * (uint64_t)layout->n_kv_heads : 2u;
+    const int64_t T = layout->n_tokens;
+    uint64_t payload = 0;
+    for (int64_t seg = 0; seg < nseg; ++seg) {
+        uint64_t seg_bytes = 0;
+        for (int64_t t = 0; t < T; ++t) {
+            const uint32_t r = record_bytes(layout->head_dim, bits_host ? bits_host[seg * T + t] : 16);
+            if (r == 0) return QKVS_ERR_BAD_BITS;
+            seg_bytes += r;
+        }
+        payload += seg_bytes * streams_per_seg;
+    }
+    *out_bytes = (size_t)(sec.payload_off + payload);
+    return QKVS_OK;
+}
+
+qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K_layers, const void *const *V_layers,
+                               const uint8_t *bits_dev, const qkvs_card_meta_t *meta, void *card_dev,
+                               size_t card_capacity, void *stream)
+{
+    qkvs_status_t st = check_shape(layout);
+    if (st != QKVS_OK) return st;
+    if (!K_layers || !V_layers || !card_dev || (!bits_dev && layout->n_tokens > 0)) return QKVS_ERR_INVALID_ARG;
+    st = check_strides(layout, 0);
+    if (st != QKVS_OK) return st;
+    if (!aligned16(card_dev)) return QKVS_ERR_INVALID_ARG;
+    for (int l = 0; l < layout->n_layers; ++l)
+        if (!K_layers[l] || !V_layers[l] || !aligned16(K_layers[l]) || !aligned16(V_layers[l])) return QKVS_ERR_INVALID_ARG;
+    const Sections sec = card_sections(layout->n_layers, layout->n_kv_heads, layout->n_tokens, layout->bits_mode);
+    if (card_capacity < sec.payload_off) return QKVS_ERR_BUFFER_TOO_SMALL;
+
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    ScanParams sp;
+    sp.bits = bits_dev;
+    sp.card = static_cast<uint8_t *>(card_dev);
+    sp.capacity = card_capacity;
+    sp.n_layers = layout->n_layers;
+    sp.n_kv_heads = layout->n_kv_heads;
+    sp.head_dim = layout->head_dim;
+    sp.n_tokens = layout->n_tokens;
+    sp.bits_mode = layout->bits_mode;
+    sp.model_id = meta ? meta->model_id : 0;
+    sp.sender_id = meta ? meta->sender_id : 0;
+    sp.position_offset = meta ? meta->position_offset : 0;
+    const int nseg = layout->bits_mode == 0 ? 1 : layout->n_layers * layout->n_kv_heads;
+    if (layout->bits_mode == 1 && cudaMemsetAsync(card_dev, 0, kHeaderBytes, cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    scan_offsets_kernel<<<nseg, kScanThreads, 0, cs>>>(sp);
+    if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
+    if (layout->bits_mode == 1) {
+        finalize_kernel<<<1, kScanThreads, 0, cs>>>(sp);
+        if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
+    }
+
+    PathParams p;
+    memset(&p, 0, sizeof(p));
+    p.card = static_cast<uint8_t *>(card_dev);
+    p.card_bytes = card_capacity;
+    p.n_layers = layout->n_layers;
+    p.n_kv_heads = layout->n_kv_heads;
+    p.head_dim = layout->head_dim;
+    p.n_tokens = layout->n_tokens;
+    p.bits_mode = layout->bits_mode;
+    p.head_stride = layout->head_stride;
+    p.token_stride = layout->token_stride;
+    for (int l0 = 0; l0 < layout->n_layers; l0 += kMaxLayersPerLaunch) {
+        const int n = std::min(kMaxLayersPerLaunch, layout->n_layers - l0);
+        LayerPtrs ptrs;
+        memset(&ptrs, 0, sizeof(ptrs));
+        for (int i = 0; i < n; ++i) {
+            ptrs.k[i] = const_cast<void *>(K_layers[l0 + i]);
+            ptrs.v[i] = const_cast<void *>(V_layers[l0 + i]);
+        }
+        p.layer_begin = l0;
+        p.layer_count = n;
+        const int64_t streams = 2ll * n * layout->n_kv_heads;
+        cudaError_t e;
+        switch (layout->head_dim) {
+            case 64: e = launch_create<64>(p, ptrs, streams, cs); break;
+            case 128: e = launch_create<128>(p, ptrs, streams, cs); break;
+            case 192: e = launch_create<192>(p, ptrs, streams, cs); break;
+            default: e = launch_create<256>(p, ptrs, streams, cs); break;
+        }
+        if (e != cudaSuccess) return QKVS_ERR_CUDA;
+    }
+    return QKVS_OK;
+}
+
+qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qkvs_layout_t *dst,
+                               void *const *K_layers_out, void *const *V_layers_out, int64_t dst_token_offset,
+                               int32_t *status_dev, void *stream)
+{
+    qkvs_status_t st = check_shape(dst);
+    if (st != QKVS_OK) return st;
+    if (!card_dev || !K_layers_out || !V_layers_out) return QKVS_ERR_INVALID_ARG;
+    st = check_strides(dst, dst_token_offset);
+    if (st != QKVS_OK) return st;
+    if (!aligned16(card_dev)) return QKVS_ERR_INVALID_ARG;
+    if (card_bytes < (size_t)kHeaderBytes) return QKVS_ERR_BAD_CARD;
+    for (int l = 0; l < dst->n_layers; ++l)
+        if (!K_layers_out[l] || !V_layers_out[l] || !aligned16(K_layers_out[l]) || !aligned16(V_layers_out[l]))
+            return QKVS_ERR_INVALID_ARG;
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    if (status_dev && cudaMemsetAsync(status_dev, 0, sizeof(int32_t), cs) != cudaSuccess) return QKVS_ERR_CUDA;
+
+    PathParams p;
+    memset(&p, 0, sizeof(p));
+    p.card = const_cast<uint8_t *>(static_cast<const uint8_t *>(card_dev));
+    p.card_bytes = card_bytes;
+    p.n_layers = dst->n_layers;
+    p.n_kv_heads = dst->n_kv_heads;
+    p.head_dim = dst->head_dim;
+    p.n_tokens = dst->n_tokens;
+    p.bits_mode = 0;  // taken from the card on the device
+    p.head_stride = dst->head_stride;
+    p.token_stride = dst->token_stride;
+    p.dst_token_offset = dst_token_offset;
+    p.status_dev = status_dev;
+    for (int l0 = 0; l0 < dst->n_layers; l0 += kMaxLayersPerLaunch) {
+        const int n = std::min(kMaxLayersPerLaunch, dst->n_layers - l0);
+        LayerPtrs ptrs;
+        memset(&ptrs, 0, sizeof(ptrs));
+        for (int i = 0; i < n; ++i) {
+            ptrs.k[i] = K_layers_out[l0 + i];
+            ptrs.v[i] = V_layers_out[l0 + i];
+        }
+        p.layer_begin = l0;
+        p.layer_count = n;
+        const int64_t streams = 2ll * n * dst->n_kv_heads;
+        cudaError_t e;
+        switch (dst->head_dim) {
+            case 64: e = launch_inject<64>(p, ptrs, streams, cs); break;
+            case 128: e = launch_inject<128>(p, ptrs, streams, cs); break;
+            case 192: e = launch_inject<192>(p, ptrs, streams, cs); break;
+            default: e = launch_inject<256>(p, ptrs, streams, cs); break;
+        }
+        if (e != cudaSuccess) return QKVS_ERR_CUDA;
+    }
+    return QKVS_OK;
+}
+
+qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_card_header_t *out_host)
+{
+    if (!card_dev || !out_host) return QKVS_ERR_INVALID_ARG;
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(out_host, card_dev, kHeaderBytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    if (out_host->magic != kMagic || out_host->version != kVersion) return QKVS_ERR_BAD_CARD;
+    if (out_host->status > (uint32_t)QKVS_ERR_TIMEOUT) return QKVS_ERR_BAD_CARD;
+    return (qkvs_status_t)out_host->status;
+}
+
+const char *qkvs_status_string(qkvs_status_t status)
+{
+    switch (status) {
+        case QKVS_OK: return "ok";
+        case QKVS_ERR_INVALID_ARG: return "invalid argument";
+        case QKVS_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case QKVS_ERR_BAD_BITS: return "bit-width outside {2,4,8,16}";
+        case QKVS_ERR_BUFFER_TOO_SMALL: return "card buffer too small";
+        case QKVS_ERR_BAD_CARD: return "card header or tables do not check out";
+        case QKVS_ERR_CUDA: return "CUDA runtime error";
+        case QKVS_ERR_TIMEOUT: return "bounded wait inside a kernel gave up";
+    }
+    return "unknown status";
+}
+
+int32_t qkvs_version(void) { return 100; }
+
+}  // extern "C"

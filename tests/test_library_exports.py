@@ -1,0 +1,89 @@
+"""The C-ABI library loads and exports every symbol the public header declares (no GPU needed),
+and its host-only entry points agree with the closed forms."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2605_03884_b200 as q
+from paper_2605_03884_b200 import build as qbuild
+from golden_io import read_fixture
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    qbuild.build()
+    return q.load_library()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "qkvshare.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(qkvs_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert set(names) == set(q.binding.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_host_only_sizes(lib):
+    fx = read_fixture("card_sizes.txt")
+    for d, b, n in fx["rec"]:
+        assert q.record_bytes(int(d), int(b)) == int(n)
+    assert q.record_bytes(128, 3) == 0 and q.record_bytes(96, 4) == 0
+    a = lambda x: (x + 255) // 256 * 256
+    for L, H, d, T, c16, c8, c4, c2, payload in fx["payload"]:
+        L, H, d, T = int(L), int(H), int(d), int(T)
+        bits = np.concatenate([np.full(int(c16), 16), np.full(int(c8), 8), np.full(int(c4), 4),
+                               np.full(int(c2), 2)]).astype(np.uint8)
+        lay = q.make_layout(L, H, d, T)
+        assert q.card_size(lay, bits) == 256 + a(T) + a(4 * (T + 1)) + int(payload)
+        assert q.card_prefix_size(lay) == 256 + a(T) + a(4 * (T + 1))
+    lay = q.make_layout(2, 2, 64, 10)
+    assert q.card_size(lay, None) == q.card_size(lay, np.full(10, 16, np.uint8))
+    with pytest.raises(q.QkvsError) as e:
+        q.card_size(lay, np.array([4] * 9 + [5], np.uint8))
+    assert e.value.status == q.binding.ERR_BAD_BITS
+    with pytest.raises(q.QkvsError) as e:
+        q.card_size(q.make_layout(1, 1, 96, 4), None)
+    assert e.value.status == q.binding.ERR_UNSUPPORTED_SHAPE
+    # per-head bits: K and V of a (layer, head) share one segment
+    lay1 = q.make_layout(2, 3, 64, 5, bits_mode=1)
+    bits = np.tile(np.array([2, 4, 8, 16, 4], np.uint8), 6)
+    per_seg = 32 + 48 + 80 + 128 + 48
+    assert q.card_size(lay1, bits) == 256 + a(30) + a(4 * 6 * 6) + a(8 * 13) + 12 * per_seg
+
+
+def test_status_strings_and_version(lib):
+    assert q.version() >= 100
+    seen = {q.status_string(i) for i in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+
+
+def test_host_side_argument_checks_need_no_gpu(lib):
+    """Errors knowable on the host come back before any CUDA call."""
+    lay = q.make_layout(1, 1, 64, 4)
+    null = C.c_void_p(0)
+    arr = (C.c_void_p * 1)(0)
+    st = lib.qkvs_card_create(C.byref(lay), arr, arr, null, None, null, 0, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    bad = q.make_layout(1, 1, 64, 4, token_stride=60)
+    ptrs = (C.c_void_p * 1)(256)
+    st = lib.qkvs_card_create(C.byref(bad), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    mis = (C.c_void_p * 1)(264)
+    st = lib.qkvs_card_create(C.byref(lay), mis, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = lib.qkvs_card_create(C.byref(lay), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 100, None)
+    assert st == q.binding.ERR_BUFFER_TOO_SMALL
+    st = lib.qkvs_card_inject(C.c_void_p(256), 100, C.byref(lay), ptrs, ptrs, 0, None, None)
+    assert st == q.binding.ERR_BAD_CARD
+    st = lib.qkvs_card_inject(C.c_void_p(256), 4096, C.byref(lay), ptrs, ptrs, -1, None, None)
+    assert st == q.binding.ERR_INVALID_ARG

@@ -465,7 +465,7 @@ def test_inject_with_offset_and_padded_destination():
     Ks, Vs, lay = _cache(L, H, T, d, 66)
     bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 9)
     _, card = oracle.card_create(lay, Ks, Vs, bits)
-    Ko, Vo, dl = _cache(L, H, 64, d, 67, t_cap=64, token_stride=80)
+    Ko, Vo, dl = _cache(L, H, T, d, 67, t_cap=64, token_stride=80)
     before = [a.copy() for a in Ko]
     assert oracle.card_inject(card, dl, Ko, Vo, dst_token_offset=20) == oracle.OK
     for l in range(L):
