@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the CacheCard create + inject path.
+
+One *step* is one pass of the whole path over one synthetic cache: offset scan, fused
+quantise-pack (create), then unpack-dequantise-scatter (inject).  The default workload is the
+Llama-3.1-8B-shaped cache at 8K context with uniform 4-bit tokens; the metric is GB/s of FP16
+KV bytes carried through create + inject (KV bytes / (create time + inject time)).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2|3|4|5] [--impl ours|reference]
+
+With N > 1 (under torchrun) every rank runs an independent replica of the same workload: the
+path has no exchange step, so there is no data-path collective.  Rank 0 prints one JSON line.
+`--impl reference` times the CPU oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2605_03884_b200 import workloads as wl  # noqa: E402
+
+METRIC = "CacheCard create+inject throughput (FP16 KV bytes through create then inject)"
+UNIT = "GB/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu_index), "-lms", "50"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) < 9:
+                        continue
+                    try:
+                        sm.append(float(parts[1]))
+                        smax.append(float(parts[2]))
+                    except ValueError:
+                        continue
+                    for name, val in zip(names, parts[5:9]):
+                        if val.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def load_workload(number: int, layers=None):
+    w = wl.WORKLOADS[number]
+    Ks, Vs = [], []
+    for _, k, v in wl.kv_layers(w, layers):
+        Ks.append(k)
+        Vs.append(v)
+    return w, Ks, Vs
+
+
+def cpu_oracle_leg(w, Ks, Vs, bits, n_layers_sample: int):
+    """Times the oracle as it stands (create then inject) on the first `n_layers_sample` layers."""
+    import oracle
+    L = min(n_layers_sample, w.n_layers)
+    lay = oracle.make_layout(L, w.n_kv_heads, w.head_dim, w.n_tokens)
+    Ko = [np.zeros_like(k) for k in Ks[:L]]
+    Vo = [np.zeros_like(v) for v in Vs[:L]]
+    t0 = time.perf_counter()
+    st, card = oracle.card_create(lay, Ks[:L], Vs[:L], bits)
+    t1 = time.perf_counter()
+    st2 = oracle.card_inject(card, lay, Ko, Vo)
+    t2 = time.perf_counter()
+    assert st == 0 and st2 == 0
+    kv_bytes = 2 * L * w.n_kv_heads * w.n_tokens * w.head_dim * 2
+    return {
+        "value": kv_bytes / (t2 - t0) / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+        "sample": f"layers 0..{L - 1} of the workload ({kv_bytes} FP16 KV bytes), create then inject, "
+                  f"one repetition, OpenMP over streams",
+        "create_gbs": kv_bytes / (t1 - t0) / 1e9, "inject_gbs": kv_bytes / (t2 - t1) / 1e9,
+        "seconds": t2 - t0,
+    }
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle on the host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample_layers = 4
+    w, Ks, Vs = load_workload(args.config, range(sample_layers))
+    bits = wl.bits_for(w)
+    for _ in range(args.warmup):
+        cpu_oracle_leg(w, Ks, Vs, bits, sample_layers)
+    t0 = time.perf_counter()
+    legs = [cpu_oracle_leg(w, Ks, Vs, bits, sample_layers) for _ in range(args.steps)]
+    dt = time.perf_counter() - t0
+    kv_bytes = 2 * sample_layers * w.n_kv_heads * w.n_tokens * w.head_dim * 2
+    value = kv_bytes * args.steps / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": w.name, "sample_layers": sample_layers},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": legs[-1]["cores"], "kind": "oracle",
+                         "sample": legs[-1]["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2605_03884_b200 as q
+    from paper_2605_03884_b200 import build as qbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        qbuild.build()
+    if world > 1:
+        dist.barrier()
+    q.load_library()
+
+    w, Ks, Vs = load_workload(args.config)
+    L, H, d, T = w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens
+    hops = w.hops
+    bits_per_hop = [wl.bits_for(w, h) for h in range(hops)]
+    lay = q.make_layout(L, H, d, T)
+    sizes = [q.card_size(lay, b) for b in bits_per_hop]
+    prefix = q.card_prefix_size(lay)
+    kv_bytes = w.kv_bytes
+
+    # pinned host staging (end-to-end leg) and device buffers
+    Kh = [torch.from_numpy(k).pin_memory() for k in Ks]
+    Vh = [torch.from_numpy(v).pin_memory() for v in Vs]
+    Kd = [torch.empty_like(k, device="cuda") for k in Kh]
+    Vd = [torch.empty_like(v, device="cuda") for v in Vh]
+    Ko = [torch.empty_like(k) for k in Kd]
+    Vo = [torch.empty_like(v) for v in Vd]
+    Koh = [torch.empty_like(k).pin_memory() for k in Kh]
+    Voh = [torch.empty_like(v).pin_memory() for v in Vh]
+    bits_h = [torch.from_numpy(b).pin_memory() for b in bits_per_hop]
+    bits_d = [b.cuda() for b in bits_h]
+    card = torch.zeros(max(sizes), dtype=torch.uint8, device="cuda")
+    for dst, src in zip(Kd + Vd, Kh + Vh):
+        dst.copy_(src)
+    stream = torch.cuda.current_stream()
+
+    def one_step(record=None):
+        """create -> inject for every hop of the workload (one hop except for the chain)."""
+        src_k, src_v = Kd, Vd
+        for h in range(hops):
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e2 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            q.card_create(lay, src_k, src_v, bits_d[h], card, card_capacity=sizes[h], stream=stream)
+            e1.record(stream)
+            q.card_inject(card, lay, Ko, Vo, card_bytes=sizes[h], stream=stream)
+            e2.record(stream)
+            if record is not None:
+                record.append((h, e0, e1, e2))
+            src_k, src_v = Ko, Vo  # the next hop re-quantises this hop's output
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    torch.cuda.synchronize()
+    st, hdr = q.card_info(card)
+    if st != 0:
+        raise RuntimeError(f"card status {st}")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    records = []
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    for _ in range(args.steps):
+        one_step(records)
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    create_ms = [[] for _ in range(hops)]
+    inject_ms = [[] for _ in range(hops)]
+    for h, e0, e1, e2 in records:
+        create_ms[h].append(e0.elapsed_time(e1))
+        inject_ms[h].append(e1.elapsed_time(e2))
+
+    # end-to-end leg: host buffers in, host buffers out, copies inside the timed region
+    def e2e_step():
+        for dst, src in zip(Kd + Vd, Kh + Vh):
+            dst.copy_(src, non_blocking=True)
+        for bd, bh in zip(bits_d, bits_h):
+            bd.copy_(bh, non_blocking=True)
+        one_step()
+        for dst, src in zip(Koh + Voh, Ko + Vo):
+            dst.copy_(src, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e_begin = torch.cuda.Event(enable_timing=True)
+    e_end = torch.cuda.Event(enable_timing=True)
+    e_begin.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    e_end.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e_begin.elapsed_time(e_end)
+    clocks = sampler.stop() if rank == 0 else None
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peaks()
+    ms_per_step = total_ms / args.steps
+    units = kv_bytes * hops * world  # FP16 KV bytes carried through create+inject per step, all ranks
+    value = units / (ms_per_step * 1e-3) / 1e9
+    e2e_value = units / (e2e_ms / args.steps * 1e-3) / 1e9
+    med = statistics.median
+    per_hop = []
+    for h in range(hops):
+        payload = sizes[h] - prefix
+        c, i = med(create_ms[h]), med(inject_ms[h])
+        per_hop.append({
+            "hop": h, "card_bytes": sizes[h], "avg_code_bits": float(bits_per_hop[h].astype(np.float64).mean()),
+            "create_ms": c, "inject_ms": i,
+            "create_kv_gbs": kv_bytes / (c * 1e-3) / 1e9, "inject_kv_gbs": kv_bytes / (i * 1e-3) / 1e9,
+            "create_hbm_frac": (kv_bytes + payload) / (c * 1e-3) / 1e9 / peak,
+            "inject_hbm_frac": (kv_bytes + payload) / (i * 1e-3) / 1e9 / peak,
+        })
+    # dominant kernel: the slower of the two halves on hop 0
+    payload0 = sizes[0] - prefix
+    c0 = sum(create_ms[0]) / len(create_ms[0])
+    i0 = sum(inject_ms[0]) / len(inject_ms[0])
+    if c0 >= i0:
+        dom, dom_ms = "create_kernel (timed together with the offset scan that precedes it)", c0
+    else:
+        dom, dom_ms = "inject_kernel", i0
+    achieved = (kv_bytes + payload0) / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                "algorithmic_bytes_per_launch": kv_bytes + payload0, "avg_launch_ms": dom_ms}
+
+    launches_per_step = hops * (2 + 1) * ((L + 63) // 64) - hops * (((L + 63) // 64) - 1)
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu = cpu_oracle_leg(w, Ks, Vs, bits_per_hop[0], L)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "n_layers": L, "n_kv_heads": H, "head_dim": d, "n_tokens": T,
+                   "hops": hops, "fp16_kv_bytes": kv_bytes, "replicas": world,
+                   "l2": "inputs (1 GiB FP16 KV per pass) exceed the 126 MB L2; no flush"
+                   if kv_bytes > 4 * 126e6 else "working set comparable to L2; L2 helps"},
+        "per_hop": per_hop,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": kv_bytes + sum(int(b.numel()) for b in bits_h),
+                "d2h_bytes_per_step": kv_bytes, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3, choices=[2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
