@@ -100,8 +100,10 @@ class ClockSampler:
         return out
 
 
-def load_workload(number: int, layers=None):
+def load_workload(number: int, layers=None, n_layers=None):
     w = wl.WORKLOADS[number]
+    if n_layers:
+        w = w.scaled(n_layers=n_layers)   # reduced case for profiler captures only
     Ks, Vs = [], []
     for _, k, v in wl.kv_layers(w, layers):
         Ks.append(k)
@@ -181,7 +183,7 @@ def run_ours(args):
         dist.barrier()
     q.load_library()
 
-    w, Ks, Vs = load_workload(args.config)
+    w, Ks, Vs = load_workload(args.config, n_layers=args.layers)
     L, H, d, T = w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens
     hops = w.hops
     bits_per_hop = [wl.bits_for(w, h) for h in range(hops)]
@@ -262,18 +264,20 @@ def run_ours(args):
         for dst, src in zip(Koh + Voh, Ko + Vo):
             dst.copy_(src, non_blocking=True)
 
-    e2e_step()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    e_begin = torch.cuda.Event(enable_timing=True)
-    e_end = torch.cuda.Event(enable_timing=True)
-    e_begin.record(stream)
-    for _ in range(args.steps):
+    e2e_ms = float("nan")
+    if not args.skip_e2e:
         e2e_step()
-    e_end.record(stream)
-    torch.cuda.synchronize()
-    e2e_ms = e_begin.elapsed_time(e_end)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        e_begin = torch.cuda.Event(enable_timing=True)
+        e_end = torch.cuda.Event(enable_timing=True)
+        e_begin.record(stream)
+        for _ in range(args.steps):
+            e2e_step()
+        e_end.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms = e_begin.elapsed_time(e_end)
     clocks = sampler.stop() if rank == 0 else None
 
     if world > 1:
@@ -290,7 +294,7 @@ def run_ours(args):
     ms_per_step = total_ms / args.steps
     units = kv_bytes * hops * world  # FP16 KV bytes carried through create+inject per step, all ranks
     value = units / (ms_per_step * 1e-3) / 1e9
-    e2e_value = units / (e2e_ms / args.steps * 1e-3) / 1e9
+    e2e_value = None if args.skip_e2e else units / (e2e_ms / args.steps * 1e-3) / 1e9
     med = statistics.median
     per_hop = []
     for h in range(hops):
@@ -327,6 +331,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "n_layers": L, "n_kv_heads": H, "head_dim": d, "n_tokens": T,
                    "hops": hops, "fp16_kv_bytes": kv_bytes, "replicas": world,
+                   "reduced_for_profiling": bool(args.layers),
                    "l2": "inputs (1 GiB FP16 KV per pass) exceed the 126 MB L2; no flush"
                    if kv_bytes > 4 * 126e6 else "working set comparable to L2; L2 helps"},
         "per_hop": per_hop,
@@ -334,7 +339,8 @@ def run_ours(args):
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": kv_bytes + sum(int(b.numel()) for b in bits_h),
-                "d2h_bytes_per_step": kv_bytes, "ms_per_step": e2e_ms / args.steps},
+                "d2h_bytes_per_step": kv_bytes,
+                "ms_per_step": None if args.skip_e2e else e2e_ms / args.steps},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
     }
@@ -351,6 +357,9 @@ def main():
     ap.add_argument("--config", type=int, default=3, choices=[2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="reduced case for profiler captures: keep the workload's recipe at this many layers")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

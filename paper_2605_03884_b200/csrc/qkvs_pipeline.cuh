@@ -1,0 +1,440 @@
+// The two streaming kernels of the path, written as persistent, warp-specialised pipelines.
+//
+// A *tile* is TB consecutive tokens of one stream (one (layer, K|V, head) matrix).  On the FP16
+// side a tile is TB rows of 2*D bytes; on the card side it is one contiguous, 16-byte aligned
+// span of records whose length follows from the offset table.  Each CTA loops over tiles
+// (tile = blockIdx.x, blockIdx.x + gridDim.x, ...) with
+//   one producer warp   reads the tile's slice of the bits / offset tables, publishes per-row
+//                       record positions in shared memory and issues the bulk asynchronous
+//                       copy (TMA) of the tile's input into a ring of NS shared-memory stages;
+//   NW consumer warps   wait on the stage's mbarrier, transform 16 bytes per lane per pass and
+//                       hand the stage back through a second mbarrier.
+// create: consumer warp w owns RPW consecutive rows of the tile, writes their records into its
+//         own shared-memory buffer and one lane sends that contiguous span to the card with a
+//         bulk store (double buffered per warp, so no CTA-wide barrier is needed).
+// inject: consumers read records from the staged span and store FP16 rows straight to the
+//         destination, 512 contiguous bytes per warp and pass.
+// No wait is unbounded: see mbar_wait.
+#pragma once
+
+#include "qkvs_common.cuh"
+
+namespace qkvs {
+
+template <int D>
+struct PipeCfg {
+    static constexpr int NW = 8;                        // consumer warps
+    static constexpr int THREADS = (NW + 1) * 32;       // + one producer warp
+    static constexpr int CPR = D / 8;                   // 16-byte chunks (lanes) per token row
+    static constexpr int RPP = 32 / CPR;                // rows a warp covers per pass
+    static constexpr int LANES = RPP * CPR;             // lanes that carry data (24 for D = 192)
+    static constexpr int TB = D == 192 ? 32 : 8192 / D; // tokens per tile
+    static constexpr int RPW = TB / NW;                 // rows per consumer warp
+    static constexpr int PASSES = RPW / RPP;
+    static constexpr int ROW_BYTES = 2 * D;
+    static constexpr int TILE_BYTES = TB * ROW_BYTES;
+    static constexpr int G = D / kGroup;
+    static_assert(RPP >= 1 && RPW % RPP == 0 && TB % NW == 0, "tile shape");
+};
+
+struct StreamInfo {
+    int layer_local;   // layer index inside this launch's pointer block
+    int kv, head;
+    int64_t seg;       // segment whose bits / offsets the stream uses
+    uint64_t base;     // byte offset of the stream inside the card
+};
+
+__device__ __forceinline__ StreamInfo locate_stream(const PathParams &p, const Sections &sec, int bits_mode,
+                                                    int64_t s_local, uint64_t stream_bytes)
+{
+    StreamInfo si;
+    const int H = p.n_kv_heads;
+    si.head = (int)(s_local % H);
+    si.kv = (int)((s_local / H) & 1);
+    si.layer_local = (int)(s_local / (2 * H));
+    const int64_t layer = p.layer_begin + si.layer_local;
+    const int64_t s = (layer * 2 + si.kv) * H + si.head;
+    if (bits_mode == 0) {
+        si.seg = 0;
+        si.base = sec.payload_off + (uint64_t)s * stream_bytes;
+    } else {
+        si.seg = layer * H + si.head;
+        si.base = sec.payload_off + reinterpret_cast<const uint64_t *>(p.card + sec.sbase_off)[s];
+    }
+    return si;
+}
+
+// ---------------------------------------------------------------------------------------------
+// create: FP16 rows -> records
+
+template <int D, int NS>
+struct CreateSmem {
+    using C = PipeCfg<D>;
+    alignas(128) uint8_t in[NS][C::TILE_BYTES];
+    alignas(128) uint8_t out[C::NW][2][C::RPW * C::ROW_BYTES];
+    uint2 info[NS][C::TB];          // per row: {record offset inside its warp's span, bit-width}
+    uint64_t span_dst[NS][C::NW];   // per consumer warp: global address of its span
+    uint32_t span_bytes[NS][C::NW];
+    uint32_t uniform_bits[NS][C::NW];  // bit-width shared by all rows of the warp, else 0
+    int32_t rows[NS];
+    uint32_t off_tmp[C::TB + 1];    // producer scratch
+    uint64_t full[NS];
+    uint64_t empty[NS];
+    int abort_flag;
+};
+
+// One chunk: 8 FP16 values (group minimum / maximum already known) -> metadata and codes written
+// into the record at `rec` (shared memory).  B is the warp-uniform bit-width, or 0 when lanes
+// may differ (then `b` is used).
+template <int D, int B>
+__device__ __forceinline__ void encode_chunk(const uint4 &v, float mn, float mx, int b, uint8_t *rec, int pos)
+{
+    constexpr int G = D / kGroup;
+    const int bb = B ? B : b;
+    if (bb == 16) {
+        *reinterpret_cast<uint4 *>(rec + pos * 16) = v;
+        return;
+    }
+    const GroupParams g = group_params(mn, mx, bb);
+    uint32_t lo, hi;
+    quantize_chunk_bytes(v, g, lo, hi);
+    uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * bb;  // 8 codes of b bits = b bytes
+    if ((pos & 3) == 0) *reinterpret_cast<float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup) = make_float2(g.scale, g.zero);
+    if (bb == 8) {
+        *reinterpret_cast<uint2 *>(codes) = make_uint2(lo, hi);
+    } else {
+        const uint32_t w = pack_nibbles(lo, hi);
+        if (bb == 4) *reinterpret_cast<uint32_t *>(codes) = w;
+        else *reinterpret_cast<uint16_t *>(codes) = (uint16_t)pack_crumbs(w);
+    }
+}
+
+template <int D, int NS, int B>
+__device__ __forceinline__ void create_tile_body(const CreateSmem<D, NS> &sm, int stage, int warp, int lane,
+                                                 int rows_t, uint8_t *obuf)
+{
+    using C = PipeCfg<D>;
+    const uint8_t *tin = sm.in[stage];
+    uint4 v[C::PASSES];
+    uint2 inf[C::PASSES];
+    const int sub = lane / C::CPR, pos = lane % C::CPR;
+#pragma unroll
+    for (int j = 0; j < C::PASSES; ++j) {
+        const int row = warp * C::RPW + j * C::RPP + sub;
+        const bool valid = lane < C::LANES && row < rows_t;
+        v[j] = make_uint4(0, 0, 0, 0);
+        inf[j] = make_uint2(0, 0);  // bit-width 0 marks a lane without data
+        if (valid) {
+            v[j] = *reinterpret_cast<const uint4 *>(tin + row * C::ROW_BYTES + pos * 16);
+            inf[j] = sm.info[stage][row];
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < C::PASSES; ++j) {
+        float mn, mx;
+        group_min_max(v[j], mn, mx);  // shuffles: every lane takes part, with or without data
+        if (inf[j].y != 0) encode_chunk<D, B>(v[j], mn, mx, (int)inf[j].y, obuf + inf[j].x, pos);
+    }
+}
+
+template <int D, int NS>
+__global__ void __launch_bounds__(PipeCfg<D>::THREADS) create_kernel(PathParams p, LayerPtrs ptrs, int64_t n_tiles)
+{
+    using C = PipeCfg<D>;
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    CreateSmem<D, NS> &sm = *reinterpret_cast<CreateSmem<D, NS> *>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    qkvs_card_header_t *hdr = reinterpret_cast<qkvs_card_header_t *>(p.card);
+    if (hdr->status != QKVS_OK) return;  // bad bits or short buffer: no payload is written
+    const uint64_t stream_bytes = hdr->stream_bytes;
+    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], C::NW);
+        }
+        sm.abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    volatile int *abort_flag = &sm.abort_flag;
+
+    if (warp == C::NW) {
+        // ---------------- producer
+        const int64_t T = p.n_tokens;
+        const bool contiguous = p.token_stride == D;
+        uint32_t k = 0;
+        for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            const int stage = k % NS;
+            if (!mbar_wait(&sm.empty[stage], ((k / NS) & 1) ^ 1, abort_flag)) break;
+            const int64_t s_local = tile / p.tiles_per_stream;
+            const int64_t t0 = (tile % p.tiles_per_stream) * C::TB;
+            const int rows = (int)min((int64_t)C::TB, T - t0);
+            const StreamInfo si = locate_stream(p, sec, p.bits_mode, s_local, stream_bytes);
+            const uint8_t *bits = p.card + sec.bits_off + (uint64_t)si.seg * (uint64_t)T + t0;
+            const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) +
+                                   (uint64_t)si.seg * (uint64_t)(T + 1) + t0;
+            for (int r = lane; r <= rows; r += 32) sm.off_tmp[r] = offs[r];
+            __syncwarp();
+            for (int r = lane; r < rows; r += 32)
+                sm.info[stage][r] = make_uint2(sm.off_tmp[r] - sm.off_tmp[(r / C::RPW) * C::RPW], bits[r]);
+            if (lane < C::NW) {
+                const int r0 = min(lane * C::RPW, rows), r1 = min(r0 + C::RPW, rows);
+                sm.span_dst[stage][lane] = reinterpret_cast<uint64_t>(p.card + si.base + sm.off_tmp[r0]);
+                sm.span_bytes[stage][lane] = sm.off_tmp[r1] - sm.off_tmp[r0];
+                uint32_t ub = r0 < r1 ? bits[r0] : 0u;
+                for (int r = r0 + 1; r < r1; ++r) ub = bits[r] == ub ? ub : 0u;
+                sm.uniform_bits[stage][lane] = (r1 - r0 == C::RPW) ? ub : 0u;
+            }
+            if (lane == 0) sm.rows[stage] = rows;
+            __syncwarp();
+            const __half *src = reinterpret_cast<const __half *>(si.kv == 0 ? ptrs.k[si.layer_local] : ptrs.v[si.layer_local]) +
+                                (int64_t)si.head * p.head_stride + t0 * p.token_stride;
+            if (lane == 0) mbar_arrive_expect_tx(&sm.full[stage], (uint32_t)rows * C::ROW_BYTES);
+            __syncwarp();
+            if (contiguous) {
+                if (lane == 0) bulk_load(sm.in[stage], src, (uint32_t)rows * C::ROW_BYTES, &sm.full[stage]);
+            } else {
+                for (int r = lane; r < rows; r += 32)
+                    bulk_load(sm.in[stage] + r * C::ROW_BYTES, src + (int64_t)r * p.token_stride, C::ROW_BYTES, &sm.full[stage]);
+            }
+        }
+        // After an abandoned wait, stages may still have copies in flight: let them land
+        // (bounded) before the CTA gives its shared memory back.
+        if (*abort_flag) {
+            for (uint32_t j = 0; j < (uint32_t)NS && j < k; ++j) {
+                const uint32_t kk = k - 1 - j;
+                mbar_wait(&sm.full[kk % NS], (kk / NS) & 1, abort_flag);
+            }
+            if (lane == 0) atomicMax(&hdr->status, (uint32_t)QKVS_ERR_TIMEOUT);
+        }
+    } else {
+        // ---------------- consumers
+        uint32_t k = 0;
+        for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            const int stage = k % NS;
+            if (!mbar_wait(&sm.full[stage], (k / NS) & 1, abort_flag)) break;
+            const int rows_t = sm.rows[stage];
+            uint8_t *obuf = sm.out[warp][k & 1];
+            if (lane == 0) bulk_wait_read<1>();  // the store that last used this buffer has read it
+            __syncwarp();
+            switch (sm.uniform_bits[stage][warp]) {
+                case 4: create_tile_body<D, NS, 4>(sm, stage, warp, lane, rows_t, obuf); break;
+                case 2: create_tile_body<D, NS, 2>(sm, stage, warp, lane, rows_t, obuf); break;
+                case 8: create_tile_body<D, NS, 8>(sm, stage, warp, lane, rows_t, obuf); break;
+                case 16: create_tile_body<D, NS, 16>(sm, stage, warp, lane, rows_t, obuf); break;
+                default: create_tile_body<D, NS, 0>(sm, stage, warp, lane, rows_t, obuf); break;
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+                const uint64_t dst = sm.span_dst[stage][warp];
+                const uint32_t bytes = sm.span_bytes[stage][warp];
+                mbar_arrive(&sm.empty[stage]);
+                if (bytes) bulk_store(reinterpret_cast<void *>(dst), obuf, bytes);
+                bulk_commit();
+            }
+        }
+        if (lane == 0) bulk_wait<0>();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// inject: records -> FP16 rows
+
+template <int D, int NS>
+struct InjectSmem {
+    using C = PipeCfg<D>;
+    alignas(128) uint8_t in[NS][C::TILE_BYTES];
+    uint2 info[NS][C::TB];          // per row: {record offset inside the tile's span, bit-width}
+    uint64_t dst_row0[NS];          // global address of the tile's first destination row
+    uint32_t uniform_bits[NS][C::NW];
+    int32_t rows[NS];               // 0 when the tile's table entries did not check out
+    uint32_t off_tmp[C::TB + 1];
+    uint64_t full[NS];
+    uint64_t empty[NS];
+    int abort_flag;
+    int header_ok;
+    uint32_t bits_mode;
+    uint64_t stream_bytes, total_bytes;
+};
+
+template <int D, int B>
+__device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos)
+{
+    constexpr int G = D / kGroup;
+    const int bb = B ? B : b;
+    if (bb == 16) return *reinterpret_cast<const uint4 *>(rec + pos * 16);
+    const float2 m = *reinterpret_cast<const float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup);
+    const uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * bb;
+    uint32_t lo, hi;
+    if (bb == 8) {
+        const uint2 w = *reinterpret_cast<const uint2 *>(codes);
+        lo = w.x;
+        hi = w.y;
+    } else {
+        uint32_t w;
+        if (bb == 4) w = *reinterpret_cast<const uint32_t *>(codes);
+        else w = unpack_crumbs(*reinterpret_cast<const uint16_t *>(codes));
+        unpack_nibbles(w, lo, hi);
+    }
+    return dequantize_chunk(lo, hi, m.x, m.y);
+}
+
+template <int D, int NS, int B>
+__device__ __forceinline__ void inject_tile_body(const InjectSmem<D, NS> &sm, int stage, int warp, int lane,
+                                                 int rows_t, int64_t token_stride)
+{
+    using C = PipeCfg<D>;
+    const uint8_t *tin = sm.in[stage];
+    const int sub = lane / C::CPR, pos = lane % C::CPR;
+    __half *dst0 = reinterpret_cast<__half *>(sm.dst_row0[stage]);
+#pragma unroll
+    for (int j = 0; j < C::PASSES; ++j) {
+        const int row = warp * C::RPW + j * C::RPP + sub;
+        if (lane < C::LANES && row < rows_t) {
+            const uint2 inf = sm.info[stage][row];
+            const uint4 out = decode_chunk<D, B>(tin + inf.x, (int)inf.y, pos);
+            __stcs(reinterpret_cast<uint4 *>(dst0 + (int64_t)row * token_stride + pos * 8), out);
+        }
+    }
+}
+
+// The card is untrusted input: nothing is read beyond card_bytes and no row is written unless the
+// header and the tile's table entries are consistent with the destination shape.
+__device__ __forceinline__ bool header_matches(const qkvs_card_header_t *h, const PathParams &p, int bits_mode,
+                                               const Sections &sec)
+{
+    bool ok = h->magic == kMagic && h->version == kVersion && h->status == QKVS_OK;
+    ok = ok && h->n_layers == p.n_layers && h->n_kv_heads == p.n_kv_heads && h->head_dim == p.head_dim;
+    ok = ok && h->n_tokens == p.n_tokens && h->group_size == kGroup && h->meta_bytes_per_group == kMetaBytesPerGroup;
+    ok = ok && h->bits_off == sec.bits_off && h->offs_off == sec.offs_off && h->payload_off == sec.payload_off;
+    ok = ok && h->sbase_off == sec.sbase_off;
+    ok = ok && h->total_bytes <= p.card_bytes && h->total_bytes >= sec.payload_off;
+    if (ok && bits_mode == 0) {
+        const uint64_t S = 2u * (uint64_t)p.n_layers * (uint64_t)p.n_kv_heads;
+        ok = h->stream_bytes <= (uint64_t)p.n_tokens * 2u * (uint64_t)p.head_dim &&
+             sec.payload_off + S * h->stream_bytes == h->total_bytes;
+    }
+    return ok;
+}
+
+template <int D, int NS>
+__global__ void __launch_bounds__(PipeCfg<D>::THREADS) inject_kernel(PathParams p, LayerPtrs ptrs, int64_t n_tiles)
+{
+    using C = PipeCfg<D>;
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    InjectSmem<D, NS> &sm = *reinterpret_cast<InjectSmem<D, NS> *>(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const qkvs_card_header_t *hdr = reinterpret_cast<const qkvs_card_header_t *>(p.card);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], C::NW);
+        }
+        sm.abort_flag = 0;
+        fence_mbar_init();
+        const uint32_t mode = hdr->bits_mode;
+        int ok = 0;
+        if (mode <= 1u) {
+            const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, (int)mode);
+            ok = sec.payload_off <= p.card_bytes && header_matches(hdr, p, (int)mode, sec);
+        }
+        sm.header_ok = ok;
+        sm.bits_mode = mode;
+        sm.stream_bytes = hdr->stream_bytes;
+        sm.total_bytes = hdr->total_bytes;
+    }
+    __syncthreads();
+    if (!sm.header_ok) {
+        if (threadIdx.x == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
+        return;
+    }
+    volatile int *abort_flag = &sm.abort_flag;
+    const int mode = (int)sm.bits_mode;
+    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, mode);
+
+    if (warp == C::NW) {
+        // ---------------- producer
+        const int64_t T = p.n_tokens;
+        const uint64_t total = sm.total_bytes;
+        uint32_t k = 0;
+        for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            const int stage = k % NS;
+            if (!mbar_wait(&sm.empty[stage], ((k / NS) & 1) ^ 1, abort_flag)) break;
+            const int64_t s_local = tile / p.tiles_per_stream;
+            const int64_t t0 = (tile % p.tiles_per_stream) * C::TB;
+            const int rows = (int)min((int64_t)C::TB, T - t0);
+            const StreamInfo si = locate_stream(p, sec, mode, s_local, sm.stream_bytes);
+            const uint8_t *bits = p.card + sec.bits_off + (uint64_t)si.seg * (uint64_t)T + t0;
+            const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) +
+                                   (uint64_t)si.seg * (uint64_t)(T + 1) + t0;
+            for (int r = lane; r <= rows; r += 32) sm.off_tmp[r] = offs[r];
+            __syncwarp();
+            const uint32_t off0 = sm.off_tmp[0];
+            int bad = 0;
+            for (int r = lane; r < rows; r += 32) {
+                const uint32_t b = bits[r];
+                const uint32_t rec = record_bytes(D, (int)b);
+                bad |= (rec == 0u) || (sm.off_tmp[r + 1] < sm.off_tmp[r]) || (sm.off_tmp[r + 1] - sm.off_tmp[r] != rec);
+                sm.info[stage][r] = make_uint2(sm.off_tmp[r] - off0, b);
+            }
+            bad = __any_sync(0xffffffffu, bad);
+            // with consistent records the span is rows * (at most 2*D) bytes, so it fits the stage
+            const uint32_t span = sm.off_tmp[rows] - off0;
+            bad |= (off0 & 15u) != 0u || si.base < sec.payload_off || (si.base & 15u) != 0u ||
+                   si.base + (uint64_t)sm.off_tmp[rows] > total;
+            if (lane < C::NW) {
+                const int r0 = min(lane * C::RPW, rows), r1 = min(r0 + C::RPW, rows);
+                uint32_t ub = r0 < r1 ? bits[r0] : 0u;
+                for (int r = r0 + 1; r < r1; ++r) ub = bits[r] == ub ? ub : 0u;
+                sm.uniform_bits[stage][lane] = (r1 - r0 == C::RPW) ? ub : 0u;
+            }
+            if (lane == 0) {
+                sm.rows[stage] = bad ? 0 : rows;
+                __half *dst = reinterpret_cast<__half *>(si.kv == 0 ? ptrs.k[si.layer_local] : ptrs.v[si.layer_local]) +
+                              (int64_t)si.head * p.head_stride + (p.dst_token_offset + t0) * p.token_stride;
+                sm.dst_row0[stage] = reinterpret_cast<uint64_t>(dst);
+                if (bad && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                if (!bad && span) {
+                    mbar_arrive_expect_tx(&sm.full[stage], span);
+                    bulk_load(sm.in[stage], p.card + si.base + off0, span, &sm.full[stage]);
+                } else {
+                    mbar_arrive(&sm.full[stage]);
+                }
+            }
+        }
+        if (*abort_flag) {
+            for (uint32_t j = 0; j < (uint32_t)NS && j < k; ++j) {
+                const uint32_t kk = k - 1 - j;
+                mbar_wait(&sm.full[kk % NS], (kk / NS) & 1, abort_flag);
+            }
+            if (lane == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_TIMEOUT);
+        }
+    } else {
+        // ---------------- consumers
+        uint32_t k = 0;
+        for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            const int stage = k % NS;
+            if (!mbar_wait(&sm.full[stage], (k / NS) & 1, abort_flag)) break;
+            const int rows_t = sm.rows[stage];
+            switch (sm.uniform_bits[stage][warp]) {
+                case 4: inject_tile_body<D, NS, 4>(sm, stage, warp, lane, rows_t, p.token_stride); break;
+                case 2: inject_tile_body<D, NS, 2>(sm, stage, warp, lane, rows_t, p.token_stride); break;
+                case 8: inject_tile_body<D, NS, 8>(sm, stage, warp, lane, rows_t, p.token_stride); break;
+                case 16: inject_tile_body<D, NS, 16>(sm, stage, warp, lane, rows_t, p.token_stride); break;
+                default: inject_tile_body<D, NS, 0>(sm, stage, warp, lane, rows_t, p.token_stride); break;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[stage]);
+        }
+    }
+}
+
+}  // namespace qkvs

@@ -2,12 +2,10 @@
 //
 // Three kernels make up the path:
 //   scan_offsets_kernel   per-segment exclusive prefix sum of record sizes over the bit-width
-//                         vector; writes the card's header, bits and offset tables
-//   create_kernel         fused group min/max -> scale/zero -> quantise -> bit-pack; one CTA
-//                         turns a tile of consecutive tokens of one stream into one contiguous
-//                         span of the card, staged in shared memory and stored 16 bytes a lane
-//   inject_kernel         reads records, unpacks, dequantises and writes FP16 rows into the
-//                         destination cache layout
+//                         vector; writes the card's header, bits and offset tables (this file)
+//   create_kernel         fused group min/max -> scale/zero -> quantise -> bit-pack
+//   inject_kernel         unpack -> dequantise -> scatter into the destination cache layout
+// The last two are the persistent TMA pipelines of qkvs_pipeline.cuh.
 // A stream is one (layer, K|V, head) matrix [tokens, head_dim].
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -17,6 +15,7 @@
 #include <cstring>
 
 #include "qkvs_common.cuh"
+#include "qkvs_pipeline.cuh"
 
 namespace qkvs {
 
@@ -249,246 +248,6 @@ __global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Stream bookkeeping shared by create and inject
-
-struct StreamInfo {
-    int layer_local;   // layer index inside this launch's pointer block
-    int kv, head;
-    int64_t seg;       // segment whose bits / offsets the stream uses
-    uint64_t base;     // byte offset of the stream inside the card
-};
-
-__device__ __forceinline__ StreamInfo locate_stream(const PathParams &p, const Sections &sec, int64_t s_local,
-                                                    uint64_t stream_bytes)
-{
-    StreamInfo si;
-    const int H = p.n_kv_heads;
-    si.head = (int)(s_local % H);
-    si.kv = (int)((s_local / H) & 1);
-    si.layer_local = (int)(s_local / (2 * H));
-    const int64_t layer = p.layer_begin + si.layer_local;
-    const int64_t s = (layer * 2 + si.kv) * H + si.head;
-    if (p.bits_mode == 0) {
-        si.seg = 0;
-        si.base = sec.payload_off + (uint64_t)s * stream_bytes;
-    } else {
-        si.seg = layer * H + si.head;
-        si.base = sec.payload_off + reinterpret_cast<const uint64_t *>(p.card + sec.sbase_off)[s];
-    }
-    return si;
-}
-
-// ---------------------------------------------------------------------------------------------
-// Card creation: fused min/max -> scale/zero -> quantise -> pack
-
-template <int D, int TB, int THREADS>
-__global__ void __launch_bounds__(THREADS) create_kernel(PathParams p, LayerPtrs ptrs)
-{
-    constexpr int CPR = D / 8;  // chunks (threads) per token row
-    constexpr int G = D / kGroup;
-    constexpr int ITER = (TB * CPR + THREADS - 1) / THREADS;
-    static_assert((TB * CPR) % THREADS == 0, "tile must be a whole number of passes");
-    __shared__ __align__(16) uint8_t s_out[TB * 2 * D];
-    __shared__ uint32_t s_off[TB + 1];
-    __shared__ uint8_t s_bits[TB];
-
-    const qkvs_card_header_t *hdr = reinterpret_cast<const qkvs_card_header_t *>(p.card);
-    if (hdr->status != QKVS_OK) return;  // bad bits or short buffer: no payload is written
-    const uint64_t stream_bytes = hdr->stream_bytes;
-    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
-
-    const int64_t s_local = blockIdx.x / p.tiles_per_stream;
-    const int64_t t0 = (int64_t)(blockIdx.x % p.tiles_per_stream) * TB;
-    const int rows = (int)min((int64_t)TB, (int64_t)p.n_tokens - t0);
-    const StreamInfo si = locate_stream(p, sec, s_local, stream_bytes);
-    const int64_t T = p.n_tokens;
-    const uint8_t *bits = p.card + sec.bits_off + (uint64_t)si.seg * (uint64_t)T + t0;
-    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) + (uint64_t)si.seg * (uint64_t)(T + 1) + t0;
-    for (int i = threadIdx.x; i <= rows; i += THREADS) {
-        s_off[i] = offs[i];
-        if (i < rows) s_bits[i] = bits[i];
-    }
-    __syncthreads();
-    const uint32_t off0 = s_off[0];
-
-    const __half *src = reinterpret_cast<const __half *>(si.kv == 0 ? ptrs.k[si.layer_local] : ptrs.v[si.layer_local]) +
-                        (int64_t)si.head * p.head_stride + t0 * p.token_stride;
-
-    uint4 v[ITER];
-#pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-        const int c = it * THREADS + threadIdx.x;
-        const int row = c / CPR, pos = c % CPR;
-        v[it] = make_uint4(0, 0, 0, 0);
-        if (row < rows) v[it] = __ldg(reinterpret_cast<const uint4 *>(src + (int64_t)row * p.token_stride + pos * 8));
-    }
-#pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-        const int c = it * THREADS + threadIdx.x;
-        const int row = c / CPR, pos = c % CPR;
-        const bool valid = row < rows;
-        const int b = valid ? s_bits[row] : 16;
-        float mn, mx;
-        group_min_max(v[it], mn, mx);
-        if (!valid) continue;
-        uint8_t *rec = s_out + (s_off[row] - off0);
-        if (b == 16) {
-            *reinterpret_cast<uint4 *>(rec + pos * 16) = v[it];
-            continue;
-        }
-        const int qmax = (1 << b) - 1;
-        const GroupParams g = group_params(mn, mx, (float)qmax);
-        if ((pos & 3) == 0) *reinterpret_cast<float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup) = make_float2(g.scale, g.zero);
-        uint32_t q[8];
-        quantize_chunk(v[it], g, qmax, q);
-        uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * b;  // 8 codes of b bits = b bytes
-        if (b == 4) {
-            uint32_t w = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) w |= q[i] << (4 * i);
-            *reinterpret_cast<uint32_t *>(codes) = w;
-        } else if (b == 2) {
-            uint32_t w = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) w |= q[i] << (2 * i);
-            *reinterpret_cast<uint16_t *>(codes) = (uint16_t)w;
-        } else {
-            const uint32_t w0 = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
-            const uint32_t w1 = q[4] | (q[5] << 8) | (q[6] << 16) | (q[7] << 24);
-            *reinterpret_cast<uint2 *>(codes) = make_uint2(w0, w1);
-        }
-    }
-    __syncthreads();
-    const uint32_t n16 = (s_off[rows] - off0) >> 4;
-    uint4 *dst = reinterpret_cast<uint4 *>(p.card + si.base + off0);
-    const uint4 *so = reinterpret_cast<const uint4 *>(s_out);
-    for (uint32_t i = threadIdx.x; i < n16; i += THREADS) dst[i] = so[i];
-}
-
-// ---------------------------------------------------------------------------------------------
-// Injection: unpack -> dequantise -> scatter
-
-__device__ __forceinline__ bool header_matches(const qkvs_card_header_t *h, const PathParams &p, const Sections &sec)
-{
-    bool ok = h->magic == kMagic && h->version == kVersion && h->status == QKVS_OK;
-    ok = ok && h->bits_mode == (uint32_t)p.bits_mode;
-    ok = ok && h->n_layers == p.n_layers && h->n_kv_heads == p.n_kv_heads && h->head_dim == p.head_dim;
-    ok = ok && h->n_tokens == p.n_tokens && h->group_size == kGroup && h->meta_bytes_per_group == kMetaBytesPerGroup;
-    ok = ok && h->bits_off == sec.bits_off && h->offs_off == sec.offs_off && h->payload_off == sec.payload_off;
-    ok = ok && h->sbase_off == sec.sbase_off;
-    ok = ok && h->total_bytes <= p.card_bytes && h->total_bytes >= sec.payload_off;
-    return ok;
-}
-
-template <int D, int TB, int THREADS>
-__global__ void __launch_bounds__(THREADS) inject_kernel(PathParams p, LayerPtrs ptrs)
-{
-    constexpr int CPR = D / 8;
-    constexpr int G = D / kGroup;
-    constexpr int ITER = (TB * CPR + THREADS - 1) / THREADS;
-    static_assert((TB * CPR) % THREADS == 0, "tile must be a whole number of passes");
-    __shared__ uint32_t s_off[TB + 1];
-    __shared__ uint8_t s_bits[TB];
-    __shared__ int s_ok;
-    __shared__ uint64_t s_base;
-
-    const qkvs_card_header_t *hdr = reinterpret_cast<const qkvs_card_header_t *>(p.card);
-    const int64_t s_local = blockIdx.x / p.tiles_per_stream;
-    const int64_t t0 = (int64_t)(blockIdx.x % p.tiles_per_stream) * TB;
-    const int rows = (int)min((int64_t)TB, (int64_t)p.n_tokens - t0);
-    const int64_t T = p.n_tokens;
-
-    // The card is untrusted input: nothing is read beyond card_bytes and no row is written
-    // unless the header and this tile's table entries are consistent.
-    if (threadIdx.x == 0) {
-        int ok = 0;
-        uint64_t base = 0;
-        const uint32_t mode = hdr->bits_mode;
-        if (mode <= 1u) {
-            PathParams q = p;
-            q.bits_mode = (int32_t)mode;
-            const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, (int)mode);
-            if (sec.payload_off <= p.card_bytes && header_matches(hdr, q, sec)) {
-                const uint64_t total = hdr->total_bytes;
-                const StreamInfo si = locate_stream(q, sec, s_local, hdr->stream_bytes);
-                base = si.base;
-                ok = base >= sec.payload_off && base <= total && (base & 15u) == 0;
-            }
-        }
-        s_ok = ok;
-        s_base = base;
-    }
-    __syncthreads();
-    if (!s_ok) {
-        if (threadIdx.x == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
-        return;
-    }
-    const int mode = (int)hdr->bits_mode;
-    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, mode);
-    const int H = p.n_kv_heads;
-    const int head = (int)(s_local % H), kv = (int)((s_local / H) & 1), layer_local = (int)(s_local / (2 * H));
-    const int64_t seg = mode == 0 ? 0 : (int64_t)(p.layer_begin + layer_local) * H + head;
-    const uint8_t *bits = p.card + sec.bits_off + (uint64_t)seg * (uint64_t)T + t0;
-    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) + (uint64_t)seg * (uint64_t)(T + 1) + t0;
-    for (int i = threadIdx.x; i <= rows; i += THREADS) {
-        s_off[i] = offs[i];
-        if (i < rows) s_bits[i] = bits[i];
-    }
-    __syncthreads();
-    int bad = 0;
-    for (int i = threadIdx.x; i < rows; i += THREADS) {
-        const uint32_t r = record_bytes(D, s_bits[i]);
-        bad |= (r == 0u) || (s_off[i + 1] - s_off[i] != r) || (s_off[i + 1] < s_off[i]);
-    }
-    if (threadIdx.x == 0) bad |= (s_base + (uint64_t)s_off[rows] > hdr->total_bytes) || (s_off[0] & 15u);
-    if (__syncthreads_or(bad)) {
-        if (threadIdx.x == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
-        return;
-    }
-
-    const uint8_t *stream = p.card + s_base;
-    __half *dst = reinterpret_cast<__half *>(kv == 0 ? ptrs.k[layer_local] : ptrs.v[layer_local]) +
-                  (int64_t)head * p.head_stride + (p.dst_token_offset + t0) * p.token_stride;
-#pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-        const int c = it * THREADS + threadIdx.x;
-        const int row = c / CPR, pos = c % CPR;
-        if (row >= rows) continue;
-        const int b = s_bits[row];
-        const uint8_t *rec = stream + s_off[row];
-        uint4 out;
-        if (b == 16) {
-            out = __ldg(reinterpret_cast<const uint4 *>(rec + pos * 16));
-        } else {
-            const float2 m = __ldg(reinterpret_cast<const float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup));
-            const uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * b;
-            uint32_t q[8];
-            if (b == 4) {
-                const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(codes));
-#pragma unroll
-                for (int i = 0; i < 8; ++i) q[i] = (w >> (4 * i)) & 15u;
-            } else if (b == 2) {
-                const uint32_t w = __ldg(reinterpret_cast<const uint16_t *>(codes));
-#pragma unroll
-                for (int i = 0; i < 8; ++i) q[i] = (w >> (2 * i)) & 3u;
-            } else {
-                const uint2 w = __ldg(reinterpret_cast<const uint2 *>(codes));
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    q[i] = (w.x >> (8 * i)) & 255u;
-                    q[4 + i] = (w.y >> (8 * i)) & 255u;
-                }
-            }
-            out.x = pack_half2(dequantize_one(q[0], m.x, m.y), dequantize_one(q[1], m.x, m.y));
-            out.y = pack_half2(dequantize_one(q[2], m.x, m.y), dequantize_one(q[3], m.x, m.y));
-            out.z = pack_half2(dequantize_one(q[4], m.x, m.y), dequantize_one(q[5], m.x, m.y));
-            out.w = pack_half2(dequantize_one(q[6], m.x, m.y), dequantize_one(q[7], m.x, m.y));
-        }
-        *reinterpret_cast<uint4 *>(dst + (int64_t)row * p.token_stride + pos * 8) = out;
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
 // Host side
 
 static qkvs_status_t check_shape(const qkvs_layout_t *l)
@@ -518,37 +277,58 @@ static qkvs_status_t check_strides(const qkvs_layout_t *l, int64_t first_row)
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Tile of consecutive tokens handled by one CTA: 1024 chunks (4 passes of 256 threads), except
-// head_dim 192 where 32 tokens give 768 chunks (3 passes).
-template <int D>
-struct TileCfg {
-    static constexpr int THREADS = 256;
-    static constexpr int TB = D == 192 ? 32 : 8192 / D;
-};
+constexpr int kStagesCreate = 4;
+constexpr int kStagesInject = 4;
+
+// Persistent grid: as many CTAs as fit on the device at once, never more than there are tiles.
+template <typename Kernel>
+static cudaError_t persistent_grid(Kernel kernel, int threads, size_t smem, int64_t n_tiles, unsigned *grid)
+{
+    int dev = 0, sms = 0, per_sm = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorInvalidConfiguration;
+    *grid = (unsigned)std::min<int64_t>(n_tiles, (int64_t)sms * per_sm);
+    return cudaSuccess;
+}
 
 template <int D>
 static cudaError_t launch_create(const PathParams &pp, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    using C = TileCfg<D>;
+    using C = PipeCfg<D>;
     PathParams p = pp;
     p.tiles_per_stream = (uint32_t)((p.n_tokens + C::TB - 1) / C::TB);
-    const int64_t blocks = streams * p.tiles_per_stream;
-    if (blocks == 0) return cudaSuccess;
-    if (blocks > 0x7fffffffll) return cudaErrorInvalidConfiguration;
-    create_kernel<D, C::TB, C::THREADS><<<(unsigned)blocks, C::THREADS, 0, st>>>(p, ptrs);
+    const int64_t n_tiles = streams * p.tiles_per_stream;
+    if (n_tiles == 0) return cudaSuccess;
+    auto kernel = create_kernel<D, kStagesCreate>;
+    const size_t smem = sizeof(CreateSmem<D, kStagesCreate>);
+    unsigned grid = 0;
+    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, n_tiles, &grid);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs, n_tiles);
     return cudaGetLastError();
 }
 
 template <int D>
 static cudaError_t launch_inject(const PathParams &pp, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    using C = TileCfg<D>;
+    using C = PipeCfg<D>;
     PathParams p = pp;
     p.tiles_per_stream = (uint32_t)((p.n_tokens + C::TB - 1) / C::TB);
-    const int64_t blocks = streams * p.tiles_per_stream;
-    if (blocks == 0) return cudaSuccess;
-    if (blocks > 0x7fffffffll) return cudaErrorInvalidConfiguration;
-    inject_kernel<D, C::TB, C::THREADS><<<(unsigned)blocks, C::THREADS, 0, st>>>(p, ptrs);
+    const int64_t n_tiles = streams * p.tiles_per_stream;
+    if (n_tiles == 0) return cudaSuccess;
+    auto kernel = inject_kernel<D, kStagesInject>;
+    const size_t smem = sizeof(InjectSmem<D, kStagesInject>);
+    unsigned grid = 0;
+    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, n_tiles, &grid);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs, n_tiles);
     return cudaGetLastError();
 }
 
