@@ -64,6 +64,75 @@ __device__ __forceinline__ StreamInfo locate_stream(const PathParams &p, const S
     return si;
 }
 
+// What the producer needs to know about one tile, gathered one loop iteration ahead so that the
+// global-memory latency of the table reads overlaps the previous tile.  Lane l holds table entries
+// l, l + 32, ...
+template <int TB>
+struct TileFetch {
+    static constexpr int NOFF = TB / 32 + 1;
+    static constexpr int NBITS = (TB + 31) / 32;
+    int64_t t0;
+    int rows;
+    int layer_local, kv, head;
+    uint64_t base;
+    uint32_t off[NOFF];
+    uint32_t bits[NBITS];
+};
+
+template <int TB>
+__device__ __forceinline__ void fetch_tile(TileFetch<TB> &f, const PathParams &p, const Sections &sec, int bits_mode,
+                                           uint64_t stream_bytes, int64_t tile, int lane)
+{
+    const int64_t T = p.n_tokens;
+    const int64_t s_local = tile / p.tiles_per_stream;
+    f.t0 = (tile % p.tiles_per_stream) * TB;
+    f.rows = (int)min((int64_t)TB, T - f.t0);
+    const StreamInfo si = locate_stream(p, sec, bits_mode, s_local, stream_bytes);
+    f.layer_local = si.layer_local;
+    f.kv = si.kv;
+    f.head = si.head;
+    f.base = si.base;
+    const uint8_t *bits = p.card + sec.bits_off + (uint64_t)si.seg * (uint64_t)T + f.t0;
+    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) +
+                           (uint64_t)si.seg * (uint64_t)(T + 1) + f.t0;
+#pragma unroll
+    for (int i = 0; i < TileFetch<TB>::NOFF; ++i) {
+        const int r = lane + 32 * i;
+        f.off[i] = r <= f.rows ? offs[r] : 0u;
+    }
+#pragma unroll
+    for (int i = 0; i < TileFetch<TB>::NBITS; ++i) {
+        const int r = lane + 32 * i;
+        f.bits[i] = r < f.rows ? (uint32_t)bits[r] : 0u;
+    }
+}
+
+// Publishes the fetched table slice in the producer's scratch arrays (all lanes call this).
+template <int TB>
+__device__ __forceinline__ void spill_tables(const TileFetch<TB> &f, uint32_t *off_tmp, uint8_t *bits_tmp, int lane)
+{
+#pragma unroll
+    for (int i = 0; i < TileFetch<TB>::NOFF; ++i) {
+        const int r = lane + 32 * i;
+        if (r <= f.rows) off_tmp[r] = f.off[i];
+    }
+#pragma unroll
+    for (int i = 0; i < TileFetch<TB>::NBITS; ++i) {
+        const int r = lane + 32 * i;
+        if (r < f.rows) bits_tmp[r] = (uint8_t)f.bits[i];
+    }
+    __syncwarp();
+}
+
+// Bit-width shared by rows [r0, r1) if they are a full warp share of RPW rows, else 0.
+__device__ __forceinline__ uint32_t uniform_bits_of(const uint8_t *bits_tmp, int r0, int r1, int rpw)
+{
+    if (r1 - r0 != rpw) return 0u;
+    uint32_t ub = bits_tmp[r0];
+    for (int r = r0 + 1; r < r1; ++r) ub = bits_tmp[r] == ub ? ub : 0u;
+    return ub;
+}
+
 // ---------------------------------------------------------------------------------------------
 // create: FP16 rows -> records
 
@@ -78,6 +147,7 @@ struct CreateSmem {
     uint32_t uniform_bits[NS][C::NW];  // bit-width shared by all rows of the warp, else 0
     int32_t rows[NS];
     uint32_t off_tmp[C::TB + 1];    // producer scratch
+    uint8_t bits_tmp[C::TB];
     uint64_t full[NS];
     uint64_t empty[NS];
     int abort_flag;
@@ -109,7 +179,8 @@ __device__ __forceinline__ void encode_chunk(const uint4 &v, float mn, float mx,
     }
 }
 
-template <int D, int NS, int B>
+// FULL: the tile has all TB rows and every lane carries data, so no validity checks are needed.
+template <int D, int NS, int B, bool FULL>
 __device__ __forceinline__ void create_tile_body(const CreateSmem<D, NS> &sm, int stage, int warp, int lane,
                                                  int rows_t, uint8_t *obuf)
 {
@@ -121,7 +192,7 @@ __device__ __forceinline__ void create_tile_body(const CreateSmem<D, NS> &sm, in
 #pragma unroll
     for (int j = 0; j < C::PASSES; ++j) {
         const int row = warp * C::RPW + j * C::RPP + sub;
-        const bool valid = lane < C::LANES && row < rows_t;
+        const bool valid = FULL || (lane < C::LANES && row < rows_t);
         v[j] = make_uint4(0, 0, 0, 0);
         inf[j] = make_uint2(0, 0);  // bit-width 0 marks a lane without data
         if (valid) {
@@ -133,7 +204,20 @@ __device__ __forceinline__ void create_tile_body(const CreateSmem<D, NS> &sm, in
     for (int j = 0; j < C::PASSES; ++j) {
         float mn, mx;
         group_min_max(v[j], mn, mx);  // shuffles: every lane takes part, with or without data
-        if (inf[j].y != 0) encode_chunk<D, B>(v[j], mn, mx, (int)inf[j].y, obuf + inf[j].x, pos);
+        if (FULL || inf[j].y != 0) encode_chunk<D, B>(v[j], mn, mx, (int)inf[j].y, obuf + inf[j].x, pos);
+    }
+}
+
+template <int D, int NS, bool FULL>
+__device__ __forceinline__ void create_tile_dispatch(const CreateSmem<D, NS> &sm, int stage, int warp, int lane,
+                                                     int rows_t, uint8_t *obuf)
+{
+    switch (sm.uniform_bits[stage][warp]) {
+        case 4: create_tile_body<D, NS, 4, FULL>(sm, stage, warp, lane, rows_t, obuf); break;
+        case 2: create_tile_body<D, NS, 2, FULL>(sm, stage, warp, lane, rows_t, obuf); break;
+        case 8: create_tile_body<D, NS, 8, FULL>(sm, stage, warp, lane, rows_t, obuf); break;
+        case 16: create_tile_body<D, NS, 16, FULL>(sm, stage, warp, lane, rows_t, obuf); break;
+        default: create_tile_body<D, NS, 0, FULL>(sm, stage, warp, lane, rows_t, obuf); break;
     }
 }
 
@@ -162,36 +246,30 @@ __global__ void __launch_bounds__(PipeCfg<D>::THREADS) create_kernel(PathParams 
     volatile int *abort_flag = &sm.abort_flag;
 
     if (warp == C::NW) {
-        // ---------------- producer
-        const int64_t T = p.n_tokens;
-        const bool contiguous = p.token_stride == D;
         uint32_t k = 0;
+        // ---------------- producer
+        const bool contiguous = p.token_stride == D;
+        TileFetch<C::TB> cur, nxt;
+        if ((int64_t)blockIdx.x < n_tiles) fetch_tile(nxt, p, sec, p.bits_mode, stream_bytes, blockIdx.x, lane);
         for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            cur = nxt;
+            if (tile + gridDim.x < n_tiles) fetch_tile(nxt, p, sec, p.bits_mode, stream_bytes, tile + gridDim.x, lane);
             const int stage = k % NS;
             if (!mbar_wait(&sm.empty[stage], ((k / NS) & 1) ^ 1, abort_flag)) break;
-            const int64_t s_local = tile / p.tiles_per_stream;
-            const int64_t t0 = (tile % p.tiles_per_stream) * C::TB;
-            const int rows = (int)min((int64_t)C::TB, T - t0);
-            const StreamInfo si = locate_stream(p, sec, p.bits_mode, s_local, stream_bytes);
-            const uint8_t *bits = p.card + sec.bits_off + (uint64_t)si.seg * (uint64_t)T + t0;
-            const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) +
-                                   (uint64_t)si.seg * (uint64_t)(T + 1) + t0;
-            for (int r = lane; r <= rows; r += 32) sm.off_tmp[r] = offs[r];
-            __syncwarp();
+            const int rows = cur.rows;
+            spill_tables(cur, sm.off_tmp, sm.bits_tmp, lane);
             for (int r = lane; r < rows; r += 32)
-                sm.info[stage][r] = make_uint2(sm.off_tmp[r] - sm.off_tmp[(r / C::RPW) * C::RPW], bits[r]);
+                sm.info[stage][r] = make_uint2(sm.off_tmp[r] - sm.off_tmp[(r / C::RPW) * C::RPW], sm.bits_tmp[r]);
             if (lane < C::NW) {
                 const int r0 = min(lane * C::RPW, rows), r1 = min(r0 + C::RPW, rows);
-                sm.span_dst[stage][lane] = reinterpret_cast<uint64_t>(p.card + si.base + sm.off_tmp[r0]);
+                sm.span_dst[stage][lane] = reinterpret_cast<uint64_t>(p.card + cur.base + sm.off_tmp[r0]);
                 sm.span_bytes[stage][lane] = sm.off_tmp[r1] - sm.off_tmp[r0];
-                uint32_t ub = r0 < r1 ? bits[r0] : 0u;
-                for (int r = r0 + 1; r < r1; ++r) ub = bits[r] == ub ? ub : 0u;
-                sm.uniform_bits[stage][lane] = (r1 - r0 == C::RPW) ? ub : 0u;
+                sm.uniform_bits[stage][lane] = uniform_bits_of(sm.bits_tmp, r0, r1, C::RPW);
             }
             if (lane == 0) sm.rows[stage] = rows;
             __syncwarp();
-            const __half *src = reinterpret_cast<const __half *>(si.kv == 0 ? ptrs.k[si.layer_local] : ptrs.v[si.layer_local]) +
-                                (int64_t)si.head * p.head_stride + t0 * p.token_stride;
+            const __half *src = reinterpret_cast<const __half *>(cur.kv == 0 ? ptrs.k[cur.layer_local] : ptrs.v[cur.layer_local]) +
+                                (int64_t)cur.head * p.head_stride + cur.t0 * p.token_stride;
             if (lane == 0) mbar_arrive_expect_tx(&sm.full[stage], (uint32_t)rows * C::ROW_BYTES);
             __syncwarp();
             if (contiguous) {
@@ -220,13 +298,8 @@ __global__ void __launch_bounds__(PipeCfg<D>::THREADS) create_kernel(PathParams 
             uint8_t *obuf = sm.out[warp][k & 1];
             if (lane == 0) bulk_wait_read<1>();  // the store that last used this buffer has read it
             __syncwarp();
-            switch (sm.uniform_bits[stage][warp]) {
-                case 4: create_tile_body<D, NS, 4>(sm, stage, warp, lane, rows_t, obuf); break;
-                case 2: create_tile_body<D, NS, 2>(sm, stage, warp, lane, rows_t, obuf); break;
-                case 8: create_tile_body<D, NS, 8>(sm, stage, warp, lane, rows_t, obuf); break;
-                case 16: create_tile_body<D, NS, 16>(sm, stage, warp, lane, rows_t, obuf); break;
-                default: create_tile_body<D, NS, 0>(sm, stage, warp, lane, rows_t, obuf); break;
-            }
+            if (C::LANES == 32 && rows_t == C::TB) create_tile_dispatch<D, NS, true>(sm, stage, warp, lane, rows_t, obuf);
+            else create_tile_dispatch<D, NS, false>(sm, stage, warp, lane, rows_t, obuf);
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) {
@@ -252,7 +325,8 @@ struct InjectSmem {
     uint64_t dst_row0[NS];          // global address of the tile's first destination row
     uint32_t uniform_bits[NS][C::NW];
     int32_t rows[NS];               // 0 when the tile's table entries did not check out
-    uint32_t off_tmp[C::TB + 1];
+    uint32_t off_tmp[C::TB + 1];    // producer scratch
+    uint8_t bits_tmp[C::TB];
     uint64_t full[NS];
     uint64_t empty[NS];
     int abort_flag;
@@ -283,7 +357,7 @@ __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos
     return dequantize_chunk(lo, hi, m.x, m.y);
 }
 
-template <int D, int NS, int B>
+template <int D, int NS, int B, bool FULL>
 __device__ __forceinline__ void inject_tile_body(const InjectSmem<D, NS> &sm, int stage, int warp, int lane,
                                                  int rows_t, int64_t token_stride)
 {
@@ -294,11 +368,24 @@ __device__ __forceinline__ void inject_tile_body(const InjectSmem<D, NS> &sm, in
 #pragma unroll
     for (int j = 0; j < C::PASSES; ++j) {
         const int row = warp * C::RPW + j * C::RPP + sub;
-        if (lane < C::LANES && row < rows_t) {
+        if (FULL || (lane < C::LANES && row < rows_t)) {
             const uint2 inf = sm.info[stage][row];
             const uint4 out = decode_chunk<D, B>(tin + inf.x, (int)inf.y, pos);
             __stcs(reinterpret_cast<uint4 *>(dst0 + (int64_t)row * token_stride + pos * 8), out);
         }
+    }
+}
+
+template <int D, int NS, bool FULL>
+__device__ __forceinline__ void inject_tile_dispatch(const InjectSmem<D, NS> &sm, int stage, int warp, int lane,
+                                                     int rows_t, int64_t token_stride)
+{
+    switch (sm.uniform_bits[stage][warp]) {
+        case 4: inject_tile_body<D, NS, 4, FULL>(sm, stage, warp, lane, rows_t, token_stride); break;
+        case 2: inject_tile_body<D, NS, 2, FULL>(sm, stage, warp, lane, rows_t, token_stride); break;
+        case 8: inject_tile_body<D, NS, 8, FULL>(sm, stage, warp, lane, rows_t, token_stride); break;
+        case 16: inject_tile_body<D, NS, 16, FULL>(sm, stage, warp, lane, rows_t, token_stride); break;
+        default: inject_tile_body<D, NS, 0, FULL>(sm, stage, warp, lane, rows_t, token_stride); break;
     }
 }
 
@@ -358,26 +445,23 @@ __global__ void __launch_bounds__(PipeCfg<D>::THREADS) inject_kernel(PathParams 
     const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, mode);
 
     if (warp == C::NW) {
-        // ---------------- producer
-        const int64_t T = p.n_tokens;
-        const uint64_t total = sm.total_bytes;
         uint32_t k = 0;
+        // ---------------- producer
+        const uint64_t total = sm.total_bytes;
+        const uint64_t stream_bytes = sm.stream_bytes;
+        TileFetch<C::TB> cur, nxt;
+        if ((int64_t)blockIdx.x < n_tiles) fetch_tile(nxt, p, sec, mode, stream_bytes, blockIdx.x, lane);
         for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++k) {
+            cur = nxt;
+            if (tile + gridDim.x < n_tiles) fetch_tile(nxt, p, sec, mode, stream_bytes, tile + gridDim.x, lane);
             const int stage = k % NS;
             if (!mbar_wait(&sm.empty[stage], ((k / NS) & 1) ^ 1, abort_flag)) break;
-            const int64_t s_local = tile / p.tiles_per_stream;
-            const int64_t t0 = (tile % p.tiles_per_stream) * C::TB;
-            const int rows = (int)min((int64_t)C::TB, T - t0);
-            const StreamInfo si = locate_stream(p, sec, mode, s_local, sm.stream_bytes);
-            const uint8_t *bits = p.card + sec.bits_off + (uint64_t)si.seg * (uint64_t)T + t0;
-            const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) +
-                                   (uint64_t)si.seg * (uint64_t)(T + 1) + t0;
-            for (int r = lane; r <= rows; r += 32) sm.off_tmp[r] = offs[r];
-            __syncwarp();
+            const int rows = cur.rows;
+            spill_tables(cur, sm.off_tmp, sm.bits_tmp, lane);
             const uint32_t off0 = sm.off_tmp[0];
             int bad = 0;
             for (int r = lane; r < rows; r += 32) {
-                const uint32_t b = bits[r];
+                const uint32_t b = sm.bits_tmp[r];
                 const uint32_t rec = record_bytes(D, (int)b);
                 bad |= (rec == 0u) || (sm.off_tmp[r + 1] < sm.off_tmp[r]) || (sm.off_tmp[r + 1] - sm.off_tmp[r] != rec);
                 sm.info[stage][r] = make_uint2(sm.off_tmp[r] - off0, b);
@@ -385,18 +469,16 @@ __global__ void __launch_bounds__(PipeCfg<D>::THREADS) inject_kernel(PathParams 
             bad = __any_sync(0xffffffffu, bad);
             // with consistent records the span is rows * (at most 2*D) bytes, so it fits the stage
             const uint32_t span = sm.off_tmp[rows] - off0;
-            bad |= (off0 & 15u) != 0u || si.base < sec.payload_off || (si.base & 15u) != 0u ||
-                   si.base + (uint64_t)sm.off_tmp[rows] > total;
+            bad |= (off0 & 15u) != 0u || cur.base < sec.payload_off || (cur.base & 15u) != 0u ||
+                   cur.base + (uint64_t)sm.off_tmp[rows] > total;
             if (lane < C::NW) {
                 const int r0 = min(lane * C::RPW, rows), r1 = min(r0 + C::RPW, rows);
-                uint32_t ub = r0 < r1 ? bits[r0] : 0u;
-                for (int r = r0 + 1; r < r1; ++r) ub = bits[r] == ub ? ub : 0u;
-                sm.uniform_bits[stage][lane] = (r1 - r0 == C::RPW) ? ub : 0u;
+                sm.uniform_bits[stage][lane] = uniform_bits_of(sm.bits_tmp, r0, r1, C::RPW);
             }
             if (lane == 0) {
                 sm.rows[stage] = bad ? 0 : rows;
-                __half *dst = reinterpret_cast<__half *>(si.kv == 0 ? ptrs.k[si.layer_local] : ptrs.v[si.layer_local]) +
-                              (int64_t)si.head * p.head_stride + (p.dst_token_offset + t0) * p.token_stride;
+                __half *dst = reinterpret_cast<__half *>(cur.kv == 0 ? ptrs.k[cur.layer_local] : ptrs.v[cur.layer_local]) +
+                              (int64_t)cur.head * p.head_stride + (p.dst_token_offset + cur.t0) * p.token_stride;
                 sm.dst_row0[stage] = reinterpret_cast<uint64_t>(dst);
                 if (bad && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
             }
@@ -404,7 +486,7 @@ __global__ void __launch_bounds__(PipeCfg<D>::THREADS) inject_kernel(PathParams 
             if (lane == 0) {
                 if (!bad && span) {
                     mbar_arrive_expect_tx(&sm.full[stage], span);
-                    bulk_load(sm.in[stage], p.card + si.base + off0, span, &sm.full[stage]);
+                    bulk_load(sm.in[stage], p.card + cur.base + off0, span, &sm.full[stage]);
                 } else {
                     mbar_arrive(&sm.full[stage]);
                 }
@@ -424,13 +506,8 @@ __global__ void __launch_bounds__(PipeCfg<D>::THREADS) inject_kernel(PathParams 
             const int stage = k % NS;
             if (!mbar_wait(&sm.full[stage], (k / NS) & 1, abort_flag)) break;
             const int rows_t = sm.rows[stage];
-            switch (sm.uniform_bits[stage][warp]) {
-                case 4: inject_tile_body<D, NS, 4>(sm, stage, warp, lane, rows_t, p.token_stride); break;
-                case 2: inject_tile_body<D, NS, 2>(sm, stage, warp, lane, rows_t, p.token_stride); break;
-                case 8: inject_tile_body<D, NS, 8>(sm, stage, warp, lane, rows_t, p.token_stride); break;
-                case 16: inject_tile_body<D, NS, 16>(sm, stage, warp, lane, rows_t, p.token_stride); break;
-                default: inject_tile_body<D, NS, 0>(sm, stage, warp, lane, rows_t, p.token_stride); break;
-            }
+            if (C::LANES == 32 && rows_t == C::TB) inject_tile_dispatch<D, NS, true>(sm, stage, warp, lane, rows_t, p.token_stride);
+            else inject_tile_dispatch<D, NS, false>(sm, stage, warp, lane, rows_t, p.token_stride);
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.empty[stage]);
         }

@@ -119,11 +119,17 @@ __device__ __forceinline__ void fence_proxy_async()
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// fl32(float(h) - c): the FP16 operand is widened exactly, one rounding in binary32.
-__device__ __forceinline__ float sub_f32_f16(uint16_t h, float c)
+// (fl32(float(lo) - c), fl32(float(hi) - c)) for the two FP16 halves of `w`: each FP16 operand is
+// widened exactly and the difference is rounded once to binary32.
+__device__ __forceinline__ float2 sub_f32_f16x2(uint32_t w, float c)
 {
-    float d;
-    asm("sub.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(h), "f"(c));
+    float2 d;
+    asm("{\n\t.reg .b16 l, h;\n\t"
+        "mov.b32 {l, h}, %2;\n\t"
+        "sub.rn.f32.f16 %0, l, %3;\n\t"
+        "sub.rn.f32.f16 %1, h, %3;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "r"(w), "f"(c));
     return d;
 }
 
