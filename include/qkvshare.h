@@ -158,6 +158,16 @@ QKVS_API qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes,
  * (or BAD_CARD if magic/version are wrong, or CUDA on a runtime error). */
 QKVS_API qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_card_header_t *out_host);
 
+/* Self-test of the arithmetic shortcuts inside card creation.  The quantiser needs
+ * (max-min)/qmax and qmax/(max-min) correctly rounded; the kernels compute them without the
+ * generic division routine.  This call compares both shortcuts with the IEEE division for every
+ * binary32 value a difference of two FP16 numbers can take (2^-24 .. 131008) and qmax in
+ * {3, 15, 255}.  (The paper has no counterpart; Section 4.2.1 only says "quantized groups".)
+ *   mismatches_dev  device array of two uint64 (8-byte aligned), zeroed by the call;
+ *                   [0] counts mismatches of qmax/range, [1] of range/qmax.  Both must read 0.
+ * Asynchronous on `stream`; about 10^9 divisions, a few milliseconds. */
+QKVS_API qkvs_status_t qkvs_selftest_division(uint64_t *mismatches_dev, void *stream);
+
 QKVS_API const char *qkvs_status_string(qkvs_status_t status);
 
 /* Library version, major*100 + minor. */

@@ -50,7 +50,8 @@ class CardHeader(C.Structure):
 assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
-           "qkvs_card_inject", "qkvs_card_info", "qkvs_status_string", "qkvs_version")
+           "qkvs_card_inject", "qkvs_card_info", "qkvs_selftest_division", "qkvs_status_string",
+           "qkvs_version")
 
 _lib = None
 
@@ -79,6 +80,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_inject.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
     lib.qkvs_card_info.restype = C.c_int
     lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
+    lib.qkvs_selftest_division.restype = C.c_int
+    lib.qkvs_selftest_division.argtypes = [vp, vp]
     lib.qkvs_status_string.restype = C.c_char_p
     lib.qkvs_status_string.argtypes = [C.c_int]
     lib.qkvs_version.restype = C.c_int32
@@ -189,6 +192,14 @@ def card_info(card_dev, stream=None):
     hdr = CardHeader()
     st = load_library().qkvs_card_info(int(card_dev.data_ptr()), _stream_handle(stream), C.byref(hdr))
     return st, hdr
+
+
+def selftest_division(mismatches_dev, stream=None) -> int:
+    """qkvs_selftest_division.  mismatches_dev: CUDA int64 tensor of two elements."""
+    st = load_library().qkvs_selftest_division(int(mismatches_dev.data_ptr()), _stream_handle(stream))
+    if st != OK:
+        raise QkvsError(st, "qkvs_selftest_division")
+    return st
 
 
 def version() -> int:

@@ -248,6 +248,37 @@ __global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Self-test of the two division shortcuts against the IEEE division, over every range value the
+// path can produce (binary32 values from 2^-24 to 131008) and the three qmax values.
+
+__global__ void selftest_division_kernel(unsigned long long *mismatches)
+{
+    const uint32_t first = 0x33800000u;  // 2^-24
+    const uint32_t last = 0x47ffe000u;   // 131008 = 2 * 65504
+    unsigned long long bad_inv = 0, bad_scale = 0;
+    for (uint64_t u = (uint64_t)first + blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; u <= last;
+         u += (uint64_t)gridDim.x * blockDim.x) {
+        const float range = __uint_as_float((uint32_t)u);
+        const float qm[3] = {3.0f, 15.0f, 255.0f};
+        const float rc[3] = {0x1.555556p-2f, 0x1.111112p-4f, 0x1.010102p-8f};
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            bad_inv += __float_as_uint(qmax_over_range(qm[i], range)) != __float_as_uint(__fdiv_rn(qm[i], range));
+            bad_scale += __float_as_uint(divide_by_qmax(range, qm[i], rc[i])) != __float_as_uint(__fdiv_rn(range, qm[i]));
+        }
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        bad_inv += __shfl_xor_sync(0xffffffffu, bad_inv, s);
+        bad_scale += __shfl_xor_sync(0xffffffffu, bad_scale, s);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (bad_inv) atomicAdd(&mismatches[0], bad_inv);
+        if (bad_scale) atomicAdd(&mismatches[1], bad_scale);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Host side
 
 static qkvs_status_t check_shape(const qkvs_layout_t *l)
@@ -509,6 +540,15 @@ qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_card_heade
     if (out_host->magic != kMagic || out_host->version != kVersion) return QKVS_ERR_BAD_CARD;
     if (out_host->status > (uint32_t)QKVS_ERR_TIMEOUT) return QKVS_ERR_BAD_CARD;
     return (qkvs_status_t)out_host->status;
+}
+
+qkvs_status_t qkvs_selftest_division(uint64_t *mismatches_dev, void *stream)
+{
+    if (!mismatches_dev || (reinterpret_cast<uintptr_t>(mismatches_dev) & 7u)) return QKVS_ERR_INVALID_ARG;
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(mismatches_dev, 0, 2 * sizeof(uint64_t), cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    selftest_division_kernel<<<148 * 8, 256, 0, cs>>>(reinterpret_cast<unsigned long long *>(mismatches_dev));
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 
 const char *qkvs_status_string(qkvs_status_t status)

@@ -353,3 +353,13 @@ def test_config5_chain_of_four_hops_full():
     assert all(np.isfinite(errs)) and errs[0] > 0
     # error accumulates but stays bounded by a few first-hop errors (soft check)
     assert errs[-1] < 4 * errs[0] + 1e-3
+
+
+def test_division_shortcuts_equal_ieee_division_exhaustively():
+    """Both division shortcuts of the quantiser agree with the IEEE quotient on every reachable
+    operand (all binary32 ranges from 2^-24 to 131008, qmax in {3, 15, 255})."""
+    import torch
+    counts = torch.full((2,), -1, dtype=torch.int64, device="cuda")
+    q.selftest_division(counts)
+    torch.cuda.synchronize()
+    assert counts.tolist() == [0, 0]
