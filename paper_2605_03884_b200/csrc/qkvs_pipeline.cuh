@@ -9,11 +9,12 @@
 //                       copy (TMA) of the tile's input into a ring of NS shared-memory stages;
 //   NW consumer warps   wait on the stage's mbarrier, transform 16 bytes per lane per pass and
 //                       hand the stage back through a second mbarrier.
-// create: consumer warp w owns RPW consecutive rows of the tile, writes their records into its
-//         own shared-memory buffer and one lane sends that contiguous span to the card with a
-//         bulk store (double buffered per warp, so no CTA-wide barrier is needed).
-// inject: consumers read records from the staged span and store FP16 rows straight to the
-//         destination, 512 contiguous bytes per warp and pass.
+// create: consumer warp w owns RPW consecutive rows of the tile, one group of 32 channels per
+//         lane; it writes the rows' records into its own shared-memory buffer and one lane sends
+//         that contiguous span to the card with a bulk store (double buffered per warp, so no
+//         CTA-wide barrier is needed).
+// inject: consumers read records from the staged span, 16 output bytes per lane and pass, and
+//         store FP16 rows straight to the destination, 512 contiguous bytes per warp and pass.
 // No wait is unbounded: see mbar_wait.
 #pragma once
 
@@ -33,7 +34,9 @@ struct PipeCfg {
     static constexpr int PASSES = RPW / RPP;
     static constexpr int ROW_BYTES = 2 * D;
     static constexpr int TILE_BYTES = TB * ROW_BYTES;
-    static constexpr int G = D / kGroup;
+    static constexpr int G = D / kGroup;                // groups per token row
+    static constexpr int GPW = RPW * G;                 // groups per consumer warp (24 for D = 192)
+    static_assert(GPW <= 32, "one group per lane");
     static_assert(RPP >= 1 && RPW % RPP == 0 && TB % NW == 0, "tile shape");
 };
 
@@ -153,58 +156,44 @@ struct CreateSmem {
     int abort_flag;
 };
 
-// One chunk: 8 FP16 values (group minimum / maximum already known) -> metadata and codes written
-// into the record at `rec` (shared memory).  B is the warp-uniform bit-width, or 0 when lanes
-// may differ (then `b` is used).
-template <int D, int B>
-__device__ __forceinline__ void encode_chunk(const uint4 &v, float mn, float mx, int b, uint8_t *rec, int pos)
-{
-    constexpr int G = D / kGroup;
-    const int bb = B ? B : b;
-    if (bb == 16) {
-        *reinterpret_cast<uint4 *>(rec + pos * 16) = v;
-        return;
-    }
-    const GroupParams g = group_params(mn, mx, bb);
-    uint32_t lo, hi;
-    quantize_chunk_bytes(v, g, lo, hi);
-    uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * bb;  // 8 codes of b bits = b bytes
-    if ((pos & 3) == 0) *reinterpret_cast<float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup) = make_float2(g.scale, g.zero);
-    if (bb == 8) {
-        *reinterpret_cast<uint2 *>(codes) = make_uint2(lo, hi);
-    } else {
-        const uint32_t w = pack_nibbles(lo, hi);
-        if (bb == 4) *reinterpret_cast<uint32_t *>(codes) = w;
-        else *reinterpret_cast<uint16_t *>(codes) = (uint16_t)pack_crumbs(w);
-    }
-}
-
-// FULL: the tile has all TB rows and every lane carries data, so no validity checks are needed.
+// One group per thread: lane l of consumer warp w owns group l % G of row w * RPW + l / G, i.e.
+// the 64 input bytes at offset l * 64 of the warp's share of the tile.  The four chunks are read
+// in an order rotated by the lane so that the eight lanes served together by a 128-bit
+// shared-memory access fall into eight different 16-byte bank columns.
+// B is the warp-uniform bit-width, or 0 when rows of the warp differ (then the row's own
+// bit-width is used).  FULL: the tile has all TB rows and every lane has a group.
 template <int D, int NS, int B, bool FULL>
 __device__ __forceinline__ void create_tile_body(const CreateSmem<D, NS> &sm, int stage, int warp, int lane,
                                                  int rows_t, uint8_t *obuf)
 {
     using C = PipeCfg<D>;
-    const uint8_t *tin = sm.in[stage];
-    uint4 v[C::PASSES];
-    uint2 inf[C::PASSES];
-    const int sub = lane / C::CPR, pos = lane % C::CPR;
+    const int lrow = lane / C::G, g = lane % C::G;
+    const int row = warp * C::RPW + lrow;
+    if (!FULL && (lane >= C::GPW || row >= rows_t)) return;
+    const uint8_t *src = sm.in[stage] + (warp * C::RPW * C::ROW_BYTES + lane * 64);
+    const int rot = lane >> 1;
+    uint4 v[4];
 #pragma unroll
-    for (int j = 0; j < C::PASSES; ++j) {
-        const int row = warp * C::RPW + j * C::RPP + sub;
-        const bool valid = FULL || (lane < C::LANES && row < rows_t);
-        v[j] = make_uint4(0, 0, 0, 0);
-        inf[j] = make_uint2(0, 0);  // bit-width 0 marks a lane without data
-        if (valid) {
-            v[j] = *reinterpret_cast<const uint4 *>(tin + row * C::ROW_BYTES + pos * 16);
-            inf[j] = sm.info[stage][row];
-        }
+    for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(src + (((c + rot) & 3) << 4));
+    const uint2 inf = sm.info[stage][row];
+    const int b = B ? B : (int)inf.y;
+    uint8_t *rec = obuf + inf.x;
+    if (b == 16) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4 *>(rec + g * 64 + (((c + rot) & 3) << 4)) = v[c];
+        return;
     }
+    float mn, mx;
+    group_min_max(v, mn, mx);
+    const GroupParams gp = group_params(mn, mx, b);
+    *reinterpret_cast<float2 *>(rec + g * kMetaBytesPerGroup) = make_float2(gp.scale, gp.zero);
+    const uint64_t inv2 = pack_f32x2(gp.inv, gp.inv);
+    uint8_t *codes = rec + C::G * kMetaBytesPerGroup + g * (4 * b);  // 32 codes of b bits = 4b bytes
 #pragma unroll
-    for (int j = 0; j < C::PASSES; ++j) {
-        float mn, mx;
-        group_min_max(v[j], mn, mx);  // shuffles: every lane takes part, with or without data
-        if (FULL || inf[j].y != 0) encode_chunk<D, B>(v[j], mn, mx, (int)inf[j].y, obuf + inf[j].x, pos);
+    for (int c = 0; c < 4; ++c) {
+        uint32_t f[8];
+        quantize_chunk(v[c], gp.zero, inv2, f);
+        pack_store_chunk<B>(f, b, codes + ((c + rot) & 3) * b);
     }
 }
 
@@ -298,7 +287,7 @@ __global__ void __launch_bounds__(PipeCfg<D>::THREADS) create_kernel(PathParams 
             uint8_t *obuf = sm.out[warp][k & 1];
             if (lane == 0) bulk_wait_read<1>();  // the store that last used this buffer has read it
             __syncwarp();
-            if (C::LANES == 32 && rows_t == C::TB) create_tile_dispatch<D, NS, true>(sm, stage, warp, lane, rows_t, obuf);
+            if (C::GPW == 32 && rows_t == C::TB) create_tile_dispatch<D, NS, true>(sm, stage, warp, lane, rows_t, obuf);
             else create_tile_dispatch<D, NS, false>(sm, stage, warp, lane, rows_t, obuf);
             fence_proxy_async();
             __syncwarp();
