@@ -1,7 +1,8 @@
 // Thin wrappers over the sm_100a PTX used by the pipelines: mbarriers, 1-D bulk asynchronous
-// copies (TMA) between global and shared memory, the cross-proxy fence, and the mixed-precision
-// subtract.  Every wait is bounded: a wait that does not complete within kWaitLimitNs gives up
-// and reports failure so that the kernel can record an error status and return.
+// copies (TMA) between global and shared memory, the cross-proxy fence, the mixed-precision
+// subtract and packed binary32 arithmetic.  Every wait is bounded: a wait that does not complete
+// within kWaitLimitNs gives up and reports failure so that the kernel can record an error status
+// and return.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -10,6 +11,7 @@
 namespace qkvs {
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr uint32_t kWaitHintNs = 1000000u;                    // suspend hint of one poll: 1 ms
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p)
 {
@@ -37,15 +39,18 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
 }
 
+// One poll of the phase with the given parity.  The hardware may suspend the warp inside the
+// instruction until the phase completes or a time limit (the hint, in nanoseconds, or a shorter
+// system limit) runs out, so a waiting warp spends almost no issue slots.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
-        : "r"(smem_addr(bar)), "r"(parity)
+        : "r"(smem_addr(bar)), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     return done != 0;
 }
@@ -57,22 +62,15 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 
-// Waits for the phase with the given parity.  Returns false if the wait was abandoned, either
-// because it exceeded kWaitLimitNs (then *abort_flag is set) or because another thread of the
-// CTA set *abort_flag.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+// Waits for the phase with the given parity.  Returns false if the phase did not complete within
+// kWaitLimitNs; the caller then records an error status and winds down.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long start = global_timer_ns();
-    for (uint32_t it = 1;; ++it) {
+    for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - start > kWaitLimitNs) {
-                *abort_flag = 1;
-                return false;
-            }
-        }
+        if (global_timer_ns() - start > kWaitLimitNs) return false;
     }
 }
 

@@ -5,7 +5,7 @@
 //                         vector; writes the card's header, bits and offset tables (this file)
 //   create_kernel         fused group min/max -> scale/zero -> quantise -> bit-pack
 //   inject_kernel         unpack -> dequantise -> scatter into the destination cache layout
-// The last two are the persistent TMA pipelines of qkvs_pipeline.cuh.
+// The last two are the persistent per-warp TMA pipelines of qkvs_pipeline.cuh.
 // A stream is one (layer, K|V, head) matrix [tokens, head_dim].
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -308,12 +308,18 @@ static qkvs_status_t check_strides(const qkvs_layout_t *l, int64_t first_row)
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-constexpr int kStagesCreate = 4;
-constexpr int kStagesInject = 4;
+#ifndef QKVS_STAGES_CREATE
+#define QKVS_STAGES_CREATE 3
+#endif
+#ifndef QKVS_STAGES_INJECT
+#define QKVS_STAGES_INJECT 4
+#endif
+constexpr int kStagesCreate = QKVS_STAGES_CREATE;
+constexpr int kStagesInject = QKVS_STAGES_INJECT;
 
-// Persistent grid: as many CTAs as fit on the device at once, never more than there are tiles.
+// Persistent grid: as many CTAs as fit on the device at once, never more than there is work for.
 template <typename Kernel>
-static cudaError_t persistent_grid(Kernel kernel, int threads, size_t smem, int64_t n_tiles, unsigned *grid)
+static cudaError_t persistent_grid(Kernel kernel, int threads, size_t smem, int64_t max_ctas, unsigned *grid)
 {
     int dev = 0, sms = 0, per_sm = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -325,42 +331,42 @@ static cudaError_t persistent_grid(Kernel kernel, int threads, size_t smem, int6
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) return cudaErrorInvalidConfiguration;
-    *grid = (unsigned)std::min<int64_t>(n_tiles, (int64_t)sms * per_sm);
+    *grid = (unsigned)std::min<int64_t>(max_ctas, (int64_t)sms * per_sm);
     return cudaSuccess;
 }
 
-template <int D>
-static cudaError_t launch_create(const PathParams &pp, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+// Splits the sub-tiles of `streams` streams over a persistent grid and launches `kernel`.
+template <int D, typename Kernel>
+static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp, const LayerPtrs &ptrs, int64_t streams,
+                               cudaStream_t st)
 {
-    using C = PipeCfg<D>;
+    using C = WarpCfg<D>;
     PathParams p = pp;
-    p.tiles_per_stream = (uint32_t)((p.n_tokens + C::TB - 1) / C::TB);
-    const int64_t n_tiles = streams * p.tiles_per_stream;
-    if (n_tiles == 0) return cudaSuccess;
-    auto kernel = create_kernel<D, kStagesCreate>;
-    const size_t smem = sizeof(CreateSmem<D, kStagesCreate>);
+    p.subs_per_stream = (uint32_t)(((int64_t)p.n_tokens + C::R - 1) / C::R);
+    p.n_subs = (uint64_t)streams * p.subs_per_stream;
+    if (p.n_subs == 0) return cudaSuccess;
     unsigned grid = 0;
-    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, n_tiles, &grid);
+    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, (int64_t)((p.n_subs + C::WARPS - 1) / C::WARPS), &grid);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs, n_tiles);
+    p.last_rows = (uint32_t)(p.n_tokens - (int64_t)(p.subs_per_stream - 1) * C::R);
+    p.subs_per_cta = (uint32_t)(p.n_subs / grid);
+    p.subs_rem = (uint32_t)(p.n_subs % grid);
+    kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs);
     return cudaGetLastError();
 }
 
 template <int D>
-static cudaError_t launch_inject(const PathParams &pp, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+static cudaError_t launch_create(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    using C = PipeCfg<D>;
-    PathParams p = pp;
-    p.tiles_per_stream = (uint32_t)((p.n_tokens + C::TB - 1) / C::TB);
-    const int64_t n_tiles = streams * p.tiles_per_stream;
-    if (n_tiles == 0) return cudaSuccess;
-    auto kernel = inject_kernel<D, kStagesInject>;
-    const size_t smem = sizeof(InjectSmem<D, kStagesInject>);
-    unsigned grid = 0;
-    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, n_tiles, &grid);
-    if (e != cudaSuccess) return e;
-    kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs, n_tiles);
-    return cudaGetLastError();
+    return launch_path<D>(create_kernel<D, kStagesCreate>, WarpCfg<D>::WARPS * sizeof(CreateWarpSmem<D, kStagesCreate>), p,
+                          ptrs, streams, st);
+}
+
+template <int D>
+static cudaError_t launch_inject(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+{
+    return launch_path<D>(inject_kernel<D, kStagesInject>, WarpCfg<D>::WARPS * sizeof(InjectWarpSmem<D, kStagesInject>), p,
+                          ptrs, streams, st);
 }
 
 }  // namespace qkvs
