@@ -37,20 +37,27 @@ def is_stale() -> bool:
     return any(os.path.getmtime(d) > t for d in _deps())
 
 
-def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) -> str:
-    if not force and not is_stale():
+def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False,
+          defines: dict | None = None, out_path: str | None = None) -> str:
+    """Compile the library.  `defines` overrides tuning constants of the kernels (stages per
+    warp, warps per CTA, CTAs per SM) and `out_path` writes the result somewhere else than the
+    in-tree default; both exist for tuning sweeps."""
+    out = out_path or LIB_PATH
+    if not force and out_path is None and not is_stale():
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB_PATH + f".{os.getpid()}.tmp"
+    tmp = out + f".{os.getpid()}.tmp"
     cmd = [nvcc] + NVCC_FLAGS + ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    for k, v in (defines or {}).items():
+        cmd.append(f"-D{k}={v}")
     if ptxas_info:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-o", tmp] + _sources()
     if verbose:
         print(" ".join(cmd), file=sys.stderr)
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":

@@ -1,12 +1,11 @@
 // The two streaming kernels of the path, written as persistent grids of self-contained warps.
 //
-// A *sub-tile* is R consecutive tokens of one stream (one (layer, K|V, head) matrix), with R
-// chosen so that the sub-tile has one group of 32 channels per lane (R = 8 for head_dim 128).  On
-// the FP16 side a sub-tile is R rows of 2*D bytes; on the card side it is one contiguous, 16-byte
-// aligned span of records whose position and length follow from the offset table.  Every warp
-// runs its own pipeline over sub-tiles -- a CTA owns a contiguous range of them and its warps
-// take them in turn, so a warp stays inside one stream for many steps and its pointers advance
-// by constant increments:
+// A *sub-tile* is ROWS consecutive tokens of one stream (one (layer, K|V, head) matrix); ROWS is
+// chosen so that a sub-tile holds U groups of 32 channels per lane (16 tokens for head_dim 128).
+// On the FP16 side a sub-tile is ROWS rows of 2*D bytes; on the card side it is one contiguous,
+// 16-byte aligned span of records whose position and length follow from the offset table.  Every
+// warp runs its own pipeline over sub-tiles, which are dealt out to CTAs in bundles of one sub-tile
+// per warp (see my_share):
 //   - a private ring of NS shared-memory stages, each filled by one bulk asynchronous copy (TMA)
 //     that signals a private mbarrier; lane 0 re-arms a stage as soon as the warp has consumed it,
 //     so NS - 1 copies per warp are in flight while it computes;
@@ -14,8 +13,9 @@
 //     per lane, and spread with shuffles.
 // Warps never wait for one another, so many of them per SM hide the latency of each other's
 // arithmetic and waits.
-// create: one group of 32 channels per lane; records are written to a private shared-memory
-//         buffer and lane 0 sends the contiguous span to the card with a bulk store.
+// create: one group of 32 channels per lane and pass; every lane stores its group's scale / zero
+//         pair and packed codes straight into the card (neighbouring lanes complete 32-byte
+//         sectors, since a record is written by consecutive lanes).
 // inject: records are read from the staged span, 16 output bytes per lane and pass, and FP16
 //         rows are stored straight to the destination, 512 contiguous bytes per warp and pass.
 // No wait is unbounded: see mbar_wait.
@@ -25,19 +25,28 @@
 
 namespace qkvs {
 
+#ifndef QKVS_WARPS_PER_CTA
+#define QKVS_WARPS_PER_CTA 6
+#endif
+#ifndef QKVS_CTAS_PER_SM
+#define QKVS_CTAS_PER_SM 3
+#endif
+
 template <int D>
 struct WarpCfg {
-    static constexpr int WARPS = 8;                     // warps per CTA
+    static constexpr int WARPS = QKVS_WARPS_PER_CTA;    // warps per CTA
     static constexpr int THREADS = WARPS * 32;
     static constexpr int G = D / kGroup;                // groups per token row
-    static constexpr int R = 32 / G;                    // rows per sub-tile: 16, 8, 5, 4 for D = 64, 128, 192, 256
+    static constexpr int R = 32 / G;                    // rows covered by one group per lane: 16, 8, 5, 4
     static constexpr int GROUPS = R * G;                // lanes that own a group in create (30 for D = 192)
+    static constexpr int U = D == 64 ? 1 : 2;           // groups per lane and sub-tile
+    static constexpr int ROWS = U * R;                  // rows per sub-tile: 16, 16, 10, 8 for D = 64, 128, 192, 256
     static constexpr int ROW_BYTES = 2 * D;
-    static constexpr int STAGE_BYTES = R * ROW_BYTES;   // 2048 (1920 for D = 192); a record never exceeds a row
+    static constexpr int STAGE_BYTES = ROWS * ROW_BYTES;  // 2048 / 4096 / 3840 / 4096; a record never exceeds a row
     static constexpr int CPR = D / 8;                   // 16-byte chunks per row
-    static constexpr int CHUNKS = R * CPR;              // chunks per sub-tile
+    static constexpr int CHUNKS = ROWS * CPR;           // chunks per sub-tile
     static constexpr int PASSES = (CHUNKS + 31) / 32;   // inject: passes of one chunk per lane
-    static_assert(R >= 1 && GROUPS <= 32 && STAGE_BYTES % 16 == 0, "sub-tile shape");
+    static_assert(R >= 1 && GROUPS <= 32 && ROWS + 1 <= 32 && STAGE_BYTES % 16 == 0, "sub-tile shape");
 };
 
 // Position of a sub-tile: index inside its stream, kv * H + head, and layer inside the launch's
@@ -57,21 +66,23 @@ __device__ __forceinline__ Pos first_pos(const PathParams &p, uint64_t sub)
     return c;
 }
 
-// Moves on by one warp step (WARPS sub-tiles).  Returns true when that left the stream, which
-// is rare: the caller then recomputes its stream-level pointers instead of incrementing them.
-template <int WARPS>
+// Moves on by one warp step.  Returns true when that left the stream: the caller then recomputes
+// its stream-level pointers instead of incrementing them by p.step_t sub-tiles.
 __device__ __forceinline__ bool step(Pos &c, const PathParams &p)
 {
-    c.tt += WARPS;
-    if (c.tt < p.subs_per_stream) return false;
+    c.tt += p.step_t;
+    if (p.step_r == 0u && p.step_l == 0u && c.tt < p.subs_per_stream) return false;
     const uint32_t twoH = 2u * (uint32_t)p.n_kv_heads;
-    do {
+    c.r += p.step_r;
+    c.layer += p.step_l;
+    while (c.tt >= p.subs_per_stream) {
         c.tt -= p.subs_per_stream;
-        if (++c.r == twoH) {
-            c.r = 0;
-            ++c.layer;
-        }
-    } while (c.tt >= p.subs_per_stream);
+        c.r += 1u;
+    }
+    while (c.r >= twoH) {
+        c.r -= twoH;
+        c.layer += 1u;
+    }
     return true;
 }
 
@@ -98,8 +109,8 @@ struct CacheWalk {
     }
     __device__ __forceinline__ void next(const PathParams &p, const LayerPtrs &ptrs, int64_t first_row)
     {
-        if (step<WARPS>(c, p)) locate(p, ptrs, first_row);
-        else row += (int64_t)(WARPS * R) * p.token_stride;
+        if (step(c, p)) locate(p, ptrs, first_row);
+        else row += (int64_t)(p.step_t * R) * p.token_stride;
     }
 };
 
@@ -128,11 +139,11 @@ struct TableWalk {
     }
     __device__ __forceinline__ void next(const PathParams &p, const Sections &sec, int bits_mode, uint64_t stream_bytes)
     {
-        if (step<WARPS>(c, p)) {
+        if (step(c, p)) {
             locate(p, sec, bits_mode, stream_bytes);
         } else {
-            offs += WARPS * R;
-            bits += WARPS * R;
+            offs += p.step_t * R;
+            bits += p.step_t * R;
         }
     }
 };
@@ -154,16 +165,24 @@ __device__ __forceinline__ void fetch_tables(Tables &t, const TableWalk<R, WARPS
     t.bits = lane < t.rows ? (uint32_t)__ldg(w.bits + lane) : 0u;
 }
 
-// Sub-tiles of this warp: CTA b owns the contiguous range of sub-tiles
-// [b * q + min(b, rem), ...) of length q + (b < rem); inside it warp w takes the sub-tiles
-// w, w + WARPS, ...  Returns how many that is and the first one's global index.
+// Sub-tiles of this warp.  The sub-tiles are dealt out in bundles of WARPS consecutive ones (warp w
+// of a CTA takes the w-th of each bundle).  With p.interleaved, CTA b takes bundles b, b + grid,
+// ... so that at any moment the grid works on one contiguous window of the cache; otherwise CTA b
+// owns a contiguous range of bundles.  Returns how many sub-tiles the warp has and the first one.
 template <int WARPS>
 __device__ __forceinline__ uint32_t my_share(const PathParams &p, int warp, uint64_t &first)
 {
     const uint32_t b = blockIdx.x;
-    const uint32_t len = p.subs_per_cta + (b < p.subs_rem ? 1u : 0u);
-    first = (uint64_t)b * p.subs_per_cta + min(b, p.subs_rem) + (uint32_t)warp;
-    return (uint32_t)warp < len ? (len - (uint32_t)warp + WARPS - 1) / WARPS : 0u;
+    const uint32_t n = p.bundles_per_cta + (b < p.bundles_rem ? 1u : 0u);  // bundles of this CTA
+    if (n == 0u) {
+        first = 0;
+        return 0u;
+    }
+    const uint64_t first_bundle = p.interleaved ? b : (uint64_t)b * p.bundles_per_cta + min(b, p.bundles_rem);
+    const uint64_t last_bundle = p.interleaved ? b + (uint64_t)(n - 1u) * gridDim.x : first_bundle + (n - 1u);
+    first = first_bundle * WARPS + (uint32_t)warp;
+    // only the very last bundle of the launch can be short
+    return last_bundle * WARPS + (uint32_t)warp < p.n_subs ? n : n - 1u;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -173,40 +192,68 @@ template <int D, int NS>
 struct CreateWarpSmem {
     using C = WarpCfg<D>;
     alignas(128) uint8_t in[NS][C::STAGE_BYTES];
-    alignas(128) uint8_t out[C::STAGE_BYTES];
     alignas(8) uint64_t full[NS];
 };
 
-// One group per lane: lane l owns group l % G of row l / G, i.e. the 64 input bytes at offset
-// l * 64 of the stage.  The four chunks are read in an order rotated by the lane so that the
+// One group: lane l owns group l % G of row l / G of the R rows at `rows_in`, i.e. the 64 input
+// bytes at offset l * 64.  The four chunks are read in an order rotated by the lane so that the
 // eight lanes served together by a 128-bit shared-memory access fall into eight different
-// 16-byte bank columns.  B is the warp-uniform bit-width, or 0 when rows differ (then `b`).
+// 16-byte bank columns; the packed codes are put back in channel order before they are stored.
+// `rec` is the row's record in the card.  B is the warp-uniform bit-width, or 0 when rows
+// differ (then `b`).
 template <int D, int B>
-__device__ __forceinline__ void encode_group(const uint8_t *stage, uint8_t *rec, int lane, int g, int b)
+__device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *rec, int lane, int g, int b)
 {
     constexpr int G = D / kGroup;
-    const uint8_t *src = stage + lane * 64;
-    const int rot = lane >> 1;
+    const uint8_t *src = rows_in + lane * 64;
+    const int rot = (lane >> 1) & 3;
     uint4 v[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) v[c] = *reinterpret_cast<const uint4 *>(src + (((c + rot) & 3) << 4));
     const int bb = B ? B : b;
     if (bb == 16) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4 *>(rec + g * 64 + (((c + rot) & 3) << 4)) = v[c];
+        for (int c = 0; c < 4; ++c) __stcs(reinterpret_cast<uint4 *>(rec + g * 64 + (((c + rot) & 3) << 4)), v[c]);
         return;
     }
     float mn, mx;
     group_min_max(v, mn, mx);
     const GroupParams gp = group_params(mn, mx, bb);
-    *reinterpret_cast<float2 *>(rec + g * kMetaBytesPerGroup) = make_float2(gp.scale, gp.zero);
+    __stcs(reinterpret_cast<float2 *>(rec + g * kMetaBytesPerGroup), make_float2(gp.scale, gp.zero));
     const uint64_t inv2 = pack_f32x2(gp.inv, gp.inv);
-    uint8_t *codes = rec + G * kMetaBytesPerGroup + g * (4 * bb);  // 32 codes of b bits = 4b bytes
+    uint32_t lo[4], hi[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         uint32_t f[8];
         quantize_chunk(v[c], gp.zero, inv2, f);
-        pack_store_chunk<B>(f, bb, codes + ((c + rot) & 3) * bb);
+        pack_chunk<B>(f, bb, lo[c], hi[c]);
+    }
+    unrotate4(lo, rot);
+    uint8_t *codes = rec + G * kMetaBytesPerGroup + g * (4 * bb);  // 32 codes of b bits = 4b bytes
+    if (bb == 8) {
+        unrotate4(hi, rot);
+        __stcs(reinterpret_cast<uint4 *>(codes), make_uint4(lo[0], hi[0], lo[1], hi[1]));
+        __stcs(reinterpret_cast<uint4 *>(codes + 16), make_uint4(lo[2], hi[2], lo[3], hi[3]));
+    } else if (bb == 4) {
+        __stcs(reinterpret_cast<uint4 *>(codes), make_uint4(lo[0], lo[1], lo[2], lo[3]));
+    } else {
+        __stcs(reinterpret_cast<uint2 *>(codes), make_uint2(__byte_perm(lo[0], lo[1], 0x5410), __byte_perm(lo[2], lo[3], 0x5410)));
+    }
+}
+
+// All U passes of a sub-tile.  Every lane of the warp calls this (it shuffles).
+template <int D, int B>
+__device__ __forceinline__ void encode_rows(const uint8_t *in, uint8_t *stream, const Tables &t, int lane)
+{
+    using C = WarpCfg<D>;
+    const int lrow = lane / C::G, g = lane % C::G;
+#pragma unroll
+    for (int u = 0; u < C::U; ++u) {
+        const int row = u * C::R + lrow;
+        const uint32_t off_row = __shfl_sync(0xffffffffu, t.off, row);
+        const int b = B ? B : (int)__shfl_sync(0xffffffffu, t.bits, row);
+        if (lane < C::GROUPS && row < t.rows)
+            encode_group<D, B>(in + u * (C::R * C::ROW_BYTES), stream + off_row, lane, g, b);
     }
 }
 
@@ -230,7 +277,7 @@ __device__ __forceinline__ void create_issue(CreateWarpSmem<D, NS> &sm, int stag
 }
 
 template <int D, int NS>
-__global__ void __launch_bounds__(WarpCfg<D>::THREADS, 3) create_kernel(PathParams p, LayerPtrs ptrs)
+__global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -252,22 +299,21 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, 3) create_kernel(PathPara
     }
     __syncwarp();
 
-    CacheWalk<C::R, C::WARPS> ahead;  // runs NS sub-tiles ahead and starts the copies
+    CacheWalk<C::ROWS, C::WARPS> ahead;  // runs NS sub-tiles ahead and starts the copies
     ahead.c = first_pos(p, first);
     ahead.locate(p, ptrs, 0);
-    TableWalk<C::R, C::WARPS> tw;
+    TableWalk<C::ROWS, C::WARPS> tw;
     tw.c = ahead.c;
     tw.locate(p, sec, p.bits_mode, stream_bytes);
 
     uint32_t issued = 0;
     for (; issued < (uint32_t)NS && issued < n_mine; ++issued) {
-        create_issue<D, NS>(sm, (int)issued, ahead.row, rows_at<C::R>(ahead.c, p), p, lane);
+        create_issue<D, NS>(sm, (int)issued, ahead.row, rows_at<C::ROWS>(ahead.c, p), p, lane);
         if (issued + 1 < n_mine) ahead.next(p, ptrs, 0);
     }
     Tables nxt;
     fetch_tables(nxt, tw, p, lane);
 
-    const int lrow = lane / C::G, g = lane % C::G;
     int stage = 0;
     uint32_t parity = 0, k = 0;
     bool ok = true;
@@ -277,43 +323,26 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, 3) create_kernel(PathPara
             tw.next(p, sec, p.bits_mode, stream_bytes);
             fetch_tables(nxt, tw, p, lane);
         }
-
-        // what this lane's row needs, spread from the lanes that hold the table entries
-        const uint32_t off0 = __shfl_sync(0xffffffffu, cur.off, 0);
-        const uint32_t off_end = __shfl_sync(0xffffffffu, cur.off, cur.rows);
-        const uint32_t off_row = __shfl_sync(0xffffffffu, cur.off, lrow);
-        const int b = (int)__shfl_sync(0xffffffffu, cur.bits, lrow);
         const int b0 = (int)__shfl_sync(0xffffffffu, cur.bits, 0);
-        const bool mine = lane < C::GROUPS && lrow < cur.rows;
-        const bool uniform = __all_sync(0xffffffffu, !mine || b == b0);
+        const bool uniform = __all_sync(0xffffffffu, lane >= cur.rows || (int)cur.bits == b0);
 
         ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[stage], parity));
         if (!ok) break;
-        if (lane == 0) bulk_wait_read<0>();  // the previous bulk store has read the output buffer
-        __syncwarp();
-        if (mine) {
-            uint8_t *rec = sm.out + (off_row - off0);
-            const uint8_t *in = sm.in[stage];
-            if (uniform) {
-                switch (b0) {
-                    case 4: encode_group<D, 4>(in, rec, lane, g, 4); break;
-                    case 2: encode_group<D, 2>(in, rec, lane, g, 2); break;
-                    case 8: encode_group<D, 8>(in, rec, lane, g, 8); break;
-                    default: encode_group<D, 16>(in, rec, lane, g, 16); break;
-                }
-            } else {
-                encode_group<D, 0>(in, rec, lane, g, b);
+        const uint8_t *in = sm.in[stage];
+        uint8_t *stream = p.card + cur.base;
+        if (uniform) {
+            switch (b0) {
+                case 4: encode_rows<D, 4>(in, stream, cur, lane); break;
+                case 2: encode_rows<D, 2>(in, stream, cur, lane); break;
+                case 8: encode_rows<D, 8>(in, stream, cur, lane); break;
+                default: encode_rows<D, 16>(in, stream, cur, lane); break;
             }
+        } else {
+            encode_rows<D, 0>(in, stream, cur, lane);
         }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) {
-            const uint32_t bytes = off_end - off0;
-            if (bytes) bulk_store(p.card + cur.base + off0, sm.out, bytes);
-            bulk_commit();
-        }
-        if (issued < n_mine) {  // the stage is consumed: re-arm it with the sub-tile NS steps ahead
-            create_issue<D, NS>(sm, stage, ahead.row, rows_at<C::R>(ahead.c, p), p, lane);
+        __syncwarp();  // every lane has read the stage: it can be re-armed
+        if (issued < n_mine) {
+            create_issue<D, NS>(sm, stage, ahead.row, rows_at<C::ROWS>(ahead.c, p), p, lane);
             if (++issued < n_mine) ahead.next(p, ptrs, 0);
         }
         if (++stage == NS) {
@@ -333,7 +362,6 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, 3) create_kernel(PathPara
             mbar_wait(&sm.full[stage], parity);
         }
     }
-    if (lane == 0) bulk_wait<0>();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -343,9 +371,9 @@ template <int D, int NS>
 struct InjectWarpSmem {
     using C = WarpCfg<D>;
     alignas(128) uint8_t in[NS][C::STAGE_BYTES];
-    alignas(8) uint2 info[NS][C::R];   // per row: {record offset inside the span, bit-width}
+    uint32_t info[NS][C::ROWS];        // per row: record offset inside the span << 8 | bit-width
     alignas(8) uint64_t full[NS];
-    uint32_t uniform_bits[NS];         // bit-width shared by all R rows, else 0
+    uint32_t uniform_bits[NS];         // bit-width shared by all ROWS rows, else 0
     int32_t rows[NS];                  // 0 when the sub-tile's table entries did not check out
 };
 
@@ -371,7 +399,7 @@ __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos
     return dequantize_chunk(lo, hi, m.x, m.y);
 }
 
-// FULL: the sub-tile has all R rows and every lane has a chunk in every pass.
+// FULL: the sub-tile has all ROWS rows and every lane has a chunk in every pass.
 template <int D, int NS, int B, bool FULL>
 __device__ __forceinline__ void inject_rows(const InjectWarpSmem<D, NS> &sm, int stage, int lane, int rows, __half *dst0,
                                             int64_t token_stride)
@@ -383,8 +411,8 @@ __device__ __forceinline__ void inject_rows(const InjectWarpSmem<D, NS> &sm, int
         const int ci = j * 32 + lane;
         const int row = ci / C::CPR, pos = ci % C::CPR;
         if (FULL || (ci < C::CHUNKS && row < rows)) {
-            const uint2 inf = sm.info[stage][row];
-            const uint4 out = decode_chunk<D, B>(in + inf.x, (int)inf.y, pos);
+            const uint32_t inf = sm.info[stage][row];
+            const uint4 out = decode_chunk<D, B>(in + (inf >> 8), (int)(inf & 0xffu), pos);
             __stcs(reinterpret_cast<uint4 *>(dst0 + (int64_t)row * token_stride + pos * 8), out);
         }
     }
@@ -426,9 +454,9 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
     if (lane < rows) {
         const uint32_t rec = record_bytes(D, (int)t.bits);
         bad = (rec == 0u) || (off_next < t.off) || (off_next - t.off != rec);
-        sm.info[stage][lane] = make_uint2(t.off - off0, t.bits);
+        sm.info[stage][lane] = ((t.off - off0) << 8) | (t.bits & 0xffu);
     }
-    const bool uniform = rows == C::R && __all_sync(0xffffffffu, lane >= rows || t.bits == b0);
+    const bool uniform = rows == C::ROWS && __all_sync(0xffffffffu, lane >= rows || t.bits == b0);
     bad = __any_sync(0xffffffffu, bad);
     // with consistent records the span is rows * (at most 2*D) bytes, so it fits the stage
     const uint32_t span = off_end - off0;
@@ -448,7 +476,7 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
 }
 
 template <int D, int NS>
-__global__ void __launch_bounds__(WarpCfg<D>::THREADS, 3) inject_kernel(PathParams p, LayerPtrs ptrs)
+__global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) inject_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -490,10 +518,10 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, 3) inject_kernel(PathPara
 
     // The copy of a span can only start once its table entries are known, so the table reads run
     // one step ahead of the copies, which run NS steps ahead of the arithmetic.
-    TableWalk<C::R, C::WARPS> tw;
+    TableWalk<C::ROWS, C::WARPS> tw;
     tw.c = first_pos(p, first);
     tw.locate(p, sec, mode, stream_bytes);
-    CacheWalk<C::R, C::WARPS> cons;
+    CacheWalk<C::ROWS, C::WARPS> cons;
     cons.c = tw.c;
     cons.locate(p, ptrs, p.dst_token_offset);
 
@@ -518,7 +546,7 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, 3) inject_kernel(PathPara
         const int rows = sm.rows[stage];
         const uint32_t ub = sm.uniform_bits[stage];
         __half *dst0 = cons.row;
-        if (C::CHUNKS % 32 == 0 && rows == C::R) {
+        if (C::CHUNKS % 32 == 0 && rows == C::ROWS) {
             switch (ub) {
                 case 4: inject_rows<D, NS, 4, true>(sm, stage, lane, rows, dst0, p.token_stride); break;
                 case 2: inject_rows<D, NS, 2, true>(sm, stage, lane, rows, dst0, p.token_stride); break;

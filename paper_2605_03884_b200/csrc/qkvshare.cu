@@ -312,7 +312,10 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 #define QKVS_STAGES_CREATE 3
 #endif
 #ifndef QKVS_STAGES_INJECT
-#define QKVS_STAGES_INJECT 4
+#define QKVS_STAGES_INJECT 3
+#endif
+#ifndef QKVS_INTERLEAVED
+#define QKVS_INTERLEAVED 1
 #endif
 constexpr int kStagesCreate = QKVS_STAGES_CREATE;
 constexpr int kStagesInject = QKVS_STAGES_INJECT;
@@ -342,15 +345,23 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
 {
     using C = WarpCfg<D>;
     PathParams p = pp;
-    p.subs_per_stream = (uint32_t)(((int64_t)p.n_tokens + C::R - 1) / C::R);
+    p.subs_per_stream = (uint32_t)(((int64_t)p.n_tokens + C::ROWS - 1) / C::ROWS);
     p.n_subs = (uint64_t)streams * p.subs_per_stream;
     if (p.n_subs == 0) return cudaSuccess;
     unsigned grid = 0;
     cudaError_t e = persistent_grid(kernel, C::THREADS, smem, (int64_t)((p.n_subs + C::WARPS - 1) / C::WARPS), &grid);
     if (e != cudaSuccess) return e;
-    p.last_rows = (uint32_t)(p.n_tokens - (int64_t)(p.subs_per_stream - 1) * C::R);
-    p.subs_per_cta = (uint32_t)(p.n_subs / grid);
-    p.subs_rem = (uint32_t)(p.n_subs % grid);
+    p.last_rows = (uint32_t)(p.n_tokens - (int64_t)(p.subs_per_stream - 1) * C::ROWS);
+    const uint64_t n_bundles = (p.n_subs + C::WARPS - 1) / C::WARPS;
+    p.bundles_per_cta = (uint32_t)(n_bundles / grid);
+    p.bundles_rem = (uint32_t)(n_bundles % grid);
+    p.interleaved = QKVS_INTERLEAVED;
+    const uint64_t step = (uint64_t)C::WARPS * (p.interleaved ? grid : 1u);  // sub-tiles per warp step
+    const uint64_t step_s = step / p.subs_per_stream;                         // whole streams per step
+    const uint32_t twoH = 2u * (uint32_t)p.n_kv_heads;
+    p.step_t = (uint32_t)(step % p.subs_per_stream);
+    p.step_r = (uint32_t)(step_s % twoH);
+    p.step_l = (uint32_t)(step_s / twoH);
     kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs);
     return cudaGetLastError();
 }
