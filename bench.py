@@ -204,6 +204,7 @@ def run_ours(args):
     bits_h = [torch.from_numpy(b).pin_memory() for b in bits_per_hop]
     bits_d = [b.cuda() for b in bits_h]
     card = torch.zeros(max(sizes), dtype=torch.uint8, device="cuda")
+    ws = q.new_workspace()
     for dst, src in zip(Kd + Vd, Kh + Vh):
         dst.copy_(src)
     stream = torch.cuda.current_stream()
@@ -216,9 +217,9 @@ def run_ours(args):
             e1 = torch.cuda.Event(enable_timing=True)
             e2 = torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            q.card_create(lay, src_k, src_v, bits_d[h], card, card_capacity=sizes[h], stream=stream)
+            q.card_create(lay, src_k, src_v, bits_d[h], card, card_capacity=sizes[h], workspace=ws, stream=stream)
             e1.record(stream)
-            q.card_inject(card, lay, Ko, Vo, card_bytes=sizes[h], stream=stream)
+            q.card_inject(card, lay, Ko, Vo, card_bytes=sizes[h], workspace=ws, stream=stream)
             e2.record(stream)
             if record is not None:
                 record.append((h, e0, e1, e2))

@@ -32,6 +32,14 @@
  * device pointer, anything else is a host pointer.  The library allocates no device memory and
  * keeps no state between calls; every buffer belongs to the caller.  Launches are asynchronous
  * on the given CUDA stream (a cudaStream_t passed as void*; NULL is the default stream).
+ *
+ * Scratch block.  qkvs_card_create and qkvs_card_inject take an optional `workspace_dev`: a
+ * device buffer of QKVS_WORKSPACE_BYTES bytes, 16-byte aligned, owned by the caller.  Its content
+ * on entry does not matter (each call clears it on its stream).  The kernels keep in it the
+ * counters from which their warps draw work -- with them, SMs that run faster simply take more of
+ * it -- and, for injection, the status word described there.  Without a block (NULL) the work is
+ * split evenly in advance, which is a few percent slower, and injection reports no status.
+ * Two calls that may run on the GPU at the same time must not share a block.
  */
 #ifndef QKVSHARE_H_
 #define QKVSHARE_H_
@@ -48,6 +56,8 @@
 #ifdef __cplusplus
 extern "C" {
 #endif
+
+#define QKVS_WORKSPACE_BYTES 256
 
 typedef enum {
     QKVS_OK = 0,
@@ -128,6 +138,7 @@ QKVS_API qkvs_status_t qkvs_card_prefix_size(const qkvs_layout_t *layout, size_t
  *   meta                identifiers to store; NULL stores zeros
  *   card_dev            device buffer, 16-byte aligned, written from byte 0
  *   card_capacity       its size in bytes; must cover at least the prefix
+ *   workspace_dev       scratch block (see above) or NULL
  * Returns after enqueueing on `stream`.  Problems visible on the host (arguments, shape,
  * alignment, capacity below the prefix) are returned at once and nothing is launched.
  * Problems only the device can see -- a bit-width outside {2,4,8,16}, or a payload that does
@@ -137,7 +148,7 @@ QKVS_API qkvs_status_t qkvs_card_prefix_size(const qkvs_layout_t *layout, size_t
 QKVS_API qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K_layers,
                                const void *const *V_layers, const uint8_t *bits_dev,
                                const qkvs_card_meta_t *meta, void *card_dev,
-                               size_t card_capacity, void *stream);
+                               size_t card_capacity, void *workspace_dev, void *stream);
 
 /* Receiver-side injection (Section 4.2.2): unpack, dequantise and write FP16 rows so that
  * token t of the card lands on row dst_token_offset + t of every head of every layer.
@@ -146,13 +157,15 @@ QKVS_API qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void 
  *                          and n_tokens must equal the card's (checked on the device), and
  *                          (dst_token_offset + n_tokens - 1)*token_stride + head_dim <= head_stride
  *   K_layers_out, V_layers_out   HOST arrays of n_layers DEVICE pointers (16-byte aligned)
- *   status_dev             optional device int32, set to 0 by this call and raised to
- *                          BAD_CARD by the kernel if the header or its tables do not check out
- *                          (then no row is written); may be NULL
+ *   workspace_dev          scratch block (see above) or NULL.  Its first 4 bytes are an int32
+ *                          status word: 0 after a clean run, raised to BAD_CARD by the kernel if
+ *                          the header or its tables do not check out (rows whose table entries
+ *                          are inconsistent are not written; with a bad header no row is), or to
+ *                          TIMEOUT if a bounded wait gave up
  * Bytes of the destination outside the injected rows and channels are left untouched. */
 QKVS_API qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qkvs_layout_t *dst,
                                void *const *K_layers_out, void *const *V_layers_out,
-                               int64_t dst_token_offset, int32_t *status_dev, void *stream);
+                               int64_t dst_token_offset, void *workspace_dev, void *stream);
 
 /* Synchronises `stream`, copies the card's header to the host and returns its recorded status
  * (or BAD_CARD if magic/version are wrong, or CUDA on a runtime error). */

@@ -75,7 +75,7 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_prefix_size.restype = C.c_int
     lib.qkvs_card_prefix_size.argtypes = [C.POINTER(Layout), C.POINTER(C.c_size_t)]
     lib.qkvs_card_create.restype = C.c_int
-    lib.qkvs_card_create.argtypes = [C.POINTER(Layout), vp, vp, vp, C.POINTER(CardMeta), vp, C.c_size_t, vp]
+    lib.qkvs_card_create.argtypes = [C.POINTER(Layout), vp, vp, vp, C.POINTER(CardMeta), vp, C.c_size_t, vp, vp]
     lib.qkvs_card_inject.restype = C.c_int
     lib.qkvs_card_inject.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
     lib.qkvs_card_info.restype = C.c_int
@@ -155,33 +155,51 @@ def card_prefix_size(layout: Layout) -> int:
     return int(out.value)
 
 
+WORKSPACE_BYTES = 256
+
+
+def new_workspace(device="cuda"):
+    """A scratch block for card_create / card_inject: WORKSPACE_BYTES of device memory (int32)."""
+    import torch
+    return torch.zeros(WORKSPACE_BYTES // 4, dtype=torch.int32, device=device)
+
+
+def _workspace_ptr(workspace):
+    if workspace is None:
+        return None
+    if workspace.numel() * workspace.element_size() < WORKSPACE_BYTES:
+        raise ValueError(f"workspace must hold {WORKSPACE_BYTES} bytes")
+    return int(workspace.data_ptr())
+
+
 def card_create(layout: Layout, K_layers: Sequence, V_layers: Sequence, bits_dev, card_dev,
                 meta: Optional[CardMeta] = None, card_capacity: Optional[int] = None,
-                stream=None, check: bool = True) -> int:
+                workspace=None, stream=None, check: bool = True) -> int:
     """qkvs_card_create.  K_layers / V_layers: per-layer CUDA tensors (FP16); bits_dev: CUDA uint8
-    tensor; card_dev: CUDA uint8 tensor that receives the card.  Returns the status."""
+    tensor; card_dev: CUDA uint8 tensor that receives the card; workspace: CUDA tensor of
+    WORKSPACE_BYTES bytes (see new_workspace) or None.  Returns the status."""
     lib = load_library()
     kp, vp = _ptr_array(K_layers), _ptr_array(V_layers)
     cap = int(card_dev.numel() * card_dev.element_size()) if card_capacity is None else int(card_capacity)
     st = lib.qkvs_card_create(C.byref(layout), kp, vp, int(bits_dev.data_ptr()) if bits_dev is not None else None,
                               C.byref(meta) if meta is not None else None, int(card_dev.data_ptr()), cap,
-                              _stream_handle(stream))
+                              _workspace_ptr(workspace), _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_card_create")
     return st
 
 
 def card_inject(card_dev, dst_layout: Layout, K_out: Sequence, V_out: Sequence,
-                dst_token_offset: int = 0, card_bytes: Optional[int] = None, status_dev=None,
+                dst_token_offset: int = 0, card_bytes: Optional[int] = None, workspace=None,
                 stream=None, check: bool = True) -> int:
-    """qkvs_card_inject.  status_dev: optional CUDA int32 tensor of one element."""
+    """qkvs_card_inject.  workspace: CUDA int32 tensor of WORKSPACE_BYTES bytes or None; after
+    the call its element 0 is the status word the kernel recorded."""
     lib = load_library()
     kp, vp = _ptr_array(K_out), _ptr_array(V_out)
     nbytes = int(card_dev.numel() * card_dev.element_size()) if card_bytes is None else int(card_bytes)
     st = lib.qkvs_card_inject(int(card_dev.data_ptr()), nbytes, C.byref(dst_layout), kp, vp,
                               int(dst_token_offset),
-                              int(status_dev.data_ptr()) if status_dev is not None else None,
-                              _stream_handle(stream))
+                              _workspace_ptr(workspace), _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_card_inject")
     return st

@@ -4,8 +4,8 @@
 // chosen so that a sub-tile holds U groups of 32 channels per lane (16 tokens for head_dim 128).
 // On the FP16 side a sub-tile is ROWS rows of 2*D bytes; on the card side it is one contiguous,
 // 16-byte aligned span of records whose position and length follow from the offset table.  Every
-// warp runs its own pipeline over sub-tiles, which are dealt out to CTAs in bundles of one sub-tile
-// per warp (see my_share):
+// warp runs its own pipeline over sub-tiles, which it takes in chunks of eight consecutive ones
+// from a shared counter (see WorkSource):
 //   - a private ring of NS shared-memory stages, each filled by one bulk asynchronous copy (TMA)
 //     that signals a private mbarrier; lane 0 re-arms a stage as soon as the warp has consumed it,
 //     so NS - 1 copies per warp are in flight while it computes;
@@ -55,33 +55,25 @@ struct Pos {
     uint32_t tt, r, layer;
 };
 
-__device__ __forceinline__ Pos first_pos(const PathParams &p, uint64_t sub)
+__device__ __forceinline__ Pos position_of(const PathParams &p, uint32_t sub)
 {
     Pos c;
-    const uint64_t s = sub / p.subs_per_stream;
+    const uint32_t s = sub / p.subs_per_stream;
     const uint32_t twoH = 2u * (uint32_t)p.n_kv_heads;
-    c.tt = (uint32_t)(sub % p.subs_per_stream);
-    c.r = (uint32_t)(s % twoH);
-    c.layer = (uint32_t)(s / twoH);
+    c.tt = sub - s * p.subs_per_stream;
+    c.r = s % twoH;
+    c.layer = s / twoH;
     return c;
 }
 
-// Moves on by one warp step.  Returns true when that left the stream: the caller then recomputes
-// its stream-level pointers instead of incrementing them by p.step_t sub-tiles.
-__device__ __forceinline__ bool step(Pos &c, const PathParams &p)
+// Moves on to the next sub-tile.  Returns true when that left the stream.
+__device__ __forceinline__ bool next_sub_tile(Pos &c, const PathParams &p)
 {
-    c.tt += p.step_t;
-    if (p.step_r == 0u && p.step_l == 0u && c.tt < p.subs_per_stream) return false;
-    const uint32_t twoH = 2u * (uint32_t)p.n_kv_heads;
-    c.r += p.step_r;
-    c.layer += p.step_l;
-    while (c.tt >= p.subs_per_stream) {
-        c.tt -= p.subs_per_stream;
-        c.r += 1u;
-    }
-    while (c.r >= twoH) {
-        c.r -= twoH;
-        c.layer += 1u;
+    if (++c.tt < p.subs_per_stream) return false;
+    c.tt = 0;
+    if (++c.r == 2u * (uint32_t)p.n_kv_heads) {
+        c.r = 0;
+        ++c.layer;
     }
     return true;
 }
@@ -92,39 +84,108 @@ __device__ __forceinline__ int rows_at(const Pos &c, const PathParams &p)
     return c.tt + 1u == p.subs_per_stream ? (int)p.last_rows : R;
 }
 
+// Work distribution.  The sub-tiles of a launch are handed out in chunks of kChunk consecutive
+// ones.  Every warp of the grid starts with the chunk of its own index; further chunks come from
+// a counter in device memory -- first come, first served, which evens out SMs that run at
+// different speeds -- or, when the caller gave no scratch block, at a fixed stride.
+// A warp walks its sequence of sub-tiles with two cursors, one ahead of the other: the leading
+// one takes the chunks and leaves their indices in a small ring in shared memory, the trailing
+// one reads them there.  The index n_chunks marks the end of the sequence.
+constexpr uint32_t kChunk = 8;
+
+struct WorkSource {
+    uint32_t *ring;       // shared memory, 4 entries: chunk indices in the order the warp took them
+    uint32_t *counter;    // device memory, zero at launch; or null
+    uint32_t n_chunks, n_warps;
+    uint32_t last;        // last chunk taken
+};
+
+struct Cursor {
+    Pos c;
+    uint32_t left;   // sub-tiles of the current chunk after the current one
+    uint32_t nth;    // index of the current chunk in the warp's sequence
+    bool done;       // the sequence has ended; c is meaningless
+};
+
+__device__ __forceinline__ void enter_chunk(Cursor &cu, uint32_t chunk, const PathParams &p)
+{
+    const uint32_t first = chunk * kChunk;
+    cu.c = position_of(p, first);
+    cu.left = min(kChunk, (uint32_t)p.n_subs - first) - 1u;
+}
+
+// Moves a cursor to the warp's next sub-tile.  Returns false when that is simply the following
+// sub-tile of the same stream (pointers advance by a constant), true otherwise (new stream or new
+// chunk: recompute pointers, or the end: cu.done).  All lanes call it together.
+template <bool LEAD>
+__device__ __forceinline__ bool advance(Cursor &cu, WorkSource &ws, const PathParams &p, int lane)
+{
+    if (cu.left) {
+        --cu.left;
+        return next_sub_tile(cu.c, p);
+    }
+    ++cu.nth;
+    uint32_t chunk;
+    if (LEAD) {
+        if (ws.last >= ws.n_chunks) {
+            chunk = ws.n_chunks;
+        } else if (ws.counter) {
+            uint32_t v = 0;
+            if (lane == 0) v = atomicAdd(ws.counter, 1u);
+            v = __shfl_sync(0xffffffffu, v, 0);
+            chunk = v < ws.n_chunks ? min(ws.n_warps + v, ws.n_chunks) : ws.n_chunks;
+        } else {
+            chunk = ws.n_chunks - ws.last > ws.n_warps ? ws.last + ws.n_warps : ws.n_chunks;
+        }
+        ws.last = chunk;
+        if (lane == 0) ws.ring[cu.nth & 3u] = chunk;
+        __syncwarp();
+    } else {
+        chunk = ws.ring[cu.nth & 3u];
+    }
+    if (chunk >= ws.n_chunks) cu.done = true;
+    else enter_chunk(cu, chunk, p);
+    return true;
+}
+
 // Walks the caller's cache block (source of create, destination of inject): `row` points at the
 // first row of the current sub-tile.
-template <int R, int WARPS>
+template <int R, bool LEAD>
 struct CacheWalk {
-    Pos c;
+    Cursor cu;
     __half *row;
 
     __device__ __forceinline__ void locate(const PathParams &p, const LayerPtrs &ptrs, int64_t first_row)
     {
+        const Pos &c = cu.c;
         const uint32_t H = (uint32_t)p.n_kv_heads;
         const bool is_v = c.r >= H;
         const uint32_t head = is_v ? c.r - H : c.r;
         row = reinterpret_cast<__half *>(is_v ? ptrs.v[c.layer] : ptrs.k[c.layer]) + (int64_t)head * p.head_stride +
               (first_row + (int64_t)c.tt * R) * p.token_stride;
     }
-    __device__ __forceinline__ void next(const PathParams &p, const LayerPtrs &ptrs, int64_t first_row)
+    __device__ __forceinline__ void next(WorkSource &ws, const PathParams &p, const LayerPtrs &ptrs, int64_t first_row, int lane)
     {
-        if (step(c, p)) locate(p, ptrs, first_row);
-        else row += (int64_t)(p.step_t * R) * p.token_stride;
+        if (advance<LEAD>(cu, ws, p, lane)) {
+            if (!cu.done) locate(p, ptrs, first_row);
+        } else {
+            row += (int64_t)R * p.token_stride;
+        }
     }
 };
 
 // Walks the card's tables: `offs` / `bits` point at the entries of the current sub-tile's first
 // token, `base` is the byte offset of its stream inside the card.
-template <int R, int WARPS>
+template <int R, bool LEAD>
 struct TableWalk {
-    Pos c;
+    Cursor cu;
     const uint32_t *offs;
     const uint8_t *bits;
     uint64_t base;
 
     __device__ __forceinline__ void locate(const PathParams &p, const Sections &sec, int bits_mode, uint64_t stream_bytes)
     {
+        const Pos &c = cu.c;
         const uint64_t T = (uint64_t)p.n_tokens;
         const uint32_t H = (uint32_t)p.n_kv_heads;
         const uint32_t head = c.r >= H ? c.r - H : c.r;
@@ -137,13 +198,14 @@ struct TableWalk {
         if (bits_mode == 0) base = sec.payload_off + stream * stream_bytes;
         else base = sec.payload_off + __ldg(reinterpret_cast<const uint64_t *>(p.card + sec.sbase_off) + stream);
     }
-    __device__ __forceinline__ void next(const PathParams &p, const Sections &sec, int bits_mode, uint64_t stream_bytes)
+    __device__ __forceinline__ void next(WorkSource &ws, const PathParams &p, const Sections &sec, int bits_mode,
+                                         uint64_t stream_bytes, int lane)
     {
-        if (step(c, p)) {
-            locate(p, sec, bits_mode, stream_bytes);
+        if (advance<LEAD>(cu, ws, p, lane)) {
+            if (!cu.done) locate(p, sec, bits_mode, stream_bytes);
         } else {
-            offs += p.step_t * R;
-            bits += p.step_t * R;
+            offs += R;
+            bits += R;
         }
     }
 };
@@ -156,33 +218,33 @@ struct Tables {
     int rows;
 };
 
-template <int R, int WARPS>
-__device__ __forceinline__ void fetch_tables(Tables &t, const TableWalk<R, WARPS> &w, const PathParams &p, int lane)
+template <int R, bool LEAD>
+__device__ __forceinline__ void fetch_tables(Tables &t, const TableWalk<R, LEAD> &w, const PathParams &p, int lane)
 {
-    t.rows = rows_at<R>(w.c, p);
+    t.rows = rows_at<R>(w.cu.c, p);
     t.base = w.base;
     t.off = lane <= t.rows ? __ldg(w.offs + lane) : 0u;
     t.bits = lane < t.rows ? (uint32_t)__ldg(w.bits + lane) : 0u;
 }
 
-// Sub-tiles of this warp.  The sub-tiles are dealt out in bundles of WARPS consecutive ones (warp w
-// of a CTA takes the w-th of each bundle).  With p.interleaved, CTA b takes bundles b, b + grid,
-// ... so that at any moment the grid works on one contiguous window of the cache; otherwise CTA b
-// owns a contiguous range of bundles.  Returns how many sub-tiles the warp has and the first one.
+// Sets up the warp's work source and the starting state of its two cursors.  Returns false when
+// there is no chunk for this warp.
 template <int WARPS>
-__device__ __forceinline__ uint32_t my_share(const PathParams &p, int warp, uint64_t &first)
+__device__ __forceinline__ bool start_work(WorkSource &ws, Cursor &cu, uint32_t *ring, const PathParams &p, int warp, int lane)
 {
-    const uint32_t b = blockIdx.x;
-    const uint32_t n = p.bundles_per_cta + (b < p.bundles_rem ? 1u : 0u);  // bundles of this CTA
-    if (n == 0u) {
-        first = 0;
-        return 0u;
-    }
-    const uint64_t first_bundle = p.interleaved ? b : (uint64_t)b * p.bundles_per_cta + min(b, p.bundles_rem);
-    const uint64_t last_bundle = p.interleaved ? b + (uint64_t)(n - 1u) * gridDim.x : first_bundle + (n - 1u);
-    first = first_bundle * WARPS + (uint32_t)warp;
-    // only the very last bundle of the launch can be short
-    return last_bundle * WARPS + (uint32_t)warp < p.n_subs ? n : n - 1u;
+    const uint32_t me = blockIdx.x * WARPS + (uint32_t)warp;
+    ws.ring = ring;
+    ws.counter = p.work_counter;
+    ws.n_chunks = p.n_chunks;
+    ws.n_warps = gridDim.x * WARPS;
+    ws.last = me;
+    if (me >= p.n_chunks) return false;
+    if (lane == 0) ring[0] = me;
+    __syncwarp();
+    cu.nth = 0;
+    cu.done = false;
+    enter_chunk(cu, me, p);
+    return true;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -193,6 +255,8 @@ struct CreateWarpSmem {
     using C = WarpCfg<D>;
     alignas(128) uint8_t in[NS][C::STAGE_BYTES];
     alignas(8) uint64_t full[NS];
+    uint32_t ring[4];
+    static_assert(NS >= 2 && NS <= (int)kChunk, "pipeline depth");
 };
 
 // One group: lane l owns group l % G of row l / G of the R rows at `rows_in`, i.e. the 64 input
@@ -289,9 +353,13 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_
     const uint64_t stream_bytes = hdr->stream_bytes;
     const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
 
-    uint64_t first;
-    const uint32_t n_mine = my_share<C::WARPS>(p, warp, first);
-    if (n_mine == 0) return;
+    WorkSource ws;
+    CacheWalk<C::ROWS, true> ahead;  // runs NS sub-tiles ahead and starts the copies
+    if (!start_work<C::WARPS>(ws, ahead.cu, sm.ring, p, warp, lane)) return;
+    ahead.locate(p, ptrs, 0);
+    TableWalk<C::ROWS, false> tw;    // runs one sub-tile ahead and reads the tables
+    tw.cu = ahead.cu;
+    tw.locate(p, sec, p.bits_mode, stream_bytes);
 
     if (lane == 0) {
         for (int s = 0; s < NS; ++s) mbar_init(&sm.full[s], 1);
@@ -299,28 +367,22 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_
     }
     __syncwarp();
 
-    CacheWalk<C::ROWS, C::WARPS> ahead;  // runs NS sub-tiles ahead and starts the copies
-    ahead.c = first_pos(p, first);
-    ahead.locate(p, ptrs, 0);
-    TableWalk<C::ROWS, C::WARPS> tw;
-    tw.c = ahead.c;
-    tw.locate(p, sec, p.bits_mode, stream_bytes);
-
-    uint32_t issued = 0;
-    for (; issued < (uint32_t)NS && issued < n_mine; ++issued) {
-        create_issue<D, NS>(sm, (int)issued, ahead.row, rows_at<C::ROWS>(ahead.c, p), p, lane);
-        if (issued + 1 < n_mine) ahead.next(p, ptrs, 0);
+    uint32_t issued = 0, consumed = 0;
+    while (issued < (uint32_t)NS && !ahead.cu.done) {
+        create_issue<D, NS>(sm, (int)issued, ahead.row, rows_at<C::ROWS>(ahead.cu.c, p), p, lane);
+        ++issued;
+        ahead.next(ws, p, ptrs, 0, lane);
     }
     Tables nxt;
     fetch_tables(nxt, tw, p, lane);
 
     int stage = 0;
-    uint32_t parity = 0, k = 0;
+    uint32_t parity = 0;
     bool ok = true;
-    for (; k < n_mine; ++k) {
+    for (; consumed < issued; ++consumed) {
         const Tables cur = nxt;
-        if (k + 1 < n_mine) {
-            tw.next(p, sec, p.bits_mode, stream_bytes);
+        if (consumed + 1 < issued) {  // the next sub-tile, if there is one, is on its way already (NS >= 2)
+            tw.next(ws, p, sec, p.bits_mode, stream_bytes, lane);
             fetch_tables(nxt, tw, p, lane);
         }
         const int b0 = (int)__shfl_sync(0xffffffffu, cur.bits, 0);
@@ -341,9 +403,10 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_
             encode_rows<D, 0>(in, stream, cur, lane);
         }
         __syncwarp();  // every lane has read the stage: it can be re-armed
-        if (issued < n_mine) {
-            create_issue<D, NS>(sm, stage, ahead.row, rows_at<C::ROWS>(ahead.c, p), p, lane);
-            if (++issued < n_mine) ahead.next(p, ptrs, 0);
+        if (!ahead.cu.done) {
+            create_issue<D, NS>(sm, stage, ahead.row, rows_at<C::ROWS>(ahead.cu.c, p), p, lane);
+            ++issued;
+            ahead.next(ws, p, ptrs, 0, lane);
         }
         if (++stage == NS) {
             stage = 0;
@@ -354,7 +417,7 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_
         // A wait was abandoned: record it, and let the copies still in flight land (bounded)
         // before the shared memory is given back.
         if (lane == 0) atomicMax(&hdr->status, (uint32_t)QKVS_ERR_TIMEOUT);
-        for (uint32_t j = k + 1; j < issued; ++j) {
+        for (uint32_t j = consumed + 1; j < issued; ++j) {
             if (++stage == NS) {
                 stage = 0;
                 parity ^= 1u;
@@ -375,6 +438,8 @@ struct InjectWarpSmem {
     alignas(8) uint64_t full[NS];
     uint32_t uniform_bits[NS];         // bit-width shared by all ROWS rows, else 0
     int32_t rows[NS];                  // 0 when the sub-tile's table entries did not check out
+    uint32_t ring[4];
+    static_assert(NS >= 2 && NS < (int)kChunk, "pipeline depth");
 };
 
 template <int D, int B>
@@ -512,35 +577,33 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) inject_
     const uint64_t stream_bytes = s_stream_bytes, total_bytes = s_total_bytes;
     const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, mode);
 
-    uint64_t first;
-    const uint32_t n_mine = my_share<C::WARPS>(p, warp, first);
-    if (n_mine == 0) return;
-
     // The copy of a span can only start once its table entries are known, so the table reads run
     // one step ahead of the copies, which run NS steps ahead of the arithmetic.
-    TableWalk<C::ROWS, C::WARPS> tw;
-    tw.c = first_pos(p, first);
+    WorkSource ws;
+    TableWalk<C::ROWS, true> tw;
+    if (!start_work<C::WARPS>(ws, tw.cu, sm.ring, p, warp, lane)) return;
     tw.locate(p, sec, mode, stream_bytes);
-    CacheWalk<C::ROWS, C::WARPS> cons;
-    cons.c = tw.c;
+    CacheWalk<C::ROWS, false> cons;
+    cons.cu = tw.cu;
     cons.locate(p, ptrs, p.dst_token_offset);
 
     Tables nxt;
     fetch_tables(nxt, tw, p, lane);
-    uint32_t issued = 0;
-    for (; issued < (uint32_t)NS && issued < n_mine; ++issued) {
+    bool more = true;  // nxt holds a sub-tile that has not been issued yet
+    uint32_t issued = 0, consumed = 0;
+    while (issued < (uint32_t)NS && more) {
         const Tables cur = nxt;
-        if (issued + 1 < n_mine) {
-            tw.next(p, sec, mode, stream_bytes);
-            fetch_tables(nxt, tw, p, lane);
-        }
+        tw.next(ws, p, sec, mode, stream_bytes, lane);
+        more = !tw.cu.done;
+        if (more) fetch_tables(nxt, tw, p, lane);
         inject_issue<D, NS>(sm, (int)issued, cur, p, sec, total_bytes, lane);
+        ++issued;
     }
 
     int stage = 0;
-    uint32_t parity = 0, k = 0;
+    uint32_t parity = 0;
     bool ok = true;
-    for (; k < n_mine; ++k) {
+    for (; consumed < issued; ++consumed) {
         ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[stage], parity));
         if (!ok) break;
         const int rows = sm.rows[stage];
@@ -558,16 +621,15 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) inject_
             inject_rows<D, NS, 0, false>(sm, stage, lane, rows, dst0, p.token_stride);
         }
         __syncwarp();  // every lane has read the stage: it can be re-armed
-        if (k + 1 < n_mine) cons.next(p, ptrs, p.dst_token_offset);
-        if (issued < n_mine) {
+        if (more) {
             const Tables cur = nxt;
-            if (issued + 1 < n_mine) {
-                tw.next(p, sec, mode, stream_bytes);
-                fetch_tables(nxt, tw, p, lane);
-            }
+            tw.next(ws, p, sec, mode, stream_bytes, lane);
+            more = !tw.cu.done;
+            if (more) fetch_tables(nxt, tw, p, lane);
             inject_issue<D, NS>(sm, stage, cur, p, sec, total_bytes, lane);
             ++issued;
         }
+        if (consumed + 1 < issued) cons.next(ws, p, ptrs, p.dst_token_offset, lane);
         if (++stage == NS) {
             stage = 0;
             parity ^= 1u;
@@ -575,7 +637,7 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) inject_
     }
     if (!ok) {
         if (lane == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_TIMEOUT);
-        for (uint32_t j = k + 1; j < issued; ++j) {
+        for (uint32_t j = consumed + 1; j < issued; ++j) {
             if (++stage == NS) {
                 stage = 0;
                 parity ^= 1u;

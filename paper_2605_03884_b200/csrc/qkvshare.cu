@@ -32,6 +32,7 @@ struct ScanParams {
     int32_t n_layers, n_kv_heads, head_dim, n_tokens, bits_mode;
     uint64_t model_id, sender_id;
     int64_t position_offset;
+    uint32_t *workspace;  // the call's scratch block, cleared here for the kernels that follow; or null
 };
 
 // Exclusive scan of one value per thread over the block; returns the block total through
@@ -105,6 +106,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
     const int d = p.head_dim;
 
     if (threadIdx.x == 0) s_bad = 0;
+    if (p.workspace && seg == 0 && threadIdx.x < QKVS_WORKSPACE_BYTES / 4) p.workspace[threadIdx.x] = 0u;
     uint32_t carry = 0;
     uint64_t sum_bits = 0;
     bool bad = false;
@@ -308,6 +310,14 @@ static qkvs_status_t check_strides(const qkvs_layout_t *l, int64_t first_row)
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Work counter of the launch with the given index inside a call's scratch block (word 0 is the
+// status word); null when there is no block or the call makes more launches than it has counters.
+static uint32_t *work_counter(void *workspace_dev, int launch)
+{
+    if (!workspace_dev || launch + 1 >= QKVS_WORKSPACE_BYTES / 4) return nullptr;
+    return static_cast<uint32_t *>(workspace_dev) + 1 + launch;
+}
+
 #ifndef QKVS_STAGES_CREATE
 #define QKVS_STAGES_CREATE 3
 #endif
@@ -338,7 +348,7 @@ static cudaError_t persistent_grid(Kernel kernel, int threads, size_t smem, int6
     return cudaSuccess;
 }
 
-// Splits the sub-tiles of `streams` streams over a persistent grid and launches `kernel`.
+// Splits `streams` streams into sub-tiles and chunks and launches `kernel` on a persistent grid.
 template <int D, typename Kernel>
 static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp, const LayerPtrs &ptrs, int64_t streams,
                                cudaStream_t st)
@@ -346,22 +356,15 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
     using C = WarpCfg<D>;
     PathParams p = pp;
     p.subs_per_stream = (uint32_t)(((int64_t)p.n_tokens + C::ROWS - 1) / C::ROWS);
-    p.n_subs = (uint64_t)streams * p.subs_per_stream;
-    if (p.n_subs == 0) return cudaSuccess;
-    unsigned grid = 0;
-    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, (int64_t)((p.n_subs + C::WARPS - 1) / C::WARPS), &grid);
-    if (e != cudaSuccess) return e;
+    const uint64_t n_subs = (uint64_t)streams * p.subs_per_stream;
+    if (n_subs == 0) return cudaSuccess;
+    if (n_subs > 0x7fffffffull) return cudaErrorInvalidValue;
+    p.n_subs = (uint32_t)n_subs;
+    p.n_chunks = (p.n_subs + kChunk - 1) / kChunk;
     p.last_rows = (uint32_t)(p.n_tokens - (int64_t)(p.subs_per_stream - 1) * C::ROWS);
-    const uint64_t n_bundles = (p.n_subs + C::WARPS - 1) / C::WARPS;
-    p.bundles_per_cta = (uint32_t)(n_bundles / grid);
-    p.bundles_rem = (uint32_t)(n_bundles % grid);
-    p.interleaved = QKVS_INTERLEAVED;
-    const uint64_t step = (uint64_t)C::WARPS * (p.interleaved ? grid : 1u);  // sub-tiles per warp step
-    const uint64_t step_s = step / p.subs_per_stream;                         // whole streams per step
-    const uint32_t twoH = 2u * (uint32_t)p.n_kv_heads;
-    p.step_t = (uint32_t)(step % p.subs_per_stream);
-    p.step_r = (uint32_t)(step_s % twoH);
-    p.step_l = (uint32_t)(step_s / twoH);
+    unsigned grid = 0;
+    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, (int64_t)((p.n_chunks + C::WARPS - 1) / C::WARPS), &grid);
+    if (e != cudaSuccess) return e;
     kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs);
     return cudaGetLastError();
 }
@@ -426,14 +429,14 @@ qkvs_status_t qkvs_card_size(const qkvs_layout_t *layout, const uint8_t *bits_ho
 
 qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K_layers, const void *const *V_layers,
                                const uint8_t *bits_dev, const qkvs_card_meta_t *meta, void *card_dev,
-                               size_t card_capacity, void *stream)
+                               size_t card_capacity, void *workspace_dev, void *stream)
 {
     qkvs_status_t st = check_shape(layout);
     if (st != QKVS_OK) return st;
     if (!K_layers || !V_layers || !card_dev || (!bits_dev && layout->n_tokens > 0)) return QKVS_ERR_INVALID_ARG;
     st = check_strides(layout, 0);
     if (st != QKVS_OK) return st;
-    if (!aligned16(card_dev)) return QKVS_ERR_INVALID_ARG;
+    if (!aligned16(card_dev) || !aligned16(workspace_dev)) return QKVS_ERR_INVALID_ARG;
     for (int l = 0; l < layout->n_layers; ++l)
         if (!K_layers[l] || !V_layers[l] || !aligned16(K_layers[l]) || !aligned16(V_layers[l])) return QKVS_ERR_INVALID_ARG;
     const Sections sec = card_sections(layout->n_layers, layout->n_kv_heads, layout->n_tokens, layout->bits_mode);
@@ -452,6 +455,7 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
     sp.model_id = meta ? meta->model_id : 0;
     sp.sender_id = meta ? meta->sender_id : 0;
     sp.position_offset = meta ? meta->position_offset : 0;
+    sp.workspace = static_cast<uint32_t *>(workspace_dev);
     const int nseg = layout->bits_mode == 0 ? 1 : layout->n_layers * layout->n_kv_heads;
     if (layout->bits_mode == 1 && cudaMemsetAsync(card_dev, 0, kHeaderBytes, cs) != cudaSuccess) return QKVS_ERR_CUDA;
     scan_offsets_kernel<<<nseg, kScanThreads, 0, cs>>>(sp);
@@ -482,6 +486,7 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
         }
         p.layer_begin = l0;
         p.layer_count = n;
+        p.work_counter = work_counter(workspace_dev, l0 / kMaxLayersPerLaunch);
         const int64_t streams = 2ll * n * layout->n_kv_heads;
         cudaError_t e;
         switch (layout->head_dim) {
@@ -497,20 +502,20 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
 
 qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qkvs_layout_t *dst,
                                void *const *K_layers_out, void *const *V_layers_out, int64_t dst_token_offset,
-                               int32_t *status_dev, void *stream)
+                               void *workspace_dev, void *stream)
 {
     qkvs_status_t st = check_shape(dst);
     if (st != QKVS_OK) return st;
     if (!card_dev || !K_layers_out || !V_layers_out) return QKVS_ERR_INVALID_ARG;
     st = check_strides(dst, dst_token_offset);
     if (st != QKVS_OK) return st;
-    if (!aligned16(card_dev)) return QKVS_ERR_INVALID_ARG;
+    if (!aligned16(card_dev) || !aligned16(workspace_dev)) return QKVS_ERR_INVALID_ARG;
     if (card_bytes < (size_t)kHeaderBytes) return QKVS_ERR_BAD_CARD;
     for (int l = 0; l < dst->n_layers; ++l)
         if (!K_layers_out[l] || !V_layers_out[l] || !aligned16(K_layers_out[l]) || !aligned16(V_layers_out[l]))
             return QKVS_ERR_INVALID_ARG;
     cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
-    if (status_dev && cudaMemsetAsync(status_dev, 0, sizeof(int32_t), cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    if (workspace_dev && cudaMemsetAsync(workspace_dev, 0, QKVS_WORKSPACE_BYTES, cs) != cudaSuccess) return QKVS_ERR_CUDA;
 
     PathParams p;
     memset(&p, 0, sizeof(p));
@@ -524,7 +529,7 @@ qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qk
     p.head_stride = dst->head_stride;
     p.token_stride = dst->token_stride;
     p.dst_token_offset = dst_token_offset;
-    p.status_dev = status_dev;
+    p.status_dev = static_cast<int32_t *>(workspace_dev);  // word 0 of the scratch block
     for (int l0 = 0; l0 < dst->n_layers; l0 += kMaxLayersPerLaunch) {
         const int n = std::min(kMaxLayersPerLaunch, dst->n_layers - l0);
         LayerPtrs ptrs;
@@ -535,6 +540,7 @@ qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qk
         }
         p.layer_begin = l0;
         p.layer_count = n;
+        p.work_counter = work_counter(workspace_dev, l0 / kMaxLayersPerLaunch);
         const int64_t streams = 2ll * n * dst->n_kv_heads;
         cudaError_t e;
         switch (dst->head_dim) {

@@ -40,29 +40,41 @@ def to_cuda(arrs):
     return [torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in arrs]
 
 
-def gpu_create(q, lay, Ks, Vs, bits, meta=None, capacity=None, Kd=None, Vd=None):
+def dirty_workspace(q):
+    """A scratch block filled with junk: the calls must not depend on what it holds on entry."""
+    import torch
+    ws = q.new_workspace()
+    ws.fill_(0x5A5A5A5A)
+    return ws
+
+
+def gpu_create(q, lay, Ks, Vs, bits, meta=None, capacity=None, Kd=None, Vd=None, scratch=True):
     """Run qkvs_card_create into a poisoned buffer; returns (status_from_header, card_bytes_np,
-    whole_buffer_np, capacity).  The buffer has PAD canary bytes behind `capacity`."""
+    whole_buffer_np, capacity).  The buffer has PAD canary bytes behind `capacity`.  `scratch`
+    False passes no scratch block (work is then split in advance)."""
     import torch
     Kd = to_cuda(Ks) if Kd is None else Kd
     Vd = to_cuda(Vs) if Vd is None else Vd
     bits_d = torch.from_numpy(np.ascontiguousarray(bits, dtype=np.uint8)).cuda()
     cap = q.card_size(lay, None) if capacity is None else capacity
     buf = torch.full((cap + PAD,), POISON, dtype=torch.uint8, device="cuda")
-    q.card_create(lay, Kd, Vd, bits_d, buf, meta=meta, card_capacity=cap)
+    q.card_create(lay, Kd, Vd, bits_d, buf, meta=meta, card_capacity=cap,
+                  workspace=dirty_workspace(q) if scratch else None)
     st, hdr = q.card_info(buf)
     torch.cuda.synchronize()
     whole = buf.cpu().numpy()
     return st, hdr, whole, cap
 
 
-def gpu_inject(q, card_np, dst_lay, Ko_np, Vo_np, dst_token_offset=0, card_bytes=None):
-    """Upload a card and destination buffers, inject, return (device status, K_out, V_out)."""
+def gpu_inject(q, card_np, dst_lay, Ko_np, Vo_np, dst_token_offset=0, card_bytes=None, scratch=True):
+    """Upload a card and destination buffers, inject, return (device status, K_out, V_out).
+    Without a scratch block there is no status word; None is returned in its place."""
     import torch
     card_d = torch.from_numpy(np.ascontiguousarray(card_np)).cuda()
     Kd, Vd = to_cuda(Ko_np), to_cuda(Vo_np)
-    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    ws = dirty_workspace(q) if scratch else None
     q.card_inject(card_d, dst_lay, Kd, Vd, dst_token_offset=dst_token_offset,
-                  card_bytes=card_np.size if card_bytes is None else card_bytes, status_dev=status)
+                  card_bytes=card_np.size if card_bytes is None else card_bytes, workspace=ws)
     torch.cuda.synchronize()
-    return int(status.item()), [k.cpu().numpy() for k in Kd], [v.cpu().numpy() for v in Vd]
+    status = int(ws[0].item()) if scratch else None
+    return status, [k.cpu().numpy() for k in Kd], [v.cpu().numpy() for v in Vd]

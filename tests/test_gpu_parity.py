@@ -32,13 +32,13 @@ def _glay(L, H, d, T, mode=0, **strides):
     return q.make_layout(L, H, d, T, bits_mode=mode, **strides)
 
 
-def _check_card(Ks, Vs, bits, L, H, d, T, mode=0, strides=None, meta=(0, 0, 0)):
+def _check_card(Ks, Vs, bits, L, H, d, T, mode=0, strides=None, meta=(0, 0, 0), scratch=True):
     strides = strides or {}
     st_o, want = oracle.card_create(_olay(L, H, d, T, mode, **strides), Ks, Vs, bits,
                                     model_id=meta[0], sender_id=meta[1], position_offset=meta[2])
     assert st_o == oracle.OK
     st, hdr, whole, cap = gpu_create(q, _glay(L, H, d, T, mode, **strides), Ks, Vs, bits,
-                                     meta=q.CardMeta(*meta))
+                                     meta=q.CardMeta(*meta), scratch=scratch)
     assert st == q.binding.OK
     assert hdr.total_bytes == want.size
     got = whole[:want.size]
@@ -50,7 +50,7 @@ def _check_card(Ks, Vs, bits, L, H, d, T, mode=0, strides=None, meta=(0, 0, 0)):
     return want
 
 
-def _check_inject(card, L, H, d, T, dst_strides=None, t_cap=None, dst_token_offset=0):
+def _check_inject(card, L, H, d, T, dst_strides=None, t_cap=None, dst_token_offset=0, scratch=True):
     dst_strides = dst_strides or {}
     t_cap = T if t_cap is None else t_cap
     ts = dst_strides.get("token_stride", d)
@@ -59,8 +59,8 @@ def _check_inject(card, L, H, d, T, dst_strides=None, t_cap=None, dst_token_offs
     Kw, Vw = [a.copy() for a in Ko], [a.copy() for a in Vo]
     lay_kw = dict(head_stride=t_cap * ts, token_stride=ts)
     assert oracle.card_inject(card, _olay(L, H, d, T, **lay_kw), Kw, Vw, dst_token_offset) == oracle.OK
-    st, Kg, Vg = gpu_inject(q, card, _glay(L, H, d, T, **lay_kw), Ko, Vo, dst_token_offset)
-    assert st == 0
+    st, Kg, Vg = gpu_inject(q, card, _glay(L, H, d, T, **lay_kw), Ko, Vo, dst_token_offset, scratch=scratch)
+    assert st == (0 if scratch else None)
     worst = 0
     for l in range(L):
         for g, w in ((Kg[l], Kw[l]), (Vg[l], Vw[l])):
@@ -87,6 +87,28 @@ def test_mixed_bits_ragged_tiles(d, T):
     bits = wl.iid_bits(T, (0.3, 0.3, 0.2, 0.2), seed=d * 7 + T)
     card = _check_card(Ks, Vs, bits, L, H, d, T, meta=(0xABCDEF0123456789, 77, -12))
     assert _check_inject(card, L, H, d, T) == 0
+
+
+@pytest.mark.parametrize("d,T", [(64, 700), (128, 2100), (192, 333), (256, 517)])
+def test_without_scratch_block(d, T):
+    """No scratch block: the work is split in advance instead of drawn from a counter; the
+    results are the same bytes."""
+    L, H = 3, 4
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=77 + d)
+    bits = wl.iid_bits(T, (0.35, 0.35, 0.2, 0.1), seed=d + T)
+    card = _check_card(Ks, Vs, bits, L, H, d, T, scratch=False)
+    assert _check_inject(card, L, H, d, T, scratch=False) == 0
+
+
+def test_many_chunks_per_warp():
+    """More chunks than the grid has warps, so that every warp draws several from the counter
+    (and, without a scratch block, strides through several)."""
+    L, H, d, T = 4, 8, 128, 9000
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=4242)
+    bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), seed=99)
+    for scratch in (True, False):
+        card = _check_card(Ks, Vs, bits, L, H, d, T, scratch=scratch)
+        assert _check_inject(card, L, H, d, T, scratch=scratch) == 0
 
 
 @pytest.mark.parametrize("b", [2, 4, 8, 16])
@@ -287,7 +309,8 @@ def _full_parity(w, Ks, Vs, bits):
     size = q.card_size(_glay(L, H, d, T), bits)
     assert size == want.size
     buf = torch.full((size + PAD,), POISON, dtype=torch.uint8, device="cuda")
-    q.card_create(_glay(L, H, d, T), Kd, Vd, bits_d, buf, card_capacity=size)
+    ws = q.new_workspace()
+    q.card_create(_glay(L, H, d, T), Kd, Vd, bits_d, buf, card_capacity=size, workspace=ws)
     st, hdr = q.card_info(buf)
     assert st == 0 and hdr.total_bytes == size
     got = buf.cpu().numpy()
@@ -296,9 +319,8 @@ def _full_parity(w, Ks, Vs, bits):
     # inject on the GPU, oracle inject on the CPU
     Ko = [torch.zeros_like(k) for k in Kd]
     Vo = [torch.zeros_like(v) for v in Vd]
-    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
-    q.card_inject(buf, _glay(L, H, d, T), Ko, Vo, card_bytes=size, status_dev=status)
-    assert int(status.item()) == 0
+    q.card_inject(buf, _glay(L, H, d, T), Ko, Vo, card_bytes=size, workspace=ws)
+    assert int(ws[0].item()) == 0
     Kw = [np.zeros_like(k) for k in Ks]
     Vw = [np.zeros_like(v) for v in Vs]
     assert oracle.card_inject(want, _olay(L, H, d, T), Kw, Vw) == oracle.OK

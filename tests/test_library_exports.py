@@ -72,18 +72,24 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     lay = q.make_layout(1, 1, 64, 4)
     null = C.c_void_p(0)
     arr = (C.c_void_p * 1)(0)
-    st = lib.qkvs_card_create(C.byref(lay), arr, arr, null, None, null, 0, None)
+    st = lib.qkvs_card_create(C.byref(lay), arr, arr, null, None, null, 0, None, None)
     assert st == q.binding.ERR_INVALID_ARG
     bad = q.make_layout(1, 1, 64, 4, token_stride=60)
     ptrs = (C.c_void_p * 1)(256)
-    st = lib.qkvs_card_create(C.byref(bad), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20, None)
+    st = lib.qkvs_card_create(C.byref(bad), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20, None, None)
     assert st == q.binding.ERR_INVALID_ARG
     mis = (C.c_void_p * 1)(264)
-    st = lib.qkvs_card_create(C.byref(lay), mis, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20, None)
+    st = lib.qkvs_card_create(C.byref(lay), mis, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20, None, None)
     assert st == q.binding.ERR_INVALID_ARG
-    st = lib.qkvs_card_create(C.byref(lay), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 100, None)
+    st = lib.qkvs_card_create(C.byref(lay), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 100, None, None)
     assert st == q.binding.ERR_BUFFER_TOO_SMALL
     st = lib.qkvs_card_inject(C.c_void_p(256), 100, C.byref(lay), ptrs, ptrs, 0, None, None)
     assert st == q.binding.ERR_BAD_CARD
     st = lib.qkvs_card_inject(C.c_void_p(256), 4096, C.byref(lay), ptrs, ptrs, -1, None, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    # a scratch block has to be 16-byte aligned
+    st = lib.qkvs_card_inject(C.c_void_p(256), 4096, C.byref(lay), ptrs, ptrs, 0, C.c_void_p(264), None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = lib.qkvs_card_create(C.byref(lay), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20,
+                              C.c_void_p(264), None)
     assert st == q.binding.ERR_INVALID_ARG
