@@ -167,6 +167,33 @@ QKVS_API qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes,
                                void *const *K_layers_out, void *const *V_layers_out,
                                int64_t dst_token_offset, void *workspace_dev, void *stream);
 
+/* Injection for callers that cannot give the library a scratch block.  (The paper has no
+ * counterpart; this entry point exists for how the library gets embedded.)  Think of a receiver
+ * inside a serving engine that has handed every free byte of the GPU to its KV-cache pool and
+ * forbids its components to call cudaMalloc -- there is nothing left to allocate, and an
+ * allocation would stall the whole device in the middle of serving -- yet still wants the evenly
+ * loaded SMs that the work counters buy.  Same inputs, outputs and results as qkvs_card_inject;
+ * the work counters live in a small array inside the library's own device image (256 bytes,
+ * present on every GPU that has loaded the library, until the process exits).
+ *   status_dev   optional device int32 (4-byte aligned), cleared by the call; the kernel raises it
+ *                to BAD_CARD / TIMEOUT exactly like the status word of qkvs_card_inject
+ * Limits and rules:
+ *   - at most QKVS_NOALLOC_MAX_LAYERS layers per call (the array has 64 counters, one per 64
+ *     layers); more are refused with QKVS_ERR_UNSUPPORTED_SHAPE and nothing is launched;
+ *   - the call allocates and frees nothing, neither host-side nor on the device;
+ *   - all calls on a device share the one array, which still holds what the previous call left
+ *     there; each call clears it on its stream before its kernels run.  Two calls that may
+ *     execute at the same time on one GPU (different streams, or different host threads) would
+ *     disturb each other's counters: run them one after the other, or give the concurrent ones
+ *     qkvs_card_inject with blocks of their own;
+ *   - the first call on each device asks the runtime for the array's device address (with that
+ *     device current) and remembers it; make that first call outside of any stream capture. */
+#define QKVS_NOALLOC_MAX_LAYERS 4096
+QKVS_API qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t card_bytes,
+                                       const qkvs_layout_t *dst, void *const *K_layers_out,
+                                       void *const *V_layers_out, int64_t dst_token_offset,
+                                       int32_t *status_dev, void *stream);
+
 /* Synchronises `stream`, copies the card's header to the host and returns its recorded status
  * (or BAD_CARD if magic/version are wrong, or CUDA on a runtime error). */
 QKVS_API qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_card_header_t *out_host);

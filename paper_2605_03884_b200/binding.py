@@ -50,7 +50,7 @@ class CardHeader(C.Structure):
 assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
-           "qkvs_card_inject", "qkvs_card_info", "qkvs_selftest_division", "qkvs_status_string",
+           "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_card_info", "qkvs_selftest_division", "qkvs_status_string",
            "qkvs_version")
 
 _lib = None
@@ -78,6 +78,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_create.argtypes = [C.POINTER(Layout), vp, vp, vp, C.POINTER(CardMeta), vp, C.c_size_t, vp, vp]
     lib.qkvs_card_inject.restype = C.c_int
     lib.qkvs_card_inject.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
+    lib.qkvs_card_inject_noalloc.restype = C.c_int
+    lib.qkvs_card_inject_noalloc.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
     lib.qkvs_card_info.restype = C.c_int
     lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
     lib.qkvs_selftest_division.restype = C.c_int
@@ -202,6 +204,27 @@ def card_inject(card_dev, dst_layout: Layout, K_out: Sequence, V_out: Sequence,
                               _workspace_ptr(workspace), _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_card_inject")
+    return st
+
+
+NOALLOC_MAX_LAYERS = 4096
+
+
+def card_inject_noalloc(card_dev, dst_layout: Layout, K_out: Sequence, V_out: Sequence,
+                        dst_token_offset: int = 0, card_bytes: Optional[int] = None, status_dev=None,
+                        stream=None, check: bool = True) -> int:
+    """qkvs_card_inject_noalloc: injection whose work counters sit in the library's own device
+    memory, for callers that may not allocate a scratch block.  status_dev: optional CUDA int32
+    tensor of one element.  Calls on one GPU must not overlap in time."""
+    lib = load_library()
+    kp, vp = _ptr_array(K_out), _ptr_array(V_out)
+    nbytes = int(card_dev.numel() * card_dev.element_size()) if card_bytes is None else int(card_bytes)
+    st = lib.qkvs_card_inject_noalloc(int(card_dev.data_ptr()), nbytes, C.byref(dst_layout), kp, vp,
+                                      int(dst_token_offset),
+                                      int(status_dev.data_ptr()) if status_dev is not None else None,
+                                      _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_card_inject_noalloc")
     return st
 
 

@@ -13,6 +13,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "qkvs_common.cuh"
 #include "qkvs_pipeline.cuh"
@@ -383,6 +384,40 @@ static cudaError_t launch_inject(const PathParams &p, const LayerPtrs &ptrs, int
                           ptrs, streams, st);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Scratch of qkvs_card_inject_noalloc: the work counters live in the library's own device
+// memory instead of a block from the caller.  One word per kernel launch of a call (a launch
+// covers kMaxLayersPerLaunch layers).  Every GPU that loads the library holds these bytes until
+// the process exits.
+
+constexpr int kNoAllocCounters = 64;
+static_assert(kNoAllocCounters * kMaxLayersPerLaunch == QKVS_NOALLOC_MAX_LAYERS, "limit stated in the header");
+static __device__ __align__(256) uint32_t g_noalloc_counters[kNoAllocCounters];
+
+// Device address of g_noalloc_counters on the current device.  In host code the array's name only
+// stands for the symbol, it is not a device pointer; the runtime has to be asked for the address,
+// once per device, with that device current.
+static cudaError_t noalloc_counters(uint32_t **out)
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mutex;
+    static uint32_t *address[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mutex);
+    if (dev >= 0 && dev < kMaxDevices && address[dev]) {
+        *out = address[dev];
+        return cudaSuccess;
+    }
+    void *ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_noalloc_counters);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < kMaxDevices) address[dev] = static_cast<uint32_t *>(ptr);
+    *out = static_cast<uint32_t *>(ptr);
+    return cudaSuccess;
+}
+
 }  // namespace qkvs
 
 using namespace qkvs;
@@ -541,6 +576,65 @@ qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qk
         p.layer_begin = l0;
         p.layer_count = n;
         p.work_counter = work_counter(workspace_dev, l0 / kMaxLayersPerLaunch);
+        const int64_t streams = 2ll * n * dst->n_kv_heads;
+        cudaError_t e;
+        switch (dst->head_dim) {
+            case 64: e = launch_inject<64>(p, ptrs, streams, cs); break;
+            case 128: e = launch_inject<128>(p, ptrs, streams, cs); break;
+            case 192: e = launch_inject<192>(p, ptrs, streams, cs); break;
+            default: e = launch_inject<256>(p, ptrs, streams, cs); break;
+        }
+        if (e != cudaSuccess) return QKVS_ERR_CUDA;
+    }
+    return QKVS_OK;
+}
+
+qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t card_bytes, const qkvs_layout_t *dst,
+                                       void *const *K_layers_out, void *const *V_layers_out, int64_t dst_token_offset,
+                                       int32_t *status_dev, void *stream)
+{
+    qkvs_status_t st = check_shape(dst);
+    if (st != QKVS_OK) return st;
+    if (dst->n_layers > QKVS_NOALLOC_MAX_LAYERS) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (!card_dev || !K_layers_out || !V_layers_out) return QKVS_ERR_INVALID_ARG;
+    st = check_strides(dst, dst_token_offset);
+    if (st != QKVS_OK) return st;
+    if (!aligned16(card_dev) || (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QKVS_ERR_INVALID_ARG;
+    if (card_bytes < (size_t)kHeaderBytes) return QKVS_ERR_BAD_CARD;
+    for (int l = 0; l < dst->n_layers; ++l)
+        if (!K_layers_out[l] || !V_layers_out[l] || !aligned16(K_layers_out[l]) || !aligned16(V_layers_out[l]))
+            return QKVS_ERR_INVALID_ARG;
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    uint32_t *counters = nullptr;
+    if (noalloc_counters(&counters) != cudaSuccess) return QKVS_ERR_CUDA;
+    // the array keeps what the previous call left in it: the counters have to start at zero
+    if (cudaMemsetAsync(counters, 0, sizeof(uint32_t) * kNoAllocCounters, cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    if (status_dev && cudaMemsetAsync(status_dev, 0, sizeof(int32_t), cs) != cudaSuccess) return QKVS_ERR_CUDA;
+
+    PathParams p;
+    memset(&p, 0, sizeof(p));
+    p.card = const_cast<uint8_t *>(static_cast<const uint8_t *>(card_dev));
+    p.card_bytes = card_bytes;
+    p.n_layers = dst->n_layers;
+    p.n_kv_heads = dst->n_kv_heads;
+    p.head_dim = dst->head_dim;
+    p.n_tokens = dst->n_tokens;
+    p.bits_mode = 0;  // taken from the card on the device
+    p.head_stride = dst->head_stride;
+    p.token_stride = dst->token_stride;
+    p.dst_token_offset = dst_token_offset;
+    p.status_dev = status_dev;
+    for (int l0 = 0; l0 < dst->n_layers; l0 += kMaxLayersPerLaunch) {
+        const int n = std::min(kMaxLayersPerLaunch, dst->n_layers - l0);
+        LayerPtrs ptrs;
+        memset(&ptrs, 0, sizeof(ptrs));
+        for (int i = 0; i < n; ++i) {
+            ptrs.k[i] = K_layers_out[l0 + i];
+            ptrs.v[i] = V_layers_out[l0 + i];
+        }
+        p.layer_begin = l0;
+        p.layer_count = n;
+        p.work_counter = counters + l0 / kMaxLayersPerLaunch;
         const int64_t streams = 2ll * n * dst->n_kv_heads;
         cudaError_t e;
         switch (dst->head_dim) {
