@@ -44,9 +44,10 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    """nvidia-smi clock / throttle-reason samples; summarised over a wall-clock window so that
+    only samples taken while the timed work ran count."""
 
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -61,13 +62,15 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu_index), "-lms", "50"],
+                 "-i", str(self.gpu_index), "-lms", "20"],
                 stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t_begin: float, t_end: float):
+        """Summary of the samples whose timestamp lies in [t_begin, t_end] (time.time() values)."""
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "power_w_max": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -75,28 +78,30 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
+        rows = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
             with open(self.path) as f:
                 for line in f:
                     parts = [p.strip() for p in line.split(",")]
-                    if len(parts) < 9:
+                    if len(parts) < 10:
                         continue
                     try:
-                        sm.append(float(parts[1]))
-                        smax.append(float(parts[2]))
+                        ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                        rows.append((ts, float(parts[2]), float(parts[3]), float(parts[4]),
+                                     [n for n, v in zip(names, parts[6:10]) if v.lower().startswith("active")]))
                     except ValueError:
                         continue
-                    for name, val in zip(names, parts[5:9]):
-                        if val.lower().startswith("active"):
-                            reasons.add(name)
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+        inside = [r for r in rows if t_begin - 0.02 <= r[0] <= t_end + 0.02]
+        if inside:
+            reasons = set()
+            for r in inside:
+                reasons.update(r[4])
+            out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
+                       power_w_max=max(r[3] for r in inside), reasons=sorted(reasons), samples=len(inside))
         return out
 
 
@@ -182,6 +187,9 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     q.load_library()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()  # runs through set-up and both timed legs; summarised over the timed window
 
     w, Ks, Vs = load_workload(args.config, n_layers=args.layers)
     L, H, d, T = w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens
@@ -232,12 +240,10 @@ def run_ours(args):
     if st != 0:
         raise RuntimeError(f"card status {st}")
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
+    t_wall_begin = time.time()
     records = []
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
@@ -279,7 +285,8 @@ def run_ours(args):
         e_end.record(stream)
         torch.cuda.synchronize()
         e2e_ms = e_begin.elapsed_time(e_end)
-    clocks = sampler.stop() if rank == 0 else None
+    torch.cuda.synchronize()
+    clocks = sampler.stop(t_wall_begin, time.time()) if rank == 0 else None
 
     if world > 1:
         t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
@@ -353,7 +360,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=3, choices=[2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

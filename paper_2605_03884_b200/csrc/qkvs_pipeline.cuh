@@ -349,25 +349,39 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_
     CreateWarpSmem<D, NS> &sm = reinterpret_cast<CreateWarpSmem<D, NS> *>(smem_raw)[warp];
 
     qkvs_card_header_t *hdr = reinterpret_cast<qkvs_card_header_t *>(p.card);
-    if (hdr->status != QKVS_OK) return;  // bad bits or short buffer: no payload is written
-    const uint64_t stream_bytes = hdr->stream_bytes;
     const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
-
-    WorkSource ws;
-    CacheWalk<C::ROWS, true> ahead;  // runs NS sub-tiles ahead and starts the copies
-    if (!start_work<C::WARPS>(ws, ahead.cu, sm.ring, p, warp, lane)) return;
-    ahead.locate(p, ptrs, 0);
-    TableWalk<C::ROWS, false> tw;    // runs one sub-tile ahead and reads the tables
-    tw.cu = ahead.cu;
-    tw.locate(p, sec, p.bits_mode, stream_bytes);
-
     if (lane == 0) {
         for (int s = 0; s < NS; ++s) mbar_init(&sm.full[s], 1);
         fence_mbar_init();
     }
     __syncwarp();
+    WorkSource ws;
+    CacheWalk<C::ROWS, true> ahead;  // runs NS sub-tiles ahead and starts the copies
+    if (!start_work<C::WARPS>(ws, ahead.cu, sm.ring, p, warp, lane)) return;
+    ahead.locate(p, ptrs, 0);
+    const Cursor first = ahead.cu;
 
+    // The first copies need nothing but kernel parameters and the caller's cache, so they start
+    // before this kernel waits for the scan kernel (which may still be running: see
+    // grid_dependency_wait).  They stay inside the warp's first chunk, because taking another
+    // chunk needs the work counter, which the scan kernel clears.
     uint32_t issued = 0, consumed = 0;
+    const uint32_t early = min((uint32_t)NS, first.left + 1u);
+    for (; issued < early; ++issued) {
+        if (issued) ahead.next(ws, p, ptrs, 0, lane);
+        create_issue<D, NS>(sm, (int)issued, ahead.row, rows_at<C::ROWS>(ahead.cu.c, p), p, lane);
+    }
+    grid_dependency_wait();
+    if (hdr->status != QKVS_OK) {
+        // bad bits or short buffer: no payload is written; let the copies land before leaving
+        for (uint32_t j = 0; j < issued; ++j) mbar_wait(&sm.full[j], 0);
+        return;
+    }
+    const uint64_t stream_bytes = hdr->stream_bytes;
+    TableWalk<C::ROWS, false> tw;    // runs one sub-tile ahead and reads the tables
+    tw.cu = first;
+    tw.locate(p, sec, p.bits_mode, stream_bytes);
+    ahead.next(ws, p, ptrs, 0, lane);
     while (issued < (uint32_t)NS && !ahead.cu.done) {
         create_issue<D, NS>(sm, (int)issued, ahead.row, rows_at<C::ROWS>(ahead.cu.c, p), p, lane);
         ++issued;

@@ -131,6 +131,20 @@ __device__ __forceinline__ float2 sub_f32_f16x2(uint32_t w, float c)
     return d;
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute
+// may start while the kernel before it in the stream still runs; grid_dependency_wait() then
+// blocks until that kernel has completed and its writes are visible (without the attribute it
+// returns at once).  allow_dependents() in the earlier kernel lets the next one start right away.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void allow_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // Packed binary32 arithmetic: one instruction performs the operation on both halves of a 64-bit
 // register pair, each half rounded on its own exactly like the scalar instruction.
 __device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)

@@ -98,6 +98,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
 {
     __shared__ uint32_t warp_sums[33];
     __shared__ int s_bad;
+    allow_dependents();  // the create kernel may set itself up while this one runs
     const int seg = blockIdx.x;
     const int64_t T = p.n_tokens;
     const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
@@ -186,6 +187,7 @@ __global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
 {
     __shared__ uint64_t s_carry;
     __shared__ uint64_t s_warp[33];
+    allow_dependents();
     const int64_t T = p.n_tokens;
     const int H = p.n_kv_heads;
     const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
@@ -332,27 +334,43 @@ constexpr int kStagesCreate = QKVS_STAGES_CREATE;
 constexpr int kStagesInject = QKVS_STAGES_INJECT;
 
 // Persistent grid: as many CTAs as fit on the device at once, never more than there is work for.
-template <typename Kernel>
+// The occupancy of a kernel on a device does not change, so it is looked up once per device;
+// TAG tells the kernels apart (they all have the same function type).
+template <int TAG, typename Kernel>
 static cudaError_t persistent_grid(Kernel kernel, int threads, size_t smem, int64_t max_ctas, unsigned *grid)
 {
-    int dev = 0, sms = 0, per_sm = 0;
+    constexpr int kMaxDevices = 64;
+    static std::mutex mutex;
+    static int resident[kMaxDevices] = {};  // CTAs of this kernel the whole device holds; 0 = not known yet
+    int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) return cudaErrorInvalidConfiguration;
-    *grid = (unsigned)std::min<int64_t>(max_ctas, (int64_t)sms * per_sm);
+    int64_t fit = 0;
+    {
+        std::lock_guard<std::mutex> lock(mutex);
+        if (dev >= 0 && dev < kMaxDevices) fit = resident[dev];
+    }
+    if (fit == 0) {
+        int sms = 0, per_sm = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) return cudaErrorInvalidConfiguration;
+        fit = (int64_t)sms * per_sm;
+        std::lock_guard<std::mutex> lock(mutex);
+        if (dev >= 0 && dev < kMaxDevices) resident[dev] = (int)fit;
+    }
+    *grid = (unsigned)std::min<int64_t>(max_ctas, fit);
     return cudaSuccess;
 }
 
 // Splits `streams` streams into sub-tiles and chunks and launches `kernel` on a persistent grid.
-template <int D, typename Kernel>
+template <int D, int TAG, typename Kernel>
 static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp, const LayerPtrs &ptrs, int64_t streams,
-                               cudaStream_t st)
+                               cudaStream_t st, bool overlap_previous)
 {
     using C = WarpCfg<D>;
     PathParams p = pp;
@@ -364,24 +382,35 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
     p.n_chunks = (p.n_subs + kChunk - 1) / kChunk;
     p.last_rows = (uint32_t)(p.n_tokens - (int64_t)(p.subs_per_stream - 1) * C::ROWS);
     unsigned grid = 0;
-    cudaError_t e = persistent_grid(kernel, C::THREADS, smem, (int64_t)((p.n_chunks + C::WARPS - 1) / C::WARPS), &grid);
+    cudaError_t e = persistent_grid<TAG>(kernel, C::THREADS, smem, (int64_t)((p.n_chunks + C::WARPS - 1) / C::WARPS), &grid);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, C::THREADS, smem, st>>>(p, ptrs);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(C::THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    memset(&attr, 0, sizeof(attr));
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = overlap_previous ? 1 : 0;  // the kernel calls grid_dependency_wait() before it reads the card
+    return cudaLaunchKernelEx(&cfg, kernel, p, ptrs);
 }
 
 template <int D>
 static cudaError_t launch_create(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D>(create_kernel<D, kStagesCreate>, WarpCfg<D>::WARPS * sizeof(CreateWarpSmem<D, kStagesCreate>), p,
-                          ptrs, streams, st);
+    return launch_path<D, D * 2>(create_kernel<D, kStagesCreate>, WarpCfg<D>::WARPS * sizeof(CreateWarpSmem<D, kStagesCreate>), p,
+                          ptrs, streams, st, true);
 }
 
 template <int D>
 static cudaError_t launch_inject(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D>(inject_kernel<D, kStagesInject>, WarpCfg<D>::WARPS * sizeof(InjectWarpSmem<D, kStagesInject>), p,
-                          ptrs, streams, st);
+    return launch_path<D, D * 2 + 1>(inject_kernel<D, kStagesInject>, WarpCfg<D>::WARPS * sizeof(InjectWarpSmem<D, kStagesInject>), p,
+                          ptrs, streams, st, false);
 }
 
 // ---------------------------------------------------------------------------------------------
