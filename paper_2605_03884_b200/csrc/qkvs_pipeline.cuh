@@ -25,8 +25,14 @@
 
 namespace qkvs {
 
-#ifndef QKVS_WARPS_PER_CTA
-#define QKVS_WARPS_PER_CTA 6
+// Launch shape, per kernel: warps per CTA and pipeline stages per warp (CTAs per SM is what the
+// shared memory then allows: three).  Injection has the longer dependent chains per warp and gains
+// from more warps with a shallower ring; creation is the other way round.
+#ifndef QKVS_WARPS_CREATE
+#define QKVS_WARPS_CREATE 6
+#endif
+#ifndef QKVS_WARPS_INJECT
+#define QKVS_WARPS_INJECT 8
 #endif
 #ifndef QKVS_CTAS_PER_SM
 #define QKVS_CTAS_PER_SM 3
@@ -34,8 +40,6 @@ namespace qkvs {
 
 template <int D>
 struct WarpCfg {
-    static constexpr int WARPS = QKVS_WARPS_PER_CTA;    // warps per CTA
-    static constexpr int THREADS = WARPS * 32;
     static constexpr int G = D / kGroup;                // groups per token row
     static constexpr int R = 32 / G;                    // rows covered by one group per lane: 16, 8, 5, 4
     static constexpr int GROUPS = R * G;                // lanes that own a group in create (30 for D = 192)
@@ -340,8 +344,8 @@ __device__ __forceinline__ void create_issue(CreateWarpSmem<D, NS> &sm, int stag
     }
 }
 
-template <int D, int NS>
-__global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_kernel(PathParams p, LayerPtrs ptrs)
+template <int D, int NS, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) create_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -357,7 +361,7 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) create_
     __syncwarp();
     WorkSource ws;
     CacheWalk<C::ROWS, true> ahead;  // runs NS sub-tiles ahead and starts the copies
-    if (!start_work<C::WARPS>(ws, ahead.cu, sm.ring, p, warp, lane)) return;
+    if (!start_work<WARPS>(ws, ahead.cu, sm.ring, p, warp, lane)) return;
     ahead.locate(p, ptrs, 0);
     const Cursor first = ahead.cu;
 
@@ -456,6 +460,11 @@ struct InjectWarpSmem {
     static_assert(NS >= 2 && NS < (int)kChunk, "pipeline depth");
 };
 
+// One chunk (8 values) of a record.  B is the bit-width known at compile time, or 0 when it is
+// only known per lane (`b`): then the widths 2, 4 and 8 share one instruction stream -- the codes
+// are fetched as the aligned 8 bytes around them and shifted into place, and the unpacking steps
+// are applied by selection -- so that lanes of different widths do not serialise; only FP16 rows
+// branch off.
 template <int D, int B>
 __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos)
 {
@@ -465,15 +474,25 @@ __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos
     const float2 m = *reinterpret_cast<const float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup);
     const uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * bb;
     uint32_t lo, hi;
-    if (bb == 8) {
+    if (B == 8) {
         const uint2 w = *reinterpret_cast<const uint2 *>(codes);
         lo = w.x;
         hi = w.y;
+    } else if (B == 4) {
+        unpack_nibbles(*reinterpret_cast<const uint32_t *>(codes), lo, hi);
+    } else if (B == 2) {
+        unpack_nibbles(unpack_crumbs(*reinterpret_cast<const uint16_t *>(codes)), lo, hi);
     } else {
-        uint32_t w;
-        if (bb == 4) w = *reinterpret_cast<const uint32_t *>(codes);
-        else w = unpack_crumbs(*reinterpret_cast<const uint16_t *>(codes));
-        unpack_nibbles(w, lo, hi);
+        // the codes start at a multiple of b bytes: inside one aligned 8-byte window
+        const uint32_t a = smem_addr(codes);
+        const uint2 w = *reinterpret_cast<const uint2 *>(codes - (a & 7u));
+        const uint32_t sh = (a & 7u) * 8u;
+        const uint32_t x = sh >= 32u ? w.y >> (sh - 32u) : __funnelshift_r(w.x, w.y, sh);  // first 32 bits of the codes
+        const uint32_t nib = bb == 2 ? unpack_crumbs(x & 0xffffu) : x;
+        uint32_t l4, h4;
+        unpack_nibbles(nib, l4, h4);
+        lo = bb == 8 ? w.x : l4;  // 8-bit codes are 8-byte aligned: the window is the codes
+        hi = bb == 8 ? w.y : h4;
     }
     return dequantize_chunk(lo, hi, m.x, m.y);
 }
@@ -554,8 +573,8 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
     __syncwarp();
 }
 
-template <int D, int NS>
-__global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) inject_kernel(PathParams p, LayerPtrs ptrs)
+template <int D, int NS, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) inject_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -595,7 +614,7 @@ __global__ void __launch_bounds__(WarpCfg<D>::THREADS, QKVS_CTAS_PER_SM) inject_
     // one step ahead of the copies, which run NS steps ahead of the arithmetic.
     WorkSource ws;
     TableWalk<C::ROWS, true> tw;
-    if (!start_work<C::WARPS>(ws, tw.cu, sm.ring, p, warp, lane)) return;
+    if (!start_work<WARPS>(ws, tw.cu, sm.ring, p, warp, lane)) return;
     tw.locate(p, sec, mode, stream_bytes);
     CacheWalk<C::ROWS, false> cons;
     cons.cu = tw.cu;

@@ -325,7 +325,7 @@ static uint32_t *work_counter(void *workspace_dev, int launch)
 #define QKVS_STAGES_CREATE 3
 #endif
 #ifndef QKVS_STAGES_INJECT
-#define QKVS_STAGES_INJECT 3
+#define QKVS_STAGES_INJECT 2
 #endif
 #ifndef QKVS_INTERLEAVED
 #define QKVS_INTERLEAVED 1
@@ -368,7 +368,7 @@ static cudaError_t persistent_grid(Kernel kernel, int threads, size_t smem, int6
 }
 
 // Splits `streams` streams into sub-tiles and chunks and launches `kernel` on a persistent grid.
-template <int D, int TAG, typename Kernel>
+template <int D, int WARPS, int TAG, typename Kernel>
 static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp, const LayerPtrs &ptrs, int64_t streams,
                                cudaStream_t st, bool overlap_previous)
 {
@@ -382,12 +382,12 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
     p.n_chunks = (p.n_subs + kChunk - 1) / kChunk;
     p.last_rows = (uint32_t)(p.n_tokens - (int64_t)(p.subs_per_stream - 1) * C::ROWS);
     unsigned grid = 0;
-    cudaError_t e = persistent_grid<TAG>(kernel, C::THREADS, smem, (int64_t)((p.n_chunks + C::WARPS - 1) / C::WARPS), &grid);
+    cudaError_t e = persistent_grid<TAG>(kernel, WARPS * 32, smem, (int64_t)((p.n_chunks + WARPS - 1) / WARPS), &grid);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(C::THREADS);
+    cfg.blockDim = dim3(WARPS * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr;
@@ -402,15 +402,15 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
 template <int D>
 static cudaError_t launch_create(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D, D * 2>(create_kernel<D, kStagesCreate>, WarpCfg<D>::WARPS * sizeof(CreateWarpSmem<D, kStagesCreate>), p,
-                          ptrs, streams, st, true);
+    return launch_path<D, QKVS_WARPS_CREATE, D * 2>(create_kernel<D, kStagesCreate, QKVS_WARPS_CREATE>,
+                                                   QKVS_WARPS_CREATE * sizeof(CreateWarpSmem<D, kStagesCreate>), p, ptrs, streams, st, true);
 }
 
 template <int D>
 static cudaError_t launch_inject(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D, D * 2 + 1>(inject_kernel<D, kStagesInject>, WarpCfg<D>::WARPS * sizeof(InjectWarpSmem<D, kStagesInject>), p,
-                          ptrs, streams, st, false);
+    return launch_path<D, QKVS_WARPS_INJECT, D * 2 + 1>(inject_kernel<D, kStagesInject, QKVS_WARPS_INJECT>,
+                                                       QKVS_WARPS_INJECT * sizeof(InjectWarpSmem<D, kStagesInject>), p, ptrs, streams, st, false);
 }
 
 // ---------------------------------------------------------------------------------------------
