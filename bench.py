@@ -31,7 +31,7 @@ import numpy as np  # noqa: E402
 
 from paper_2605_03884_b200 import workloads as wl  # noqa: E402
 
-METRIC = "CacheCard create+inject throughput (FP16 KV bytes through create then inject)"
+METRIC = "CacheCard create+inject GB/s (FP16 KV bytes) and % of HBM peak at 8K ctx"
 UNIT = "GB/s"
 
 
@@ -122,6 +122,23 @@ class ClockSampler:
             out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
                        power_w_max=max(r[3] for r in inside), reasons=sorted(reasons), samples=len(inside))
         return out
+
+
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks of the default process group
+    (the list itself when there is no group): a replica job is as slow as its slowest rank."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def replica_throughput(kv_bytes: int, hops: int, world: int, ms_per_step: float) -> float:
+    """Whole-job GB/s of FP16 KV: every rank carries its own cache through create + inject."""
+    return kv_bytes * hops * world / (ms_per_step * 1e-3) / 1e9
 
 
 def load_workload(number: int, layers=None, n_layers=None):
@@ -307,10 +324,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     clocks = sampler.stop(t_wall_begin, time.time()) if rank == 0 else None
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device="cuda")
 
     if rank != 0:
         if world > 1:
@@ -319,9 +333,8 @@ def run_ours(args):
 
     peak, peak_src = measured_peaks()
     ms_per_step = total_ms / args.steps
-    units = kv_bytes * hops * world  # FP16 KV bytes carried through create+inject per step, all ranks
-    value = units / (ms_per_step * 1e-3) / 1e9
-    e2e_value = None if args.skip_e2e else units / (e2e_ms / args.steps * 1e-3) / 1e9
+    value = replica_throughput(kv_bytes, hops, world, ms_per_step)
+    e2e_value = None if args.skip_e2e else replica_throughput(kv_bytes, hops, world, e2e_ms / args.steps)
     med = statistics.median
     per_hop = []
     for h in range(hops):
