@@ -78,6 +78,8 @@ def lib():
                                             C.c_uint64, C.c_int64, C.c_void_p, C.c_uint64, C.c_int64, C.c_int64]
         l.orc_card_inject.restype = C.c_int
         l.orc_card_inject.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_void_p, C.c_void_p, C.c_int64]
+        l.orc_card_attend.restype = C.c_int
+        l.orc_card_attend.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_int, C.c_void_p, C.c_double, C.c_void_p]
         l.orc_num_threads.restype = C.c_int
         l.orc_set_num_threads.argtypes = [C.c_int]
         _lib = l
@@ -227,6 +229,19 @@ def card_inject(card: np.ndarray, dst: Layout, K_out: List[np.ndarray], V_out: L
     kp, vp = _ptr_array(K_out), _ptr_array(V_out)
     return lib().orc_card_inject(_ptr(card), card.size if card_bytes is None else card_bytes,
                                  C.byref(dst), kp, vp, dst_token_offset)
+
+
+def card_attend(card: np.ndarray, layout: Layout, q: np.ndarray, softmax_scale: Optional[float] = None
+                ) -> Tuple[int, np.ndarray]:
+    """Decode-step attention from the card.  q: FP16 [n_layers, n_q_heads, head_dim]; returns
+    (status, float64 [n_layers, n_q_heads, head_dim])."""
+    card = np.ascontiguousarray(card, dtype=np.uint8)
+    q = np.ascontiguousarray(q, dtype=np.float16)
+    assert q.ndim == 3 and q.shape[0] == layout.n_layers and q.shape[2] == layout.head_dim
+    scale = 1.0 / float(np.sqrt(layout.head_dim)) if softmax_scale is None else float(softmax_scale)
+    out = np.zeros(q.shape, dtype=np.float64)
+    st = lib().orc_card_attend(_ptr(card), card.size, C.byref(layout), q.shape[1], _ptr(q), scale, _ptr(out))
+    return st, out
 
 
 def num_threads() -> int:

@@ -26,12 +26,16 @@
  * Pins (see tests): closed-form size, uniform offsets, brute-force scan, FP16 round trip,
  * |x - x^| <= scale/2 (+ rounding slack), min -> code 0 / max -> code 2^b-1, monotone codes,
  * hand-worked 2-bit and 4-bit groups with exact ties, exact-rational recomputation of codes,
- * the 8-bit case against the textbook affine uint8 quantiser, all-FP16 card == memcpy.
+ * the 8-bit case against the textbook affine uint8 quantiser, all-FP16 card == memcpy;
+ * attention from the card: one token -> its value row, equal value rows -> that row, zero query
+ * -> the mean of the value rows, a card of FP16 tokens -> the library softmax attention on the
+ * original cache, one dominant key -> its value row.
  *
  * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
  */
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #ifdef _OPENMP
@@ -519,6 +523,90 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
                           T, C.head_dim, x, dst->token_stride);
     }
     return ORC_OK;
+}
+
+/* Decode-step attention straight from a card, without rebuilding the FP16 cache
+ * (Section 4.3: consuming a foreign quantised cache directly inside attention is the paper's
+ * stated goal; Section 3.1 for K, V per layer and head).  One new token per layer attends to all
+ * n_tokens of the card.  Query head j of a layer reads KV head j / (n_q_heads / n_kv_heads)
+ * (grouped-query attention; the paper's model, Llama-3.1-8B, has 32 query and 8 KV heads):
+ *     s_t  = softmax_scale * sum_c q[j][c] * K^[t][c]
+ *     p_t  = exp(s_t - max_t s_t) / sum_t exp(s_t - max_t s_t)
+ *     o[c] = sum_t p_t * V^[t][c]
+ * where K^, V^ are exactly the FP16 values injection reconstructs.  The paper gives no formula
+ * for this step; this is the textbook definition, evaluated in double precision.
+ *   q    [n_layers][n_q_heads][head_dim] FP16 bit patterns
+ *   out  [n_layers][n_q_heads][head_dim] double */
+int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *L, int n_q_heads,
+                    const uint16_t *q, double softmax_scale, double *out)
+{
+    int st = layout_ok(L);
+    if (st) return st;
+    if (n_q_heads < L->n_kv_heads || n_q_heads % L->n_kv_heads != 0) return ORC_INVALID_ARG;
+    if (card_bytes < 256) return ORC_BAD_CARD;
+    if (get_u32(card + 0) != 0x53564B51u || get_u32(card + 4) != 1u || get_u32(card + 8) != 0u) return ORC_BAD_CARD;
+    orc_layout C = *L;
+    C.bits_mode = (int32_t)get_u32(card + 12);
+    if ((int32_t)get_u32(card + 16) != L->n_layers || (int32_t)get_u32(card + 20) != L->n_kv_heads ||
+        (int32_t)get_u32(card + 24) != L->head_dim || (int32_t)get_u32(card + 28) != L->n_tokens ||
+        (C.bits_mode != 0 && C.bits_mode != 1) || get_u64(card + 112) > card_bytes)
+        return ORC_BAD_CARD;
+    const int d = C.head_dim, H = C.n_kv_heads, per_kv = n_q_heads / H;
+    const int64_t T = C.n_tokens;
+    const uint64_t bo = get_u64(card + 80), oo = get_u64(card + 88);
+    if (T == 0) {
+        memset(out, 0, sizeof(double) * (size_t)C.n_layers * (size_t)n_q_heads * (size_t)d);
+        return ORC_OK;
+    }
+    int failed = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int64_t lh = 0; lh < (int64_t)C.n_layers * H; ++lh) {
+        const int l = (int)(lh / H), h = (int)(lh % H);
+        const int64_t seg = segment_of(&C, l, h);
+        const uint8_t *bits = card + bo + (uint64_t)seg * (uint64_t)T;
+        const uint32_t *off = (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1));
+        uint16_t *kx = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)T * (size_t)d);
+        uint16_t *vx = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)T * (size_t)d);
+        double *s = (double *)malloc(sizeof(double) * (size_t)T);
+        if (!kx || !vx || !s) {
+            failed = 1;
+            free(kx);
+            free(vx);
+            free(s);
+            continue;
+        }
+        orc_decode_stream(card + stream_base(card, &C, stream_index(&C, l, 0, h)), bits, off, T, d, kx, d);
+        orc_decode_stream(card + stream_base(card, &C, stream_index(&C, l, 1, h)), bits, off, T, d, vx, d);
+        for (int jj = 0; jj < per_kv; ++jj) {
+            const int j = h * per_kv + jj;
+            const uint16_t *qv = q + ((int64_t)l * n_q_heads + j) * d;
+            double *o = out + ((int64_t)l * n_q_heads + j) * d;
+            double mx = -INFINITY;
+            for (int64_t t = 0; t < T; ++t) {
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c)
+                    acc += (double)orc_half_to_float(qv[c]) * (double)orc_half_to_float(kx[t * d + c]);
+                s[t] = softmax_scale * acc;
+                if (s[t] > mx) mx = s[t];
+            }
+            double denom = 0.0;
+            for (int64_t t = 0; t < T; ++t) {
+                s[t] = exp(s[t] - mx);
+                denom += s[t];
+            }
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int64_t t = 0; t < T; ++t) acc += s[t] * (double)orc_half_to_float(vx[t * d + c]);
+                o[c] = acc / denom;
+            }
+        }
+        free(kx);
+        free(vx);
+        free(s);
+    }
+    return failed ? ORC_INVALID_ARG : ORC_OK;
 }
 
 int orc_num_threads(void)

@@ -1,0 +1,131 @@
+"""Pins of the oracle's attention-from-the-card against what the definition fixes: special cases
+with a known answer and the library routine it reduces to.  CPU only.
+
+(The paper, Section 4.3, names consuming the quantised cache inside attention as the goal but
+prints neither a formula nor numbers for it; the definition is the textbook one.)"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2605_03884_b200 import workloads as wl
+
+
+def _card(Ks, Vs, bits, L, H, d, T, mode=0):
+    lay = oracle.make_layout(L, H, d, T, bits_mode=mode)
+    st, card = oracle.card_create(lay, Ks, Vs, bits)
+    assert st == oracle.OK
+    return lay, card
+
+
+def _cache(L, H, T, d, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    Ks = [(rng.standard_normal((H, T, d), dtype=np.float32) * scale).astype(np.float16) for _ in range(L)]
+    Vs = [(rng.standard_normal((H, T, d), dtype=np.float32) * scale).astype(np.float16) for _ in range(L)]
+    return Ks, Vs
+
+
+def _reference_attention(Kh, Vh, q, per_kv, scale):
+    """softmax(q K^T * scale) V with numpy in float64; Kh, Vh: per-layer [H, T, d]; q: [L, nq, d]."""
+    L, nq, d = q.shape
+    out = np.zeros((L, nq, d))
+    for l in range(L):
+        for j in range(nq):
+            k = Kh[l][j // per_kv].astype(np.float64)
+            v = Vh[l][j // per_kv].astype(np.float64)
+            s = k @ q[l, j].astype(np.float64) * scale
+            p = np.exp(s - s.max())
+            out[l, j] = (p / p.sum()) @ v
+    return out
+
+
+def test_single_token_returns_its_value_row():
+    L, H, d, T, nq = 2, 2, 64, 1, 4
+    Ks, Vs = _cache(L, H, T, d, 1)
+    lay, card = _card(Ks, Vs, np.full(T, 16, np.uint8), L, H, d, T)
+    q = wl.random_fp16((L, nq, d), 2)
+    st, o = oracle.card_attend(card, lay, q)
+    assert st == oracle.OK
+    for l in range(L):
+        for j in range(nq):
+            assert np.array_equal(o[l, j], Vs[l][j // 2][0].astype(np.float64))
+
+
+def test_equal_value_rows_come_back_whatever_the_query():
+    L, H, d, T, nq = 1, 2, 128, 37, 8
+    Ks, Vs = _cache(L, H, T, d, 3)
+    row = wl.random_fp16((H, 1, d), 4)
+    Vs = [np.repeat(row, T, axis=1)]
+    lay, card = _card(Ks, Vs, np.full(T, 16, np.uint8), L, H, d, T)
+    st, o = oracle.card_attend(card, lay, wl.random_fp16((L, nq, d), 5, scale=3.0))
+    assert st == oracle.OK
+    for j in range(nq):
+        np.testing.assert_allclose(o[0, j], row[j // 4, 0].astype(np.float64), rtol=1e-14, atol=1e-300)
+
+
+def test_zero_query_gives_the_mean_of_the_reconstructed_values():
+    L, H, d, T, nq = 1, 1, 64, 50, 2
+    Ks, Vs = _cache(L, H, T, d, 6)
+    bits = wl.iid_bits(T, (0.3, 0.3, 0.3, 0.1), 7)
+    lay, card = _card(Ks, Vs, bits, L, H, d, T)
+    Kr, Vr = [np.zeros_like(Ks[0])], [np.zeros_like(Vs[0])]
+    assert oracle.card_inject(card, lay, Kr, Vr) == oracle.OK
+    st, o = oracle.card_attend(card, lay, np.zeros((L, nq, d), np.float16))
+    assert st == oracle.OK
+    np.testing.assert_allclose(o[0, 0], Vr[0][0].astype(np.float64).mean(axis=0), rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(o[0, 1], o[0, 0], rtol=0, atol=0)
+
+
+def test_fp16_card_reduces_to_library_attention_on_the_original_cache():
+    L, H, d, T, nq = 2, 2, 128, 200, 8
+    Ks, Vs = _cache(L, H, T, d, 8)
+    lay, card = _card(Ks, Vs, np.full(T, 16, np.uint8), L, H, d, T)
+    q = wl.random_fp16((L, nq, d), 9)
+    st, o = oracle.card_attend(card, lay, q)
+    assert st == oracle.OK
+    want = _reference_attention(Ks, Vs, q, nq // H, 1.0 / np.sqrt(d))
+    np.testing.assert_allclose(o, want, rtol=1e-12, atol=1e-14)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_quantised_card_equals_library_attention_on_the_injected_cache(mode):
+    L, H, d, T, nq = 2, 3, 64, 150, 6
+    Ks, Vs = _cache(L, H, T, d, 10)
+    if mode == 0:
+        bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 11)
+    else:
+        bits = np.concatenate([wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 20 + s) for s in range(L * H)])
+    lay, card = _card(Ks, Vs, bits, L, H, d, T, mode)
+    Kr, Vr = [np.zeros_like(k) for k in Ks], [np.zeros_like(v) for v in Vs]
+    assert oracle.card_inject(card, lay, Kr, Vr) == oracle.OK
+    q = wl.random_fp16((L, nq, d), 12)
+    st, o = oracle.card_attend(card, lay, q, softmax_scale=0.3)
+    assert st == oracle.OK
+    np.testing.assert_allclose(o, _reference_attention(Kr, Vr, q, nq // H, 0.3), rtol=1e-12, atol=1e-14)
+
+
+def test_one_dominant_key_selects_its_value_row():
+    """K rows are +-e_0 * 8 except token 17 = +e_0 * 64: with q = 32 e_0 the softmax weight of
+    every other token is below exp(-64*32*... ) ~ 0, so the output is V[17] to double precision."""
+    L, H, d, T, nq = 1, 1, 64, 40, 1
+    K = np.zeros((H, T, d), np.float16)
+    K[0, :, 0] = 8.0
+    K[0, 17, 0] = 64.0
+    V = wl.random_fp16((H, T, d), 13)
+    lay, card = _card([K], [V], np.full(T, 16, np.uint8), L, H, d, T)
+    q = np.zeros((L, nq, d), np.float16)
+    q[0, 0, 0] = 32.0
+    st, o = oracle.card_attend(card, lay, q, softmax_scale=1.0)
+    assert st == oracle.OK
+    np.testing.assert_allclose(o[0, 0], V[0, 17].astype(np.float64), rtol=1e-12, atol=1e-300)
+
+
+def test_argument_and_card_checks():
+    L, H, d, T = 1, 2, 64, 8
+    Ks, Vs = _cache(L, H, T, d, 14)
+    lay, card = _card(Ks, Vs, np.full(T, 4, np.uint8), L, H, d, T)
+    st, _ = oracle.card_attend(card, lay, np.zeros((L, 3, d), np.float16))     # 3 query heads over 2 KV heads
+    assert st == oracle.INVALID_ARG
+    bad = card.copy()
+    bad[0] ^= 0xFF
+    st, _ = oracle.card_attend(bad, lay, np.zeros((L, 2, d), np.float16))
+    assert st == oracle.BAD_CARD
