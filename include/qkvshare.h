@@ -194,6 +194,32 @@ QKVS_API qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t car
                                        void *const *V_layers_out, int64_t dst_token_offset,
                                        int32_t *status_dev, void *stream);
 
+/* Decode-step attention straight from a card (Section 4.3 names consuming the quantised cache
+ * inside attention as the goal; the FP16 cache of Section 4.2.2 is never rebuilt).  One query
+ * token per layer attends to all n_tokens of the card, with grouped queries: query head j reads
+ * KV head j / (n_q_heads / n_kv_heads):
+ *     s_t = softmax_scale * q_j . K^_t,   p = softmax_t(s),   out_j = sum_t p_t V^_t
+ * where K^, V^ are exactly the FP16 values qkvs_card_inject would write.  Products run on the
+ * tensor cores with FP16 inputs (the probabilities are rounded to FP16) and FP32 accumulation.
+ *   layout        n_layers, n_kv_heads, head_dim, n_tokens of the card (checked against its
+ *                 header on the device); head_dim must be 128; strides are not looked at
+ *   n_q_heads     multiple of n_kv_heads, at most 8 query heads per KV head
+ *   q_dev         FP16 [n_layers][n_q_heads][head_dim], 16-byte aligned
+ *   out_dev       FP32 [n_layers][n_q_heads][head_dim], 16-byte aligned; all zeros if n_tokens is
+ *                 0 or the card does not check out
+ *   scratch_dev   device buffer of at least qkvs_attend_scratch_size() bytes, 16-byte aligned,
+ *                 content irrelevant on entry; afterwards its first int32 is the status word
+ *                 (0, BAD_CARD or TIMEOUT, as for qkvs_card_inject).  Holds the work counter and
+ *                 the per-item partial results that a second kernel merges
+ * Asynchronous on `stream`.  Errors visible on the host: INVALID_ARG, UNSUPPORTED_SHAPE,
+ * BAD_CARD (card_bytes below a header), BUFFER_TOO_SMALL (scratch), CUDA. */
+QKVS_API qkvs_status_t qkvs_attend_scratch_size(const qkvs_layout_t *layout, int32_t n_q_heads,
+                                                size_t *out_bytes);
+QKVS_API qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes,
+                               const qkvs_layout_t *layout, int32_t n_q_heads, const void *q_dev,
+                               float softmax_scale, float *out_dev, void *scratch_dev,
+                               size_t scratch_bytes, void *stream);
+
 /* Synchronises `stream`, copies the card's header to the host and returns its recorded status
  * (or BAD_CARD if magic/version are wrong, or CUDA on a runtime error). */
 QKVS_API qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_card_header_t *out_host);

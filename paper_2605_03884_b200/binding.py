@@ -50,7 +50,8 @@ class CardHeader(C.Structure):
 assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
-           "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_card_info", "qkvs_selftest_division", "qkvs_status_string",
+           "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_attend_scratch_size", "qkvs_card_attend",
+           "qkvs_card_info", "qkvs_selftest_division", "qkvs_status_string",
            "qkvs_version")
 
 _lib = None
@@ -80,6 +81,10 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_inject.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
     lib.qkvs_card_inject_noalloc.restype = C.c_int
     lib.qkvs_card_inject_noalloc.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
+    lib.qkvs_attend_scratch_size.restype = C.c_int
+    lib.qkvs_attend_scratch_size.argtypes = [C.POINTER(Layout), C.c_int32, C.POINTER(C.c_size_t)]
+    lib.qkvs_card_attend.restype = C.c_int
+    lib.qkvs_card_attend.argtypes = [vp, C.c_size_t, C.POINTER(Layout), C.c_int32, vp, C.c_float, vp, vp, C.c_size_t, vp]
     lib.qkvs_card_info.restype = C.c_int
     lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
     lib.qkvs_selftest_division.restype = C.c_int
@@ -225,6 +230,30 @@ def card_inject_noalloc(card_dev, dst_layout: Layout, K_out: Sequence, V_out: Se
                                       _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_card_inject_noalloc")
+    return st
+
+
+def attend_scratch_size(layout: Layout, n_q_heads: int) -> int:
+    out = C.c_size_t(0)
+    st = load_library().qkvs_attend_scratch_size(C.byref(layout), int(n_q_heads), C.byref(out))
+    if st != OK:
+        raise QkvsError(st, "qkvs_attend_scratch_size")
+    return int(out.value)
+
+
+def card_attend(card_dev, layout: Layout, q_dev, out_dev, scratch_dev, softmax_scale: Optional[float] = None,
+                card_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """qkvs_card_attend.  q_dev: CUDA FP16 [L, n_q_heads, d]; out_dev: CUDA FP32 of the same
+    shape; scratch_dev: CUDA uint8 tensor of attend_scratch_size() bytes (its first int32 is the
+    status word afterwards).  softmax_scale defaults to 1/sqrt(d)."""
+    nbytes = int(card_dev.numel() * card_dev.element_size()) if card_bytes is None else int(card_bytes)
+    scale = float(layout.head_dim) ** -0.5 if softmax_scale is None else float(softmax_scale)
+    st = load_library().qkvs_card_attend(int(card_dev.data_ptr()), nbytes, C.byref(layout), int(q_dev.shape[1]),
+                                         int(q_dev.data_ptr()), scale, int(out_dev.data_ptr()),
+                                         int(scratch_dev.data_ptr()),
+                                         int(scratch_dev.numel() * scratch_dev.element_size()), _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_card_attend")
     return st
 
 

@@ -17,6 +17,7 @@
 
 #include "qkvs_common.cuh"
 #include "qkvs_pipeline.cuh"
+#include "qkvs_attend.cuh"
 
 namespace qkvs {
 
@@ -675,6 +676,81 @@ qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t card_bytes, 
         if (e != cudaSuccess) return QKVS_ERR_CUDA;
     }
     return QKVS_OK;
+}
+
+// Shape of the attention work: steps of 16 tokens, items of 16 steps, per (layer, KV head).
+static qkvs_status_t attend_shape(const qkvs_layout_t *layout, int32_t n_q_heads, AttendParams *p)
+{
+    const qkvs_status_t st = check_shape(layout);
+    if (st != QKVS_OK) return st;
+    if (layout->head_dim != kAttendD) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (n_q_heads < layout->n_kv_heads || n_q_heads % layout->n_kv_heads != 0) return QKVS_ERR_INVALID_ARG;
+    if (n_q_heads / layout->n_kv_heads > kAttendMaxPerKv) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    memset(p, 0, sizeof(*p));
+    p->n_layers = layout->n_layers;
+    p->n_kv_heads = layout->n_kv_heads;
+    p->n_tokens = layout->n_tokens;
+    p->n_q_heads = n_q_heads;
+    p->subs_per_head = (uint32_t)(((int64_t)layout->n_tokens + kAttendRows - 1) / kAttendRows);
+    p->items_per_head = (p->subs_per_head + kAttendSteps - 1) / kAttendSteps;
+    const uint64_t n_items = (uint64_t)layout->n_layers * (uint64_t)layout->n_kv_heads * p->items_per_head;
+    if (n_items > 0x7fffffffull) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    p->n_items = (uint32_t)n_items;
+    p->last_rows = p->subs_per_head ? (uint32_t)(layout->n_tokens - (int64_t)(p->subs_per_head - 1) * kAttendRows) : 0u;
+    return QKVS_OK;
+}
+
+static size_t attend_scratch_bytes(const AttendParams &p)
+{
+    const size_t per_kv = (size_t)(p.n_q_heads / p.n_kv_heads);
+    return (size_t)QKVS_WORKSPACE_BYTES + (size_t)p.n_items * per_kv * kPartialFloats * sizeof(float);
+}
+
+qkvs_status_t qkvs_attend_scratch_size(const qkvs_layout_t *layout, int32_t n_q_heads, size_t *out_bytes)
+{
+    AttendParams p;
+    const qkvs_status_t st = attend_shape(layout, n_q_heads, &p);
+    if (st != QKVS_OK) return st;
+    if (!out_bytes) return QKVS_ERR_INVALID_ARG;
+    *out_bytes = attend_scratch_bytes(p);
+    return QKVS_OK;
+}
+
+qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qkvs_layout_t *layout, int32_t n_q_heads,
+                               const void *q_dev, float softmax_scale, float *out_dev, void *scratch_dev,
+                               size_t scratch_bytes, void *stream)
+{
+    constexpr int kAttendStages = 2, kAttendWarps = 4;
+    AttendParams p;
+    const qkvs_status_t st = attend_shape(layout, n_q_heads, &p);
+    if (st != QKVS_OK) return st;
+    if (!card_dev || !q_dev || !out_dev || !scratch_dev) return QKVS_ERR_INVALID_ARG;
+    if (!aligned16(card_dev) || !aligned16(q_dev) || !aligned16(out_dev) || !aligned16(scratch_dev)) return QKVS_ERR_INVALID_ARG;
+    if (card_bytes < (size_t)kHeaderBytes) return QKVS_ERR_BAD_CARD;
+    if (scratch_bytes < attend_scratch_bytes(p)) return QKVS_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(scratch_dev, 0, QKVS_WORKSPACE_BYTES, cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    p.card = static_cast<const uint8_t *>(card_dev);
+    p.card_bytes = card_bytes;
+    p.q = static_cast<const __half *>(q_dev);
+    p.scale_log2 = softmax_scale * 1.4426950408889634f;
+    p.out = out_dev;
+    p.status_dev = static_cast<int32_t *>(scratch_dev);
+    p.work_counter = static_cast<uint32_t *>(scratch_dev) + 1;
+    p.partials = reinterpret_cast<float *>(static_cast<uint8_t *>(scratch_dev) + QKVS_WORKSPACE_BYTES);
+    if (p.n_items > 0) {
+        auto kernel = attend_kernel<kAttendStages, kAttendWarps>;
+        const size_t smem = kAttendWarps * sizeof(AttendWarpSmem<kAttendStages>);
+        unsigned grid = 0;
+        if (persistent_grid<1000>(kernel, kAttendWarps * 32, smem, (int64_t)((p.n_items + kAttendWarps - 1) / kAttendWarps), &grid) !=
+            cudaSuccess)
+            return QKVS_ERR_CUDA;
+        kernel<<<grid, kAttendWarps * 32, smem, cs>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
+    }
+    const unsigned rows = (unsigned)p.n_layers * (unsigned)p.n_q_heads;
+    attend_merge_kernel<<<(rows + 3) / 4, 128, 0, cs>>>(p);
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 
 qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_card_header_t *out_host)

@@ -1,0 +1,156 @@
+"""Attention straight from the card: CUDA path against the oracle, through the C-ABI, on a B200.
+
+Tolerance.  Both sides use exactly the same reconstructed K^, V^ (FP16).  The CUDA path rounds
+the softmax weights to FP16 (relative 2^-11) before the tensor-core product with V^, accumulates
+in FP32 and uses the hardware exp2 (relative 2^-22); everything else is below that.  A convex
+combination of values with weights off by 2^-11 relative moves by at most 2^-11 * max|V^| (twice
+that when numerator and denominator are counted separately): the tests allow
+2^-9 * max|V^| of the head + 1e-6, a fourfold margin.
+"""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2605_03884_b200 as q
+from paper_2605_03884_b200 import build as qbuild
+from paper_2605_03884_b200 import workloads as wl
+from gpu_utils import padded_cache
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    qbuild.build()
+    q.load_library()
+
+
+def _gpu_attend(card_np, L, H, d, T, qh, scale=None, card_bytes=None):
+    import torch
+    lay = q.make_layout(L, H, d, T)
+    card = torch.from_numpy(np.ascontiguousarray(card_np)).cuda()
+    qd = torch.from_numpy(qh).cuda()
+    out = torch.full(qh.shape, 7.0, dtype=torch.float32, device="cuda")
+    scratch = torch.full((q.attend_scratch_size(lay, qh.shape[1]),), 0x5A, dtype=torch.uint8, device="cuda")
+    q.card_attend(card, lay, qd, out, scratch, softmax_scale=scale, card_bytes=card_bytes)
+    torch.cuda.synchronize()
+    status = int(scratch[:4].view(torch.int32).item())
+    return status, out.cpu().numpy()
+
+
+def _check(Ks, Vs, bits, L, H, d, T, nq, mode=0, scale=None, qscale=1.0, seed=0):
+    olay = oracle.make_layout(L, H, d, T, bits_mode=mode)
+    st, card = oracle.card_create(olay, Ks, Vs, bits)
+    assert st == oracle.OK
+    qh = wl.random_fp16((L, nq, d), 900 + seed, scale=qscale)
+    st, want = oracle.card_attend(card, olay, qh, softmax_scale=scale)
+    assert st == oracle.OK
+    status, got = _gpu_attend(card, L, H, d, T, qh, scale)
+    assert status == 0
+    # bound per (layer, KV head): the largest reconstructed value
+    Kr, Vr = [np.zeros_like(k) for k in Ks], [np.zeros_like(v) for v in Vs]
+    assert oracle.card_inject(card, olay, Kr, Vr) == oracle.OK
+    per_kv = nq // H
+    worst = 0.0
+    for l in range(L):
+        for j in range(nq):
+            vmax = float(np.abs(Vr[l][j // per_kv][:T, :d].astype(np.float64)).max()) if T else 0.0
+            err = float(np.abs(got[l, j] - want[l, j]).max())
+            assert err <= 2.0 ** -9 * vmax + 1e-6, (l, j, err, vmax)
+            worst = max(worst, err / (vmax + 1e-30))
+    return worst
+
+
+@pytest.mark.parametrize("T", [1, 15, 16, 17, 255, 256, 257, 1000])
+def test_mixed_bits_ragged_lengths(T):
+    L, H, d, nq = 2, 2, 128, 8
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=300 + T)
+    bits = wl.iid_bits(T, (0.3, 0.3, 0.2, 0.2), seed=T)
+    _check(Ks, Vs, bits, L, H, d, T, nq, seed=T)
+
+
+@pytest.mark.parametrize("b", [2, 4, 8, 16])
+def test_uniform_bits(b):
+    L, H, d, T, nq = 1, 2, 128, 700, 8
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=310 + b)
+    _check(Ks, Vs, np.full(T, b, np.uint8), L, H, d, T, nq, seed=b)
+
+
+@pytest.mark.parametrize("per_kv", [1, 2, 4, 8])
+def test_query_group_sizes(per_kv):
+    L, H, d, T = 2, 3, 128, 530
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=320 + per_kv)
+    bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), seed=per_kv)
+    _check(Ks, Vs, bits, L, H, d, T, H * per_kv, seed=per_kv)
+
+
+def test_sharp_and_flat_softmax():
+    L, H, d, T, nq = 1, 2, 128, 900, 8
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=330)
+    bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), seed=331)
+    _check(Ks, Vs, bits, L, H, d, T, nq, scale=1.0, qscale=2.0, seed=1)    # a few tokens take all the weight
+    _check(Ks, Vs, bits, L, H, d, T, nq, scale=1e-4, seed=2)                # nearly the mean of the values
+    _check(Ks, Vs, bits, L, H, d, T, nq, scale=0.0, seed=3)                 # exactly the mean
+
+
+def test_per_head_bits_mode():
+    L, H, d, T, nq = 2, 2, 128, 300, 4
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=340)
+    bits = np.concatenate([wl.iid_bits(T, (0.3, 0.3, 0.2, 0.2), 341 + s) for s in range(L * H)])
+    _check(Ks, Vs, bits, L, H, d, T, nq, mode=1, seed=4)
+
+
+def test_no_tokens_and_bad_arguments():
+    import torch
+    L, H, d, nq = 1, 2, 128, 4
+    olay = oracle.make_layout(L, H, d, 0, head_stride=d)
+    st, card = oracle.card_create(olay, [np.zeros((H, 1, d), np.float16)], [np.zeros((H, 1, d), np.float16)], np.zeros(0, np.uint8))
+    assert st == oracle.OK
+    status, got = _gpu_attend(card, L, H, d, 0, wl.random_fp16((L, nq, d), 1))
+    assert status == 0 and np.all(got == 0.0)
+    lay64 = q.make_layout(1, 2, 64, 16)
+    with pytest.raises(q.QkvsError) as e:
+        q.attend_scratch_size(lay64, 4)
+    assert e.value.status == q.binding.ERR_UNSUPPORTED_SHAPE
+    lay = q.make_layout(1, 2, 128, 16)
+    with pytest.raises(q.QkvsError) as e:
+        q.attend_scratch_size(lay, 3)
+    assert e.value.status == q.binding.ERR_INVALID_ARG
+    with pytest.raises(q.QkvsError) as e:
+        q.attend_scratch_size(lay, 32)       # 16 query heads per KV head
+    assert e.value.status == q.binding.ERR_UNSUPPORTED_SHAPE
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    st = q.card_attend(torch.zeros(4096, dtype=torch.uint8, device="cuda"), lay,
+                       torch.zeros((1, 4, 128), dtype=torch.float16, device="cuda"),
+                       torch.zeros((1, 4, 128), dtype=torch.float32, device="cuda"), small, check=False)
+    assert st == q.binding.ERR_BUFFER_TOO_SMALL
+
+
+def test_damaged_cards_give_zeros_and_a_status():
+    L, H, d, T, nq = 1, 2, 128, 100, 4
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=350)
+    bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 351)
+    olay = oracle.make_layout(L, H, d, T)
+    _, card = oracle.card_create(olay, Ks, Vs, bits)
+    hd = oracle.parse_header(card)
+    qh = wl.random_fp16((L, nq, d), 352)
+    for off, val in ((0, 0), (8, 3), (28, 99), (hd["bits_off"] + 10, 3), (hd["offs_off"] + 80, card[hd["offs_off"] + 80] ^ 0x10)):
+        c = card.copy()
+        c[off] = val
+        status, got = _gpu_attend(c, L, H, d, T, qh)
+        assert status == q.binding.ERR_BAD_CARD
+        assert np.all(got == 0.0)
+    status, got = _gpu_attend(card, L, H, d, T, qh, card_bytes=card.size - 16)
+    assert status == q.binding.ERR_BAD_CARD and np.all(got == 0.0)
+
+
+@pytest.mark.parametrize("number", [3, 4])
+def test_full_size_llama_8k(number):
+    """The benchmark's size and launch configuration: 32 layers, 8 KV heads, 32 query heads, 8192 tokens."""
+    w = wl.WORKLOADS[number]
+    Ks, Vs = [], []
+    for _, k, v in wl.kv_layers(w):
+        Ks.append(k)
+        Vs.append(v)
+    worst = _check(Ks, Vs, wl.bits_for(w), w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens, 32, seed=number)
+    assert worst <= 2.0 ** -9
