@@ -55,6 +55,7 @@ struct AttendWarpSmem {
     uint32_t info[NS][kAttendRows];  // per token: record offset inside the span << 8 | bit-width
     alignas(8) uint64_t full[NS];
     int32_t rows[NS];                // 0 when the step's table entries did not check out
+    uint32_t uniform_bits[NS];       // bit-width shared by all 16 rows, else 0
 };
 
 __device__ __forceinline__ void mma_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -77,6 +78,55 @@ __device__ __forceinline__ uint32_t word_of(const uint4 &v, int i)
     return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
 }
 
+// N consecutive chunks (pos0 .. pos0 + N - 1, all inside one group of a row whose record is `rec`)
+// -> N x 8 FP16 values, bit for bit what injection reconstructs.  With the bit-width B known at
+// compile time the group's scale / zero pair and its codes are fetched once for the whole run;
+// B = 0 decodes chunk by chunk with the row's own width `b`.
+template <int B, int N>
+__device__ __forceinline__ void decode_run(const uint8_t *rec, int b, int pos0, uint4 (&out)[N])
+{
+    constexpr int G = kAttendD / kGroup;
+    if (B == 0) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) out[i] = decode_chunk<kAttendD, 0>(rec, b, pos0 + i);
+        return;
+    }
+    if (B == 16) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) out[i] = *reinterpret_cast<const uint4 *>(rec + (pos0 + i) * 16);
+        return;
+    }
+    const float2 m = *reinterpret_cast<const float2 *>(rec + (pos0 >> 2) * kMetaBytesPerGroup);
+    const Dequant dq = make_dequant(m.x, m.y);
+    const uint8_t *codes = rec + G * kMetaBytesPerGroup + pos0 * B;  // N * B bytes, aligned to their size
+    uint32_t w[N * B / 4 > 0 ? N * B / 4 : 1];
+    if (N * B == 32) {
+        const uint4 a = *reinterpret_cast<const uint4 *>(codes), c = *reinterpret_cast<const uint4 *>(codes + 16);
+        w[0] = a.x, w[1] = a.y, w[2] = a.z, w[3] = a.w, w[4] = c.x, w[5] = c.y, w[6] = c.z, w[7] = c.w;
+    } else if (N * B == 16) {
+        const uint4 a = *reinterpret_cast<const uint4 *>(codes);
+        w[0] = a.x, w[1] = a.y, w[2] = a.z, w[3] = a.w;
+    } else if (N * B == 8) {
+        const uint2 a = *reinterpret_cast<const uint2 *>(codes);
+        w[0] = a.x, w[1] = a.y;
+    } else {
+        w[0] = *reinterpret_cast<const uint32_t *>(codes);
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        uint32_t lo, hi;
+        if (B == 8) {
+            lo = w[2 * i];
+            hi = w[2 * i + 1];
+        } else if (B == 4) {
+            unpack_nibbles(w[i], lo, hi);
+        } else {
+            unpack_nibbles(unpack_crumbs((w[i >> 1] >> (16 * (i & 1))) & 0xffffu), lo, hi);
+        }
+        out[i] = dequantize_chunk(lo, hi, dq);
+    }
+}
+
 // Checks a step's table entries, publishes the per-token record positions and starts the copies
 // of its K and V spans (same offsets, two streams).  All lanes call it.
 template <int NS>
@@ -94,11 +144,14 @@ __device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, 
         sm.info[stage][lane] = ((t.off - off0) << 8) | (t.bits & 0xffu);
     }
     bad = __any_sync(0xffffffffu, bad);
+    const uint32_t b0 = __shfl_sync(0xffffffffu, t.bits, 0);
+    const bool uniform = rows == kAttendRows && __all_sync(0xffffffffu, lane >= rows || t.bits == b0);
     const uint32_t span = off_end - off0;  // consistent records: at most rows * 256 bytes, fits the stage
     bad |= (off0 & 15u) != 0u || base_k < sec.payload_off || base_v < sec.payload_off || ((base_k | base_v) & 15u) != 0u ||
            base_k + (uint64_t)off_end > total_bytes || base_v + (uint64_t)off_end > total_bytes;
     if (lane == 0) {
         sm.rows[stage] = bad ? 0 : rows;
+        sm.uniform_bits[stage] = uniform ? b0 : 0u;
         if (bad && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
         if (!bad && span) {
             mbar_arrive_expect_tx(&sm.full[stage], 2u * span);
@@ -109,6 +162,93 @@ __device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, 
         }
     }
     __syncwarp();
+}
+
+// One step: 16 tokens of K and V staged in `stage` against the group's queries.  Updates the
+// running maximum / sum of head g and the output accumulators.  B is the bit-width shared by all
+// 16 rows, or 0 when they differ or the step is short.
+template <int NS, int B>
+__device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int stage, int rows, int gid, int tig, float scale_log2,
+                                            const uint32_t (&qa0)[8], const uint32_t (&qa2)[8], float &m_run, float &l_run,
+                                            float (&acc)[8][4])
+{
+    // ---- scores of 2 x 8 tokens for the heads of the group
+    float sacc[2][4];
+#pragma unroll
+    for (int bi = 0; bi < 2; ++bi) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sacc[bi][i] = 0.0f;
+        const int tok = 8 * bi + gid;
+        uint4 kq[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) kq[c] = make_uint4(0, 0, 0, 0);  // lanes without a token feed zeros
+        if (tok < rows) {
+            const uint32_t inf = sm.info[stage][tok];
+            const uint8_t *rec = sm.k[stage] + (inf >> 8);
+            decode_run<B, 4>(rec, (int)(inf & 0xffu), 4 * tig, kq);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {  // the whole warp executes every mma together
+            mma_m16n8k16(sacc[bi], qa0[2 * c], 0u, qa2[2 * c], 0u, kq[c].x, kq[c].y);
+            mma_m16n8k16(sacc[bi], qa0[2 * c + 1], 0u, qa2[2 * c + 1], 0u, kq[c].z, kq[c].w);
+        }
+    }
+    // ---- running softmax for head g over tokens 8bi + 2t + e
+    float x[2][2];
+    float m_loc = -INFINITY;
+#pragma unroll
+    for (int bi = 0; bi < 2; ++bi)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            x[bi][e] = (8 * bi + 2 * tig + e) < rows ? sacc[bi][e] * scale_log2 : -INFINITY;
+            m_loc = fmaxf(m_loc, x[bi][e]);
+        }
+    m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 1));
+    m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 2));
+    const float m_new = fmaxf(m_run, m_loc);
+    const float m_ref = m_new == -INFINITY ? 0.0f : m_new;
+    const float alpha = exp2_approx(m_run - m_ref);  // 0 on the first tokens of the item
+    float pr[2][2];
+#pragma unroll
+    for (int bi = 0; bi < 2; ++bi)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) pr[bi][e] = exp2_approx(x[bi][e] - m_ref);
+    l_run = l_run * alpha + (pr[0][0] + pr[0][1]) + (pr[1][0] + pr[1][1]);
+    m_run = m_new;
+    const uint32_t pb0 = as_u32(__floats2half2_rn(pr[0][0], pr[0][1]));
+    const uint32_t pb1 = as_u32(__floats2half2_rn(pr[1][0], pr[1][1]));
+    // the accumulators of this lane belong to heads 2t and 2t + 1, whose factors other lanes hold
+    const float a_lo = __shfl_sync(0xffffffffu, alpha, 8 * tig);
+    const float a_hi = __shfl_sync(0xffffffffu, alpha, 8 * tig + 4);
+    if (__any_sync(0xffffffffu, a_lo != 1.0f || a_hi != 1.0f)) {
+#pragma unroll
+        for (int mb = 0; mb < 8; ++mb) {
+            acc[mb][0] *= a_lo;
+            acc[mb][1] *= a_hi;
+            acc[mb][2] *= a_lo;
+            acc[mb][3] *= a_hi;
+        }
+    }
+    // ---- values: channels 16g .. 16g+15 of tokens 2t, 2t+1, 2t+8, 2t+9
+    uint4 vq[4][2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int tok = 2 * tig + (i & 1) + 8 * (i >> 1);
+        vq[i][0] = make_uint4(0, 0, 0, 0);
+        vq[i][1] = make_uint4(0, 0, 0, 0);
+        if (tok < rows) {
+            const uint32_t inf = sm.info[stage][tok];
+            const uint8_t *rec = sm.v[stage] + (inf >> 8);
+            decode_run<B, 2>(rec, (int)(inf & 0xffu), 2 * gid, vq[i]);
+        }
+    }
+#pragma unroll
+    for (int mb = 0; mb < 8; ++mb) {
+        const uint32_t wa = word_of(vq[0][mb >> 2], mb & 3), wb = word_of(vq[1][mb >> 2], mb & 3);
+        const uint32_t wc = word_of(vq[2][mb >> 2], mb & 3), wd = word_of(vq[3][mb >> 2], mb & 3);
+        mma_m16n8k16(acc[mb], __byte_perm(wa, wb, 0x5410), __byte_perm(wa, wb, 0x7632), __byte_perm(wc, wd, 0x5410),
+                     __byte_perm(wc, wd, 0x7632), pb0, pb1);
+    }
 }
 
 template <int NS, int WARPS>
@@ -221,84 +361,12 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             if (!ok) break;
             const int rows = sm.rows[stage];
 
-            // ---- scores of 2 x 8 tokens for the heads of the group
-            float sacc[2][4];
-#pragma unroll
-            for (int bi = 0; bi < 2; ++bi) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) sacc[bi][i] = 0.0f;
-                const int tok = 8 * bi + gid;
-                uint4 kq[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) kq[c] = make_uint4(0, 0, 0, 0);  // lanes without a token feed zeros
-                if (tok < rows) {
-                    const uint32_t inf = sm.info[stage][tok];
-                    const uint8_t *rec = sm.k[stage] + (inf >> 8);
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) kq[c] = decode_chunk<kAttendD, 0>(rec, (int)(inf & 0xffu), 4 * tig + c);
-                }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {  // the whole warp executes every mma together
-                    mma_m16n8k16(sacc[bi], qa0[2 * c], 0u, qa2[2 * c], 0u, kq[c].x, kq[c].y);
-                    mma_m16n8k16(sacc[bi], qa0[2 * c + 1], 0u, qa2[2 * c + 1], 0u, kq[c].z, kq[c].w);
-                }
-            }
-            // ---- running softmax for head g over tokens 8bi + 2t + e
-            float x[2][2];
-            float m_loc = -INFINITY;
-#pragma unroll
-            for (int bi = 0; bi < 2; ++bi)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    x[bi][e] = (8 * bi + 2 * tig + e) < rows ? sacc[bi][e] * p.scale_log2 : -INFINITY;
-                    m_loc = fmaxf(m_loc, x[bi][e]);
-                }
-            m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 1));
-            m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 2));
-            const float m_new = fmaxf(m_run, m_loc);
-            const float m_ref = m_new == -INFINITY ? 0.0f : m_new;
-            const float alpha = exp2_approx(m_run - m_ref);  // 0 on the first tokens of the item
-            float pr[2][2];
-#pragma unroll
-            for (int bi = 0; bi < 2; ++bi)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) pr[bi][e] = exp2_approx(x[bi][e] - m_ref);
-            l_run = l_run * alpha + (pr[0][0] + pr[0][1]) + (pr[1][0] + pr[1][1]);
-            m_run = m_new;
-            const uint32_t pb0 = as_u32(__floats2half2_rn(pr[0][0], pr[0][1]));
-            const uint32_t pb1 = as_u32(__floats2half2_rn(pr[1][0], pr[1][1]));
-            // the accumulators of this lane belong to heads 2t and 2t + 1, whose factors other lanes hold
-            const float a_lo = __shfl_sync(0xffffffffu, alpha, 8 * tig);
-            const float a_hi = __shfl_sync(0xffffffffu, alpha, 8 * tig + 4);
-            if (__any_sync(0xffffffffu, a_lo != 1.0f || a_hi != 1.0f)) {
-#pragma unroll
-                for (int mb = 0; mb < 8; ++mb) {
-                    acc[mb][0] *= a_lo;
-                    acc[mb][1] *= a_hi;
-                    acc[mb][2] *= a_lo;
-                    acc[mb][3] *= a_hi;
-                }
-            }
-            // ---- values: channels 16g .. 16g+15 of tokens 2t, 2t+1, 2t+8, 2t+9
-            uint4 vq[4][2];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int tok = 2 * tig + (i & 1) + 8 * (i >> 1);
-                vq[i][0] = make_uint4(0, 0, 0, 0);
-                vq[i][1] = make_uint4(0, 0, 0, 0);
-                if (tok < rows) {
-                    const uint32_t inf = sm.info[stage][tok];
-                    const uint8_t *rec = sm.v[stage] + (inf >> 8);
-                    vq[i][0] = decode_chunk<kAttendD, 0>(rec, (int)(inf & 0xffu), 2 * gid);
-                    vq[i][1] = decode_chunk<kAttendD, 0>(rec, (int)(inf & 0xffu), 2 * gid + 1);
-                }
-            }
-#pragma unroll
-            for (int mb = 0; mb < 8; ++mb) {
-                const uint32_t wa = word_of(vq[0][mb >> 2], mb & 3), wb = word_of(vq[1][mb >> 2], mb & 3);
-                const uint32_t wc = word_of(vq[2][mb >> 2], mb & 3), wd = word_of(vq[3][mb >> 2], mb & 3);
-                mma_m16n8k16(acc[mb], __byte_perm(wa, wb, 0x5410), __byte_perm(wa, wb, 0x7632), __byte_perm(wc, wd, 0x5410),
-                             __byte_perm(wc, wd, 0x7632), pb0, pb1);
+            switch (sm.uniform_bits[stage]) {  // all 16 rows of one width: the specialised body
+                case 4: attend_step<NS, 4>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
+                case 2: attend_step<NS, 2>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
+                case 8: attend_step<NS, 8>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
+                case 16: attend_step<NS, 16>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
+                default: attend_step<NS, 0>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
             }
             __syncwarp();  // every lane has read the stage: it can be re-armed
             if (issued < n_steps) {
