@@ -324,6 +324,29 @@ def run_ours(args):
     torch.cuda.synchronize()
     clocks = sampler.stop(t_wall_begin, time.time()) if rank == 0 else None
 
+    # attention straight from the card (the row after the hot path): one decode step, 32 query
+    # heads, over the card the last create left behind; reported beside the main metric
+    attend = None
+    if d == 128 and not args.skip_attend:
+        n_q = 4 * H
+        qd = torch.randn((L, n_q, d), device="cuda").half()
+        od = torch.zeros((L, n_q, d), dtype=torch.float32, device="cuda")
+        scratch = torch.zeros(q.attend_scratch_size(lay, n_q), dtype=torch.uint8, device="cuda")
+        ev = []
+        for _ in range(25):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            q.card_attend(card, lay, qd, od, scratch, card_bytes=sizes[-1], stream=stream)
+            b.record(stream)
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        if int(scratch[:4].view(torch.int32).item()) != 0:
+            raise RuntimeError("attention from the card reported a bad card")
+        a_ms = statistics.median(x.elapsed_time(y) for x, y in ev[5:])
+        payload = sizes[-1] - prefix
+        attend = {"what": "decode-step attention straight from the card, all layers, 4 query heads per KV head",
+                  "ms": a_ms, "card_payload_bytes": payload, "card_gbs": payload / (a_ms * 1e-3) / 1e9}
+
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device="cuda")
 
     if rank != 0:
@@ -384,7 +407,10 @@ def run_ours(args):
                 "ms_per_step": None if args.skip_e2e else e2e_ms / args.steps},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
+        "attend_from_card": attend,
     }
+    if attend is not None:
+        attend["hbm_frac"] = attend["card_gbs"] / peak
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -399,6 +425,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
+    ap.add_argument("--skip-attend", action="store_true", help="skip the attention-from-the-card measurement")
     ap.add_argument("--layers", type=int, default=0,
                     help="reduced case for profiler captures: keep the workload's recipe at this many layers")
     args = ap.parse_args()
