@@ -78,6 +78,8 @@ def lib():
                                             C.c_uint64, C.c_int64, C.c_void_p, C.c_uint64, C.c_int64, C.c_int64]
         l.orc_card_inject.restype = C.c_int
         l.orc_card_inject.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_void_p, C.c_void_p, C.c_int64]
+        l.orc_bits_from_scores.restype = C.c_int
+        l.orc_bits_from_scores.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]
         l.orc_card_attend.restype = C.c_int
         l.orc_card_attend.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_int, C.c_void_p, C.c_double, C.c_void_p]
         l.orc_num_threads.restype = C.c_int
@@ -242,6 +244,14 @@ def card_attend(card: np.ndarray, layout: Layout, q: np.ndarray, softmax_scale: 
     out = np.zeros(q.shape, dtype=np.float64)
     st = lib().orc_card_attend(_ptr(card), card.size, C.byref(layout), q.shape[1], _ptr(q), scale, _ptr(out))
     return st, out
+
+
+def bits_from_scores(scores: np.ndarray, n_fp16: int, n_8bit: int, n_4bit: int) -> Tuple[int, np.ndarray]:
+    """Per-token bit-widths from float32 scores [T] by rank (see orc_bits_from_scores)."""
+    scores = np.ascontiguousarray(scores, dtype=np.float32)
+    bits = np.zeros(scores.size, dtype=np.uint8)
+    st = lib().orc_bits_from_scores(_ptr(scores), scores.size, n_fp16, n_8bit, n_4bit, _ptr(bits))
+    return st, bits
 
 
 def num_threads() -> int:

@@ -609,6 +609,46 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
     return failed ? ORC_INVALID_ARG : ORC_OK;
 }
 
+/* Bit-width assignment from per-token importance scores, the step in front of card creation
+ * (Section 3.3: tokens that matter more get more bits, under a budget; Section 4.1.2: the
+ * controller outputs b(t) in {2, 4, 8, 16}).  The paper's controller is a trained network that is
+ * not available; what is restated here is the rank rule of the benchmark's adaptive
+ * configuration: order the tokens by score, highest first, equal scores by lower token index
+ * first; the first n_fp16 tokens keep FP16, the next n_8bit get 8 bits, the next n_4bit get
+ * 4 bits, all others 2 bits.  Plain sort on (score descending, index ascending). */
+typedef struct { float score; int64_t index; } orc_ranked;
+
+static int ranked_before(const void *a, const void *b)
+{
+    const orc_ranked *x = (const orc_ranked *)a, *y = (const orc_ranked *)b;
+    if (x->score > y->score) return -1;
+    if (x->score < y->score) return 1;
+    return x->index < y->index ? -1 : (x->index > y->index ? 1 : 0);
+}
+
+int orc_bits_from_scores(const float *scores, int64_t n_tokens, int64_t n_fp16, int64_t n_8bit,
+                         int64_t n_4bit, uint8_t *bits)
+{
+    if (n_tokens < 0 || n_fp16 < 0 || n_8bit < 0 || n_4bit < 0 || n_fp16 + n_8bit + n_4bit > n_tokens)
+        return ORC_INVALID_ARG;
+    orc_ranked *r = (orc_ranked *)malloc(sizeof(orc_ranked) * (size_t)(n_tokens > 0 ? n_tokens : 1));
+    if (!r) return ORC_INVALID_ARG;
+    for (int64_t t = 0; t < n_tokens; ++t) {
+        r[t].score = scores[t];
+        r[t].index = t;
+    }
+    qsort(r, (size_t)n_tokens, sizeof(orc_ranked), ranked_before);
+    for (int64_t k = 0; k < n_tokens; ++k) {
+        uint8_t b = 2;
+        if (k < n_fp16) b = 16;
+        else if (k < n_fp16 + n_8bit) b = 8;
+        else if (k < n_fp16 + n_8bit + n_4bit) b = 4;
+        bits[r[k].index] = b;
+    }
+    free(r);
+    return ORC_OK;
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP

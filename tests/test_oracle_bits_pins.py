@@ -1,0 +1,70 @@
+"""Pins of the oracle's rank-based bit-width assignment (CPU only): class counts, order
+property, tie rule, brute-force ranks on small inputs, the library sort, and the counts the
+adaptive benchmark configuration fixes (410 / 1228 / 3277 / 3277 of 8192 tokens)."""
+import numpy as np
+import pytest
+
+import oracle
+from golden_io import read_fixture
+from paper_2605_03884_b200 import workloads as wl
+
+
+def _cuts(T):
+    c16 = int(np.floor(0.05 * T + 0.5)); c8 = int(np.floor(0.20 * T + 0.5)); c4 = int(np.floor(0.60 * T + 0.5))
+    return c16, c8 - c16, c4 - c8
+
+
+def test_counts_of_the_adaptive_configuration():
+    T = 8192
+    scores = np.random.default_rng(1007).lognormal(0.0, 1.0, size=T).astype(np.float32)
+    n16, n8, n4 = _cuts(T)
+    assert (n16, n8, n4, T - n16 - n8 - n4) == (410, 1228, 3277, 3277)
+    st, bits = oracle.bits_from_scores(scores, n16, n8, n4)
+    assert st == oracle.OK
+    assert [(bits == b).sum() for b in (16, 8, 4, 2)] == [410, 1228, 3277, 3277]
+    assert bits.astype(np.float64).mean() == pytest.approx(4.40, abs=0.005)
+
+
+@pytest.mark.parametrize("T", [1, 2, 7, 64, 1000])
+def test_higher_scores_never_get_fewer_bits_and_counts_hold(T):
+    scores = np.random.default_rng(T).standard_normal(T).astype(np.float32)
+    n16, n8, n4 = _cuts(T)
+    st, bits = oracle.bits_from_scores(scores, n16, n8, n4)
+    assert st == oracle.OK
+    assert (bits == 16).sum() == n16 and (bits == 8).sum() == n8 and (bits == 4).sum() == n4
+    order = np.argsort(-scores, kind="stable")
+    assert np.all(np.diff(bits[order].astype(int)) <= 0)
+
+
+def test_brute_force_rank_with_many_ties():
+    T = 300
+    scores = np.random.default_rng(5).integers(0, 6, size=T).astype(np.float32)   # six levels only
+    n16, n8, n4 = 31, 77, 101
+    st, bits = oracle.bits_from_scores(scores, n16, n8, n4)
+    assert st == oracle.OK
+    for t in range(T):
+        rank = int((scores > scores[t]).sum() + (scores[:t] == scores[t]).sum())
+        want = 16 if rank < n16 else 8 if rank < n16 + n8 else 4 if rank < n16 + n8 + n4 else 2
+        assert bits[t] == want
+
+
+def test_equal_scores_favour_the_lower_index():
+    st, bits = oracle.bits_from_scores(np.zeros(10, np.float32), 2, 3, 1)
+    assert st == oracle.OK and bits.tolist() == [16, 16, 8, 8, 8, 4, 2, 2, 2, 2]
+
+
+def test_matches_the_library_sort_of_the_workload_generator():
+    """Same rule as workloads.quantile_bits (numpy lexsort), on scores that are exact in float32."""
+    T = 4096
+    scores = np.random.default_rng(77).lognormal(0.0, 1.0, size=T).astype(np.float32)
+    order = np.lexsort((np.arange(T), -scores.astype(np.float64)))
+    n16, n8, n4 = _cuts(T)
+    want = np.empty(T, np.uint8)
+    want[order[:n16]] = 16; want[order[n16:n16 + n8]] = 8; want[order[n16 + n8:n16 + n8 + n4]] = 4; want[order[n16 + n8 + n4:]] = 2
+    st, bits = oracle.bits_from_scores(scores, n16, n8, n4)
+    assert st == oracle.OK and np.array_equal(bits, want)
+
+
+def test_bad_counts_are_rejected():
+    st, _ = oracle.bits_from_scores(np.zeros(4, np.float32), 3, 2, 0)
+    assert st == oracle.INVALID_ARG
