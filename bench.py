@@ -440,6 +440,22 @@ def run_ours(args):
     if not args.no_cpu_baseline:
         cpu = cpu_oracle_leg(w, Ks, Vs, bits_per_hop[0], L)
 
+    # the step in front of the path: bit-widths from importance scores by rank (config 4's recipe)
+    rank_us = None
+    if not args.skip_attend:
+        sc = torch.randn(T, device="cuda").exp()
+        bd = torch.zeros(T, dtype=torch.uint8, device="cuda")
+        c16, c8, c4 = int(0.05 * T + 0.5), int(0.20 * T + 0.5), int(0.60 * T + 0.5)
+        ev = []
+        for _ in range(25):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            q.bits_from_scores(sc, c16, c8 - c16, c4 - c8, bd, stream=stream)
+            b.record(stream)
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        rank_us = statistics.median(x.elapsed_time(y) for x, y in ev[5:]) * 1e3
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -462,6 +478,7 @@ def run_ours(args):
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
         "attend_from_card": attend,
+        "bits_from_scores_us": rank_us,
     }
     if attend is not None:
         attend["hbm_frac"] = attend["card_gbs"] / peak

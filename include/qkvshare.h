@@ -131,6 +131,19 @@ QKVS_API qkvs_status_t qkvs_card_size(const qkvs_layout_t *layout, const uint8_t
  * hold at least this much for qkvs_card_create to start.  Host only. */
 QKVS_API qkvs_status_t qkvs_card_prefix_size(const qkvs_layout_t *layout, size_t *out_bytes);
 
+/* Bit-widths from importance scores (the step in front of card creation; Section 3.3: tokens
+ * that matter more get more bits; Section 4.1.2: b(t) in {2, 4, 8, 16}).  The paper's controller
+ * is a trained network; this is the rank rule of an adaptive budget: order the tokens of a
+ * segment by score, highest first, equal scores by lower token index first; the first n_fp16 keep
+ * FP16, the next n_8bit get 8 bits, the next n_4bit get 4 bits, the rest 2 bits.
+ *   scores_dev   device float32 [n_segments][n_tokens], finite values
+ *   bits_dev     device uint8  [n_segments][n_tokens]: ready to be passed to qkvs_card_create
+ *                (n_segments = 1 for bits_mode 0, n_layers * n_kv_heads for bits_mode 1)
+ * The result is exact (integer ranks).  n_tokens up to 2^20.  Asynchronous on `stream`. */
+QKVS_API qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_segments,
+                                    int32_t n_tokens, int32_t n_fp16, int32_t n_8bit,
+                                    int32_t n_4bit, uint8_t *bits_dev, void *stream);
+
 /* Card creation (Section 4.2.1): offset scan over the bit-widths, then fused
  * min/max -> scale/zero -> quantise -> bit-pack of every (layer, K|V, head) stream.
  *   K_layers, V_layers  HOST arrays of n_layers DEVICE pointers to FP16 blocks (16-byte aligned)

@@ -51,7 +51,7 @@ assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
            "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_attend_scratch_size", "qkvs_card_attend",
-           "qkvs_card_info", "qkvs_selftest_division", "qkvs_status_string",
+           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_selftest_division", "qkvs_status_string",
            "qkvs_version")
 
 _lib = None
@@ -85,6 +85,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_attend_scratch_size.argtypes = [C.POINTER(Layout), C.c_int32, C.POINTER(C.c_size_t)]
     lib.qkvs_card_attend.restype = C.c_int
     lib.qkvs_card_attend.argtypes = [vp, C.c_size_t, C.POINTER(Layout), C.c_int32, vp, C.c_float, vp, vp, C.c_size_t, vp]
+    lib.qkvs_bits_from_scores.restype = C.c_int
+    lib.qkvs_bits_from_scores.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp]
     lib.qkvs_card_info.restype = C.c_int
     lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
     lib.qkvs_selftest_division.restype = C.c_int
@@ -254,6 +256,18 @@ def card_attend(card_dev, layout: Layout, q_dev, out_dev, scratch_dev, softmax_s
                                          int(scratch_dev.numel() * scratch_dev.element_size()), _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_card_attend")
+    return st
+
+
+def bits_from_scores(scores_dev, n_fp16: int, n_8bit: int, n_4bit: int, bits_dev, stream=None, check: bool = True) -> int:
+    """qkvs_bits_from_scores.  scores_dev: CUDA float32 [T] or [n_segments, T]; bits_dev: CUDA uint8
+    of the same shape."""
+    n_seg = 1 if scores_dev.dim() == 1 else int(scores_dev.shape[0])
+    n_tok = int(scores_dev.shape[-1])
+    st = load_library().qkvs_bits_from_scores(int(scores_dev.data_ptr()), n_seg, n_tok, int(n_fp16), int(n_8bit),
+                                              int(n_4bit), int(bits_dev.data_ptr()), _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_bits_from_scores")
     return st
 
 

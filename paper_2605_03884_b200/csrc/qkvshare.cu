@@ -254,6 +254,47 @@ __global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Bit-widths from importance scores by rank (the step in front of the offset scan).
+// rank(t) = #{s : score_s > score_t} + #{s < t : score_s == score_t}; the first n16 ranks keep
+// FP16, the next n8 get 8 bits, the next n4 get 4 bits, the rest 2 bits.  Exact and order-free:
+// every token counts for itself.  A CTA ranks 64 tokens, four threads per token, each thread
+// against a quarter of every 1024-score tile staged in shared memory.
+
+constexpr int kRankThreads = 256;
+constexpr int kRankTile = 1024;
+
+__global__ void __launch_bounds__(kRankThreads) bits_from_scores_kernel(const float *scores, int64_t T, uint32_t n16,
+                                                                        uint32_t n8, uint32_t n4, uint8_t *bits)
+{
+    __shared__ __align__(16) float tile[kRankTile];
+    scores += (int64_t)blockIdx.y * T;
+    bits += (int64_t)blockIdx.y * T;
+    const int part = threadIdx.x & 3;
+    const int64_t t = (int64_t)blockIdx.x * (kRankThreads / 4) + (threadIdx.x >> 2);
+    const float mine = t < T ? scores[t] : 0.0f;
+    uint32_t rank = 0;
+    for (int64_t base = 0; base < T; base += kRankTile) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < kRankTile; i += kRankThreads) tile[i] = base + i < T ? scores[base + i] : -INFINITY;
+        __syncthreads();
+        // padding is -inf and sits behind every real index, so it never counts
+        const int64_t first = base + part * (kRankTile / 4);
+#pragma unroll 4
+        for (int i = 0; i < kRankTile / 4; i += 4) {
+            const float4 s = *reinterpret_cast<const float4 *>(&tile[part * (kRankTile / 4) + i]);
+            const int64_t idx = first + i;
+            rank += (s.x > mine) || (s.x == mine && idx < t);
+            rank += (s.y > mine) || (s.y == mine && idx + 1 < t);
+            rank += (s.z > mine) || (s.z == mine && idx + 2 < t);
+            rank += (s.w > mine) || (s.w == mine && idx + 3 < t);
+        }
+    }
+    rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+    rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+    if (part == 0 && t < T) bits[t] = rank < n16 ? 16 : (rank < n16 + n8 ? 8 : (rank < n16 + n8 + n4 ? 4 : 2));
+}
+
+// ---------------------------------------------------------------------------------------------
 // Self-test of the two division shortcuts against the IEEE division, over every range value the
 // path can produce (binary32 values from 2^-24 to 131008) and the three qmax values.
 
@@ -750,6 +791,20 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
     }
     const unsigned rows = (unsigned)p.n_layers * (unsigned)p.n_q_heads;
     attend_merge_kernel<<<(rows + 3) / 4, 128, 0, cs>>>(p);
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+}
+
+qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_segments, int32_t n_tokens, int32_t n_fp16,
+                                    int32_t n_8bit, int32_t n_4bit, uint8_t *bits_dev, void *stream)
+{
+    if (n_segments < 1 || n_tokens < 0 || n_fp16 < 0 || n_8bit < 0 || n_4bit < 0) return QKVS_ERR_INVALID_ARG;
+    if ((int64_t)n_fp16 + n_8bit + n_4bit > n_tokens) return QKVS_ERR_INVALID_ARG;
+    if (n_tokens > (1 << 20) || n_segments > 65535) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (n_tokens == 0) return QKVS_OK;
+    if (!scores_dev || !bits_dev || (reinterpret_cast<uintptr_t>(scores_dev) & 3u)) return QKVS_ERR_INVALID_ARG;
+    const dim3 grid((unsigned)((n_tokens + kRankThreads / 4 - 1) / (kRankThreads / 4)), (unsigned)n_segments);
+    bits_from_scores_kernel<<<grid, kRankThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        scores_dev, n_tokens, (uint32_t)n_fp16, (uint32_t)n_8bit, (uint32_t)n_4bit, bits_dev);
     return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 

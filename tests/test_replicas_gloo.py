@@ -37,7 +37,7 @@ def _rank_main(rank, world, port, out):
 
 def test_two_replicas_report_the_slowest_rank_and_the_sum_of_the_work():
     world = 2
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_rank_main, args=(world, _free_port(), out), nprocs=world, join=True)
         res = dict(out)
