@@ -525,16 +525,36 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
     return ORC_OK;
 }
 
+/* The values a record stands for, as real numbers: code * scale + zero for a quantised row,
+ * the FP16 values themselves for a 16-bit row.  No rounding to FP16: that rounding belongs to
+ * injection, which has to hand an FP16 cache to the receiving framework (Section 4.2.2); attention
+ * that reads the card itself (Section 4.3) has no FP16 copy to round into. */
+static void reconstruct_record(const uint8_t *rec, int d, int b, double *row)
+{
+    if (b == 16) {
+        for (int i = 0; i < d; ++i) row[i] = (double)orc_half_to_float((uint16_t)(rec[2 * i] | (rec[2 * i + 1] << 8)));
+        return;
+    }
+    int G = d / 32;
+    uint8_t q[32];
+    for (int g = 0; g < G; ++g) {
+        double scale = (double)get_f32(rec + 8 * g);
+        double zero = (double)get_f32(rec + 8 * g + 4);
+        orc_unpack_codes(rec + 8 * G + (size_t)g * 32 * b / 8, 32, b, q);
+        for (int i = 0; i < 32; ++i) row[32 * g + i] = (double)q[i] * scale + zero;
+    }
+}
+
 /* Decode-step attention straight from a card, without rebuilding the FP16 cache
  * (Section 4.3: consuming a foreign quantised cache directly inside attention is the paper's
  * stated goal; Section 3.1 for K, V per layer and head).  One new token per layer attends to all
  * n_tokens of the card.  Query head j of a layer reads KV head j / (n_q_heads / n_kv_heads)
  * (grouped-query attention; the paper's model, Llama-3.1-8B, has 32 query and 8 KV heads):
- *     s_t  = softmax_scale * sum_c q[j][c] * K^[t][c]
+ *     s_t  = softmax_scale * sum_c q[j][c] * K~[t][c]
  *     p_t  = exp(s_t - max_t s_t) / sum_t exp(s_t - max_t s_t)
- *     o[c] = sum_t p_t * V^[t][c]
- * where K^, V^ are exactly the FP16 values injection reconstructs.  The paper gives no formula
- * for this step; this is the textbook definition, evaluated in double precision.
+ *     o[c] = sum_t p_t * V~[t][c]
+ * where K~, V~ are the values the records stand for (reconstruct_record).  The paper gives no
+ * formula for this step; this is the textbook definition, evaluated in double precision.
  *   q    [n_layers][n_q_heads][head_dim] FP16 bit patterns
  *   out  [n_layers][n_q_heads][head_dim] double */
 int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *L, int n_q_heads,
@@ -567,8 +587,8 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
         const int64_t seg = segment_of(&C, l, h);
         const uint8_t *bits = card + bo + (uint64_t)seg * (uint64_t)T;
         const uint32_t *off = (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1));
-        uint16_t *kx = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)T * (size_t)d);
-        uint16_t *vx = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)T * (size_t)d);
+        double *kx = (double *)malloc(sizeof(double) * (size_t)T * (size_t)d);
+        double *vx = (double *)malloc(sizeof(double) * (size_t)T * (size_t)d);
         double *s = (double *)malloc(sizeof(double) * (size_t)T);
         if (!kx || !vx || !s) {
             failed = 1;
@@ -577,8 +597,12 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
             free(s);
             continue;
         }
-        orc_decode_stream(card + stream_base(card, &C, stream_index(&C, l, 0, h)), bits, off, T, d, kx, d);
-        orc_decode_stream(card + stream_base(card, &C, stream_index(&C, l, 1, h)), bits, off, T, d, vx, d);
+        const uint8_t *ks = card + stream_base(card, &C, stream_index(&C, l, 0, h));
+        const uint8_t *vs = card + stream_base(card, &C, stream_index(&C, l, 1, h));
+        for (int64_t t = 0; t < T; ++t) {
+            reconstruct_record(ks + off[t], d, bits[t], kx + t * d);
+            reconstruct_record(vs + off[t], d, bits[t], vx + t * d);
+        }
         for (int jj = 0; jj < per_kv; ++jj) {
             const int j = h * per_kv + jj;
             const uint16_t *qv = q + ((int64_t)l * n_q_heads + j) * d;
@@ -587,7 +611,7 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
             for (int64_t t = 0; t < T; ++t) {
                 double acc = 0.0;
                 for (int c = 0; c < d; ++c)
-                    acc += (double)orc_half_to_float(qv[c]) * (double)orc_half_to_float(kx[t * d + c]);
+                    acc += (double)orc_half_to_float(qv[c]) * kx[t * d + c];
                 s[t] = softmax_scale * acc;
                 if (s[t] > mx) mx = s[t];
             }
@@ -598,7 +622,7 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
             }
             for (int c = 0; c < d; ++c) {
                 double acc = 0.0;
-                for (int64_t t = 0; t < T; ++t) acc += s[t] * (double)orc_half_to_float(vx[t * d + c]);
+                for (int64_t t = 0; t < T; ++t) acc += s[t] * vx[t * d + c];
                 o[c] = acc / denom;
             }
         }

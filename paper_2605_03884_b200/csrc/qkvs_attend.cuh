@@ -1,24 +1,27 @@
 // Decode-step attention straight from a card: one query token per layer attends to every token
-// of the card, reading the records themselves -- the FP16 cache is never written out.
+// of the card, reading the records themselves -- no FP16 cache is written or even formed.
 //
-//     s_t = softmax_scale * q . K^_t,   p = softmax(s),   o = sum_t p_t V^_t
+//     s_t = softmax_scale * q . K~_t,   p = softmax(s),   o = sum_t p_t V~_t
 //
-// with K^, V^ exactly the FP16 values injection reconstructs (the same decode_chunk), grouped
-// queries (query head j reads KV head j / per_kv), head_dim 128.
+// with K~, V~ the values the records stand for (code * scale + zero per group of 32 channels, or
+// the FP16 value of a 16-bit row), grouped queries (query head j reads KV head j / per_kv),
+// head_dim 128.  Scale and zero never touch the elements: with D = sum_c q_c code_c per group,
+//     q . K~_t   = sum_g scale_tg * D_tg + zero_tg * (sum_{c in g} q_c)
+//     sum_t p_t V~_tc = sum_t (p_t scale_tg) code_tc + sum_t p_t zero_tg        (c in group g)
+// so both contractions run on the tensor cores over the integer codes themselves (exact in FP16;
+// mma.sync m16n8k16, FP32 accumulation) and the group parameters enter once per token and group.
 //
 // Work item: 256 consecutive tokens of one (layer, KV head), taken by one warp from a counter.
 // The warp walks them in steps of 16 tokens; the spans of K and V records of a step are staged by
-// two bulk copies (TMA) on one mbarrier, NS steps ahead.  Both products run on the tensor cores
-// (mma.sync m16n8k16, FP16 inputs, FP32 accumulation) with operands laid out so that every lane
-// decodes exactly the values its own fragments need -- nothing passes through shared memory
-// after decoding:
-//   scores   S = Q K^T : rows = query heads of the group (up to 8 of 16 used), columns = 8 tokens
-//            per instruction; lane (g, t) supplies token g's group t (channels 32t .. 32t+31,
-//            four per k-step), and holds the matching channels of Q;
-//   outputs  O^T = V^T P^T : rows = channels, columns = query heads; lane (g, t) supplies channels
-//            16g .. 16g+15 of the four tokens 2t, 2t+1, 2t+8, 2t+9, and the probabilities it
-//            computed itself from S are already the B fragment.
-// Softmax is the usual running maximum / running sum; every item leaves (max, sum, o) per query
+// two bulk copies (TMA) on one mbarrier, NS steps ahead.  Operand layouts are chosen -- the order
+// of channels inside a group and of tokens inside a step is free in a contraction -- so that every
+// lane builds its fragments from a few bytes of its own with shifts and masks:
+//   scores   rows = query heads of the group (up to 8 of 16 used), columns = 8 tokens; lane (g, t)
+//            supplies 8 codes of token g from each group and holds the matching channels of Q;
+//   outputs  rows = channels, columns = query heads; lane (g, t) supplies 4 channels per group of
+//            the four tokens 2t, 2t+1, 2t+8, 2t+9, and the probabilities it computed itself, times
+//            the tokens' scales, are already the B fragment.
+// Softmax is the usual running maximum / running sum; every item leaves (o, max, sum) per query
 // head in the scratch buffer and a second small kernel merges the items of a head.
 #pragma once
 
@@ -78,55 +81,6 @@ __device__ __forceinline__ uint32_t word_of(const uint4 &v, int i)
     return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
 }
 
-// N consecutive chunks (pos0 .. pos0 + N - 1, all inside one group of a row whose record is `rec`)
-// -> N x 8 FP16 values, bit for bit what injection reconstructs.  With the bit-width B known at
-// compile time the group's scale / zero pair and its codes are fetched once for the whole run;
-// B = 0 decodes chunk by chunk with the row's own width `b`.
-template <int B, int N>
-__device__ __forceinline__ void decode_run(const uint8_t *rec, int b, int pos0, uint4 (&out)[N])
-{
-    constexpr int G = kAttendD / kGroup;
-    if (B == 0) {
-#pragma unroll
-        for (int i = 0; i < N; ++i) out[i] = decode_chunk<kAttendD, 0>(rec, b, pos0 + i);
-        return;
-    }
-    if (B == 16) {
-#pragma unroll
-        for (int i = 0; i < N; ++i) out[i] = *reinterpret_cast<const uint4 *>(rec + (pos0 + i) * 16);
-        return;
-    }
-    const float2 m = *reinterpret_cast<const float2 *>(rec + (pos0 >> 2) * kMetaBytesPerGroup);
-    const Dequant dq = make_dequant(m.x, m.y);
-    const uint8_t *codes = rec + G * kMetaBytesPerGroup + pos0 * B;  // N * B bytes, aligned to their size
-    uint32_t w[N * B / 4 > 0 ? N * B / 4 : 1];
-    if (N * B == 32) {
-        const uint4 a = *reinterpret_cast<const uint4 *>(codes), c = *reinterpret_cast<const uint4 *>(codes + 16);
-        w[0] = a.x, w[1] = a.y, w[2] = a.z, w[3] = a.w, w[4] = c.x, w[5] = c.y, w[6] = c.z, w[7] = c.w;
-    } else if (N * B == 16) {
-        const uint4 a = *reinterpret_cast<const uint4 *>(codes);
-        w[0] = a.x, w[1] = a.y, w[2] = a.z, w[3] = a.w;
-    } else if (N * B == 8) {
-        const uint2 a = *reinterpret_cast<const uint2 *>(codes);
-        w[0] = a.x, w[1] = a.y;
-    } else {
-        w[0] = *reinterpret_cast<const uint32_t *>(codes);
-    }
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-        uint32_t lo, hi;
-        if (B == 8) {
-            lo = w[2 * i];
-            hi = w[2 * i + 1];
-        } else if (B == 4) {
-            unpack_nibbles(w[i], lo, hi);
-        } else {
-            unpack_nibbles(unpack_crumbs((w[i >> 1] >> (16 * (i & 1))) & 0xffffu), lo, hi);
-        }
-        out[i] = dequantize_chunk(lo, hi, dq);
-    }
-}
-
 // Checks a step's table entries, publishes the per-token record positions and starts the copies
 // of its K and V spans (same offsets, two streams).  All lanes call it.
 template <int NS>
@@ -164,90 +118,231 @@ __device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, 
     __syncwarp();
 }
 
-// One step: 16 tokens of K and V staged in `stage` against the group's queries.  Updates the
-// running maximum / sum of head g and the output accumulators.  B is the bit-width shared by all
-// 16 rows, or 0 when they differ or the step is short.
-template <int NS, int B>
-__device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int stage, int rows, int gid, int tig, float scale_log2,
-                                            const uint32_t (&qa0)[8], const uint32_t (&qa2)[8], float &m_run, float &l_run,
-                                            float (&acc)[8][4])
+constexpr uint32_t kHalfMagic = 0x64006400u;  // two FP16 1024.0: 1024 + n has n in its low mantissa bits
+
+// Two small integers, found in `word` under `mask` (one in each 16-bit half), as an FP16 pair:
+// (word & mask) | 1024.0 puts them into the low mantissa bits of 1024 + n; minus 1024 is exact.
+__device__ __forceinline__ uint32_t int_pair(uint32_t word, uint32_t mask)
 {
-    // ---- scores of 2 x 8 tokens for the heads of the group
-    float sacc[2][4];
+    uint32_t f;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(f) : "r"(word), "r"(mask), "r"(kHalfMagic));  // (a & b) | c
+    return as_u32(__hsub2(as_half2(f), as_half2(kHalfMagic)));
+}
+
+// Key side.  The lane's 8 channels of group g of one token (channels 32g + 8t + 0..7) as four
+// FP16 pairs e[k] = (value k, value k + 4) -- codes for a quantised row, the FP16 values for a
+// 16-bit row.  The query fragments pair channels the same way.
+template <int B>
+__device__ __forceinline__ void key_pairs(const uint8_t *rec, int b, int g, int tig, uint32_t (&e)[4])
+{
+    const int bb = B ? B : b;
+    if (bb == 16) {
+        const uint4 h = *reinterpret_cast<const uint4 *>(rec + 64 * g + 16 * tig);
+        e[0] = __byte_perm(h.x, h.z, 0x5410);
+        e[1] = __byte_perm(h.x, h.z, 0x7632);
+        e[2] = __byte_perm(h.y, h.w, 0x5410);
+        e[3] = __byte_perm(h.y, h.w, 0x7632);
+        return;
+    }
+    const uint8_t *codes = rec + 4 * kMetaBytesPerGroup + (4 * g + tig) * bb;  // the lane's 8 codes: b bytes
+    if (bb == 4) {
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(codes);  // nibble k and k + 4 are 16 bits apart
 #pragma unroll
-    for (int bi = 0; bi < 2; ++bi) {
+        for (int k = 0; k < 4; ++k) e[k] = int_pair(w >> (4 * k), 0x000f000fu);
+    } else if (bb == 8) {
+        const uint2 w = *reinterpret_cast<const uint2 *>(codes);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) sacc[bi][i] = 0.0f;
-        const int tok = 8 * bi + gid;
-        uint4 kq[4];
+        for (int k = 0; k < 4; ++k) e[k] = int_pair(__byte_perm(w.x, w.y, 0x0011u * k + 0x1100u * (4 + k)), 0x00ff00ffu);
+    } else {
+        const uint32_t w = *reinterpret_cast<const uint16_t *>(codes);
+        const uint32_t y = __byte_perm(w, 0u, 0x4140);  // codes 0..3 in byte 0, codes 4..7 in byte 2
 #pragma unroll
-        for (int c = 0; c < 4; ++c) kq[c] = make_uint4(0, 0, 0, 0);  // lanes without a token feed zeros
-        if (tok < rows) {
-            const uint32_t inf = sm.info[stage][tok];
-            const uint8_t *rec = sm.k[stage] + (inf >> 8);
-            decode_run<B, 4>(rec, (int)(inf & 0xffu), 4 * tig, kq);
-        }
+        for (int k = 0; k < 4; ++k) e[k] = int_pair(y >> (2 * k), 0x00030003u);
+    }
+}
+
+// Value side, one token: the lane's 4 channels of group g (channels 32g + 4gid + 0..3) as two FP16
+// pairs (value 0, value 1), (value 2, value 3).
+__device__ __forceinline__ void value_quad(const uint8_t *rec, int b, int g, int gid, uint32_t &p01, uint32_t &p23)
+{
+    if (b == 16) {
+        const uint2 h = *reinterpret_cast<const uint2 *>(rec + 64 * g + 8 * gid);
+        p01 = h.x;
+        p23 = h.y;
+    } else if (b == 4) {
+        const uint32_t w = *reinterpret_cast<const uint16_t *>(rec + 32 + 16 * g + 2 * gid);
+        p01 = int_pair(w | (w << 12), 0x000f000fu);
+        p23 = int_pair((w >> 8) | (w << 4), 0x000f000fu);
+    } else if (b == 8) {
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(rec + 32 + 32 * g + 4 * gid);
+        p01 = int_pair(__byte_perm(w, 0u, 0x4140), 0x00ff00ffu);
+        p23 = int_pair(__byte_perm(w, 0u, 0x4342), 0x00ff00ffu);
+    } else {
+        const uint32_t w = *(rec + 32 + 8 * g + gid);
+        p01 = int_pair(w | (w << 14), 0x00030003u);
+        p23 = int_pair((w >> 4) | (w << 10), 0x00030003u);
+    }
+}
+
+// Value side, two tokens of one known width B at once: the lane's 4 channels of group g as four
+// FP16 pairs e[k] = (token a's value k, token b's value k).
+template <int B>
+__device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t *rec_b, int g, int gid, uint32_t (&e)[4])
+{
+    if (B == 16) {
+        const uint2 ha = *reinterpret_cast<const uint2 *>(rec_a + 64 * g + 8 * gid);
+        const uint2 hb = *reinterpret_cast<const uint2 *>(rec_b + 64 * g + 8 * gid);
+        e[0] = __byte_perm(ha.x, hb.x, 0x5410);
+        e[1] = __byte_perm(ha.x, hb.x, 0x7632);
+        e[2] = __byte_perm(ha.y, hb.y, 0x5410);
+        e[3] = __byte_perm(ha.y, hb.y, 0x7632);
+    } else if (B == 4) {
+        const uint32_t wa = *reinterpret_cast<const uint16_t *>(rec_a + 32 + 16 * g + 2 * gid);
+        const uint32_t wb = *reinterpret_cast<const uint16_t *>(rec_b + 32 + 16 * g + 2 * gid);
+        const uint32_t x = wa | (wb << 16);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {  // the whole warp executes every mma together
-            mma_m16n8k16(sacc[bi], qa0[2 * c], 0u, qa2[2 * c], 0u, kq[c].x, kq[c].y);
-            mma_m16n8k16(sacc[bi], qa0[2 * c + 1], 0u, qa2[2 * c + 1], 0u, kq[c].z, kq[c].w);
+        for (int k = 0; k < 4; ++k) e[k] = int_pair(x >> (4 * k), 0x000f000fu);
+    } else if (B == 8) {
+        const uint32_t wa = *reinterpret_cast<const uint32_t *>(rec_a + 32 + 32 * g + 4 * gid);
+        const uint32_t wb = *reinterpret_cast<const uint32_t *>(rec_b + 32 + 32 * g + 4 * gid);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) e[k] = int_pair(__byte_perm(wa, wb, 0x0011u * k + 0x1100u * (4 + k)), 0x00ff00ffu);
+    } else {
+        const uint32_t x = (uint32_t)*(rec_a + 32 + 8 * g + gid) | ((uint32_t)*(rec_b + 32 + 8 * g + gid) << 16);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) e[k] = int_pair(x >> (2 * k), 0x00030003u);
+    }
+}
+
+// Scale / zero pairs of a token's four groups; (1, 0) for a 16-bit row, (0, 0) for no token.
+// B != 0: the width is B and the token exists.
+template <int B>
+__device__ __forceinline__ void group_params_of(const uint8_t *rec, int b, bool valid, float (&sc)[4], float (&ze)[4])
+{
+    if (B ? B != 16 : (valid && b != 16)) {
+        const uint4 m0 = *reinterpret_cast<const uint4 *>(rec), m1 = *reinterpret_cast<const uint4 *>(rec + 16);
+        sc[0] = __uint_as_float(m0.x), ze[0] = __uint_as_float(m0.y), sc[1] = __uint_as_float(m0.z), ze[1] = __uint_as_float(m0.w);
+        sc[2] = __uint_as_float(m1.x), ze[2] = __uint_as_float(m1.y), sc[3] = __uint_as_float(m1.z), ze[3] = __uint_as_float(m1.w);
+    } else {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            sc[g] = (B || valid) ? 1.0f : 0.0f;
+            ze[g] = 0.0f;
         }
     }
-    // ---- running softmax for head g over tokens 8bi + 2t + e
-    float x[2][2];
-    float m_loc = -INFINITY;
+}
+
+// One step: 16 tokens of K and V staged in `stage` against the group's queries.  Updates the
+// running maximum / sum of head g, the zero-point sums and the output accumulators.  B is the
+// bit-width shared by all 16 rows, or 0 when they differ or the step is short.
+//   qa[g][k]    query fragments: head gid, channels 32g + 8tig + k and + k + 4
+//   qsum[g]     sum of head gid's query over group g
+//   zacc[g]     sum_t p_t zero_tg for head gid, over the tokens this lane has seen
+//   acc[g][h]   channels 32g + 4gid + 2h (+1) x heads 2tig, 2tig + 1, without the zero-point part
+template <int NS, int B>
+__device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int stage, int rows, int gid, int tig, float scale_log2,
+                                            const uint32_t (&qa)[4][4], const float (&qsum)[4], float &m_run, float &l_run,
+                                            float (&zacc)[4], float (&acc)[4][2][4])
+{
+    // the lane's four tokens (the same ones on the score side and on the value side)
+    int tok[4], bw[4];
+    uint32_t off[4];
 #pragma unroll
-    for (int bi = 0; bi < 2; ++bi)
+    for (int i = 0; i < 4; ++i) {
+        tok[i] = 2 * tig + (i & 1) + 8 * (i >> 1);
+        const uint32_t inf = (B || tok[i] < rows) ? sm.info[stage][tok[i]] : 0u;
+        off[i] = inf >> 8;
+        bw[i] = B ? B : (int)(inf & 0xffu);
+    }
+    // ---- scores: per group, sum_c q_c code_c for the heads of the group x 2 blocks of 8 tokens
+    float x[4];  // logits (base 2) of head gid for the lane's four tokens
+    {
+        float sacc[2][4][4];
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            x[bi][e] = (8 * bi + 2 * tig + e) < rows ? sacc[bi][e] * scale_log2 : -INFINITY;
-            m_loc = fmaxf(m_loc, x[bi][e]);
+        for (int bi = 0; bi < 2; ++bi) {
+            const int t = 8 * bi + gid;
+            const uint32_t inf = (B || t < rows) ? sm.info[stage][t] : 0u;
+            const uint8_t *rec = sm.k[stage] + (inf >> 8);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                uint32_t e[4] = {0u, 0u, 0u, 0u};  // lanes without a token feed zeros
+                if (B || t < rows) key_pairs<B>(rec, (int)(inf & 0xffu), g, tig, e);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sacc[bi][g][i] = 0.0f;
+                mma_m16n8k16(sacc[bi][g], qa[g][0], 0u, qa[g][1], 0u, e[0], e[1]);  // the whole warp, together
+                mma_m16n8k16(sacc[bi][g], qa[g][2], 0u, qa[g][3], 0u, e[2], e[3]);
+            }
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float sc[4], ze[4];
+            group_params_of<B>(sm.k[stage] + off[i], bw[i], tok[i] < rows, sc, ze);
+            float dot = 0.0f;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) dot = fmaf(sc[g], sacc[i >> 1][g][i & 1], fmaf(ze[g], qsum[g], dot));
+            x[i] = (B || tok[i] < rows) ? dot * scale_log2 : -INFINITY;
+        }
+    }
+    // ---- running softmax for head gid
+    float m_loc = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
     m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 1));
     m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 2));
     const float m_new = fmaxf(m_run, m_loc);
     const float m_ref = m_new == -INFINITY ? 0.0f : m_new;
     const float alpha = exp2_approx(m_run - m_ref);  // 0 on the first tokens of the item
-    float pr[2][2];
+    float pr[4];
 #pragma unroll
-    for (int bi = 0; bi < 2; ++bi)
-#pragma unroll
-        for (int e = 0; e < 2; ++e) pr[bi][e] = exp2_approx(x[bi][e] - m_ref);
-    l_run = l_run * alpha + (pr[0][0] + pr[0][1]) + (pr[1][0] + pr[1][1]);
+    for (int i = 0; i < 4; ++i) pr[i] = exp2_approx(x[i] - m_ref);
+    l_run = fmaf(l_run, alpha, (pr[0] + pr[1]) + (pr[2] + pr[3]));
     m_run = m_new;
-    const uint32_t pb0 = as_u32(__floats2half2_rn(pr[0][0], pr[0][1]));
-    const uint32_t pb1 = as_u32(__floats2half2_rn(pr[1][0], pr[1][1]));
     // the accumulators of this lane belong to heads 2t and 2t + 1, whose factors other lanes hold
     const float a_lo = __shfl_sync(0xffffffffu, alpha, 8 * tig);
     const float a_hi = __shfl_sync(0xffffffffu, alpha, 8 * tig + 4);
-    if (__any_sync(0xffffffffu, a_lo != 1.0f || a_hi != 1.0f)) {
+    if (__any_sync(0xffffffffu, a_lo != 1.0f || a_hi != 1.0f || alpha != 1.0f)) {
 #pragma unroll
-        for (int mb = 0; mb < 8; ++mb) {
-            acc[mb][0] *= a_lo;
-            acc[mb][1] *= a_hi;
-            acc[mb][2] *= a_lo;
-            acc[mb][3] *= a_hi;
+        for (int g = 0; g < 4; ++g) {
+            zacc[g] *= alpha;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                acc[g][h][0] *= a_lo;
+                acc[g][h][1] *= a_hi;
+                acc[g][h][2] *= a_lo;
+                acc[g][h][3] *= a_hi;
+            }
         }
     }
-    // ---- values: channels 16g .. 16g+15 of tokens 2t, 2t+1, 2t+8, 2t+9
-    uint4 vq[4][2];
+    // ---- values: probabilities times the tokens' scales against the codes; zero points aside
+    float vs[4][4];  // [token][group]
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const int tok = 2 * tig + (i & 1) + 8 * (i >> 1);
-        vq[i][0] = make_uint4(0, 0, 0, 0);
-        vq[i][1] = make_uint4(0, 0, 0, 0);
-        if (tok < rows) {
-            const uint32_t inf = sm.info[stage][tok];
-            const uint8_t *rec = sm.v[stage] + (inf >> 8);
-            decode_run<B, 2>(rec, (int)(inf & 0xffu), 2 * gid, vq[i]);
-        }
+        float ze[4];
+        group_params_of<B>(sm.v[stage] + off[i], bw[i], tok[i] < rows, vs[i], ze);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) zacc[g] = fmaf(pr[i], ze[g], zacc[g]);
     }
 #pragma unroll
-    for (int mb = 0; mb < 8; ++mb) {
-        const uint32_t wa = word_of(vq[0][mb >> 2], mb & 3), wb = word_of(vq[1][mb >> 2], mb & 3);
-        const uint32_t wc = word_of(vq[2][mb >> 2], mb & 3), wd = word_of(vq[3][mb >> 2], mb & 3);
-        mma_m16n8k16(acc[mb], __byte_perm(wa, wb, 0x5410), __byte_perm(wa, wb, 0x7632), __byte_perm(wc, wd, 0x5410),
-                     __byte_perm(wc, wd, 0x7632), pb0, pb1);
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t pb0 = as_u32(__floats2half2_rn(pr[0] * vs[0][g], pr[1] * vs[1][g]));
+        const uint32_t pb1 = as_u32(__floats2half2_rn(pr[2] * vs[2][g], pr[3] * vs[3][g]));
+        uint32_t eab[4], ecd[4];
+        if (B) {
+            value_pairs<B>(sm.v[stage] + off[0], sm.v[stage] + off[1], g, gid, eab);
+            value_pairs<B>(sm.v[stage] + off[2], sm.v[stage] + off[3], g, gid, ecd);
+        } else {
+            uint32_t q01[4], q23[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                q01[i] = 0u;
+                q23[i] = 0u;
+                if (tok[i] < rows) value_quad(sm.v[stage] + off[i], bw[i], g, gid, q01[i], q23[i]);
+            }
+            eab[0] = __byte_perm(q01[0], q01[1], 0x5410), eab[1] = __byte_perm(q01[0], q01[1], 0x7632);
+            eab[2] = __byte_perm(q23[0], q23[1], 0x5410), eab[3] = __byte_perm(q23[0], q23[1], 0x7632);
+            ecd[0] = __byte_perm(q01[2], q01[3], 0x5410), ecd[1] = __byte_perm(q01[2], q01[3], 0x7632);
+            ecd[2] = __byte_perm(q23[2], q23[3], 0x5410), ecd[3] = __byte_perm(q23[2], q23[3], 0x7632);
+        }
+        mma_m16n8k16(acc[g][0], eab[0], eab[1], ecd[0], ecd[1], pb0, pb1);
+        mma_m16n8k16(acc[g][1], eab[2], eab[3], ecd[2], ecd[3], pb0, pb1);
     }
 }
 
@@ -328,22 +423,37 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             t.bits = lane < t.rows ? (uint32_t)__ldg(bits_tab + step * kAttendRows + lane) : 0u;
         };
 
-        // the group's queries as A fragments: lane (g, t) holds head g, channels 32t + 4kk + {0,1 | 2,3}
-        uint32_t qa0[8], qa2[8];
+        // the group's queries as A fragments: lane (gid, tig) holds head gid, per group the channels
+        // 32g + 8tig + k paired with + k + 4 (the pairing of key_pairs), and the query's sum over the group
+        uint32_t qa[4][4];
+        float qsum[4];
         {
-            const __half *qrow = p.q + ((uint64_t)layer * p.n_q_heads + (uint64_t)head * per_kv + gid) * kAttendD + 32 * tig;
+            const __half *qrow = p.q + ((uint64_t)layer * p.n_q_heads + (uint64_t)head * per_kv + gid) * kAttendD + 8 * tig;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                qa0[kk] = gid < per_kv ? __ldg(reinterpret_cast<const uint32_t *>(qrow + 4 * kk)) : 0u;
-                qa2[kk] = gid < per_kv ? __ldg(reinterpret_cast<const uint32_t *>(qrow + 4 * kk + 2)) : 0u;
+            for (int g = 0; g < 4; ++g) {
+                uint4 h = make_uint4(0u, 0u, 0u, 0u);
+                if (gid < per_kv) h = __ldg(reinterpret_cast<const uint4 *>(qrow + 32 * g));
+                qa[g][0] = __byte_perm(h.x, h.z, 0x5410);
+                qa[g][1] = __byte_perm(h.x, h.z, 0x7632);
+                qa[g][2] = __byte_perm(h.y, h.w, 0x5410);
+                qa[g][3] = __byte_perm(h.y, h.w, 0x7632);
+                const float2 f0 = __half22float2(as_half2(h.x)), f1 = __half22float2(as_half2(h.y));
+                const float2 f2 = __half22float2(as_half2(h.z)), f3 = __half22float2(as_half2(h.w));
+                float sum = ((f0.x + f0.y) + (f1.x + f1.y)) + ((f2.x + f2.y) + (f3.x + f3.y));
+                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                qsum[g] = sum;
             }
         }
-        float m_run = -INFINITY, l_run = 0.0f;  // of head g (same in the four lanes of a g, l_run summed at the end)
-        float acc[8][4];                        // O^T: channels 16g + 2mb (+1) x heads 2t, 2t + 1
+        float m_run = -INFINITY, l_run = 0.0f;  // of head gid (same in the four lanes of a gid; l_run summed at the end)
+        float zacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        float acc[4][2][4];
 #pragma unroll
-        for (int mb = 0; mb < 8; ++mb)
+        for (int g = 0; g < 4; ++g)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[mb][i] = 0.0f;
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[g][h][i] = 0.0f;
 
         Tables nxt;
         fetch(nxt, 0);
@@ -362,11 +472,11 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             const int rows = sm.rows[stage];
 
             switch (sm.uniform_bits[stage]) {  // all 16 rows of one width: the specialised body
-                case 4: attend_step<NS, 4>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
-                case 2: attend_step<NS, 2>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
-                case 8: attend_step<NS, 8>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
-                case 16: attend_step<NS, 16>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
-                default: attend_step<NS, 0>(sm, stage, rows, gid, tig, p.scale_log2, qa0, qa2, m_run, l_run, acc); break;
+                case 4: attend_step<NS, 4>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                case 2: attend_step<NS, 2>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                case 8: attend_step<NS, 8>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                case 16: attend_step<NS, 16>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                default: attend_step<NS, 0>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
             }
             __syncwarp();  // every lane has read the stage: it can be re-armed
             if (issued < n_steps) {
@@ -382,20 +492,33 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
         }
         if (!ok) break;
 
-        // ---- what the item found, per query head: running maximum, running sum, unnormalised o
+        // ---- what the item found, per query head: unnormalised o (zero-point part added), maximum, sum
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        float z_lo[4], z_hi[4];  // of heads 2tig and 2tig + 1
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            float z = zacc[g];
+            z += __shfl_xor_sync(0xffffffffu, z, 1);
+            z += __shfl_xor_sync(0xffffffffu, z, 2);
+            z_lo[g] = __shfl_sync(0xffffffffu, z, 8 * tig);
+            z_hi[g] = __shfl_sync(0xffffffffu, z, 8 * tig + 4);
+        }
         float *part = p.partials + (uint64_t)item * per_kv * kPartialFloats;
         if (tig == 0 && gid < per_kv) {
             part[gid * kPartialFloats + kAttendD] = m_run;
             part[gid * kPartialFloats + kAttendD + 1] = l_run;
         }
 #pragma unroll
-        for (int mb = 0; mb < 8; ++mb) {
-            const int ch = 16 * gid + 2 * mb;
-            if (2 * tig < per_kv) *reinterpret_cast<float2 *>(part + (2 * tig) * kPartialFloats + ch) = make_float2(acc[mb][0], acc[mb][2]);
-            if (2 * tig + 1 < per_kv) *reinterpret_cast<float2 *>(part + (2 * tig + 1) * kPartialFloats + ch) = make_float2(acc[mb][1], acc[mb][3]);
-        }
+        for (int g = 0; g < 4; ++g)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int ch = 32 * g + 4 * gid + 2 * h;
+                if (2 * tig < per_kv)
+                    *reinterpret_cast<float2 *>(part + (2 * tig) * kPartialFloats + ch) = make_float2(acc[g][h][0] + z_lo[g], acc[g][h][2] + z_lo[g]);
+                if (2 * tig + 1 < per_kv)
+                    *reinterpret_cast<float2 *>(part + (2 * tig + 1) * kPartialFloats + ch) = make_float2(acc[g][h][1] + z_hi[g], acc[g][h][3] + z_hi[g]);
+            }
 
         uint32_t v = 0;
         if (lane == 0) v = atomicAdd(p.work_counter, 1u);
