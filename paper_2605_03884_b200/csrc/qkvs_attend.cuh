@@ -136,7 +136,7 @@ template <int B>
 __device__ __forceinline__ void key_pairs(const uint8_t *rec, int b, int g, int tig, uint32_t (&e)[4])
 {
     const int bb = B ? B : b;
-    if (bb == 16) {
+    if (B == 16 || (B == 0 && bb == 16)) {
         const uint4 h = *reinterpret_cast<const uint4 *>(rec + 64 * g + 16 * tig);
         e[0] = __byte_perm(h.x, h.z, 0x5410);
         e[1] = __byte_perm(h.x, h.z, 0x7632);
@@ -145,19 +145,34 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int b, int g, int 
         return;
     }
     const uint8_t *codes = rec + 4 * kMetaBytesPerGroup + (4 * g + tig) * bb;  // the lane's 8 codes: b bytes
-    if (bb == 4) {
+    if constexpr (B == 4) {
         const uint32_t w = *reinterpret_cast<const uint32_t *>(codes);  // nibble k and k + 4 are 16 bits apart
 #pragma unroll
         for (int k = 0; k < 4; ++k) e[k] = int_pair(w >> (4 * k), 0x000f000fu);
-    } else if (bb == 8) {
+    } else if constexpr (B == 8) {
         const uint2 w = *reinterpret_cast<const uint2 *>(codes);
 #pragma unroll
         for (int k = 0; k < 4; ++k) e[k] = int_pair(__byte_perm(w.x, w.y, 0x0011u * k + 0x1100u * (4 + k)), 0x00ff00ffu);
-    } else {
+    } else if constexpr (B == 2) {
         const uint32_t w = *reinterpret_cast<const uint16_t *>(codes);
         const uint32_t y = __byte_perm(w, 0u, 0x4140);  // codes 0..3 in byte 0, codes 4..7 in byte 2
 #pragma unroll
         for (int k = 0; k < 4; ++k) e[k] = int_pair(y >> (2 * k), 0x00030003u);
+    } else if constexpr (B == 0) {
+        // width known per lane only: one instruction stream for 2, 4 and 8 bits.  The b bytes sit
+        // inside one aligned 8-byte window; codes 0..3 end up in `lo`, codes 4..7 in `hi`, each
+        // at k * b bits, and a pair is (lo >> k*b) & mask | ((hi >> k*b) & mask) << 16.
+        const uint32_t a = smem_addr(codes);
+        const uint2 win = *reinterpret_cast<const uint2 *>(codes - (a & 7u));
+        const uint32_t sh = (a & 7u) * 8u;
+        const uint32_t lo = sh >= 32u ? win.y >> (sh - 32u) : __funnelshift_r(win.x, win.y, sh);  // first 32 bits of the codes
+        const uint32_t hi = bb == 8 ? win.y : lo >> (4 * bb);                                         // from code 4 on
+        const uint32_t mask = (1u << bb) - 1u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t pair = ((lo >> (k * bb)) & mask) | (((hi >> (k * bb)) & mask) << 16);
+            e[k] = int_pair(pair, 0x00ff00ffu);
+        }
     }
 }
 
@@ -169,18 +184,15 @@ __device__ __forceinline__ void value_quad(const uint8_t *rec, int b, int g, int
         const uint2 h = *reinterpret_cast<const uint2 *>(rec + 64 * g + 8 * gid);
         p01 = h.x;
         p23 = h.y;
-    } else if (b == 4) {
-        const uint32_t w = *reinterpret_cast<const uint16_t *>(rec + 32 + 16 * g + 2 * gid);
-        p01 = int_pair(w | (w << 12), 0x000f000fu);
-        p23 = int_pair((w >> 8) | (w << 4), 0x000f000fu);
-    } else if (b == 8) {
-        const uint32_t w = *reinterpret_cast<const uint32_t *>(rec + 32 + 32 * g + 4 * gid);
-        p01 = int_pair(__byte_perm(w, 0u, 0x4140), 0x00ff00ffu);
-        p23 = int_pair(__byte_perm(w, 0u, 0x4342), 0x00ff00ffu);
     } else {
-        const uint32_t w = *(rec + 32 + 8 * g + gid);
-        p01 = int_pair(w | (w << 14), 0x00030003u);
-        p23 = int_pair((w >> 4) | (w << 10), 0x00030003u);
+        // one instruction stream for 2, 4 and 8 bits: the lane's 4 codes are b/2 bytes inside one
+        // aligned 4-byte word
+        const uint8_t *codes = rec + 4 * kMetaBytesPerGroup + (8 * g) * (b / 2) + gid * (b / 2);
+        const uint32_t a = smem_addr(codes);
+        const uint32_t x = *reinterpret_cast<const uint32_t *>(codes - (a & 3u)) >> ((a & 3u) * 8u);
+        const uint32_t mask = (1u << b) - 1u;
+        p01 = int_pair((x & mask) | (((x >> b) & mask) << 16), 0x00ff00ffu);
+        p23 = int_pair(((x >> (2 * b)) & mask) | (((x >> (3 * b)) & mask) << 16), 0x00ff00ffu);
     }
 }
 
