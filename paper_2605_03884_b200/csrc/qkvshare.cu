@@ -279,14 +279,30 @@ __global__ void __launch_bounds__(kRankThreads) bits_from_scores_kernel(const fl
         __syncthreads();
         // padding is -inf and sits behind every real index, so it never counts
         const int64_t first = base + part * (kRankTile / 4);
-#pragma unroll 4
-        for (int i = 0; i < kRankTile / 4; i += 4) {
-            const float4 s = *reinterpret_cast<const float4 *>(&tile[part * (kRankTile / 4) + i]);
-            const int64_t idx = first + i;
-            rank += (s.x > mine) || (s.x == mine && idx < t);
-            rank += (s.y > mine) || (s.y == mine && idx + 1 < t);
-            rank += (s.z > mine) || (s.z == mine && idx + 2 < t);
-            rank += (s.w > mine) || (s.w == mine && idx + 3 < t);
+        const float4 *quarter = reinterpret_cast<const float4 *>(&tile[part * (kRankTile / 4)]);
+        if (first + kRankTile / 4 <= t) {
+            // the whole quarter lies in front of the token: equal scores count too
+#pragma unroll 8
+            for (int i = 0; i < kRankTile / 16; ++i) {
+                const float4 s = quarter[i];
+                rank += (s.x >= mine) + (s.y >= mine) + (s.z >= mine) + (s.w >= mine);
+            }
+        } else if (first > t) {
+            // the whole quarter lies behind it: only larger scores count
+#pragma unroll 8
+            for (int i = 0; i < kRankTile / 16; ++i) {
+                const float4 s = quarter[i];
+                rank += (s.x > mine) + (s.y > mine) + (s.z > mine) + (s.w > mine);
+            }
+        } else {
+            for (int i = 0; i < kRankTile / 16; ++i) {
+                const float4 s = quarter[i];
+                const int64_t idx = first + 4 * i;
+                rank += (s.x > mine) || (s.x == mine && idx < t);
+                rank += (s.y > mine) || (s.y == mine && idx + 1 < t);
+                rank += (s.z > mine) || (s.z == mine && idx + 2 < t);
+                rank += (s.w > mine) || (s.w == mine && idx + 3 < t);
+            }
         }
     }
     rank += __shfl_xor_sync(0xffffffffu, rank, 1);
