@@ -53,12 +53,10 @@ struct AttendParams {
 
 template <int NS>
 struct AttendWarpSmem {
-    alignas(128) uint8_t k[NS][kAttendRows * 2 * kAttendD];
+    alignas(128) uint8_t k[NS][kAttendRows * 2 * kAttendD];  // up to 16 records, packed one after another
     alignas(128) uint8_t v[NS][kAttendRows * 2 * kAttendD];
-    uint32_t info[NS][kAttendRows];  // per token: record offset inside the span << 8 | bit-width
+    uint32_t list[kAttendRows * kAttendSteps];  // record offsets of the item's tokens, grouped by bit-width
     alignas(8) uint64_t full[NS];
-    int32_t rows[NS];                // 0 when the step's table entries did not check out
-    uint32_t uniform_bits[NS];       // bit-width shared by all 16 rows, else 0
 };
 
 __device__ __forceinline__ void mma_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -81,41 +79,61 @@ __device__ __forceinline__ uint32_t word_of(const uint4 &v, int i)
     return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
 }
 
-// Checks a step's table entries, publishes the per-token record positions and starts the copies
-// of its K and V spans (same offsets, two streams).  All lanes call it.
+// The order of tokens does not matter to attention, so a warp regroups the (up to) 256 tokens of
+// its item by bit-width and walks them one width at a time: every step then deals with a single
+// width and runs the body compiled for it, however the widths are mixed in the card.
+
+// Bit-width classes in the order they are walked: 2, 4, 8, 16 bits.
+__device__ __forceinline__ uint32_t class_width(int c) { return c == 0 ? 2u : (c == 1 ? 4u : (c == 2 ? 8u : 16u)); }
+
+// The item's steps, in order: class c, tokens [s0, s0 + n) of that class's part of the list.
+struct StepIter {
+    uint32_t s1, s2, s3, s4;  // where classes 1, 2, 3 begin in the list (class 0 begins at 0) and where it ends
+    int c;
+    uint32_t s0;
+
+    __device__ __forceinline__ uint32_t end_of(int cls) const { return cls == 0 ? s1 : (cls == 1 ? s2 : (cls == 2 ? s3 : s4)); }
+    __device__ __forceinline__ void skip_empty()
+    {
+        while (c < 4 && s0 >= end_of(c)) ++c;  // the next class begins where this one ends
+    }
+    __device__ __forceinline__ void begin()
+    {
+        c = 0;
+        s0 = 0;
+        skip_empty();
+    }
+    __device__ __forceinline__ bool done() const { return c >= 4; }
+    __device__ __forceinline__ int rows() const { return (int)min((uint32_t)kAttendRows, end_of(c) - s0); }
+    __device__ __forceinline__ void next()
+    {
+        s0 = min(s0 + kAttendRows, end_of(c));
+        skip_empty();
+    }
+};
+
+// Starts the copies of one step's K and V records into `stage`, packed in list order: one copy
+// per stream when the tokens are neighbours in the card, else one per record.  All lanes call it.
 template <int NS>
-__device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, const Tables &t, uint64_t base_k, uint64_t base_v,
-                                             const AttendParams &p, const Sections &sec, uint64_t total_bytes, int lane)
+__device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, const StepIter &it, uint64_t base_k,
+                                             uint64_t base_v, const AttendParams &p, int lane)
 {
-    const int rows = t.rows;
-    const uint32_t off0 = __shfl_sync(0xffffffffu, t.off, 0);
-    const uint32_t off_next = __shfl_down_sync(0xffffffffu, t.off, 1);
-    const uint32_t off_end = __shfl_sync(0xffffffffu, t.off, rows);
-    int bad = 0;
-    if (lane < rows) {
-        const uint32_t rec = record_bytes(kAttendD, (int)t.bits);
-        bad = (rec == 0u) || (off_next < t.off) || (off_next - t.off != rec);
-        sm.info[stage][lane] = ((t.off - off0) << 8) | (t.bits & 0xffu);
-    }
-    bad = __any_sync(0xffffffffu, bad);
-    const uint32_t b0 = __shfl_sync(0xffffffffu, t.bits, 0);
-    const bool uniform = rows == kAttendRows && __all_sync(0xffffffffu, lane >= rows || t.bits == b0);
-    const uint32_t span = off_end - off0;  // consistent records: at most rows * 256 bytes, fits the stage
-    bad |= (off0 & 15u) != 0u || base_k < sec.payload_off || base_v < sec.payload_off || ((base_k | base_v) & 15u) != 0u ||
-           base_k + (uint64_t)off_end > total_bytes || base_v + (uint64_t)off_end > total_bytes;
-    if (lane == 0) {
-        sm.rows[stage] = bad ? 0 : rows;
-        sm.uniform_bits[stage] = uniform ? b0 : 0u;
-        if (bad && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
-        if (!bad && span) {
-            mbar_arrive_expect_tx(&sm.full[stage], 2u * span);
-            bulk_load(sm.k[stage], p.card + base_k + off0, span, &sm.full[stage]);
-            bulk_load(sm.v[stage], p.card + base_v + off0, span, &sm.full[stage]);
-        } else {
-            mbar_arrive(&sm.full[stage]);
-        }
-    }
+    const int n = it.rows();
+    const uint32_t rec = record_bytes(kAttendD, (int)class_width(it.c));
+    const uint32_t mine = lane < n ? sm.list[it.s0 + lane] : 0u;
+    const uint32_t first = __shfl_sync(0xffffffffu, mine, 0);
+    const bool neighbours = __all_sync(0xffffffffu, lane >= n || mine == first + (uint32_t)lane * rec);
+    if (lane == 0) mbar_arrive_expect_tx(&sm.full[stage], 2u * (uint32_t)n * rec);
     __syncwarp();
+    if (neighbours) {
+        if (lane == 0) {
+            bulk_load(sm.k[stage], p.card + base_k + first, (uint32_t)n * rec, &sm.full[stage]);
+            bulk_load(sm.v[stage], p.card + base_v + first, (uint32_t)n * rec, &sm.full[stage]);
+        }
+    } else if (lane < n) {
+        bulk_load(sm.k[stage] + lane * rec, p.card + base_k + mine, rec, &sm.full[stage]);
+        bulk_load(sm.v[stage] + lane * rec, p.card + base_v + mine, rec, &sm.full[stage]);
+    }
 }
 
 constexpr uint32_t kHalfMagic = 0x64006400u;  // two FP16 1024.0: 1024 + n has n in its low mantissa bits
@@ -133,10 +151,10 @@ __device__ __forceinline__ uint32_t int_pair(uint32_t word, uint32_t mask)
 // FP16 pairs e[k] = (value k, value k + 4) -- codes for a quantised row, the FP16 values for a
 // 16-bit row.  The query fragments pair channels the same way.
 template <int B>
-__device__ __forceinline__ void key_pairs(const uint8_t *rec, int b, int g, int tig, uint32_t (&e)[4])
+__device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, uint32_t (&e)[4])
 {
-    const int bb = B ? B : b;
-    if (B == 16 || (B == 0 && bb == 16)) {
+    constexpr int bb = B;
+    if (B == 16) {
         const uint4 h = *reinterpret_cast<const uint4 *>(rec + 64 * g + 16 * tig);
         e[0] = __byte_perm(h.x, h.z, 0x5410);
         e[1] = __byte_perm(h.x, h.z, 0x7632);
@@ -158,46 +176,11 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int b, int g, int 
         const uint32_t y = __byte_perm(w, 0u, 0x4140);  // codes 0..3 in byte 0, codes 4..7 in byte 2
 #pragma unroll
         for (int k = 0; k < 4; ++k) e[k] = int_pair(y >> (2 * k), 0x00030003u);
-    } else if constexpr (B == 0) {
-        // width known per lane only: one instruction stream for 2, 4 and 8 bits.  The b bytes sit
-        // inside one aligned 8-byte window; codes 0..3 end up in `lo`, codes 4..7 in `hi`, each
-        // at k * b bits, and a pair is (lo >> k*b) & mask | ((hi >> k*b) & mask) << 16.
-        const uint32_t a = smem_addr(codes);
-        const uint2 win = *reinterpret_cast<const uint2 *>(codes - (a & 7u));
-        const uint32_t sh = (a & 7u) * 8u;
-        const uint32_t lo = sh >= 32u ? win.y >> (sh - 32u) : __funnelshift_r(win.x, win.y, sh);  // first 32 bits of the codes
-        const uint32_t hi = bb == 8 ? win.y : lo >> (4 * bb);                                         // from code 4 on
-        const uint32_t mask = (1u << bb) - 1u;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint32_t pair = ((lo >> (k * bb)) & mask) | (((hi >> (k * bb)) & mask) << 16);
-            e[k] = int_pair(pair, 0x00ff00ffu);
-        }
     }
 }
 
-// Value side, one token: the lane's 4 channels of group g (channels 32g + 4gid + 0..3) as two FP16
-// pairs (value 0, value 1), (value 2, value 3).
-__device__ __forceinline__ void value_quad(const uint8_t *rec, int b, int g, int gid, uint32_t &p01, uint32_t &p23)
-{
-    if (b == 16) {
-        const uint2 h = *reinterpret_cast<const uint2 *>(rec + 64 * g + 8 * gid);
-        p01 = h.x;
-        p23 = h.y;
-    } else {
-        // one instruction stream for 2, 4 and 8 bits: the lane's 4 codes are b/2 bytes inside one
-        // aligned 4-byte word
-        const uint8_t *codes = rec + 4 * kMetaBytesPerGroup + (8 * g) * (b / 2) + gid * (b / 2);
-        const uint32_t a = smem_addr(codes);
-        const uint32_t x = *reinterpret_cast<const uint32_t *>(codes - (a & 3u)) >> ((a & 3u) * 8u);
-        const uint32_t mask = (1u << b) - 1u;
-        p01 = int_pair((x & mask) | (((x >> b) & mask) << 16), 0x00ff00ffu);
-        p23 = int_pair(((x >> (2 * b)) & mask) | (((x >> (3 * b)) & mask) << 16), 0x00ff00ffu);
-    }
-}
-
-// Value side, two tokens of one known width B at once: the lane's 4 channels of group g as four
-// FP16 pairs e[k] = (token a's value k, token b's value k).
+// Value side, two tokens at once: the lane's 4 channels of group g (channels 32g + 4gid + 0..3)
+// as four FP16 pairs e[k] = (token a's value k, token b's value k).
 template <int B>
 __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t *rec_b, int g, int gid, uint32_t (&e)[4])
 {
@@ -227,45 +210,39 @@ __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t 
 }
 
 // Scale / zero pairs of a token's four groups; (1, 0) for a 16-bit row, (0, 0) for no token.
-// B != 0: the width is B and the token exists.
 template <int B>
-__device__ __forceinline__ void group_params_of(const uint8_t *rec, int b, bool valid, float (&sc)[4], float (&ze)[4])
+__device__ __forceinline__ void group_params_of(const uint8_t *rec, bool valid, float (&sc)[4], float (&ze)[4])
 {
-    if (B ? B != 16 : (valid && b != 16)) {
+    if (B != 16 && valid) {
         const uint4 m0 = *reinterpret_cast<const uint4 *>(rec), m1 = *reinterpret_cast<const uint4 *>(rec + 16);
         sc[0] = __uint_as_float(m0.x), ze[0] = __uint_as_float(m0.y), sc[1] = __uint_as_float(m0.z), ze[1] = __uint_as_float(m0.w);
         sc[2] = __uint_as_float(m1.x), ze[2] = __uint_as_float(m1.y), sc[3] = __uint_as_float(m1.z), ze[3] = __uint_as_float(m1.w);
     } else {
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            sc[g] = (B || valid) ? 1.0f : 0.0f;
+            sc[g] = valid ? 1.0f : 0.0f;
             ze[g] = 0.0f;
         }
     }
 }
 
-// One step: 16 tokens of K and V staged in `stage` against the group's queries.  Updates the
-// running maximum / sum of head g, the zero-point sums and the output accumulators.  B is the
-// bit-width shared by all 16 rows, or 0 when they differ or the step is short.
+// One step: up to 16 tokens of one bit-width B, their K and V records packed one after another in
+// `stage`, against the group's queries.  Updates the running maximum / sum of head gid, the
+// zero-point sums and the output accumulators.  FULL: all 16 tokens are there.
 //   qa[g][k]    query fragments: head gid, channels 32g + 8tig + k and + k + 4
 //   qsum[g]     sum of head gid's query over group g
 //   zacc[g]     sum_t p_t zero_tg for head gid, over the tokens this lane has seen
 //   acc[g][h]   channels 32g + 4gid + 2h (+1) x heads 2tig, 2tig + 1, without the zero-point part
-template <int NS, int B>
+template <int NS, int B, bool FULL>
 __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int stage, int rows, int gid, int tig, float scale_log2,
                                             const uint32_t (&qa)[4][4], const float (&qsum)[4], float &m_run, float &l_run,
                                             float (&zacc)[4], float (&acc)[4][2][4])
 {
+    constexpr int REC = B == 16 ? 2 * kAttendD : kAttendD * B / 8 + 4 * kMetaBytesPerGroup;
     // the lane's four tokens (the same ones on the score side and on the value side)
-    int tok[4], bw[4];
-    uint32_t off[4];
+    int tok[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        tok[i] = 2 * tig + (i & 1) + 8 * (i >> 1);
-        const uint32_t inf = (B || tok[i] < rows) ? sm.info[stage][tok[i]] : 0u;
-        off[i] = inf >> 8;
-        bw[i] = B ? B : (int)(inf & 0xffu);
-    }
+    for (int i = 0; i < 4; ++i) tok[i] = 2 * tig + (i & 1) + 8 * (i >> 1);
     // ---- scores: per group, sum_c q_c code_c for the heads of the group x 2 blocks of 8 tokens
     float x[4];  // logits (base 2) of head gid for the lane's four tokens
     {
@@ -273,12 +250,11 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
 #pragma unroll
         for (int bi = 0; bi < 2; ++bi) {
             const int t = 8 * bi + gid;
-            const uint32_t inf = (B || t < rows) ? sm.info[stage][t] : 0u;
-            const uint8_t *rec = sm.k[stage] + (inf >> 8);
+            const uint8_t *rec = sm.k[stage] + t * REC;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 uint32_t e[4] = {0u, 0u, 0u, 0u};  // lanes without a token feed zeros
-                if (B || t < rows) key_pairs<B>(rec, (int)(inf & 0xffu), g, tig, e);
+                if (FULL || t < rows) key_pairs<B>(rec, g, tig, e);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) sacc[bi][g][i] = 0.0f;
                 mma_m16n8k16(sacc[bi][g], qa[g][0], 0u, qa[g][1], 0u, e[0], e[1]);  // the whole warp, together
@@ -288,11 +264,11 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             float sc[4], ze[4];
-            group_params_of<B>(sm.k[stage] + off[i], bw[i], tok[i] < rows, sc, ze);
+            group_params_of<B>(sm.k[stage] + tok[i] * REC, FULL || tok[i] < rows, sc, ze);
             float dot = 0.0f;
 #pragma unroll
             for (int g = 0; g < 4; ++g) dot = fmaf(sc[g], sacc[i >> 1][g][i & 1], fmaf(ze[g], qsum[g], dot));
-            x[i] = (B || tok[i] < rows) ? dot * scale_log2 : -INFINITY;
+            x[i] = (FULL || tok[i] < rows) ? dot * scale_log2 : -INFINITY;
         }
     }
     // ---- running softmax for head gid
@@ -328,31 +304,22 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         float ze[4];
-        group_params_of<B>(sm.v[stage] + off[i], bw[i], tok[i] < rows, vs[i], ze);
+        group_params_of<B>(sm.v[stage] + tok[i] * REC, FULL || tok[i] < rows, vs[i], ze);
 #pragma unroll
         for (int g = 0; g < 4; ++g) zacc[g] = fmaf(pr[i], ze[g], zacc[g]);
     }
+    // records of tokens that are not there hold stale bytes: their probabilities are zero, and so
+    // that nothing non-finite can come out of stale FP16 patterns their rows are read from token 0
+    const uint8_t *rv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) rv[i] = sm.v[stage] + ((FULL || tok[i] < rows) ? tok[i] : 0) * REC;
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
         const uint32_t pb0 = as_u32(__floats2half2_rn(pr[0] * vs[0][g], pr[1] * vs[1][g]));
         const uint32_t pb1 = as_u32(__floats2half2_rn(pr[2] * vs[2][g], pr[3] * vs[3][g]));
         uint32_t eab[4], ecd[4];
-        if (B) {
-            value_pairs<B>(sm.v[stage] + off[0], sm.v[stage] + off[1], g, gid, eab);
-            value_pairs<B>(sm.v[stage] + off[2], sm.v[stage] + off[3], g, gid, ecd);
-        } else {
-            uint32_t q01[4], q23[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                q01[i] = 0u;
-                q23[i] = 0u;
-                if (tok[i] < rows) value_quad(sm.v[stage] + off[i], bw[i], g, gid, q01[i], q23[i]);
-            }
-            eab[0] = __byte_perm(q01[0], q01[1], 0x5410), eab[1] = __byte_perm(q01[0], q01[1], 0x7632);
-            eab[2] = __byte_perm(q23[0], q23[1], 0x5410), eab[3] = __byte_perm(q23[0], q23[1], 0x7632);
-            ecd[0] = __byte_perm(q01[2], q01[3], 0x5410), ecd[1] = __byte_perm(q01[2], q01[3], 0x7632);
-            ecd[2] = __byte_perm(q23[2], q23[3], 0x5410), ecd[3] = __byte_perm(q23[2], q23[3], 0x7632);
-        }
+        value_pairs<B>(rv[0], rv[1], g, gid, eab);
+        value_pairs<B>(rv[2], rv[3], g, gid, ecd);
         mma_m16n8k16(acc[g][0], eab[0], eab[1], ecd[0], ecd[1], pb0, pb1);
         mma_m16n8k16(acc[g][1], eab[2], eab[3], ecd[2], ecd[3], pb0, pb1);
     }
@@ -413,7 +380,6 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
         const uint32_t lh = item / p.items_per_head, ck = item - lh * p.items_per_head;
         const uint32_t layer = lh / H, head = lh - layer * H;
         const uint32_t sub0 = ck * kAttendSteps;
-        const int n_steps = (int)min((uint32_t)kAttendSteps, p.subs_per_head - sub0);
 
         const uint64_t seg = mode == 0 ? 0u : lh;
         const uint8_t *bits_tab = p.card + sec.bits_off + seg * T + (uint64_t)sub0 * kAttendRows;
@@ -428,12 +394,68 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             base_k = sec.payload_off + __ldg(sbase + stream_k);
             base_v = sec.payload_off + __ldg(sbase + stream_v);
         }
-        auto fetch = [&](Tables &t, int step) {
-            t.rows = (sub0 + (uint32_t)step + 1u == p.subs_per_head) ? (int)p.last_rows : kAttendRows;
-            t.base = 0;
-            t.off = lane <= t.rows ? __ldg(offs_tab + step * kAttendRows + lane) : 0u;
-            t.bits = lane < t.rows ? (uint32_t)__ldg(bits_tab + step * kAttendRows + lane) : 0u;
-        };
+        // ---- the item's tokens, eight per lane: check the table entries, sort by width into the list
+        const uint32_t tok0 = sub0 * kAttendRows;
+        const int n_tok = (int)min((uint64_t)(kAttendRows * kAttendSteps), T - tok0);
+        uint32_t my_off[8];
+        int my_cls[8];
+        uint32_t counts = 0, counts_hi = 0;  // tokens of this lane per class: 16-bit fields (2 | 4 bits), (8 | 16 bits)
+        {
+            const bool base_ok = base_k >= sec.payload_off && base_v >= sec.payload_off && ((base_k | base_v) & 15u) == 0u;
+            bool bad = false;
+            uint32_t o_next = 8 * lane <= n_tok ? __ldg(offs_tab + 8 * lane) : 0u;
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                const int j = 8 * lane + r;
+                const uint32_t o = o_next;
+                o_next = j + 1 <= n_tok ? __ldg(offs_tab + j + 1) : 0u;
+                my_off[r] = o;
+                my_cls[r] = 4;
+                if (j < n_tok) {
+                    const uint32_t b = __ldg(bits_tab + j);
+                    const uint32_t rec = record_bytes(kAttendD, (int)b);
+                    const bool fine = base_ok && rec != 0u && o_next >= o && o_next - o == rec && (o & 15u) == 0u &&
+                                      base_k + (uint64_t)o_next <= total_bytes && base_v + (uint64_t)o_next <= total_bytes;
+                    bad |= !fine;
+                    if (fine) {
+                        my_cls[r] = b == 2u ? 0 : (b == 4u ? 1 : (b == 8u ? 2 : 3));
+                        if (my_cls[r] < 2) counts += 1u << (16 * my_cls[r]);
+                        else counts_hi += 1u << (16 * (my_cls[r] - 2));
+                    }
+                }
+            }
+            if (__any_sync(0xffffffffu, bad) && lane == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
+        }
+        StepIter iss;
+        {
+            // positions: class-major, then lane, then the lane's own order
+            uint32_t inc = counts, inc_hi = counts_hi;
+#pragma unroll
+            for (int sft = 1; sft < 32; sft <<= 1) {
+                const uint32_t a = __shfl_up_sync(0xffffffffu, inc, sft), bq = __shfl_up_sync(0xffffffffu, inc_hi, sft);
+                if (lane >= sft) {
+                    inc += a;
+                    inc_hi += bq;
+                }
+            }
+            const uint32_t tot = __shfl_sync(0xffffffffu, inc, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
+            iss.s1 = tot & 0xffffu;
+            iss.s2 = iss.s1 + (tot >> 16);
+            iss.s3 = iss.s2 + (tot_hi & 0xffffu);
+            iss.s4 = iss.s3 + (tot_hi >> 16);
+            const uint32_t before = inc - counts, before_hi = inc_hi - counts_hi;  // in lower lanes
+            uint32_t pos[4] = {before & 0xffffu, iss.s1 + (before >> 16), iss.s2 + (before_hi & 0xffffu), iss.s3 + (before_hi >> 16)};
+            __syncwarp();  // the previous item's list is no longer read
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (my_cls[r] == c) sm.list[pos[c]++] = my_off[r];
+            }
+            __syncwarp();
+        }
+        iss.begin();
+        StepIter con = iss;
 
         // the group's queries as A fragments: lane (gid, tig) holds head gid, per group the channels
         // 32g + 8tig + k paired with + k + 4 (the pairing of key_pairs), and the query's sum over the group
@@ -467,35 +489,37 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[g][h][i] = 0.0f;
 
-        Tables nxt;
-        fetch(nxt, 0);
-        int issued = 0;
-        for (; issued < NS && issued < n_steps; ++issued) {
-            const Tables cur = nxt;
-            if (issued + 1 < n_steps) fetch(nxt, issued + 1);
-            int st = stage + issued;
+        int in_flight = 0;
+        for (; in_flight < NS && !iss.done(); ++in_flight) {
+            int st = stage + in_flight;
             if (st >= NS) st -= NS;
-            attend_issue<NS>(sm, st, cur, base_k, base_v, p, sec, total_bytes, lane);
+            attend_issue<NS>(sm, st, iss, base_k, base_v, p, lane);
+            iss.next();
         }
-
-        for (int step = 0; step < n_steps; ++step) {
+        while (!con.done()) {
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[stage], parity));
             if (!ok) break;
-            const int rows = sm.rows[stage];
-
-            switch (sm.uniform_bits[stage]) {  // all 16 rows of one width: the specialised body
-                case 4: attend_step<NS, 4>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                case 2: attend_step<NS, 2>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                case 8: attend_step<NS, 8>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                case 16: attend_step<NS, 16>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                default: attend_step<NS, 0>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+            const int rows = con.rows();
+            if (rows == kAttendRows) {
+                switch (con.c) {
+                    case 0: attend_step<NS, 2, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 1: attend_step<NS, 4, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 2: attend_step<NS, 8, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    default: attend_step<NS, 16, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                }
+            } else {
+                switch (con.c) {
+                    case 0: attend_step<NS, 2, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 1: attend_step<NS, 4, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 2: attend_step<NS, 8, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    default: attend_step<NS, 16, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                }
             }
+            con.next();
             __syncwarp();  // every lane has read the stage: it can be re-armed
-            if (issued < n_steps) {
-                const Tables cur = nxt;
-                if (issued + 1 < n_steps) fetch(nxt, issued + 1);
-                attend_issue<NS>(sm, stage, cur, base_k, base_v, p, sec, total_bytes, lane);
-                ++issued;
+            if (!iss.done()) {
+                attend_issue<NS>(sm, stage, iss, base_k, base_v, p, lane);
+                iss.next();
             }
             if (++stage == NS) {
                 stage = 0;
