@@ -32,6 +32,7 @@ namespace qkvs {
 constexpr int kAttendD = 128;
 constexpr int kAttendRows = 16;          // tokens per step
 constexpr int kAttendSteps = 16;         // steps per work item
+constexpr int kAttendPerLane = kAttendRows * kAttendSteps / 32;  // tokens of an item per lane when they are sorted
 constexpr int kAttendMaxPerKv = 8;       // query heads per KV head
 constexpr int kPartialFloats = kAttendD + 4;  // o[128], running maximum (base-2 exponent), running sum, padding
 
@@ -394,19 +395,19 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             base_k = sec.payload_off + __ldg(sbase + stream_k);
             base_v = sec.payload_off + __ldg(sbase + stream_v);
         }
-        // ---- the item's tokens, eight per lane: check the table entries, sort by width into the list
+        // ---- the item's tokens, a run of kAttendPerLane per lane: check the table entries, sort by width into the list
         const uint32_t tok0 = sub0 * kAttendRows;
         const int n_tok = (int)min((uint64_t)(kAttendRows * kAttendSteps), T - tok0);
-        uint32_t my_off[8];
-        int my_cls[8];
+        uint32_t my_off[kAttendPerLane];
+        int my_cls[kAttendPerLane];
         uint32_t counts = 0, counts_hi = 0;  // tokens of this lane per class: 16-bit fields (2 | 4 bits), (8 | 16 bits)
         {
             const bool base_ok = base_k >= sec.payload_off && base_v >= sec.payload_off && ((base_k | base_v) & 15u) == 0u;
             bool bad = false;
-            uint32_t o_next = 8 * lane <= n_tok ? __ldg(offs_tab + 8 * lane) : 0u;
+            uint32_t o_next = kAttendPerLane * lane <= n_tok ? __ldg(offs_tab + kAttendPerLane * lane) : 0u;
 #pragma unroll
-            for (int r = 0; r < 8; ++r) {
-                const int j = 8 * lane + r;
+            for (int r = 0; r < kAttendPerLane; ++r) {
+                const int j = kAttendPerLane * lane + r;
                 const uint32_t o = o_next;
                 o_next = j + 1 <= n_tok ? __ldg(offs_tab + j + 1) : 0u;
                 my_off[r] = o;
@@ -447,7 +448,7 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             uint32_t pos[4] = {before & 0xffffu, iss.s1 + (before >> 16), iss.s2 + (before_hi & 0xffffu), iss.s3 + (before_hi >> 16)};
             __syncwarp();  // the previous item's list is no longer read
 #pragma unroll
-            for (int r = 0; r < 8; ++r) {
+            for (int r = 0; r < kAttendPerLane; ++r) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
                     if (my_cls[r] == c) sm.list[pos[c]++] = my_off[r];
