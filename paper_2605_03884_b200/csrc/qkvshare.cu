@@ -257,11 +257,13 @@ __global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
 // Bit-widths from importance scores by rank (the step in front of the offset scan).
 // rank(t) = #{s : score_s > score_t} + #{s < t : score_s == score_t}; the first n16 ranks keep
 // FP16, the next n8 get 8 bits, the next n4 get 4 bits, the rest 2 bits.  Exact and order-free:
-// every token counts for itself.  A CTA ranks 64 tokens, four threads per token, each thread
-// against a quarter of every 1024-score tile staged in shared memory.
+// every token counts for itself.  A CTA ranks 32 tokens, eight threads per token, each thread
+// against an eighth of every tile of up to 8192 scores staged in shared memory.
 
 constexpr int kRankThreads = 256;
-constexpr int kRankTile = 1024;
+constexpr int kRankSplit = 8;       // threads per token
+constexpr int kRankTile = 8192;     // scores per tile (32 KB of shared memory)
+constexpr int kRankBlock = 256;     // scores per block inside a tile
 
 __global__ void __launch_bounds__(kRankThreads) bits_from_scores_kernel(const float *scores, int64_t T, uint32_t n16,
                                                                         uint32_t n8, uint32_t n4, uint8_t *bits)
@@ -269,44 +271,49 @@ __global__ void __launch_bounds__(kRankThreads) bits_from_scores_kernel(const fl
     __shared__ __align__(16) float tile[kRankTile];
     scores += (int64_t)blockIdx.y * T;
     bits += (int64_t)blockIdx.y * T;
-    const int part = threadIdx.x & 3;
-    const int64_t t = (int64_t)blockIdx.x * (kRankThreads / 4) + (threadIdx.x >> 2);
+    const int part = threadIdx.x % kRankSplit;
+    const int64_t t = (int64_t)blockIdx.x * (kRankThreads / kRankSplit) + threadIdx.x / kRankSplit;
     const float mine = t < T ? scores[t] : 0.0f;
     uint32_t rank = 0;
     for (int64_t base = 0; base < T; base += kRankTile) {
+        const int n = (int)min((int64_t)kRankTile, T - base);
+        const int n_pad = (n + kRankBlock - 1) / kRankBlock * kRankBlock;
         __syncthreads();
-        for (int i = threadIdx.x; i < kRankTile; i += kRankThreads) tile[i] = base + i < T ? scores[base + i] : -INFINITY;
+        for (int i = threadIdx.x; i < n_pad; i += kRankThreads) tile[i] = i < n ? scores[base + i] : -INFINITY;
         __syncthreads();
-        // padding is -inf and sits behind every real index, so it never counts
-        const int64_t first = base + part * (kRankTile / 4);
-        const float4 *quarter = reinterpret_cast<const float4 *>(&tile[part * (kRankTile / 4)]);
-        if (first + kRankTile / 4 <= t) {
-            // the whole quarter lies in front of the token: equal scores count too
-#pragma unroll 8
-            for (int i = 0; i < kRankTile / 16; ++i) {
-                const float4 s = quarter[i];
-                rank += (s.x >= mine) + (s.y >= mine) + (s.z >= mine) + (s.w >= mine);
-            }
-        } else if (first > t) {
-            // the whole quarter lies behind it: only larger scores count
-#pragma unroll 8
-            for (int i = 0; i < kRankTile / 16; ++i) {
-                const float4 s = quarter[i];
-                rank += (s.x > mine) + (s.y > mine) + (s.z > mine) + (s.w > mine);
-            }
-        } else {
-            for (int i = 0; i < kRankTile / 16; ++i) {
-                const float4 s = quarter[i];
-                const int64_t idx = first + 4 * i;
-                rank += (s.x > mine) || (s.x == mine && idx < t);
-                rank += (s.y > mine) || (s.y == mine && idx + 1 < t);
-                rank += (s.z > mine) || (s.z == mine && idx + 2 < t);
-                rank += (s.w > mine) || (s.w == mine && idx + 3 < t);
+        // padding is -inf and sits behind every real index, so it never counts.  The eight threads
+        // of a token read neighbouring 16-byte pieces (no bank conflicts); a block of 256 scores
+        // that lies wholly in front of the token, or wholly behind it, needs one comparison per score.
+        const float4 *tile4 = reinterpret_cast<const float4 *>(tile);
+        for (int blk = 0; blk < n_pad / kRankBlock; ++blk) {
+            const int64_t first = base + (int64_t)blk * kRankBlock;
+            const float4 *piece = tile4 + blk * (kRankBlock / 4) + part;
+            if (first + kRankBlock <= t) {
+#pragma unroll
+                for (int i = 0; i < kRankBlock / 4 / kRankSplit; ++i) {
+                    const float4 s = piece[i * kRankSplit];
+                    rank += (s.x >= mine) + (s.y >= mine) + (s.z >= mine) + (s.w >= mine);
+                }
+            } else if (first > t) {
+#pragma unroll
+                for (int i = 0; i < kRankBlock / 4 / kRankSplit; ++i) {
+                    const float4 s = piece[i * kRankSplit];
+                    rank += (s.x > mine) + (s.y > mine) + (s.z > mine) + (s.w > mine);
+                }
+            } else {
+                for (int i = 0; i < kRankBlock / 4 / kRankSplit; ++i) {
+                    const float4 s = piece[i * kRankSplit];
+                    const int64_t idx = first + 4 * (i * kRankSplit + part);
+                    rank += (s.x > mine) || (s.x == mine && idx < t);
+                    rank += (s.y > mine) || (s.y == mine && idx + 1 < t);
+                    rank += (s.z > mine) || (s.z == mine && idx + 2 < t);
+                    rank += (s.w > mine) || (s.w == mine && idx + 3 < t);
+                }
             }
         }
     }
-    rank += __shfl_xor_sync(0xffffffffu, rank, 1);
-    rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+#pragma unroll
+    for (int s = 1; s < kRankSplit; s <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, s);
     if (part == 0 && t < T) bits[t] = rank < n16 ? 16 : (rank < n16 + n8 ? 8 : (rank < n16 + n8 + n4 ? 4 : 2));
 }
 
@@ -818,7 +825,7 @@ qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_segments,
     if (n_tokens > (1 << 20) || n_segments > 65535) return QKVS_ERR_UNSUPPORTED_SHAPE;
     if (n_tokens == 0) return QKVS_OK;
     if (!scores_dev || !bits_dev || (reinterpret_cast<uintptr_t>(scores_dev) & 3u)) return QKVS_ERR_INVALID_ARG;
-    const dim3 grid((unsigned)((n_tokens + kRankThreads / 4 - 1) / (kRankThreads / 4)), (unsigned)n_segments);
+    const dim3 grid((unsigned)((n_tokens + kRankThreads / kRankSplit - 1) / (kRankThreads / kRankSplit)), (unsigned)n_segments);
     bits_from_scores_kernel<<<grid, kRankThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
         scores_dev, n_tokens, (uint32_t)n_fp16, (uint32_t)n_8bit, (uint32_t)n_4bit, bits_dev);
     return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
