@@ -24,7 +24,8 @@ OK, INVALID_ARG, UNSUPPORTED_SHAPE, BAD_BITS, BUFFER_TOO_SMALL, BAD_CARD = range
 class Layout(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("n_tokens", C.c_int32), ("group_size", C.c_int32), ("bits_mode", C.c_int32),
-                ("head_stride", C.c_int64), ("token_stride", C.c_int64)]
+                ("head_stride", C.c_int64), ("token_stride", C.c_int64),
+                ("meta_bytes", C.c_int32), ("reserved_", C.c_int32)]
 
 
 def build(force: bool = False) -> str:
@@ -54,13 +55,17 @@ def lib():
         l.orc_float_to_half.restype = C.c_uint16
         l.orc_float_to_half.argtypes = [C.c_float]
         l.orc_record_bytes.restype = C.c_int64
-        l.orc_record_bytes.argtypes = [C.c_int, C.c_int]
+        l.orc_record_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         l.orc_scan_offsets.restype = C.c_int
-        l.orc_scan_offsets.argtypes = [C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(C.c_uint64)]
+        l.orc_scan_offsets.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(C.c_uint64)]
         l.orc_card_size.restype = C.c_int
         l.orc_card_size.argtypes = [C.POINTER(Layout), C.c_void_p, C.POINTER(C.c_uint64)]
         l.orc_quantize_group.restype = None
         l.orc_quantize_group.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_void_p]
+        l.orc_quantize_group_compact.restype = None
+        l.orc_quantize_group_compact.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16), C.c_void_p]
+        l.orc_float_to_half_up.restype = C.c_uint16
+        l.orc_float_to_half_up.argtypes = [C.c_float]
         l.orc_dequantize_group.restype = None
         l.orc_dequantize_group.argtypes = [C.c_void_p, C.c_float, C.c_float, C.c_void_p]
         l.orc_pack_codes.restype = None
@@ -68,9 +73,9 @@ def lib():
         l.orc_unpack_codes.restype = None
         l.orc_unpack_codes.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
         l.orc_encode_stream.restype = None
-        l.orc_encode_stream.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.orc_encode_stream.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         l.orc_decode_stream.restype = None
-        l.orc_decode_stream.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_int64]
+        l.orc_decode_stream.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p, C.c_int64]
         l.orc_write_prefix.restype = C.c_int
         l.orc_write_prefix.argtypes = [C.POINTER(Layout), C.c_void_p, C.c_uint64, C.c_uint64, C.c_int64, C.c_void_p, C.c_uint64]
         l.orc_card_create_range.restype = C.c_int
@@ -93,10 +98,10 @@ def _ptr(a: np.ndarray) -> int:
 
 
 def make_layout(n_layers, n_kv_heads, head_dim, n_tokens, bits_mode=0, head_stride=None,
-                token_stride=None) -> Layout:
+                token_stride=None, meta_bytes=8) -> Layout:
     ts = head_dim if token_stride is None else token_stride
     hs = n_tokens * ts if head_stride is None else head_stride
-    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, 32, bits_mode, hs, ts)
+    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, 32, bits_mode, hs, ts, meta_bytes, 0)
 
 
 def half_to_float(h: int) -> float:
@@ -107,15 +112,15 @@ def float_to_half(f: float) -> int:
     return int(lib().orc_float_to_half(C.c_float(f)))
 
 
-def record_bytes(head_dim: int, b: int) -> int:
-    return int(lib().orc_record_bytes(head_dim, b))
+def record_bytes(head_dim: int, b: int, meta_bytes: int = 8) -> int:
+    return int(lib().orc_record_bytes(head_dim, b, meta_bytes))
 
 
-def scan_offsets(head_dim: int, bits: np.ndarray) -> Tuple[int, np.ndarray, int]:
+def scan_offsets(head_dim: int, bits: np.ndarray, meta_bytes: int = 8) -> Tuple[int, np.ndarray, int]:
     bits = np.ascontiguousarray(bits, dtype=np.uint8)
     off = np.zeros(bits.size + 1, dtype=np.uint32)
     sb = C.c_uint64(0)
-    st = lib().orc_scan_offsets(head_dim, _ptr(bits), bits.size, _ptr(off), C.byref(sb))
+    st = lib().orc_scan_offsets(head_dim, meta_bytes, _ptr(bits), bits.size, _ptr(off), C.byref(sb))
     return st, off, int(sb.value)
 
 
@@ -135,6 +140,21 @@ def quantize_group(x: np.ndarray, b: int) -> Tuple[float, float, np.ndarray]:
     s, z = C.c_float(0), C.c_float(0)
     lib().orc_quantize_group(_ptr(x), b, C.byref(s), C.byref(z), _ptr(q))
     return np.float32(s.value), np.float32(z.value), q
+
+
+def quantize_group_compact(x: np.ndarray, b: int) -> Tuple[np.float16, np.float16, np.ndarray]:
+    """x: 32 FP16 values -> (scale, zero, codes[32]) with scale and zero as FP16 values."""
+    x = np.ascontiguousarray(x).view(np.uint16)
+    assert x.size == 32
+    q = np.zeros(32, dtype=np.uint8)
+    s, z = C.c_uint16(0), C.c_uint16(0)
+    lib().orc_quantize_group_compact(_ptr(x), b, C.byref(s), C.byref(z), _ptr(q))
+    return (np.array([s.value], dtype=np.uint16).view(np.float16)[0],
+            np.array([z.value], dtype=np.uint16).view(np.float16)[0], q)
+
+
+def float_to_half_up(f: float) -> int:
+    return int(lib().orc_float_to_half_up(C.c_float(f)))
 
 
 def dequantize_group(q: np.ndarray, scale, zero) -> np.ndarray:
@@ -158,28 +178,28 @@ def unpack_codes(packed: np.ndarray, n: int, b: int) -> np.ndarray:
     return q
 
 
-def encode_stream(x: np.ndarray, bits: np.ndarray) -> np.ndarray:
+def encode_stream(x: np.ndarray, bits: np.ndarray, meta_bytes: int = 8) -> np.ndarray:
     """One [T, d] FP16 matrix + bits[T] -> the stream's payload bytes."""
     x = np.ascontiguousarray(x).view(np.uint16)
     t, d = x.shape
-    st, off, _ = scan_offsets(d, bits)
+    st, off, _ = scan_offsets(d, bits, meta_bytes)
     if st:
         raise ValueError(f"bad bits (status {st})")
     bits = np.ascontiguousarray(bits, dtype=np.uint8)
     out = np.zeros(int(off[-1]), dtype=np.uint8)
-    lib().orc_encode_stream(_ptr(x), d, t, d, _ptr(bits), _ptr(off), _ptr(out))
+    lib().orc_encode_stream(_ptr(x), d, t, d, meta_bytes, _ptr(bits), _ptr(off), _ptr(out))
     return out
 
 
-def decode_stream(payload: np.ndarray, bits: np.ndarray, d: int) -> np.ndarray:
+def decode_stream(payload: np.ndarray, bits: np.ndarray, d: int, meta_bytes: int = 8) -> np.ndarray:
     payload = np.ascontiguousarray(payload, dtype=np.uint8)
     bits = np.ascontiguousarray(bits, dtype=np.uint8)
-    st, off, _ = scan_offsets(d, bits)
+    st, off, _ = scan_offsets(d, bits, meta_bytes)
     if st:
         raise ValueError(f"bad bits (status {st})")
     assert payload.size == int(off[-1])
     x = np.zeros((bits.size, d), dtype=np.uint16)
-    lib().orc_decode_stream(_ptr(payload), _ptr(bits), _ptr(off), bits.size, d, _ptr(x), d)
+    lib().orc_decode_stream(_ptr(payload), _ptr(bits), _ptr(off), bits.size, d, meta_bytes, _ptr(x), d)
     return x.view(np.float16)
 
 

@@ -19,7 +19,10 @@
  *     binary32 operation per step, round-to-nearest-even everywhere, nothing fused;
  *   - a constant group has scale = inv = 0 and all-zero codes; a zero minimum is stored +0;
  *   - reconstruction x^ = fp16_rne( fl32(fl32(q) * scale) + zero );
- *   - the byte layout described at write_prefix() / encode_record() below.
+ *   - the byte layout described at write_prefix() / encode_record() below;
+ *   - a compact variant that stores {scale, zero} as two FP16 values (zero exactly, scale rounded
+ *     up), defined at orc_quantize_group_compact(); the paper's "about 0.5 bytes per element at
+ *     4 bits" (Section 3.1) leaves no room for 8 bytes of metadata per 32 elements.
  * NaN or infinity inside a quantised (b < 16) token is outside the definition (codes are
  * then unspecified); inside an FP16 token the bit patterns are preserved.
  *
@@ -52,7 +55,11 @@ typedef struct {
     int32_t bits_mode;  /* 0: one bits[T] for the whole model; 1: bits[L*H][T] */
     int64_t head_stride;  /* elements between heads  */
     int64_t token_stride; /* elements between tokens */
+    int32_t meta_bytes;   /* bytes of {scale, zero} per group: 8 (fp32 pair; 0 means 8) or 4 (FP16 pair) */
+    int32_t reserved_;
 } orc_layout;
+
+static int meta_of(const orc_layout *L) { return L->meta_bytes == 0 ? 8 : L->meta_bytes; }
 
 /* ------------------------------------------------------------------ FP16 <-> FP32 */
 
@@ -101,13 +108,14 @@ uint16_t orc_float_to_half(float f)
 
 static uint64_t round_up_256(uint64_t x) { return (x + 255u) / 256u * 256u; }
 
-/* Bytes of one token row inside one stream: G (scale, zero) fp32 pairs then the packed
- * codes; an FP16 token is the row itself.  Code bytes alone are d*b/8 (Section 3.1's
- * bytes-per-element law). */
-int64_t orc_record_bytes(int head_dim, int b)
+/* Bytes of one token row inside one stream: G (scale, zero) pairs of `meta` bytes each (8: two
+ * fp32; 4: two FP16) then the packed codes; an FP16 token is the row itself.  Code bytes alone
+ * are d*b/8 (Section 3.1's bytes-per-element law). */
+int64_t orc_record_bytes(int head_dim, int b, int meta)
 {
+    if (meta != 8 && meta != 4) return -1;
     if (b == 16) return 2 * (int64_t)head_dim;
-    if (b == 2 || b == 4 || b == 8) return (int64_t)head_dim * b / 8 + 8 * (int64_t)(head_dim / 32);
+    if (b == 2 || b == 4 || b == 8) return (int64_t)head_dim * b / 8 + meta * (int64_t)(head_dim / 32);
     return -1;
 }
 
@@ -118,6 +126,9 @@ static int layout_ok(const orc_layout *L)
     if (L->bits_mode != 0 && L->bits_mode != 1) return ORC_INVALID_ARG;
     if (L->group_size != 32) return ORC_UNSUPPORTED_SHAPE;
     if (L->head_dim < 64 || L->head_dim % 64 != 0) return ORC_UNSUPPORTED_SHAPE;
+    if (meta_of(L) != 8 && meta_of(L) != 4) return ORC_INVALID_ARG;
+    /* records stay multiples of 16 bytes: FP16 pairs need head_dim to be a multiple of 128 */
+    if (meta_of(L) == 4 && L->head_dim % 128 != 0) return ORC_UNSUPPORTED_SHAPE;
     return ORC_OK;
 }
 
@@ -139,13 +150,14 @@ static int64_t segment_of(const orc_layout *L, int l, int h)
 
 /* Exclusive prefix sum of record sizes over one segment: off[0] = 0,
  * off[t+1] = off[t] + rec(b_t).  Returns ORC_BAD_BITS on a value outside {2,4,8,16}. */
-int orc_scan_offsets(int head_dim, const uint8_t *bits, int64_t n_tokens, uint32_t *off,
+int orc_scan_offsets(int head_dim, int meta, const uint8_t *bits, int64_t n_tokens, uint32_t *off,
                      uint64_t *sum_bits)
 {
+    if (meta != 8 && meta != 4) return ORC_INVALID_ARG;
     uint64_t run = 0, sb = 0;
     off[0] = 0;
     for (int64_t t = 0; t < n_tokens; ++t) {
-        int64_t r = orc_record_bytes(head_dim, bits[t]);
+        int64_t r = orc_record_bytes(head_dim, bits[t], meta);
         if (r < 0) return ORC_BAD_BITS;
         run += (uint64_t)r;
         sb += bits[t];
@@ -186,7 +198,7 @@ int orc_card_size(const orc_layout *L, const uint8_t *bits, uint64_t *out_bytes)
     for (int64_t seg = 0; seg < nseg; ++seg) {
         uint64_t seg_bytes = 0;
         for (int64_t t = 0; t < L->n_tokens; ++t) {
-            int64_t r = orc_record_bytes(L->head_dim, bits ? bits[seg * L->n_tokens + t] : 16);
+            int64_t r = orc_record_bytes(L->head_dim, bits ? bits[seg * L->n_tokens + t] : 16, meta_of(L));
             if (r < 0) return ORC_BAD_BITS;
             seg_bytes += (uint64_t)r;
         }
@@ -232,6 +244,12 @@ static float get_f32(const uint8_t *p)
     memcpy(&f, &b, 4);
     return f;
 }
+static void put_u16(uint8_t *p, uint16_t v)
+{
+    p[0] = (uint8_t)(v & 0xff);
+    p[1] = (uint8_t)(v >> 8);
+}
+static uint16_t get_u16(const uint8_t *p) { return (uint16_t)(p[0] | (p[1] << 8)); }
 
 /* ------------------------------------------------------------------ one group of 32 */
 
@@ -271,6 +289,63 @@ void orc_quantize_group(const uint16_t *x, int b, float *scale_out, float *zero_
     *zero_out = mn;
 }
 
+/* Smallest FP16 value that is >= f, for finite f >= 0 not above the largest FP16 value:
+ * round to nearest, then step one FP16 value up if that landed below f. */
+uint16_t orc_float_to_half_up(float f)
+{
+    uint16_t h = orc_float_to_half(f);
+    if (orc_half_to_float(h) < f) h = (uint16_t)(h + 1); /* positive FP16 values order like their bit patterns */
+    return h;
+}
+
+/* Compact-metadata variant: the group stores {scale, zero} as two FP16 values.
+ *   zero  = the group minimum, which is an FP16 value already (kept exactly; -0 stored as +0);
+ *   scale = (max-min)/(2^b-1) computed in binary32 as above, then rounded UP to FP16, so that
+ *           (x-zero)/scale never exceeds 2^b-1 by more than rounding;
+ *   inv   = fl32(1 / scale) with the stored scale, so that the codes are the ones the receiver's
+ *           scale implies: q = clamp(rint(fl32((x-zero) * inv)), 0, 2^b-1);
+ *   a constant group has scale = inv = 0 and all-zero codes.
+ * The largest possible scale, (65504+65504)/3, is below the largest FP16 value, so the rounding
+ * up never overflows; the smallest, 2^-24/255, rounds up to the smallest FP16 subnormal 2^-24.
+ * Reconstruction is orc_dequantize_group() with the two FP16 values widened to binary32. */
+void orc_quantize_group_compact(const uint16_t *x, int b, uint16_t *scale_out, uint16_t *zero_out,
+                                uint8_t *q)
+{
+    float xf[32];
+    for (int i = 0; i < 32; ++i) xf[i] = orc_half_to_float(x[i]);
+    float mn = xf[0], mx = xf[0];
+    uint16_t mn_bits = x[0];
+    for (int i = 1; i < 32; ++i) {
+        if (xf[i] < mn) { mn = xf[i]; mn_bits = x[i]; }
+        if (xf[i] > mx) mx = xf[i];
+    }
+    if (mn == 0.0f) { /* a zero minimum is stored as +0 whatever sign it carried */
+        mn = 0.0f;
+        mn_bits = 0;
+    }
+    int qmax = (1 << b) - 1;
+    float qmaxf = (float)qmax;
+    float range = mx - mn;
+    uint16_t scale16 = 0;
+    float inv = 0.0f;
+    if (range > 0.0f) {
+        scale16 = orc_float_to_half_up(range / qmaxf);
+        inv = 1.0f / orc_half_to_float(scale16);
+    }
+    for (int i = 0; i < 32; ++i) {
+        float t = xf[i] - mn;
+        float u = t * inv;
+        float r = nearbyintf(u); /* ties to even (default rounding mode) */
+        int qi;
+        if (!(r >= 0.0f)) qi = 0;
+        else if (r > qmaxf) qi = qmax;
+        else qi = (int)r;
+        q[i] = (uint8_t)qi;
+    }
+    *scale_out = scale16;
+    *zero_out = mn_bits;
+}
+
 /* Reconstruct 32 FP16 values: multiply, then add, each rounded to binary32, then to FP16. */
 void orc_dequantize_group(const uint8_t *q, float scale, float zero, uint16_t *out)
 {
@@ -301,10 +376,10 @@ void orc_unpack_codes(const uint8_t *in, int n, int b, uint8_t *q)
 
 /* ------------------------------------------------------------------ one token row */
 
-/* Record of a b<16 token: G pairs {scale_g, zero_g} (fp32, little-endian), group g covering
- * channels 32g..32g+31, then the d*b/8 code bytes of the whole row.  b == 16: the row's
- * FP16 bit patterns verbatim. */
-static void encode_record(const uint16_t *row, int d, int b, uint8_t *rec)
+/* Record of a b<16 token: G pairs {scale_g, zero_g} (little-endian; two fp32 when meta == 8,
+ * two FP16 when meta == 4), group g covering channels 32g..32g+31, then the d*b/8 code bytes of
+ * the whole row.  b == 16: the row's FP16 bit patterns verbatim. */
+static void encode_record(const uint16_t *row, int d, int b, int meta, uint8_t *rec)
 {
     if (b == 16) {
         for (int i = 0; i < d; ++i) {
@@ -316,15 +391,34 @@ static void encode_record(const uint16_t *row, int d, int b, uint8_t *rec)
     int G = d / 32;
     uint8_t q[32];
     for (int g = 0; g < G; ++g) {
-        float scale, zero;
-        orc_quantize_group(row + 32 * g, b, &scale, &zero, q);
-        put_f32(rec + 8 * g, scale);
-        put_f32(rec + 8 * g + 4, zero);
-        orc_pack_codes(q, 32, b, rec + 8 * G + (size_t)g * 32 * b / 8);
+        if (meta == 8) {
+            float scale, zero;
+            orc_quantize_group(row + 32 * g, b, &scale, &zero, q);
+            put_f32(rec + 8 * g, scale);
+            put_f32(rec + 8 * g + 4, zero);
+        } else {
+            uint16_t scale16, zero16;
+            orc_quantize_group_compact(row + 32 * g, b, &scale16, &zero16, q);
+            put_u16(rec + 4 * g, scale16);
+            put_u16(rec + 4 * g + 2, zero16);
+        }
+        orc_pack_codes(q, 32, b, rec + meta * G + (size_t)g * 32 * b / 8);
     }
 }
 
-static void decode_record(const uint8_t *rec, int d, int b, uint16_t *row)
+/* {scale, zero} of group g as binary32 (widening an FP16 pair is exact) */
+static void group_meta(const uint8_t *rec, int g, int meta, float *scale, float *zero)
+{
+    if (meta == 8) {
+        *scale = get_f32(rec + 8 * g);
+        *zero = get_f32(rec + 8 * g + 4);
+    } else {
+        *scale = orc_half_to_float(get_u16(rec + 4 * g));
+        *zero = orc_half_to_float(get_u16(rec + 4 * g + 2));
+    }
+}
+
+static void decode_record(const uint8_t *rec, int d, int b, int meta, uint16_t *row)
 {
     if (b == 16) {
         for (int i = 0; i < d; ++i) row[i] = (uint16_t)(rec[2 * i] | (rec[2 * i + 1] << 8));
@@ -333,26 +427,26 @@ static void decode_record(const uint8_t *rec, int d, int b, uint16_t *row)
     int G = d / 32;
     uint8_t q[32];
     for (int g = 0; g < G; ++g) {
-        float scale = get_f32(rec + 8 * g);
-        float zero = get_f32(rec + 8 * g + 4);
-        orc_unpack_codes(rec + 8 * G + (size_t)g * 32 * b / 8, 32, b, q);
+        float scale, zero;
+        group_meta(rec, g, meta, &scale, &zero);
+        orc_unpack_codes(rec + meta * G + (size_t)g * 32 * b / 8, 32, b, q);
         orc_dequantize_group(q, scale, zero, row + 32 * g);
     }
 }
 
 /* One stream (a [T, d] matrix with a row stride) -> its payload bytes. */
-void orc_encode_stream(const uint16_t *x, int64_t token_stride, int64_t n_tokens, int d,
+void orc_encode_stream(const uint16_t *x, int64_t token_stride, int64_t n_tokens, int d, int meta,
                        const uint8_t *bits, const uint32_t *off, uint8_t *out)
 {
     for (int64_t t = 0; t < n_tokens; ++t)
-        encode_record(x + t * token_stride, d, bits[t], out + off[t]);
+        encode_record(x + t * token_stride, d, bits[t], meta, out + off[t]);
 }
 
 void orc_decode_stream(const uint8_t *in, const uint8_t *bits, const uint32_t *off,
-                       int64_t n_tokens, int d, uint16_t *x, int64_t token_stride)
+                       int64_t n_tokens, int d, int meta, uint16_t *x, int64_t token_stride)
 {
     for (int64_t t = 0; t < n_tokens; ++t)
-        decode_record(in + off[t], d, bits[t], x + t * token_stride);
+        decode_record(in + off[t], d, bits[t], meta, x + t * token_stride);
 }
 
 /* ------------------------------------------------------------------ whole card */
@@ -360,7 +454,7 @@ void orc_decode_stream(const uint8_t *in, const uint8_t *bits, const uint32_t *o
 /* Header (256 bytes, little-endian, fields at these byte offsets, everything else zero):
  *   0 magic "QKVS" = 0x53564B51   4 version = 1     8 status        12 bits_mode
  *  16 n_layers  20 n_kv_heads  24 head_dim  28 n_tokens  32 group_size
- *  36 meta_bytes_per_group = 8    40 model_id u64   48 sender_id u64
+ *  36 meta_bytes_per_group (8|4)  40 model_id u64   48 sender_id u64
  *  56 position_offset i64 (placeholder)  64 sum_bits u64   72 avg_code_bits f32
  *  80 bits_off u64   88 offs_off u64   96 payload_off u64
  * 104 stream_bytes u64 (mode 0: bytes of one stream; mode 1: 0)   112 total_bytes u64
@@ -387,7 +481,7 @@ int orc_write_prefix(const orc_layout *L, const uint8_t *bits, uint64_t model_id
         uint32_t *off_tmp = (uint32_t *)(void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1));
         /* the host is little-endian, so writing uint32_t in place equals put_u32 */
         uint64_t sb = 0;
-        status = orc_scan_offsets(L->head_dim, bits + seg * T, T, off_tmp, &sb);
+        status = orc_scan_offsets(L->head_dim, meta_of(L), bits + seg * T, T, off_tmp, &sb);
         sum_bits += sb;
         memcpy(card + bo + (uint64_t)seg * (uint64_t)T, bits + seg * T, (size_t)T);
     }
@@ -417,7 +511,7 @@ int orc_write_prefix(const orc_layout *L, const uint8_t *bits, uint64_t model_id
     put_u32(card + 24, (uint32_t)L->head_dim);
     put_u32(card + 28, (uint32_t)L->n_tokens);
     put_u32(card + 32, (uint32_t)L->group_size);
-    put_u32(card + 36, 8u);
+    put_u32(card + 36, (uint32_t)meta_of(L));
     put_u64(card + 40, model_id);
     put_u64(card + 48, sender_id);
     put_u64(card + 56, (uint64_t)position_offset);
@@ -466,7 +560,7 @@ int orc_card_create_range(const orc_layout *L, const uint16_t *const *K_layers,
         int l = (int)(s / (2 * L->n_kv_heads));
         int64_t seg = segment_of(L, l, h);
         const uint16_t *x = (kv == 0 ? K_layers[l] : V_layers[l]) + (int64_t)h * L->head_stride;
-        orc_encode_stream(x, L->token_stride, T, L->head_dim, card + bo + (uint64_t)seg * (uint64_t)T,
+        orc_encode_stream(x, L->token_stride, T, L->head_dim, meta_of(L), card + bo + (uint64_t)seg * (uint64_t)T,
                           (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1)),
                           card + stream_base(card, L, s));
     }
@@ -498,7 +592,7 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
     C.n_tokens = (int32_t)get_u32(card + 28);
     if ((int32_t)get_u32(card + 16) != dst->n_layers || (int32_t)get_u32(card + 20) != dst->n_kv_heads ||
         (int32_t)get_u32(card + 24) != dst->head_dim || get_u32(card + 32) != 32u ||
-        get_u32(card + 36) != 8u || (C.bits_mode != 0 && C.bits_mode != 1) ||
+        get_u32(card + 36) != (uint32_t)meta_of(dst) || (C.bits_mode != 0 && C.bits_mode != 1) ||
         C.n_tokens != dst->n_tokens)
         return ORC_BAD_CARD;
     if (get_u64(card + 112) > card_bytes) return ORC_BAD_CARD;
@@ -520,7 +614,7 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
                       dst_token_offset * dst->token_stride;
         orc_decode_stream(card + stream_base(card, &C, s), card + bo + (uint64_t)seg * (uint64_t)T,
                           (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1)),
-                          T, C.head_dim, x, dst->token_stride);
+                          T, C.head_dim, meta_of(&C), x, dst->token_stride);
     }
     return ORC_OK;
 }
@@ -529,7 +623,7 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
  * the FP16 values themselves for a 16-bit row.  No rounding to FP16: that rounding belongs to
  * injection, which has to hand an FP16 cache to the receiving framework (Section 4.2.2); attention
  * that reads the card itself (Section 4.3) has no FP16 copy to round into. */
-static void reconstruct_record(const uint8_t *rec, int d, int b, double *row)
+static void reconstruct_record(const uint8_t *rec, int d, int b, int meta, double *row)
 {
     if (b == 16) {
         for (int i = 0; i < d; ++i) row[i] = (double)orc_half_to_float((uint16_t)(rec[2 * i] | (rec[2 * i + 1] << 8)));
@@ -538,10 +632,10 @@ static void reconstruct_record(const uint8_t *rec, int d, int b, double *row)
     int G = d / 32;
     uint8_t q[32];
     for (int g = 0; g < G; ++g) {
-        double scale = (double)get_f32(rec + 8 * g);
-        double zero = (double)get_f32(rec + 8 * g + 4);
-        orc_unpack_codes(rec + 8 * G + (size_t)g * 32 * b / 8, 32, b, q);
-        for (int i = 0; i < 32; ++i) row[32 * g + i] = (double)q[i] * scale + zero;
+        float scale, zero;
+        group_meta(rec, g, meta, &scale, &zero);
+        orc_unpack_codes(rec + meta * G + (size_t)g * 32 * b / 8, 32, b, q);
+        for (int i = 0; i < 32; ++i) row[32 * g + i] = (double)q[i] * (double)scale + (double)zero;
     }
 }
 
@@ -569,7 +663,7 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
     C.bits_mode = (int32_t)get_u32(card + 12);
     if ((int32_t)get_u32(card + 16) != L->n_layers || (int32_t)get_u32(card + 20) != L->n_kv_heads ||
         (int32_t)get_u32(card + 24) != L->head_dim || (int32_t)get_u32(card + 28) != L->n_tokens ||
-        (C.bits_mode != 0 && C.bits_mode != 1) || get_u64(card + 112) > card_bytes)
+        get_u32(card + 36) != (uint32_t)meta_of(L) || (C.bits_mode != 0 && C.bits_mode != 1) || get_u64(card + 112) > card_bytes)
         return ORC_BAD_CARD;
     const int d = C.head_dim, H = C.n_kv_heads, per_kv = n_q_heads / H;
     const int64_t T = C.n_tokens;
@@ -600,8 +694,8 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
         const uint8_t *ks = card + stream_base(card, &C, stream_index(&C, l, 0, h));
         const uint8_t *vs = card + stream_base(card, &C, stream_index(&C, l, 1, h));
         for (int64_t t = 0; t < T; ++t) {
-            reconstruct_record(ks + off[t], d, bits[t], kx + t * d);
-            reconstruct_record(vs + off[t], d, bits[t], vx + t * d);
+            reconstruct_record(ks + off[t], d, bits[t], meta_of(&C), kx + t * d);
+            reconstruct_record(vs + off[t], d, bits[t], meta_of(&C), vx + t * d);
         }
         for (int jj = 0; jj < per_kv; ++jj) {
             const int j = h * per_kv + jj;
