@@ -152,11 +152,11 @@ def load_workload(number: int, layers=None, n_layers=None):
     return w, Ks, Vs
 
 
-def cpu_oracle_leg(w, Ks, Vs, bits, n_layers_sample: int):
+def cpu_oracle_leg(w, Ks, Vs, bits, n_layers_sample: int, meta_bytes: int = 8):
     """Times the oracle as it stands (create then inject) on the first `n_layers_sample` layers."""
     import oracle
     L = min(n_layers_sample, w.n_layers)
-    lay = oracle.make_layout(L, w.n_kv_heads, w.head_dim, w.n_tokens)
+    lay = oracle.make_layout(L, w.n_kv_heads, w.head_dim, w.n_tokens, meta_bytes=meta_bytes)
     Ko = [np.zeros_like(k) for k in Ks[:L]]
     Vo = [np.zeros_like(v) for v in Vs[:L]]
     t0 = time.perf_counter()
@@ -184,9 +184,9 @@ def run_reference(args):
     w, Ks, Vs = load_workload(args.config, range(sample_layers))
     bits = wl.bits_for(w)
     for _ in range(args.warmup):
-        cpu_oracle_leg(w, Ks, Vs, bits, sample_layers)
+        cpu_oracle_leg(w, Ks, Vs, bits, sample_layers, args.meta_bytes)
     t0 = time.perf_counter()
-    legs = [cpu_oracle_leg(w, Ks, Vs, bits, sample_layers) for _ in range(args.steps)]
+    legs = [cpu_oracle_leg(w, Ks, Vs, bits, sample_layers, args.meta_bytes) for _ in range(args.steps)]
     dt = time.perf_counter() - t0
     kv_bytes = 2 * sample_layers * w.n_kv_heads * w.n_tokens * w.head_dim * 2
     value = kv_bytes * args.steps / dt / 1e9
@@ -194,7 +194,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": w.name, "sample_layers": sample_layers},
+        "data": "synthetic", "config": {"workload": w.name, "sample_layers": sample_layers,
+                                        "meta_bytes_per_group": args.meta_bytes},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": legs[-1]["cores"], "kind": "oracle",
                          "sample": legs[-1]["sample"]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -231,7 +232,7 @@ def run_ours(args):
     L, H, d, T = w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens
     hops = w.hops
     bits_per_hop = [wl.bits_for(w, h) for h in range(hops)]
-    lay = q.make_layout(L, H, d, T)
+    lay = q.make_layout(L, H, d, T, meta_bytes=args.meta_bytes)
     sizes = [q.card_size(lay, b) for b in bits_per_hop]
     prefix = q.card_prefix_size(lay)
     kv_bytes = w.kv_bytes
@@ -430,7 +431,7 @@ def run_ours(args):
     else:
         dom, dom_ms, dom_key = "inject_kernel", i0, "inject_kernel"
     achieved = (kv_bytes + payload0) / (dom_ms * 1e-3) / 1e9
-    traffic = captured_traffic(dom_key, L) if w.number == 3 else None
+    traffic = captured_traffic(dom_key, L) if w.number == 3 and args.meta_bytes == 8 else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src, "traffic": traffic,
                 "algorithmic_bytes_per_launch": kv_bytes + payload0, "avg_launch_ms": dom_ms}
@@ -438,7 +439,7 @@ def run_ours(args):
     launches_per_step = hops * (2 + 1) * ((L + 63) // 64) - hops * (((L + 63) // 64) - 1)
     cpu = None
     if not args.no_cpu_baseline:
-        cpu = cpu_oracle_leg(w, Ks, Vs, bits_per_hop[0], L)
+        cpu = cpu_oracle_leg(w, Ks, Vs, bits_per_hop[0], L, args.meta_bytes)
 
     # the step in front of the path: bit-widths from importance scores by rank (config 4's recipe)
     rank_us = None
@@ -462,6 +463,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "n_layers": L, "n_kv_heads": H, "head_dim": d, "n_tokens": T,
                    "hops": hops, "fp16_kv_bytes": kv_bytes, "replicas": world,
+                   "meta_bytes_per_group": args.meta_bytes,
                    "reduced_for_profiling": bool(args.layers),
                    "l2": "inputs (1 GiB FP16 KV per pass) exceed the 126 MB L2; no flush"
                    if kv_bytes > 4 * 126e6 else "working set comparable to L2; L2 helps"},
@@ -497,6 +499,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiler captures)")
     ap.add_argument("--skip-attend", action="store_true", help="skip the attention-from-the-card measurement")
+    ap.add_argument("--meta-bytes", type=int, default=8, choices=[8, 4],
+                    help="bytes of scale and zero per group in the card: 8 = two fp32 (the headline format), "
+                         "4 = two FP16 (compact variant)")
     ap.add_argument("--layers", type=int, default=0,
                     help="reduced case for profiler captures: keep the workload's recipe at this many layers")
     args = ap.parse_args()

@@ -15,6 +15,15 @@
  *   code = round-to-nearest-even((x - zero) * ((2^b - 1) / (max - min))), clamped to [0, 2^b - 1];
  *   reconstruction = fp16_rne(fl32(code * scale) + zero);  every step one IEEE binary32
  *   operation, never fused; a constant group has scale 0 and all-zero codes.
+ * Compact metadata (qkvs_layout_t.meta_bytes = 4).  Section 3.1 counts a 4-bit cache at about
+ * 0.5 bytes per element, which eight bytes of scale and zero per 32 elements (two more bits per
+ * element) do not leave room for; the paper says nothing on how the metadata is kept.  In this
+ * variant a group keeps an FP16 pair: zero, a group minimum, is an FP16 value already and is kept
+ * exactly; scale = (max - min) / (2^b - 1) computed as above and then rounded UP to FP16, so that
+ * the largest value still maps inside the code range; the codes are taken against the stored
+ * scale, code = round-to-nearest-even((x - zero) * fl32(1 / scale)), and reconstruction is the
+ * same formula with the two FP16 values widened.  One more bit per element instead of two:
+ * 5 / 3 / 9 effective bits at 4 / 2 / 8.  Needs head_dim to be a multiple of 128.
  *
  * Card bytes (little-endian; every section padded with zeros to a multiple of 256):
  *   [0, 256)        qkvs_card_header_t
@@ -23,10 +32,12 @@
  *   sbase_off       sbase[0..S] u64            (bits_mode 1 only) start of each stream in the payload
  *   payload_off     streams one after another, stream index s = (layer*2 + kv)*H + head,
  *                   kv 0 = K, 1 = V; token t's record sits at off[seg][t] inside its stream.
- *   record, b < 16: d/32 pairs {fp32 scale, fp32 zero}, then d*b/8 code bytes; the code of
+ *   record, b < 16: d/32 pairs {scale, zero} (two fp32, or two FP16 in the compact variant), then
+ *                   d*b/8 code bytes, which therefore start on a 16-byte boundary; the code of
  *                   channel i occupies bits [i*b, i*b + b) of the code bytes read as a
  *                   little-endian bit string.  record, b = 16: the d FP16 values verbatim.
- *   record size:    d*b/8 + 8*(d/32) bytes for b in {2,4,8};  2*d bytes for b = 16.
+ *   record size:    d*b/8 + meta_bytes*(d/32) bytes for b in {2,4,8};  2*d bytes for b = 16;
+ *                   always a multiple of 16.
  *
  * All entry points return a qkvs_status_t.  Unless stated otherwise a pointer named *_dev is a
  * device pointer, anything else is a host pointer.  The library allocates no device memory and
@@ -62,7 +73,8 @@ extern "C" {
 typedef enum {
     QKVS_OK = 0,
     QKVS_ERR_INVALID_ARG = 1,      /* null pointer, negative size, misaligned pointer or stride */
-    QKVS_ERR_UNSUPPORTED_SHAPE = 2,/* head_dim not in {64,128,192,256}, group_size != 32 */
+    QKVS_ERR_UNSUPPORTED_SHAPE = 2,/* head_dim not in {64,128,192,256}, group_size != 32, compact
+                                      metadata with a head_dim that is not a multiple of 128 */
     QKVS_ERR_BAD_BITS = 3,         /* a bit-width outside {2,4,8,16} */
     QKVS_ERR_BUFFER_TOO_SMALL = 4, /* card capacity below what the bit-widths need */
     QKVS_ERR_BAD_CARD = 5,         /* header magic/version/shape/status/size does not check out */
@@ -83,6 +95,11 @@ typedef struct {
                              vector); 1: bits[n_layers*n_kv_heads][n_tokens] */
     int64_t head_stride;  /* elements between heads; multiple of 8 */
     int64_t token_stride; /* elements between tokens; >= head_dim, multiple of 8 */
+    int32_t meta_bytes;   /* bytes of {scale, zero} per group in the card: 8 (or 0) = two fp32,
+                             4 = two FP16 (compact variant above).  A card is read back with the
+                             value it was made with: the header records it and a mismatch is a
+                             BAD_CARD. */
+    int32_t reserved_;    /* 0 */
 } qkvs_layout_t;
 
 /* Identifiers carried in the card (Section 4.2.1).  position_offset is the placeholder the
@@ -100,7 +117,7 @@ typedef struct {
     uint32_t status;               /* qkvs_status_t recorded on the device; 0 = usable card */
     uint32_t bits_mode;
     int32_t n_layers, n_kv_heads, head_dim, n_tokens, group_size;
-    uint32_t meta_bytes_per_group; /* 8 */
+    uint32_t meta_bytes_per_group; /* 8 or 4 */
     uint64_t model_id;
     uint64_t sender_id;
     int64_t position_offset;
@@ -114,9 +131,11 @@ typedef struct {
     uint8_t reserved_[128];
 } qkvs_card_header_t;
 
-/* Record size in bytes of one token row of `head_dim` channels at bit-width b, or 0 if b is
- * not one of {2,4,8,16}.  Host only.  (Closed form above; Section 3.1 for the code bytes.) */
-QKVS_API size_t qkvs_record_bytes(int32_t head_dim, int32_t b);
+/* Record size in bytes of one token row of `head_dim` channels at bit-width b with meta_bytes
+ * (8, 0 for 8, or 4) of scale and zero per group; 0 if b is not one of {2,4,8,16} or the
+ * combination of head_dim and meta_bytes is not supported.  Host only.  (Closed form above;
+ * Section 3.1 for the code bytes.) */
+QKVS_API size_t qkvs_record_bytes(int32_t head_dim, int32_t b, int32_t meta_bytes);
 
 /* Exact size of the card for a bit-width vector (Section 4.2.1: the card is variable-length,
  * its size follows from b(t)).  Host only, no GPU work.
@@ -212,10 +231,14 @@ QKVS_API qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t car
  * token per layer attends to all n_tokens of the card, with grouped queries: query head j reads
  * KV head j / (n_q_heads / n_kv_heads):
  *     s_t = softmax_scale * q_j . K^_t,   p = softmax_t(s),   out_j = sum_t p_t V^_t
- * where K^, V^ are exactly the FP16 values qkvs_card_inject would write.  Products run on the
- * tensor cores with FP16 inputs (the probabilities are rounded to FP16) and FP32 accumulation.
- *   layout        n_layers, n_kv_heads, head_dim, n_tokens of the card (checked against its
- *                 header on the device); head_dim must be 128; strides are not looked at
+ * where K^, V^ are the values the records stand for, code * scale + zero (an FP16 token: its
+ * values), without the rounding to FP16 that injection ends with: that rounding belongs to
+ * handing an FP16 cache to the receiving framework (Section 4.2.2), which is not done here.
+ * Products run on the tensor cores with FP16 inputs (the integer codes, exact in FP16, and the
+ * probabilities times the scales, rounded to FP16) and FP32 accumulation; scale and zero are
+ * applied outside the products.
+ *   layout        n_layers, n_kv_heads, head_dim, n_tokens and meta_bytes of the card (checked
+ *                 against its header on the device); head_dim must be 128; strides are not looked at
  *   n_q_heads     multiple of n_kv_heads, at most 8 query heads per KV head
  *   q_dev         FP16 [n_layers][n_q_heads][head_dim], 16-byte aligned
  *   out_dev       FP32 [n_layers][n_q_heads][head_dim], 16-byte aligned; all zeros if n_tokens is

@@ -27,7 +27,8 @@ class Layout(C.Structure):
     """qkvs_layout_t"""
     _fields_ = [("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("n_tokens", C.c_int32), ("group_size", C.c_int32), ("bits_mode", C.c_int32),
-                ("head_stride", C.c_int64), ("token_stride", C.c_int64)]
+                ("head_stride", C.c_int64), ("token_stride", C.c_int64),
+                ("meta_bytes", C.c_int32), ("reserved_", C.c_int32)]
 
 
 class CardMeta(C.Structure):
@@ -70,7 +71,7 @@ def load_library(path: Optional[str] = None):
     lib = C.CDLL(p)
     vp = C.c_void_p
     lib.qkvs_record_bytes.restype = C.c_size_t
-    lib.qkvs_record_bytes.argtypes = [C.c_int32, C.c_int32]
+    lib.qkvs_record_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
     lib.qkvs_card_size.restype = C.c_int
     lib.qkvs_card_size.argtypes = [C.POINTER(Layout), vp, C.POINTER(C.c_size_t)]
     lib.qkvs_card_prefix_size.restype = C.c_int
@@ -104,13 +105,15 @@ def status_string(status: int) -> str:
 
 
 def make_layout(n_layers: int, n_kv_heads: int, head_dim: int, n_tokens: int, bits_mode: int = 0,
-                head_stride: Optional[int] = None, token_stride: Optional[int] = None) -> Layout:
+                head_stride: Optional[int] = None, token_stride: Optional[int] = None,
+                meta_bytes: int = 8) -> Layout:
     ts = head_dim if token_stride is None else token_stride
     hs = n_tokens * ts if head_stride is None else head_stride
-    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, 32, bits_mode, hs, ts)
+    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, 32, bits_mode, hs, ts, meta_bytes, 0)
 
 
-def layout_of(tensors: Sequence, n_tokens: Optional[int] = None, bits_mode: int = 0) -> Layout:
+def layout_of(tensors: Sequence, n_tokens: Optional[int] = None, bits_mode: int = 0,
+              meta_bytes: int = 8) -> Layout:
     """Layout of a list of per-layer torch tensors shaped [H, T_cap, d] or [1, H, T_cap, d]."""
     t = tensors[0]
     if t.dim() == 4:
@@ -121,7 +124,7 @@ def layout_of(tensors: Sequence, n_tokens: Optional[int] = None, bits_mode: int 
         raise ValueError("expected [H, T, d] with unit channel stride")
     h, tcap, d = t.shape
     return Layout(len(tensors), h, d, tcap if n_tokens is None else n_tokens, 32, bits_mode,
-                  t.stride(0), t.stride(1))
+                  t.stride(0), t.stride(1), meta_bytes, 0)
 
 
 def _ptr_array(tensors: Sequence):
@@ -137,8 +140,8 @@ def _stream_handle(stream) -> int:
     return int(stream.cuda_stream)
 
 
-def record_bytes(head_dim: int, b: int) -> int:
-    return int(load_library().qkvs_record_bytes(head_dim, b))
+def record_bytes(head_dim: int, b: int, meta_bytes: int = 8) -> int:
+    return int(load_library().qkvs_record_bytes(head_dim, b, meta_bytes))
 
 
 def card_size(layout: Layout, bits_host=None) -> int:

@@ -40,6 +40,7 @@ struct AttendParams {
     const uint8_t *card;
     uint64_t card_bytes;
     int32_t n_layers, n_kv_heads, n_tokens, n_q_heads;
+    int32_t meta_bytes;      // 8 or 4: bytes of {scale, zero} per group in the card's records
     const __half *q;         // [n_layers][n_q_heads][128]
     float scale_log2;        // softmax_scale * log2(e)
     float *partials;         // [n_items][per_kv][kPartialFloats]
@@ -115,12 +116,12 @@ struct StepIter {
 
 // Starts the copies of one step's K and V records into `stage`, packed in list order: one copy
 // per stream when the tokens are neighbours in the card, else one per record.  All lanes call it.
-template <int NS>
+template <int NS, int META>
 __device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, const StepIter &it, uint64_t base_k,
                                              uint64_t base_v, const AttendParams &p, int lane)
 {
     const int n = it.rows();
-    const uint32_t rec = record_bytes(kAttendD, (int)class_width(it.c));
+    const uint32_t rec = record_bytes(kAttendD, (int)class_width(it.c), META);
     const uint32_t mine = lane < n ? sm.list[it.s0 + lane] : 0u;
     const uint32_t first = __shfl_sync(0xffffffffu, mine, 0);
     const bool neighbours = __all_sync(0xffffffffu, lane >= n || mine == first + (uint32_t)lane * rec);
@@ -151,7 +152,7 @@ __device__ __forceinline__ uint32_t int_pair(uint32_t word, uint32_t mask)
 // Key side.  The lane's 8 channels of group g of one token (channels 32g + 8t + 0..7) as four
 // FP16 pairs e[k] = (value k, value k + 4) -- codes for a quantised row, the FP16 values for a
 // 16-bit row.  The query fragments pair channels the same way.
-template <int B>
+template <int B, int META>
 __device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, uint32_t (&e)[4])
 {
     constexpr int bb = B;
@@ -163,7 +164,7 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, ui
         e[3] = __byte_perm(h.y, h.w, 0x7632);
         return;
     }
-    const uint8_t *codes = rec + 4 * kMetaBytesPerGroup + (4 * g + tig) * bb;  // the lane's 8 codes: b bytes
+    const uint8_t *codes = rec + 4 * META + (4 * g + tig) * bb;  // the lane's 8 codes: b bytes
     if constexpr (B == 4) {
         const uint32_t w = *reinterpret_cast<const uint32_t *>(codes);  // nibble k and k + 4 are 16 bits apart
 #pragma unroll
@@ -182,9 +183,10 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, ui
 
 // Value side, two tokens at once: the lane's 4 channels of group g (channels 32g + 4gid + 0..3)
 // as four FP16 pairs e[k] = (token a's value k, token b's value k).
-template <int B>
+template <int B, int META>
 __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t *rec_b, int g, int gid, uint32_t (&e)[4])
 {
+    constexpr int CODES = 4 * META;  // the code bytes follow the four {scale, zero} pairs
     if (B == 16) {
         const uint2 ha = *reinterpret_cast<const uint2 *>(rec_a + 64 * g + 8 * gid);
         const uint2 hb = *reinterpret_cast<const uint2 *>(rec_b + 64 * g + 8 * gid);
@@ -193,28 +195,37 @@ __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t 
         e[2] = __byte_perm(ha.y, hb.y, 0x5410);
         e[3] = __byte_perm(ha.y, hb.y, 0x7632);
     } else if (B == 4) {
-        const uint32_t wa = *reinterpret_cast<const uint16_t *>(rec_a + 32 + 16 * g + 2 * gid);
-        const uint32_t wb = *reinterpret_cast<const uint16_t *>(rec_b + 32 + 16 * g + 2 * gid);
+        const uint32_t wa = *reinterpret_cast<const uint16_t *>(rec_a + CODES + 16 * g + 2 * gid);
+        const uint32_t wb = *reinterpret_cast<const uint16_t *>(rec_b + CODES + 16 * g + 2 * gid);
         const uint32_t x = wa | (wb << 16);
 #pragma unroll
         for (int k = 0; k < 4; ++k) e[k] = int_pair(x >> (4 * k), 0x000f000fu);
     } else if (B == 8) {
-        const uint32_t wa = *reinterpret_cast<const uint32_t *>(rec_a + 32 + 32 * g + 4 * gid);
-        const uint32_t wb = *reinterpret_cast<const uint32_t *>(rec_b + 32 + 32 * g + 4 * gid);
+        const uint32_t wa = *reinterpret_cast<const uint32_t *>(rec_a + CODES + 32 * g + 4 * gid);
+        const uint32_t wb = *reinterpret_cast<const uint32_t *>(rec_b + CODES + 32 * g + 4 * gid);
 #pragma unroll
         for (int k = 0; k < 4; ++k) e[k] = int_pair(__byte_perm(wa, wb, 0x0011u * k + 0x1100u * (4 + k)), 0x00ff00ffu);
     } else {
-        const uint32_t x = (uint32_t)*(rec_a + 32 + 8 * g + gid) | ((uint32_t)*(rec_b + 32 + 8 * g + gid) << 16);
+        const uint32_t x = (uint32_t)*(rec_a + CODES + 8 * g + gid) | ((uint32_t)*(rec_b + CODES + 8 * g + gid) << 16);
 #pragma unroll
         for (int k = 0; k < 4; ++k) e[k] = int_pair(x >> (2 * k), 0x00030003u);
     }
 }
 
 // Scale / zero pairs of a token's four groups; (1, 0) for a 16-bit row, (0, 0) for no token.
-template <int B>
+template <int B, int META>
 __device__ __forceinline__ void group_params_of(const uint8_t *rec, bool valid, float (&sc)[4], float (&ze)[4])
 {
-    if (B != 16 && valid) {
+    if (B != 16 && valid && META == kMetaFp16) {
+        const uint4 m = *reinterpret_cast<const uint4 *>(rec);  // four FP16 pairs
+        const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const float2 f = __half22float2(as_half2(w[g]));
+            sc[g] = f.x;
+            ze[g] = f.y;
+        }
+    } else if (B != 16 && valid) {
         const uint4 m0 = *reinterpret_cast<const uint4 *>(rec), m1 = *reinterpret_cast<const uint4 *>(rec + 16);
         sc[0] = __uint_as_float(m0.x), ze[0] = __uint_as_float(m0.y), sc[1] = __uint_as_float(m0.z), ze[1] = __uint_as_float(m0.w);
         sc[2] = __uint_as_float(m1.x), ze[2] = __uint_as_float(m1.y), sc[3] = __uint_as_float(m1.z), ze[3] = __uint_as_float(m1.w);
@@ -234,12 +245,12 @@ __device__ __forceinline__ void group_params_of(const uint8_t *rec, bool valid, 
 //   qsum[g]     sum of head gid's query over group g
 //   zacc[g]     sum_t p_t zero_tg for head gid, over the tokens this lane has seen
 //   acc[g][h]   channels 32g + 4gid + 2h (+1) x heads 2tig, 2tig + 1, without the zero-point part
-template <int NS, int B, bool FULL>
+template <int NS, int B, bool FULL, int META>
 __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int stage, int rows, int gid, int tig, float scale_log2,
                                             const uint32_t (&qa)[4][4], const float (&qsum)[4], float &m_run, float &l_run,
                                             float (&zacc)[4], float (&acc)[4][2][4])
 {
-    constexpr int REC = B == 16 ? 2 * kAttendD : kAttendD * B / 8 + 4 * kMetaBytesPerGroup;
+    constexpr int REC = B == 16 ? 2 * kAttendD : kAttendD * B / 8 + 4 * META;
     // the lane's four tokens (the same ones on the score side and on the value side)
     int tok[4];
 #pragma unroll
@@ -255,7 +266,7 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 uint32_t e[4] = {0u, 0u, 0u, 0u};  // lanes without a token feed zeros
-                if (FULL || t < rows) key_pairs<B>(rec, g, tig, e);
+                if (FULL || t < rows) key_pairs<B, META>(rec, g, tig, e);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) sacc[bi][g][i] = 0.0f;
                 mma_m16n8k16(sacc[bi][g], qa[g][0], 0u, qa[g][1], 0u, e[0], e[1]);  // the whole warp, together
@@ -265,7 +276,7 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             float sc[4], ze[4];
-            group_params_of<B>(sm.k[stage] + tok[i] * REC, FULL || tok[i] < rows, sc, ze);
+            group_params_of<B, META>(sm.k[stage] + tok[i] * REC, FULL || tok[i] < rows, sc, ze);
             float dot = 0.0f;
 #pragma unroll
             for (int g = 0; g < 4; ++g) dot = fmaf(sc[g], sacc[i >> 1][g][i & 1], fmaf(ze[g], qsum[g], dot));
@@ -305,7 +316,7 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         float ze[4];
-        group_params_of<B>(sm.v[stage] + tok[i] * REC, FULL || tok[i] < rows, vs[i], ze);
+        group_params_of<B, META>(sm.v[stage] + tok[i] * REC, FULL || tok[i] < rows, vs[i], ze);
 #pragma unroll
         for (int g = 0; g < 4; ++g) zacc[g] = fmaf(pr[i], ze[g], zacc[g]);
     }
@@ -319,14 +330,14 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
         const uint32_t pb0 = as_u32(__floats2half2_rn(pr[0] * vs[0][g], pr[1] * vs[1][g]));
         const uint32_t pb1 = as_u32(__floats2half2_rn(pr[2] * vs[2][g], pr[3] * vs[3][g]));
         uint32_t eab[4], ecd[4];
-        value_pairs<B>(rv[0], rv[1], g, gid, eab);
-        value_pairs<B>(rv[2], rv[3], g, gid, ecd);
+        value_pairs<B, META>(rv[0], rv[1], g, gid, eab);
+        value_pairs<B, META>(rv[2], rv[3], g, gid, ecd);
         mma_m16n8k16(acc[g][0], eab[0], eab[1], ecd[0], ecd[1], pb0, pb1);
         mma_m16n8k16(acc[g][1], eab[2], eab[3], ecd[2], ecd[3], pb0, pb1);
     }
 }
 
-template <int NS, int WARPS>
+template <int NS, int WARPS, int META>
 __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -345,6 +356,7 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
         hp.n_kv_heads = p.n_kv_heads;
         hp.head_dim = kAttendD;
         hp.n_tokens = p.n_tokens;
+        hp.meta_bytes = META;
         const uint32_t mode = hdr->bits_mode;
         int ok = 0;
         if (mode <= 1u) {
@@ -414,7 +426,7 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
                 my_cls[r] = 4;
                 if (j < n_tok) {
                     const uint32_t b = __ldg(bits_tab + j);
-                    const uint32_t rec = record_bytes(kAttendD, (int)b);
+                    const uint32_t rec = record_bytes(kAttendD, (int)b, META);
                     const bool fine = base_ok && rec != 0u && o_next >= o && o_next - o == rec && (o & 15u) == 0u &&
                                       base_k + (uint64_t)o_next <= total_bytes && base_v + (uint64_t)o_next <= total_bytes;
                     bad |= !fine;
@@ -494,7 +506,7 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
         for (; in_flight < NS && !iss.done(); ++in_flight) {
             int st = stage + in_flight;
             if (st >= NS) st -= NS;
-            attend_issue<NS>(sm, st, iss, base_k, base_v, p, lane);
+            attend_issue<NS, META>(sm, st, iss, base_k, base_v, p, lane);
             iss.next();
         }
         while (!con.done()) {
@@ -503,23 +515,23 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             const int rows = con.rows();
             if (rows == kAttendRows) {
                 switch (con.c) {
-                    case 0: attend_step<NS, 2, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 1: attend_step<NS, 4, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 2: attend_step<NS, 8, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    default: attend_step<NS, 16, true>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 0: attend_step<NS, 2, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 1: attend_step<NS, 4, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 2: attend_step<NS, 8, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    default: attend_step<NS, 16, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                 }
             } else {
                 switch (con.c) {
-                    case 0: attend_step<NS, 2, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 1: attend_step<NS, 4, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 2: attend_step<NS, 8, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    default: attend_step<NS, 16, false>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 0: attend_step<NS, 2, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 1: attend_step<NS, 4, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 2: attend_step<NS, 8, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    default: attend_step<NS, 16, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                 }
             }
             con.next();
             __syncwarp();  // every lane has read the stage: it can be re-armed
             if (!iss.done()) {
-                attend_issue<NS>(sm, stage, iss, base_k, base_v, p, lane);
+                attend_issue<NS, META>(sm, stage, iss, base_k, base_v, p, lane);
                 iss.next();
             }
             if (++stage == NS) {

@@ -268,8 +268,8 @@ struct CreateWarpSmem {
 // eight lanes served together by a 128-bit shared-memory access fall into eight different
 // 16-byte bank columns; the packed codes are put back in channel order before they are stored.
 // `rec` is the row's record in the card.  B is the warp-uniform bit-width, or 0 when rows
-// differ (then `b`).
-template <int D, int B>
+// differ (then `b`); META the bytes of {scale, zero} per group.
+template <int D, int B, int META>
 __device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *rec, int lane, int g, int b)
 {
     constexpr int G = D / kGroup;
@@ -286,8 +286,11 @@ __device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *re
     }
     float mn, mx;
     group_min_max(v, mn, mx);
-    const GroupParams gp = group_params(mn, mx, bb);
-    __stcs(reinterpret_cast<float2 *>(rec + g * kMetaBytesPerGroup), make_float2(gp.scale, gp.zero));
+    const GroupParams gp = group_params<META>(mn, mx, bb);
+    if (META == kMetaFp16)  // both are FP16 values: the conversion is exact
+        __stcs(reinterpret_cast<uint32_t *>(rec + g * META), as_u32(__floats2half2_rn(gp.scale, gp.zero)));
+    else
+        __stcs(reinterpret_cast<float2 *>(rec + g * META), make_float2(gp.scale, gp.zero));
     const uint64_t inv2 = pack_f32x2(gp.inv, gp.inv);
     uint32_t lo[4], hi[4];
 #pragma unroll
@@ -297,7 +300,7 @@ __device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *re
         pack_chunk<B>(f, bb, lo[c], hi[c]);
     }
     unrotate4(lo, rot);
-    uint8_t *codes = rec + G * kMetaBytesPerGroup + g * (4 * bb);  // 32 codes of b bits = 4b bytes
+    uint8_t *codes = rec + G * META + g * (4 * bb);  // 32 codes of b bits = 4b bytes
     if (bb == 8) {
         unrotate4(hi, rot);
         __stcs(reinterpret_cast<uint4 *>(codes), make_uint4(lo[0], hi[0], lo[1], hi[1]));
@@ -310,7 +313,7 @@ __device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *re
 }
 
 // All U passes of a sub-tile.  Every lane of the warp calls this (it shuffles).
-template <int D, int B>
+template <int D, int B, int META>
 __device__ __forceinline__ void encode_rows(const uint8_t *in, uint8_t *stream, const Tables &t, int lane)
 {
     using C = WarpCfg<D>;
@@ -321,7 +324,7 @@ __device__ __forceinline__ void encode_rows(const uint8_t *in, uint8_t *stream, 
         const uint32_t off_row = __shfl_sync(0xffffffffu, t.off, row);
         const int b = B ? B : (int)__shfl_sync(0xffffffffu, t.bits, row);
         if (lane < C::GROUPS && row < t.rows)
-            encode_group<D, B>(in + u * (C::R * C::ROW_BYTES), stream + off_row, lane, g, b);
+            encode_group<D, B, META>(in + u * (C::R * C::ROW_BYTES), stream + off_row, lane, g, b);
     }
 }
 
@@ -344,7 +347,7 @@ __device__ __forceinline__ void create_issue(CreateWarpSmem<D, NS> &sm, int stag
     }
 }
 
-template <int D, int NS, int WARPS>
+template <int D, int NS, int WARPS, int META>
 __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) create_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
@@ -412,13 +415,13 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) create_kernel(Pa
         uint8_t *stream = p.card + cur.base;
         if (uniform) {
             switch (b0) {
-                case 4: encode_rows<D, 4>(in, stream, cur, lane); break;
-                case 2: encode_rows<D, 2>(in, stream, cur, lane); break;
-                case 8: encode_rows<D, 8>(in, stream, cur, lane); break;
-                default: encode_rows<D, 16>(in, stream, cur, lane); break;
+                case 4: encode_rows<D, 4, META>(in, stream, cur, lane); break;
+                case 2: encode_rows<D, 2, META>(in, stream, cur, lane); break;
+                case 8: encode_rows<D, 8, META>(in, stream, cur, lane); break;
+                default: encode_rows<D, 16, META>(in, stream, cur, lane); break;
             }
         } else {
-            encode_rows<D, 0>(in, stream, cur, lane);
+            encode_rows<D, 0, META>(in, stream, cur, lane);
         }
         __syncwarp();  // every lane has read the stage: it can be re-armed
         if (!ahead.cu.done) {
@@ -464,15 +467,18 @@ struct InjectWarpSmem {
 // only known per lane (`b`): then the widths 2, 4 and 8 share one instruction stream -- the codes
 // are fetched as the aligned 8 bytes around them and shifted into place, and the unpacking steps
 // are applied by selection -- so that lanes of different widths do not serialise; only FP16 rows
-// branch off.
-template <int D, int B>
+// branch off.  META: bytes of {scale, zero} per group (the code bytes start 16-byte aligned either
+// way, see qkvs_card_create).
+template <int D, int B, int META>
 __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos)
 {
     constexpr int G = D / kGroup;
     const int bb = B ? B : b;
     if (bb == 16) return *reinterpret_cast<const uint4 *>(rec + pos * 16);
-    const float2 m = *reinterpret_cast<const float2 *>(rec + (pos >> 2) * kMetaBytesPerGroup);
-    const uint8_t *codes = rec + G * kMetaBytesPerGroup + pos * bb;
+    float2 m;
+    if (META == kMetaFp16) m = __half22float2(*reinterpret_cast<const __half2 *>(rec + (pos >> 2) * META));
+    else m = *reinterpret_cast<const float2 *>(rec + (pos >> 2) * META);
+    const uint8_t *codes = rec + G * META + pos * bb;
     uint32_t lo, hi;
     if (B == 8) {
         const uint2 w = *reinterpret_cast<const uint2 *>(codes);
@@ -498,7 +504,7 @@ __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos
 }
 
 // FULL: the sub-tile has all ROWS rows and every lane has a chunk in every pass.
-template <int D, int NS, int B, bool FULL>
+template <int D, int NS, int B, bool FULL, int META>
 __device__ __forceinline__ void inject_rows(const InjectWarpSmem<D, NS> &sm, int stage, int lane, int rows, __half *dst0,
                                             int64_t token_stride)
 {
@@ -510,7 +516,7 @@ __device__ __forceinline__ void inject_rows(const InjectWarpSmem<D, NS> &sm, int
         const int row = ci / C::CPR, pos = ci % C::CPR;
         if (FULL || (ci < C::CHUNKS && row < rows)) {
             const uint32_t inf = sm.info[stage][row];
-            const uint4 out = decode_chunk<D, B>(in + (inf >> 8), (int)(inf & 0xffu), pos);
+            const uint4 out = decode_chunk<D, B, META>(in + (inf >> 8), (int)(inf & 0xffu), pos);
             __stcs(reinterpret_cast<uint4 *>(dst0 + (int64_t)row * token_stride + pos * 8), out);
         }
     }
@@ -523,7 +529,7 @@ __device__ __forceinline__ bool header_matches(const qkvs_card_header_t *h, cons
 {
     bool ok = h->magic == kMagic && h->version == kVersion && h->status == QKVS_OK;
     ok = ok && h->n_layers == p.n_layers && h->n_kv_heads == p.n_kv_heads && h->head_dim == p.head_dim;
-    ok = ok && h->n_tokens == p.n_tokens && h->group_size == kGroup && h->meta_bytes_per_group == kMetaBytesPerGroup;
+    ok = ok && h->n_tokens == p.n_tokens && h->group_size == kGroup && h->meta_bytes_per_group == (uint32_t)p.meta_bytes;
     ok = ok && h->bits_off == sec.bits_off && h->offs_off == sec.offs_off && h->payload_off == sec.payload_off;
     ok = ok && h->sbase_off == sec.sbase_off;
     ok = ok && h->total_bytes <= p.card_bytes && h->total_bytes >= sec.payload_off;
@@ -550,7 +556,7 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
     const uint32_t b0 = __shfl_sync(0xffffffffu, t.bits, 0);
     int bad = 0;
     if (lane < rows) {
-        const uint32_t rec = record_bytes(D, (int)t.bits);
+        const uint32_t rec = record_bytes(D, (int)t.bits, p.meta_bytes);
         bad = (rec == 0u) || (off_next < t.off) || (off_next - t.off != rec);
         sm.info[stage][lane] = ((t.off - off0) << 8) | (t.bits & 0xffu);
     }
@@ -573,7 +579,7 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
     __syncwarp();
 }
 
-template <int D, int NS, int WARPS>
+template <int D, int NS, int WARPS, int META>
 __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) inject_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
@@ -644,14 +650,14 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) inject_kernel(Pa
         __half *dst0 = cons.row;
         if (C::CHUNKS % 32 == 0 && rows == C::ROWS) {
             switch (ub) {
-                case 4: inject_rows<D, NS, 4, true>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                case 2: inject_rows<D, NS, 2, true>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                case 8: inject_rows<D, NS, 8, true>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                case 16: inject_rows<D, NS, 16, true>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                default: inject_rows<D, NS, 0, true>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 4: inject_rows<D, NS, 4, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 2: inject_rows<D, NS, 2, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 8: inject_rows<D, NS, 8, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 16: inject_rows<D, NS, 16, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                default: inject_rows<D, NS, 0, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
             }
         } else {
-            inject_rows<D, NS, 0, false>(sm, stage, lane, rows, dst0, p.token_stride);
+            inject_rows<D, NS, 0, false, META>(sm, stage, lane, rows, dst0, p.token_stride);
         }
         __syncwarp();  // every lane has read the stage: it can be re-armed
         if (more) {

@@ -32,6 +32,7 @@ struct ScanParams {
     uint8_t *card;
     uint64_t capacity;
     int32_t n_layers, n_kv_heads, head_dim, n_tokens, bits_mode;
+    int32_t meta_bytes;   // 8 or 4
     uint64_t model_id, sender_id;
     int64_t position_offset;
     uint32_t *workspace;  // the call's scratch block, cleared here for the kernels that follow; or null
@@ -77,7 +78,7 @@ __device__ __forceinline__ void write_header_static(qkvs_card_header_t *h, const
     h->head_dim = p.head_dim;
     h->n_tokens = p.n_tokens;
     h->group_size = kGroup;
-    h->meta_bytes_per_group = kMetaBytesPerGroup;
+    h->meta_bytes_per_group = (uint32_t)p.meta_bytes;
     h->model_id = p.model_id;
     h->sender_id = p.sender_id;
     h->position_offset = p.position_offset;
@@ -124,7 +125,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
             bv[i] = 0;
             if (t0 + i < T) {
                 bv[i] = bits[t0 + i];
-                rec[i] = record_bytes(d, bv[i]);
+                rec[i] = record_bytes(d, bv[i], p.meta_bytes);
                 bad |= rec[i] == 0u;
                 sum_bits += bv[i];
                 mine += rec[i];
@@ -362,6 +363,10 @@ static qkvs_status_t check_shape(const qkvs_layout_t *l)
     // offsets inside a stream are 32-bit
     if ((uint64_t)l->n_tokens * 2u * (uint64_t)l->head_dim > 0xffffffffull) return QKVS_ERR_UNSUPPORTED_SHAPE;
     if ((uint64_t)l->n_layers * (uint64_t)l->n_kv_heads > (1u << 24)) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    const int meta = meta_bytes_of(l->meta_bytes);
+    if (meta == 0) return QKVS_ERR_INVALID_ARG;
+    // records must stay multiples of 16 bytes: four bytes per group need groups in fours
+    if (meta == kMetaFp16 && l->head_dim % 128 != 0) return QKVS_ERR_UNSUPPORTED_SHAPE;
     return QKVS_OK;
 }
 
@@ -464,18 +469,46 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
     return cudaLaunchKernelEx(&cfg, kernel, p, ptrs);
 }
 
-template <int D>
+template <int D, int META>
 static cudaError_t launch_create(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D, QKVS_WARPS_CREATE, D * 2>(create_kernel<D, kStagesCreate, QKVS_WARPS_CREATE>,
-                                                   QKVS_WARPS_CREATE * sizeof(CreateWarpSmem<D, kStagesCreate>), p, ptrs, streams, st, true);
+    return launch_path<D, QKVS_WARPS_CREATE, D * 4 + META>(create_kernel<D, kStagesCreate, QKVS_WARPS_CREATE, META>,
+                                                          QKVS_WARPS_CREATE * sizeof(CreateWarpSmem<D, kStagesCreate>), p, ptrs, streams, st, true);
 }
 
-template <int D>
+template <int D, int META>
 static cudaError_t launch_inject(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D, QKVS_WARPS_INJECT, D * 2 + 1>(inject_kernel<D, kStagesInject, QKVS_WARPS_INJECT>,
-                                                       QKVS_WARPS_INJECT * sizeof(InjectWarpSmem<D, kStagesInject>), p, ptrs, streams, st, false);
+    return launch_path<D, QKVS_WARPS_INJECT, D * 4 + META + 1>(inject_kernel<D, kStagesInject, QKVS_WARPS_INJECT, META>,
+                                                              QKVS_WARPS_INJECT * sizeof(InjectWarpSmem<D, kStagesInject>), p, ptrs, streams, st, false);
+}
+
+// The kernel instance for a checked shape: every head_dim with fp32 pairs, 128 and 256 with FP16
+// pairs.
+static cudaError_t launch_create_for(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+{
+    if (p.meta_bytes == kMetaFp16)
+        return p.head_dim == 128 ? launch_create<128, kMetaFp16>(p, ptrs, streams, st)
+                                 : launch_create<256, kMetaFp16>(p, ptrs, streams, st);
+    switch (p.head_dim) {
+        case 64: return launch_create<64, kMetaFp32>(p, ptrs, streams, st);
+        case 128: return launch_create<128, kMetaFp32>(p, ptrs, streams, st);
+        case 192: return launch_create<192, kMetaFp32>(p, ptrs, streams, st);
+        default: return launch_create<256, kMetaFp32>(p, ptrs, streams, st);
+    }
+}
+
+static cudaError_t launch_inject_for(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+{
+    if (p.meta_bytes == kMetaFp16)
+        return p.head_dim == 128 ? launch_inject<128, kMetaFp16>(p, ptrs, streams, st)
+                                 : launch_inject<256, kMetaFp16>(p, ptrs, streams, st);
+    switch (p.head_dim) {
+        case 64: return launch_inject<64, kMetaFp32>(p, ptrs, streams, st);
+        case 128: return launch_inject<128, kMetaFp32>(p, ptrs, streams, st);
+        case 192: return launch_inject<192, kMetaFp32>(p, ptrs, streams, st);
+        default: return launch_inject<256, kMetaFp32>(p, ptrs, streams, st);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -518,10 +551,12 @@ using namespace qkvs;
 
 extern "C" {
 
-size_t qkvs_record_bytes(int32_t head_dim, int32_t b)
+size_t qkvs_record_bytes(int32_t head_dim, int32_t b, int32_t meta_bytes)
 {
-    if (head_dim <= 0 || head_dim % 64 != 0) return 0;
-    return record_bytes(head_dim, b);
+    const int meta = meta_bytes_of(meta_bytes);
+    if (head_dim <= 0 || head_dim % 64 != 0 || meta == 0) return 0;
+    if (meta == kMetaFp16 && head_dim % 128 != 0) return 0;
+    return record_bytes(head_dim, b, meta);
 }
 
 qkvs_status_t qkvs_card_prefix_size(const qkvs_layout_t *layout, size_t *out_bytes)
@@ -546,7 +581,7 @@ qkvs_status_t qkvs_card_size(const qkvs_layout_t *layout, const uint8_t *bits_ho
     for (int64_t seg = 0; seg < nseg; ++seg) {
         uint64_t seg_bytes = 0;
         for (int64_t t = 0; t < T; ++t) {
-            const uint32_t r = record_bytes(layout->head_dim, bits_host ? bits_host[seg * T + t] : 16);
+            const uint32_t r = record_bytes(layout->head_dim, bits_host ? bits_host[seg * T + t] : 16, meta_bytes_of(layout->meta_bytes));
             if (r == 0) return QKVS_ERR_BAD_BITS;
             seg_bytes += r;
         }
@@ -581,6 +616,7 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
     sp.head_dim = layout->head_dim;
     sp.n_tokens = layout->n_tokens;
     sp.bits_mode = layout->bits_mode;
+    sp.meta_bytes = meta_bytes_of(layout->meta_bytes);
     sp.model_id = meta ? meta->model_id : 0;
     sp.sender_id = meta ? meta->sender_id : 0;
     sp.position_offset = meta ? meta->position_offset : 0;
@@ -603,6 +639,7 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
     p.head_dim = layout->head_dim;
     p.n_tokens = layout->n_tokens;
     p.bits_mode = layout->bits_mode;
+    p.meta_bytes = meta_bytes_of(layout->meta_bytes);
     p.head_stride = layout->head_stride;
     p.token_stride = layout->token_stride;
     for (int l0 = 0; l0 < layout->n_layers; l0 += kMaxLayersPerLaunch) {
@@ -617,14 +654,7 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
         p.layer_count = n;
         p.work_counter = work_counter(workspace_dev, l0 / kMaxLayersPerLaunch);
         const int64_t streams = 2ll * n * layout->n_kv_heads;
-        cudaError_t e;
-        switch (layout->head_dim) {
-            case 64: e = launch_create<64>(p, ptrs, streams, cs); break;
-            case 128: e = launch_create<128>(p, ptrs, streams, cs); break;
-            case 192: e = launch_create<192>(p, ptrs, streams, cs); break;
-            default: e = launch_create<256>(p, ptrs, streams, cs); break;
-        }
-        if (e != cudaSuccess) return QKVS_ERR_CUDA;
+        if (launch_create_for(p, ptrs, streams, cs) != cudaSuccess) return QKVS_ERR_CUDA;
     }
     return QKVS_OK;
 }
@@ -655,6 +685,7 @@ qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qk
     p.head_dim = dst->head_dim;
     p.n_tokens = dst->n_tokens;
     p.bits_mode = 0;  // taken from the card on the device
+    p.meta_bytes = meta_bytes_of(dst->meta_bytes);  // the card's header must say the same
     p.head_stride = dst->head_stride;
     p.token_stride = dst->token_stride;
     p.dst_token_offset = dst_token_offset;
@@ -671,14 +702,7 @@ qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qk
         p.layer_count = n;
         p.work_counter = work_counter(workspace_dev, l0 / kMaxLayersPerLaunch);
         const int64_t streams = 2ll * n * dst->n_kv_heads;
-        cudaError_t e;
-        switch (dst->head_dim) {
-            case 64: e = launch_inject<64>(p, ptrs, streams, cs); break;
-            case 128: e = launch_inject<128>(p, ptrs, streams, cs); break;
-            case 192: e = launch_inject<192>(p, ptrs, streams, cs); break;
-            default: e = launch_inject<256>(p, ptrs, streams, cs); break;
-        }
-        if (e != cudaSuccess) return QKVS_ERR_CUDA;
+        if (launch_inject_for(p, ptrs, streams, cs) != cudaSuccess) return QKVS_ERR_CUDA;
     }
     return QKVS_OK;
 }
@@ -714,6 +738,7 @@ qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t card_bytes, 
     p.head_dim = dst->head_dim;
     p.n_tokens = dst->n_tokens;
     p.bits_mode = 0;  // taken from the card on the device
+    p.meta_bytes = meta_bytes_of(dst->meta_bytes);  // the card's header must say the same
     p.head_stride = dst->head_stride;
     p.token_stride = dst->token_stride;
     p.dst_token_offset = dst_token_offset;
@@ -730,14 +755,7 @@ qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t card_bytes, 
         p.layer_count = n;
         p.work_counter = counters + l0 / kMaxLayersPerLaunch;
         const int64_t streams = 2ll * n * dst->n_kv_heads;
-        cudaError_t e;
-        switch (dst->head_dim) {
-            case 64: e = launch_inject<64>(p, ptrs, streams, cs); break;
-            case 128: e = launch_inject<128>(p, ptrs, streams, cs); break;
-            case 192: e = launch_inject<192>(p, ptrs, streams, cs); break;
-            default: e = launch_inject<256>(p, ptrs, streams, cs); break;
-        }
-        if (e != cudaSuccess) return QKVS_ERR_CUDA;
+        if (launch_inject_for(p, ptrs, streams, cs) != cudaSuccess) return QKVS_ERR_CUDA;
     }
     return QKVS_OK;
 }
@@ -755,6 +773,7 @@ static qkvs_status_t attend_shape(const qkvs_layout_t *layout, int32_t n_q_heads
     p->n_kv_heads = layout->n_kv_heads;
     p->n_tokens = layout->n_tokens;
     p->n_q_heads = n_q_heads;
+    p->meta_bytes = meta_bytes_of(layout->meta_bytes);
     p->subs_per_head = (uint32_t)(((int64_t)layout->n_tokens + kAttendRows - 1) / kAttendRows);
     p->items_per_head = (p->subs_per_head + kAttendSteps - 1) / kAttendSteps;
     const uint64_t n_items = (uint64_t)layout->n_layers * (uint64_t)layout->n_kv_heads * p->items_per_head;
@@ -803,10 +822,12 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
     p.work_counter = static_cast<uint32_t *>(scratch_dev) + 1;
     p.partials = reinterpret_cast<float *>(static_cast<uint8_t *>(scratch_dev) + QKVS_WORKSPACE_BYTES);
     if (p.n_items > 0) {
-        auto kernel = attend_kernel<kAttendStages, kAttendWarps>;
+        const bool compact = p.meta_bytes == kMetaFp16;
+        auto kernel = compact ? attend_kernel<kAttendStages, kAttendWarps, kMetaFp16> : attend_kernel<kAttendStages, kAttendWarps, kMetaFp32>;
         const size_t smem = kAttendWarps * sizeof(AttendWarpSmem<kAttendStages>);
         unsigned grid = 0;
-        if (persistent_grid<1000>(kernel, kAttendWarps * 32, smem, (int64_t)((p.n_items + kAttendWarps - 1) / kAttendWarps), &grid) !=
+        if ((compact ? persistent_grid<1001>(kernel, kAttendWarps * 32, smem, (int64_t)((p.n_items + kAttendWarps - 1) / kAttendWarps), &grid)
+                     : persistent_grid<1000>(kernel, kAttendWarps * 32, smem, (int64_t)((p.n_items + kAttendWarps - 1) / kAttendWarps), &grid)) !=
             cudaSuccess)
             return QKVS_ERR_CUDA;
         kernel<<<grid, kAttendWarps * 32, smem, cs>>>(p);

@@ -59,6 +59,22 @@ def test_host_only_sizes(lib):
     bits = np.tile(np.array([2, 4, 8, 16, 4], np.uint8), 6)
     per_seg = 32 + 48 + 80 + 128 + 48
     assert q.card_size(lay1, bits) == 256 + a(30) + a(4 * 6 * 6) + a(8 * 13) + 12 * per_seg
+    # compact metadata: four bytes per group, head_dim a multiple of 128
+    for d, b, n in fx["crec"]:
+        assert q.record_bytes(int(d), int(b), 4) == int(n)
+    assert q.record_bytes(64, 4, 4) == 0 and q.record_bytes(128, 4, 3) == 0
+    assert q.record_bytes(128, 4, 0) == q.record_bytes(128, 4, 8)
+    for L, H, d, T, c16, c8, c4, c2, payload in fx["cpayload"]:
+        L, H, d, T = int(L), int(H), int(d), int(T)
+        bits = np.concatenate([np.full(int(c16), 16), np.full(int(c8), 8), np.full(int(c4), 4),
+                               np.full(int(c2), 2)]).astype(np.uint8)
+        assert q.card_size(q.make_layout(L, H, d, T, meta_bytes=4), bits) == 256 + a(T) + a(4 * (T + 1)) + int(payload)
+    with pytest.raises(q.QkvsError) as e:
+        q.card_size(q.make_layout(1, 1, 64, 4, meta_bytes=4), None)
+    assert e.value.status == q.binding.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(q.QkvsError) as e:
+        q.card_size(q.make_layout(1, 1, 128, 4, meta_bytes=16), None)
+    assert e.value.status == q.binding.ERR_INVALID_ARG
 
 
 def test_status_strings_and_version(lib):
