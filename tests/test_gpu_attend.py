@@ -1,7 +1,8 @@
 """Attention straight from the card: CUDA path against the oracle, through the C-ABI, on a B200.
 
-Tolerance.  Both sides use exactly the same reconstructed K^, V^ (FP16).  The CUDA path rounds
-the softmax weights to FP16 (relative 2^-11) before the tensor-core product with V^, accumulates
+Tolerance.  Both sides attend to the values the records stand for (code * scale + zero, not
+rounded to FP16).  The CUDA path rounds the softmax weights, times the scale, to FP16 (relative
+2^-11) before the tensor-core product with the codes, accumulates
 in FP32 and uses the hardware exp2 (relative 2^-22); everything else is below that.  A convex
 combination of values with weights off by 2^-11 relative moves by at most 2^-11 * max|V^| (twice
 that when numerator and denominator are counted separately): the tests allow
