@@ -231,8 +231,11 @@ def run_ours(args):
     w, Ks, Vs = load_workload(args.config, n_layers=args.layers)
     L, H, d, T = w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens
     hops = w.hops
-    bits_per_hop = [wl.bits_for(w, h) for h in range(hops)]
-    lay = q.make_layout(L, H, d, T, meta_bytes=args.meta_bytes)
+    if args.bits_mode == 1:
+        bits_per_hop = [wl.bits_per_head(w, h) for h in range(hops)]
+    else:
+        bits_per_hop = [wl.bits_for(w, h) for h in range(hops)]
+    lay = q.make_layout(L, H, d, T, bits_mode=args.bits_mode, meta_bytes=args.meta_bytes)
     sizes = [q.card_size(lay, b) for b in bits_per_hop]
     prefix = q.card_prefix_size(lay)
     kv_bytes = w.kv_bytes
@@ -431,15 +434,17 @@ def run_ours(args):
     else:
         dom, dom_ms, dom_key = "inject_kernel", i0, "inject_kernel"
     achieved = (kv_bytes + payload0) / (dom_ms * 1e-3) / 1e9
-    traffic = captured_traffic(dom_key, L) if w.number == 3 and args.meta_bytes == 8 else None
+    traffic = captured_traffic(dom_key, L) if w.number == 3 and args.meta_bytes == 8 and args.bits_mode == 0 else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src, "traffic": traffic,
                 "algorithmic_bytes_per_launch": kv_bytes + payload0, "avg_launch_ms": dom_ms}
 
-    launches_per_step = hops * (2 + 1) * ((L + 63) // 64) - hops * (((L + 63) // 64) - 1)
+    # per hop: the offset scan (plus its second stage with per-head bit-widths), then one create
+    # and one inject launch per block of 64 layers
+    launches_per_step = hops * (1 + args.bits_mode + 2 * ((L + 63) // 64))
     cpu = None
     if not args.no_cpu_baseline:
-        cpu = cpu_oracle_leg(w, Ks, Vs, bits_per_hop[0], L, args.meta_bytes)
+        cpu = cpu_oracle_leg(w, Ks, Vs, bits_per_hop[0][:T], L, args.meta_bytes)
 
     # the step in front of the path: bit-widths from importance scores by rank (config 4's recipe)
     rank_us = None
@@ -463,7 +468,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "n_layers": L, "n_kv_heads": H, "head_dim": d, "n_tokens": T,
                    "hops": hops, "fp16_kv_bytes": kv_bytes, "replicas": world,
-                   "meta_bytes_per_group": args.meta_bytes,
+                   "meta_bytes_per_group": args.meta_bytes, "bits_mode": args.bits_mode,
                    "reduced_for_profiling": bool(args.layers),
                    "l2": "inputs (1 GiB FP16 KV per pass) exceed the 126 MB L2; no flush"
                    if kv_bytes > 4 * 126e6 else "working set comparable to L2; L2 helps"},
@@ -502,6 +507,8 @@ def main():
     ap.add_argument("--meta-bytes", type=int, default=8, choices=[8, 4],
                     help="bytes of scale and zero per group in the card: 8 = two fp32 (the headline format), "
                          "4 = two FP16 (compact variant)")
+    ap.add_argument("--bits-mode", type=int, default=0, choices=[0, 1],
+                    help="0: one bit-width vector for the whole model (the paper's); 1: one per (layer, KV head)")
     ap.add_argument("--layers", type=int, default=0,
                     help="reduced case for profiler captures: keep the workload's recipe at this many layers")
     args = ap.parse_args()

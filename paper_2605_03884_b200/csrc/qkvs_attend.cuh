@@ -16,11 +16,13 @@
 // two bulk copies (TMA) on one mbarrier, NS steps ahead.  Operand layouts are chosen -- the order
 // of channels inside a group and of tokens inside a step is free in a contraction -- so that every
 // lane builds its fragments from a few bytes of its own with shifts and masks:
-//   scores   rows = query heads of the group (up to 8 of 16 used), columns = 8 tokens; lane (g, t)
-//            supplies 8 codes of token g from each group and holds the matching channels of Q;
+//   scores   rows = the 16 tokens of a step, columns = the query heads of the group (up to 8);
+//            lane (g, t) supplies 8 codes per group of the tokens g and g + 8 and holds the matching
+//            channels of head g's query; it receives the scores of its two tokens for heads 2t, 2t+1;
 //   outputs  rows = channels, columns = query heads; lane (g, t) supplies 4 channels per group of
-//            the four tokens 2t, 2t+1, 2t+8, 2t+9, and the probabilities it computed itself, times
-//            the tokens' scales, are already the B fragment.
+//            the four tokens 2t, 2t+1, 2t+8, 2t+9; the weights (probabilities times the tokens'
+//            scales, FP16) are moved from the score layout into the B fragment by an 8 x 8
+//            transpose inside the warp (movmatrix); the accumulators are again heads 2t, 2t+1.
 // Softmax is the usual running maximum / running sum; every item leaves (o, max, sum) per query
 // head in the scratch buffer and a second small kernel merges the items of a head.
 #pragma once
@@ -67,6 +69,25 @@ __device__ __forceinline__ void mma_m16n8k16(float (&c)[4], uint32_t a0, uint32_
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// The same product with a zero accumulator coming in.
+__device__ __forceinline__ void mma_m16n8k16_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                                   uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
+}
+
+// Transposes an 8 x 8 matrix of 16-bit elements held one row per group of four lanes, two
+// neighbouring columns per lane: afterwards lane (gid, tig) holds what was in rows 2tig, 2tig + 1
+// of column gid.
+__device__ __forceinline__ uint32_t transpose_8x8(uint32_t v)
+{
+    uint32_t r;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(r) : "r"(v));
+    return r;
 }
 
 __device__ __forceinline__ float exp2_approx(float x)
@@ -239,101 +260,119 @@ __device__ __forceinline__ void group_params_of(const uint8_t *rec, bool valid, 
 }
 
 // One step: up to 16 tokens of one bit-width B, their K and V records packed one after another in
-// `stage`, against the group's queries.  Updates the running maximum / sum of head gid, the
-// zero-point sums and the output accumulators.  FULL: all 16 tokens are there.
-//   qa[g][k]    query fragments: head gid, channels 32g + 8tig + k and + k + 4
-//   qsum[g]     sum of head gid's query over group g
-//   zacc[g]     sum_t p_t zero_tg for head gid, over the tokens this lane has seen
-//   acc[g][h]   channels 32g + 4gid + 2h (+1) x heads 2tig, 2tig + 1, without the zero-point part
+// `stage`, against the group's queries.  Lane (gid, tig) owns the tokens gid and gid + 8 of the
+// step on the score side and the query heads 2tig and 2tig + 1 throughout, so that the running
+// maximum and sum of a head, the factors that rescale its accumulators and the accumulators
+// themselves sit in the same lane.  FULL: all 16 tokens are there.
+//   qb[g][k]     query fragments (B operand): head gid, channels 32g + 8tig + k and + k + 4
+//   qsum[g][h]   sum of head 2tig + h's query over group g
+//   m_run[h], l_run[h]   running maximum of head 2tig + h (the same in all lanes of a tig) and this
+//                lane's share of its running sum (tokens gid, gid + 8 of every step)
+//   zacc[g][h]   this lane's share of sum_t p_t zero_tg for head 2tig + h
+//   acc[g][j][.] channels 32g + 4gid + 2j (+1) x heads 2tig, 2tig + 1, without the zero-point part
 template <int NS, int B, bool FULL, int META>
 __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int stage, int rows, int gid, int tig, float scale_log2,
-                                            const uint32_t (&qa)[4][4], const float (&qsum)[4], float &m_run, float &l_run,
-                                            float (&zacc)[4], float (&acc)[4][2][4])
+                                            const uint32_t (&qb)[4][4], const float (&qsum)[4][2], float (&m_run)[2],
+                                            float (&l_run)[2], float (&zacc)[4][2], float (&acc)[4][2][4])
 {
     constexpr int REC = B == 16 ? 2 * kAttendD : kAttendD * B / 8 + 4 * META;
-    // the lane's four tokens (the same ones on the score side and on the value side)
-    int tok[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) tok[i] = 2 * tig + (i & 1) + 8 * (i >> 1);
-    // ---- scores: per group, sum_c q_c code_c for the heads of the group x 2 blocks of 8 tokens
-    float x[4];  // logits (base 2) of head gid for the lane's four tokens
+    const bool have[2] = {FULL || gid < rows, FULL || gid + 8 < rows};
+    const uint8_t *krec[2] = {sm.k[stage] + gid * REC, sm.k[stage] + (gid + 8) * REC};
+    const uint8_t *vrec[2] = {sm.v[stage] + gid * REC, sm.v[stage] + (gid + 8) * REC};
+    // ---- scores: rows = the 16 tokens, columns = the group's heads; per group of 32 channels
+    // sum_c code_c q_c, two products of 16 channels each
+    float x[2][2];  // logits (base 2): [token gid + 8k][head 2tig + h]
     {
-        float sacc[2][4][4];
-#pragma unroll
-        for (int bi = 0; bi < 2; ++bi) {
-            const int t = 8 * bi + gid;
-            const uint8_t *rec = sm.k[stage] + t * REC;
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                uint32_t e[4] = {0u, 0u, 0u, 0u};  // lanes without a token feed zeros
-                if (FULL || t < rows) key_pairs<B, META>(rec, g, tig, e);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) sacc[bi][g][i] = 0.0f;
-                mma_m16n8k16(sacc[bi][g], qa[g][0], 0u, qa[g][1], 0u, e[0], e[1]);  // the whole warp, together
-                mma_m16n8k16(sacc[bi][g], qa[g][2], 0u, qa[g][3], 0u, e[2], e[3]);
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float sc[4], ze[4];
-            group_params_of<B, META>(sm.k[stage] + tok[i] * REC, FULL || tok[i] < rows, sc, ze);
-            float dot = 0.0f;
-#pragma unroll
-            for (int g = 0; g < 4; ++g) dot = fmaf(sc[g], sacc[i >> 1][g][i & 1], fmaf(ze[g], qsum[g], dot));
-            x[i] = (FULL || tok[i] < rows) ? dot * scale_log2 : -INFINITY;
-        }
-    }
-    // ---- running softmax for head gid
-    float m_loc = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
-    m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 1));
-    m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 2));
-    const float m_new = fmaxf(m_run, m_loc);
-    const float m_ref = m_new == -INFINITY ? 0.0f : m_new;
-    const float alpha = exp2_approx(m_run - m_ref);  // 0 on the first tokens of the item
-    float pr[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) pr[i] = exp2_approx(x[i] - m_ref);
-    l_run = fmaf(l_run, alpha, (pr[0] + pr[1]) + (pr[2] + pr[3]));
-    m_run = m_new;
-    // the accumulators of this lane belong to heads 2t and 2t + 1, whose factors other lanes hold
-    const float a_lo = __shfl_sync(0xffffffffu, alpha, 8 * tig);
-    const float a_hi = __shfl_sync(0xffffffffu, alpha, 8 * tig + 4);
-    if (__any_sync(0xffffffffu, a_lo != 1.0f || a_hi != 1.0f || alpha != 1.0f)) {
+        float sacc[4][4];
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            zacc[g] *= alpha;
+            uint32_t ea[4] = {0u, 0u, 0u, 0u}, eb[4] = {0u, 0u, 0u, 0u};  // lanes without a token feed zeros
+            if (have[0]) key_pairs<B, META>(krec[0], g, tig, ea);
+            if (have[1]) key_pairs<B, META>(krec[1], g, tig, eb);
+            mma_m16n8k16_first(sacc[g], ea[0], eb[0], ea[1], eb[1], qb[g][0], qb[g][1]);  // the whole warp, together
+            mma_m16n8k16(sacc[g], ea[2], eb[2], ea[3], eb[3], qb[g][2], qb[g][3]);
+        }
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            float sc[4], ze[4];
+            group_params_of<B, META>(krec[k], have[k], sc, ze);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                acc[g][h][0] *= a_lo;
-                acc[g][h][1] *= a_hi;
-                acc[g][h][2] *= a_lo;
-                acc[g][h][3] *= a_hi;
+                float dot = 0.0f;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) dot = fmaf(sc[g], sacc[g][2 * k + h], fmaf(ze[g], qsum[g][h], dot));
+                x[k][h] = have[k] ? dot * scale_log2 : -INFINITY;
             }
         }
     }
-    // ---- values: probabilities times the tokens' scales against the codes; zero points aside
-    float vs[4][4];  // [token][group]
+    // ---- running softmax of heads 2tig and 2tig + 1 (the maximum goes over all 16 tokens: the
+    // eight lanes of a tig)
+    float pr[2][2], alpha[2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float ze[4];
-        group_params_of<B, META>(sm.v[stage] + tok[i] * REC, FULL || tok[i] < rows, vs[i], ze);
-#pragma unroll
-        for (int g = 0; g < 4; ++g) zacc[g] = fmaf(pr[i], ze[g], zacc[g]);
+    for (int h = 0; h < 2; ++h) {
+        float m_loc = fmaxf(x[0][h], x[1][h]);
+        m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 4));
+        m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 8));
+        m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 16));
+        const float m_new = fmaxf(m_run[h], m_loc);
+        const float m_ref = m_new == -INFINITY ? 0.0f : m_new;
+        alpha[h] = exp2_approx(m_run[h] - m_ref);  // 0 on the first tokens of the item
+        pr[0][h] = exp2_approx(x[0][h] - m_ref);
+        pr[1][h] = exp2_approx(x[1][h] - m_ref);
+        l_run[h] = fmaf(l_run[h], alpha[h], pr[0][h] + pr[1][h]);
+        m_run[h] = m_new;
     }
-    // records of tokens that are not there hold stale bytes: their probabilities are zero, and so
-    // that nothing non-finite can come out of stale FP16 patterns their rows are read from token 0
+    if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            zacc[g][0] *= alpha[0];
+            zacc[g][1] *= alpha[1];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                acc[g][j][0] *= alpha[0];
+                acc[g][j][1] *= alpha[1];
+                acc[g][j][2] *= alpha[0];
+                acc[g][j][3] *= alpha[1];
+            }
+        }
+    }
+    // ---- values.  The weights p_t * scale_tg are formed where the probabilities are (tokens gid,
+    // gid + 8 x heads 2tig, 2tig + 1), rounded to FP16 and transposed inside the warp into the B
+    // operand (tokens 2tig, 2tig + 1, 2tig + 8, 2tig + 9 x head gid); the zero points go aside.
+    uint32_t wb0[4], wb1[4];
+    {
+        float vs[2][4];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            float ze[4];
+            group_params_of<B, META>(vrec[k], have[k], vs[k], ze);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                zacc[g][0] = fmaf(pr[k][0], ze[g], zacc[g][0]);
+                zacc[g][1] = fmaf(pr[k][1], ze[g], zacc[g][1]);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            wb0[g] = transpose_8x8(as_u32(__floats2half2_rn(pr[0][0] * vs[0][g], pr[0][1] * vs[0][g])));
+            wb1[g] = transpose_8x8(as_u32(__floats2half2_rn(pr[1][0] * vs[1][g], pr[1][1] * vs[1][g])));
+        }
+    }
+    // records of tokens that are not there hold stale bytes: their weights are zero, and so that
+    // nothing non-finite can come out of stale FP16 patterns their rows are read from token 0
     const uint8_t *rv[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) rv[i] = sm.v[stage] + ((FULL || tok[i] < rows) ? tok[i] : 0) * REC;
+    for (int i = 0; i < 4; ++i) {
+        const int t = 2 * tig + (i & 1) + 8 * (i >> 1);
+        rv[i] = sm.v[stage] + ((FULL || t < rows) ? t : 0) * REC;
+    }
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
-        const uint32_t pb0 = as_u32(__floats2half2_rn(pr[0] * vs[0][g], pr[1] * vs[1][g]));
-        const uint32_t pb1 = as_u32(__floats2half2_rn(pr[2] * vs[2][g], pr[3] * vs[3][g]));
         uint32_t eab[4], ecd[4];
         value_pairs<B, META>(rv[0], rv[1], g, gid, eab);
         value_pairs<B, META>(rv[2], rv[3], g, gid, ecd);
-        mma_m16n8k16(acc[g][0], eab[0], eab[1], ecd[0], ecd[1], pb0, pb1);
-        mma_m16n8k16(acc[g][1], eab[2], eab[3], ecd[2], ecd[3], pb0, pb1);
+        mma_m16n8k16(acc[g][0], eab[0], eab[1], ecd[0], ecd[1], wb0[g], wb1[g]);
+        mma_m16n8k16(acc[g][1], eab[2], eab[3], ecd[2], ecd[3], wb0[g], wb1[g]);
     }
 }
 
@@ -470,10 +509,11 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
         iss.begin();
         StepIter con = iss;
 
-        // the group's queries as A fragments: lane (gid, tig) holds head gid, per group the channels
-        // 32g + 8tig + k paired with + k + 4 (the pairing of key_pairs), and the query's sum over the group
+        // the group's queries as B fragments: lane (gid, tig) holds head gid, per group the channels
+        // 32g + 8tig + k paired with + k + 4 (the pairing of key_pairs); and the sums over a group of
+        // the queries of the lane's own two heads
         uint32_t qa[4][4];
-        float qsum[4];
+        float qsum[4][2];
         {
             const __half *qrow = p.q + ((uint64_t)layer * p.n_q_heads + (uint64_t)head * per_kv + gid) * kAttendD + 8 * tig;
 #pragma unroll
@@ -488,12 +528,13 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
                 const float2 f2 = __half22float2(as_half2(h.z)), f3 = __half22float2(as_half2(h.w));
                 float sum = ((f0.x + f0.y) + (f1.x + f1.y)) + ((f2.x + f2.y) + (f3.x + f3.y));
                 sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-                qsum[g] = sum;
+                sum += __shfl_xor_sync(0xffffffffu, sum, 2);  // head gid's, in all four lanes of the gid
+                qsum[g][0] = __shfl_sync(0xffffffffu, sum, 8 * tig);
+                qsum[g][1] = __shfl_sync(0xffffffffu, sum, 8 * tig + 4);
             }
         }
-        float m_run = -INFINITY, l_run = 0.0f;  // of head gid (same in the four lanes of a gid; l_run summed at the end)
-        float zacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
+        float zacc[4][2] = {{0.0f, 0.0f}, {0.0f, 0.0f}, {0.0f, 0.0f}, {0.0f, 0.0f}};
         float acc[4][2][4];
 #pragma unroll
         for (int g = 0; g < 4; ++g)
@@ -542,21 +583,31 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
         if (!ok) break;
 
         // ---- what the item found, per query head: unnormalised o (zero-point part added), maximum, sum
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        float z_lo[4], z_hi[4];  // of heads 2tig and 2tig + 1
+        // the lanes of a tig each hold a share (their tokens) of the sums of heads 2tig, 2tig + 1
+        float z_lo[4], z_hi[4];
+#pragma unroll
+        for (int sft = 4; sft < 32; sft <<= 1) {
+            l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], sft);
+            l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], sft);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                zacc[g][0] += __shfl_xor_sync(0xffffffffu, zacc[g][0], sft);
+                zacc[g][1] += __shfl_xor_sync(0xffffffffu, zacc[g][1], sft);
+            }
+        }
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            float z = zacc[g];
-            z += __shfl_xor_sync(0xffffffffu, z, 1);
-            z += __shfl_xor_sync(0xffffffffu, z, 2);
-            z_lo[g] = __shfl_sync(0xffffffffu, z, 8 * tig);
-            z_hi[g] = __shfl_sync(0xffffffffu, z, 8 * tig + 4);
+            z_lo[g] = zacc[g][0];
+            z_hi[g] = zacc[g][1];
         }
         float *part = p.partials + (uint64_t)item * per_kv * kPartialFloats;
-        if (tig == 0 && gid < per_kv) {
-            part[gid * kPartialFloats + kAttendD] = m_run;
-            part[gid * kPartialFloats + kAttendD + 1] = l_run;
+        if (gid == 0) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                if (2 * tig + h < per_kv) {
+                    part[(2 * tig + h) * kPartialFloats + kAttendD] = m_run[h];
+                    part[(2 * tig + h) * kPartialFloats + kAttendD + 1] = l_run[h];
+                }
         }
 #pragma unroll
         for (int g = 0; g < 4; ++g)

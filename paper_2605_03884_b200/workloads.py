@@ -134,18 +134,26 @@ def quantile_bits(n_tokens: int, seed: int) -> np.ndarray:
     return bits
 
 
-def bits_for(w: Workload, hop: int = 0) -> np.ndarray:
-    """Per-token bit-width vector (uint8, values in {2,4,8,16}; 16 means raw FP16)."""
+def bits_for(w: Workload, hop: int = 0, segment: int = 0) -> np.ndarray:
+    """Per-token bit-width vector (uint8, values in {2,4,8,16}; 16 means raw FP16).  `segment`
+    varies the draw for the per-(layer, head) mode; segment 0 is the whole-model vector."""
     t = w.n_tokens
+    shift = 7919 * segment
     if w.bits_recipe == "uniform4":
         return np.full(t, 4, dtype=np.uint8)
     if w.bits_recipe == "iid":
-        return iid_bits(t, w.iid_probs, w.value_seed + 2)
+        return iid_bits(t, w.iid_probs, w.value_seed + 2 + shift)
     if w.bits_recipe == "quantile":
-        return quantile_bits(t, w.value_seed + 3)
+        return quantile_bits(t, w.value_seed + 3 + shift)
     if w.bits_recipe == "chain":
-        return iid_bits(t, w.iid_probs, 1000 + w.number + 10 + hop)
+        return iid_bits(t, w.iid_probs, 1000 + w.number + 10 + hop + shift)
     raise ValueError(w.bits_recipe)
+
+
+def bits_per_head(w: Workload, hop: int = 0) -> np.ndarray:
+    """bits[n_layers * n_kv_heads][n_tokens], flattened: every (layer, head) segment draws the
+    workload's recipe on its own (as a controller that scores tokens per head would)."""
+    return np.concatenate([bits_for(w, hop, seg) for seg in range(w.n_layers * w.n_kv_heads)])
 
 
 def random_fp16(shape, seed: int, scale: float = 1.0) -> np.ndarray:
