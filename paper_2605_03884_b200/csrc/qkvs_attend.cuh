@@ -33,6 +33,9 @@ namespace qkvs {
 
 constexpr int kAttendD = 128;
 constexpr int kAttendRows = 16;          // tokens per step
+constexpr int kAttendRecMax = 160;       // largest record of which a step takes 16 (8 bits, fp32 pairs)
+constexpr int kAttendStageBytes = kAttendRows * kAttendRecMax;  // per stream; 16-bit rows go 8 per step
+static_assert(kAttendStageBytes >= 8 * 2 * kAttendD && kAttendStageBytes % 128 == 0, "stage size");
 constexpr int kAttendSteps = 16;         // steps per work item
 constexpr int kAttendPerLane = kAttendRows * kAttendSteps / 32;  // tokens of an item per lane when they are sorted
 constexpr int kAttendMaxPerKv = 8;       // query heads per KV head
@@ -57,9 +60,10 @@ struct AttendParams {
 
 template <int NS>
 struct AttendWarpSmem {
-    alignas(128) uint8_t k[NS][kAttendRows * 2 * kAttendD];  // up to 16 records, packed one after another
-    alignas(128) uint8_t v[NS][kAttendRows * 2 * kAttendD];
+    alignas(128) uint8_t k[NS][kAttendStageBytes];  // the step's records, packed one after another
+    alignas(128) uint8_t v[NS][kAttendStageBytes];
     uint32_t list[kAttendRows * kAttendSteps];  // record offsets of the item's tokens, grouped by bit-width
+    uint32_t steps[64];                         // the item's step descriptors
     alignas(8) uint64_t full[NS];
 };
 
@@ -109,53 +113,69 @@ __device__ __forceinline__ uint32_t word_of(const uint4 &v, int i)
 // Bit-width classes in the order they are walked: 2, 4, 8, 16 bits.
 __device__ __forceinline__ uint32_t class_width(int c) { return c == 0 ? 2u : (c == 1 ? 4u : (c == 2 ? 8u : 16u)); }
 
-// The item's steps, in order: class c, tokens [s0, s0 + n) of that class's part of the list.
-struct StepIter {
-    uint32_t s1, s2, s3, s4;  // where classes 1, 2, 3 begin in the list (class 0 begins at 0) and where it ends
-    int c;
-    uint32_t s0;
+// The item's steps are laid out once per item, one descriptor per step, by the lanes in parallel:
+// the tokens of class c occupy [begin_c, end_c) of the list and are walked 16 at a time (16-bit
+// rows, 256 bytes each, 8 at a time: a stage holds eight of them).
+//   bits 0..8  first list position   9..13  tokens in the step   14..15  class
+//   bit 16     the step's records are neighbours in the card (one copy per stream will do)
+constexpr int kAttendMaxSteps = kAttendRows * kAttendSteps / 8 + 3;  // all 16-bit but three tokens, one per other class
 
-    __device__ __forceinline__ uint32_t end_of(int cls) const { return cls == 0 ? s1 : (cls == 1 ? s2 : (cls == 2 ? s3 : s4)); }
-    __device__ __forceinline__ void skip_empty()
-    {
-        while (c < 4 && s0 >= end_of(c)) ++c;  // the next class begins where this one ends
+__device__ __forceinline__ uint32_t step_first(uint32_t d) { return d & 511u; }
+__device__ __forceinline__ int step_rows(uint32_t d) { return (int)((d >> 9) & 31u); }
+__device__ __forceinline__ int step_class(uint32_t d) { return (int)((d >> 14) & 3u); }
+
+template <int META>
+__device__ __forceinline__ uint32_t class_record_bytes(int c)
+{
+    return c == 0 ? (uint32_t)(kAttendD / 4 + 4 * META) : (c == 1 ? (uint32_t)(kAttendD / 2 + 4 * META) : (c == 2 ? (uint32_t)(kAttendD + 4 * META) : 2u * kAttendD));
+}
+
+// Descriptor of step `idx` given where the classes end in the list (e[c], with e[-1] = 0); 0 past the last step.
+template <int META>
+__device__ __forceinline__ uint32_t make_step(uint32_t idx, const uint32_t (&e)[4], const uint32_t *list)
+{
+    uint32_t begin = 0, first_step = 0;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t per = c == 3 ? kAttendRows / 2 : kAttendRows;
+        const uint32_t n_steps = (e[c] - begin + per - 1) / per;
+        if (idx < first_step + n_steps) {
+            const uint32_t s0 = begin + (idx - first_step) * per;
+            const uint32_t rows = min(per, e[c] - s0);
+            const bool neighbours = list[s0 + rows - 1] - list[s0] == (rows - 1) * class_record_bytes<META>(c);
+            return s0 | (rows << 9) | ((uint32_t)c << 14) | (neighbours ? 1u << 16 : 0u);
+        }
+        first_step += n_steps;
+        begin = e[c];
     }
-    __device__ __forceinline__ void begin()
-    {
-        c = 0;
-        s0 = 0;
-        skip_empty();
-    }
-    __device__ __forceinline__ bool done() const { return c >= 4; }
-    __device__ __forceinline__ int rows() const { return (int)min((uint32_t)kAttendRows, end_of(c) - s0); }
-    __device__ __forceinline__ void next()
-    {
-        s0 = min(s0 + kAttendRows, end_of(c));
-        skip_empty();
-    }
-};
+    return 0u;
+}
 
 // Starts the copies of one step's K and V records into `stage`, packed in list order: one copy
-// per stream when the tokens are neighbours in the card, else one per record.  All lanes call it.
+// per stream when the tokens are neighbours in the card (the offsets grow with the token index,
+// so first and last record a step's length apart leave no room for others in between), else one
+// per record.  All lanes call it.
 template <int NS, int META>
-__device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, const StepIter &it, uint64_t base_k,
-                                             uint64_t base_v, const AttendParams &p, int lane)
+__device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, uint32_t d, uint64_t base_k, uint64_t base_v,
+                                             const AttendParams &p, int lane)
 {
-    const int n = it.rows();
-    const uint32_t rec = record_bytes(kAttendD, (int)class_width(it.c), META);
-    const uint32_t mine = lane < n ? sm.list[it.s0 + lane] : 0u;
-    const uint32_t first = __shfl_sync(0xffffffffu, mine, 0);
-    const bool neighbours = __all_sync(0xffffffffu, lane >= n || mine == first + (uint32_t)lane * rec);
-    if (lane == 0) mbar_arrive_expect_tx(&sm.full[stage], 2u * (uint32_t)n * rec);
-    __syncwarp();
-    if (neighbours) {
+    const int n = step_rows(d);
+    const uint32_t rec = class_record_bytes<META>(step_class(d));
+    if (d & (1u << 16)) {
         if (lane == 0) {
+            const uint32_t first = sm.list[step_first(d)];
+            mbar_arrive_expect_tx(&sm.full[stage], 2u * (uint32_t)n * rec);
             bulk_load(sm.k[stage], p.card + base_k + first, (uint32_t)n * rec, &sm.full[stage]);
             bulk_load(sm.v[stage], p.card + base_v + first, (uint32_t)n * rec, &sm.full[stage]);
         }
-    } else if (lane < n) {
-        bulk_load(sm.k[stage] + lane * rec, p.card + base_k + mine, rec, &sm.full[stage]);
-        bulk_load(sm.v[stage] + lane * rec, p.card + base_v + mine, rec, &sm.full[stage]);
+    } else {
+        if (lane == 0) mbar_arrive_expect_tx(&sm.full[stage], 2u * (uint32_t)n * rec);
+        __syncwarp();
+        if (lane < n) {
+            const uint32_t mine = sm.list[step_first(d) + lane];
+            bulk_load(sm.k[stage] + lane * rec, p.card + base_k + mine, rec, &sm.full[stage]);
+            bulk_load(sm.v[stage] + lane * rec, p.card + base_v + mine, rec, &sm.full[stage]);
+        }
     }
 }
 
@@ -168,6 +188,40 @@ __device__ __forceinline__ uint32_t int_pair(uint32_t word, uint32_t mask)
     uint32_t f;
     asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(f) : "r"(word), "r"(mask), "r"(kHalfMagic));  // (a & b) | c
     return as_u32(__hsub2(as_half2(f), as_half2(kHalfMagic)));
+}
+
+// The eight nibbles n0..n7 of a word as four FP16 pairs e[k] = (n_k, n_{k+4}).  The odd nibbles
+// are picked up where they sit, four bits up, as 1024 + 16 n, and (1024 + 16 n) / 16 - 64 = n is
+// exact in one fused multiply-add; so one shift serves the whole word.
+__device__ __forceinline__ void nibble_pairs(uint32_t w, uint32_t (&e)[4])
+{
+    const __half2 sixteenth = __floats2half2_rn(0.0625f, 0.0625f), minus64 = __floats2half2_rn(-64.0f, -64.0f);
+    const uint32_t hi = w >> 8;
+    uint32_t f1, f3;
+    e[0] = int_pair(w, 0x000f000fu);
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(f1) : "r"(w), "r"(0x00f000f0u), "r"(kHalfMagic));
+    e[1] = as_u32(__hfma2(as_half2(f1), sixteenth, minus64));
+    e[2] = int_pair(hi, 0x000f000fu);
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(f3) : "r"(hi), "r"(0x00f000f0u), "r"(kHalfMagic));
+    e[3] = as_u32(__hfma2(as_half2(f3), sixteenth, minus64));
+}
+
+// Four 8 x 8 matrices of 16-bit elements from shared memory, rows of 16 bytes: lane l gives the
+// address of row l % 8 of matrix l / 8; lane (gid, tig) receives from each matrix the word tig of
+// row gid -- or, transposed, the element gid of the rows 2tig (low half) and 2tig + 1 (high half).
+__device__ __forceinline__ void load_matrices(const void *row, uint32_t (&d)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+                 : "r"(smem_addr(row))
+                 : "memory");
+}
+__device__ __forceinline__ void load_matrices_transposed(const void *row, uint32_t (&d)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+                 : "r"(smem_addr(row))
+                 : "memory");
 }
 
 // Key side.  The lane's 8 channels of group g of one token (channels 32g + 8t + 0..7) as four
@@ -187,9 +241,7 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, ui
     }
     const uint8_t *codes = rec + 4 * META + (4 * g + tig) * bb;  // the lane's 8 codes: b bytes
     if constexpr (B == 4) {
-        const uint32_t w = *reinterpret_cast<const uint32_t *>(codes);  // nibble k and k + 4 are 16 bits apart
-#pragma unroll
-        for (int k = 0; k < 4; ++k) e[k] = int_pair(w >> (4 * k), 0x000f000fu);
+        nibble_pairs(*reinterpret_cast<const uint32_t *>(codes), e);  // nibble k and k + 4 are 16 bits apart
     } else if constexpr (B == 8) {
         const uint2 w = *reinterpret_cast<const uint2 *>(codes);
 #pragma unroll
@@ -218,9 +270,7 @@ __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t 
     } else if (B == 4) {
         const uint32_t wa = *reinterpret_cast<const uint16_t *>(rec_a + CODES + 16 * g + 2 * gid);
         const uint32_t wb = *reinterpret_cast<const uint16_t *>(rec_b + CODES + 16 * g + 2 * gid);
-        const uint32_t x = wa | (wb << 16);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) e[k] = int_pair(x >> (4 * k), 0x000f000fu);
+        nibble_pairs(wa | (wb << 16), e);
     } else if (B == 8) {
         const uint32_t wa = *reinterpret_cast<const uint32_t *>(rec_a + CODES + 32 * g + 4 * gid);
         const uint32_t wb = *reinterpret_cast<const uint32_t *>(rec_b + CODES + 32 * g + 4 * gid);
@@ -284,11 +334,25 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
     float x[2][2];  // logits (base 2): [token gid + 8k][head 2tig + h]
     {
         float sacc[4][4];
+        // 4-bit rows: a (token, group) is 16 bytes of codes, a matrix row; two loads hand every
+        // lane its words of all four groups of its two tokens
+        uint32_t ka[4], kb[4];
+        if (B == 4) {
+            const int l = gid * 4 + tig;
+            const uint8_t *row = sm.k[stage] + (l & 7) * REC + 4 * META + 16 * (l >> 3);
+            load_matrices(row, ka);
+            load_matrices(row + 8 * REC, kb);
+        }
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
             uint32_t ea[4] = {0u, 0u, 0u, 0u}, eb[4] = {0u, 0u, 0u, 0u};  // lanes without a token feed zeros
-            if (have[0]) key_pairs<B, META>(krec[0], g, tig, ea);
-            if (have[1]) key_pairs<B, META>(krec[1], g, tig, eb);
+            if (B == 4) {
+                if (have[0]) nibble_pairs(ka[g], ea);
+                if (have[1]) nibble_pairs(kb[g], eb);
+            } else {
+                if (have[0]) key_pairs<B, META>(krec[0], g, tig, ea);
+                if (have[1]) key_pairs<B, META>(krec[1], g, tig, eb);
+            }
             mma_m16n8k16_first(sacc[g], ea[0], eb[0], ea[1], eb[1], qb[g][0], qb[g][1]);  // the whole warp, together
             mma_m16n8k16(sacc[g], ea[2], eb[2], ea[3], eb[3], qb[g][2], qb[g][3]);
         }
@@ -366,18 +430,37 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
         const int t = 2 * tig + (i & 1) + 8 * (i >> 1);
         rv[i] = sm.v[stage] + ((FULL || t < rows) ? t : 0) * REC;
     }
+    // 4-bit rows: transposed matrix loads deliver (token 2tig, token 2tig + 1) x channels 4gid..4gid+3
+    // of a group in one word, tokens 0..7 and 8..15 of two groups per load.  Stale rows of tokens
+    // that are not there are integers like any others, and their weights are zero.
+    uint32_t va[4], vb[4];
+    if (B == 4) {
+        const int l = gid * 4 + tig;
+        const uint8_t *row = sm.v[stage] + ((l & 7) + 8 * ((l >> 3) & 1)) * REC + 4 * META + 16 * (l >> 4);
+        load_matrices_transposed(row, va);       // groups 0, 1
+        load_matrices_transposed(row + 32, vb);  // groups 2, 3
+    }
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
         uint32_t eab[4], ecd[4];
-        value_pairs<B, META>(rv[0], rv[1], g, gid, eab);
-        value_pairs<B, META>(rv[2], rv[3], g, gid, ecd);
+        if (B == 4) {
+            nibble_pairs(g < 2 ? va[2 * g] : vb[2 * g - 4], eab);
+            nibble_pairs(g < 2 ? va[2 * g + 1] : vb[2 * g - 3], ecd);
+        } else {
+            value_pairs<B, META>(rv[0], rv[1], g, gid, eab);
+            value_pairs<B, META>(rv[2], rv[3], g, gid, ecd);
+        }
         mma_m16n8k16(acc[g][0], eab[0], eab[1], ecd[0], ecd[1], wb0[g], wb1[g]);
         mma_m16n8k16(acc[g][1], eab[2], eab[3], ecd[2], ecd[3], wb0[g], wb1[g]);
     }
 }
 
+#ifndef QKVS_ATTEND_CTAS
+#define QKVS_ATTEND_CTAS 4
+#endif
+
 template <int NS, int WARPS, int META>
-__global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
+__global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(AttendParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     __shared__ int s_header_ok;
@@ -478,7 +561,7 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
             }
             if (__any_sync(0xffffffffu, bad) && lane == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
         }
-        StepIter iss;
+        uint32_t n_steps;
         {
             // positions: class-major, then lane, then the lane's own order
             uint32_t inc = counts, inc_hi = counts_hi;
@@ -491,12 +574,13 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
                 }
             }
             const uint32_t tot = __shfl_sync(0xffffffffu, inc, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
-            iss.s1 = tot & 0xffffu;
-            iss.s2 = iss.s1 + (tot >> 16);
-            iss.s3 = iss.s2 + (tot_hi & 0xffffu);
-            iss.s4 = iss.s3 + (tot_hi >> 16);
+            uint32_t ends[4];  // where each class ends in the list
+            ends[0] = tot & 0xffffu;
+            ends[1] = ends[0] + (tot >> 16);
+            ends[2] = ends[1] + (tot_hi & 0xffffu);
+            ends[3] = ends[2] + (tot_hi >> 16);
             const uint32_t before = inc - counts, before_hi = inc_hi - counts_hi;  // in lower lanes
-            uint32_t pos[4] = {before & 0xffffu, iss.s1 + (before >> 16), iss.s2 + (before_hi & 0xffffu), iss.s3 + (before_hi >> 16)};
+            uint32_t pos[4] = {before & 0xffffu, ends[0] + (before >> 16), ends[1] + (before_hi & 0xffffu), ends[2] + (before_hi >> 16)};
             __syncwarp();  // the previous item's list is no longer read
 #pragma unroll
             for (int r = 0; r < kAttendPerLane; ++r) {
@@ -505,9 +589,14 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
                     if (my_cls[r] == c) sm.list[pos[c]++] = my_off[r];
             }
             __syncwarp();
+            // the steps, two descriptors per lane
+            const uint32_t d_lo = make_step<META>((uint32_t)lane, ends, sm.list);
+            const uint32_t d_hi = make_step<META>((uint32_t)lane + 32u, ends, sm.list);
+            sm.steps[lane] = d_lo;
+            sm.steps[lane + 32] = d_hi;
+            n_steps = __popc(__ballot_sync(0xffffffffu, d_lo != 0u)) + __popc(__ballot_sync(0xffffffffu, d_hi != 0u));
+            __syncwarp();
         }
-        iss.begin();
-        StepIter con = iss;
 
         // the group's queries as B fragments: lane (gid, tig) holds head gid, per group the channels
         // 32g + 8tig + k paired with + k + 4 (the pairing of key_pairs); and the sums over a group of
@@ -543,38 +632,32 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[g][h][i] = 0.0f;
 
-        int in_flight = 0;
-        for (; in_flight < NS && !iss.done(); ++in_flight) {
-            int st = stage + in_flight;
+        for (uint32_t i = 0; i < (uint32_t)NS && i < n_steps; ++i) {
+            int st = stage + (int)i;
             if (st >= NS) st -= NS;
-            attend_issue<NS, META>(sm, st, iss, base_k, base_v, p, lane);
-            iss.next();
+            attend_issue<NS, META>(sm, st, sm.steps[i], base_k, base_v, p, lane);
         }
-        while (!con.done()) {
+        for (uint32_t i = 0; i < n_steps; ++i) {
+            const uint32_t d = sm.steps[i];
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[stage], parity));
             if (!ok) break;
-            const int rows = con.rows();
-            if (rows == kAttendRows) {
-                switch (con.c) {
+            const int rows = step_rows(d), cls = step_class(d);
+            if (rows == kAttendRows) {  // 16-bit rows come at most eight per step
+                switch (cls) {
                     case 0: attend_step<NS, 2, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                     case 1: attend_step<NS, 4, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 2: attend_step<NS, 8, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    default: attend_step<NS, 16, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    default: attend_step<NS, 8, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                 }
             } else {
-                switch (con.c) {
+                switch (cls) {
                     case 0: attend_step<NS, 2, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                     case 1: attend_step<NS, 4, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                     case 2: attend_step<NS, 8, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                     default: attend_step<NS, 16, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
                 }
             }
-            con.next();
             __syncwarp();  // every lane has read the stage: it can be re-armed
-            if (!iss.done()) {
-                attend_issue<NS, META>(sm, stage, iss, base_k, base_v, p, lane);
-                iss.next();
-            }
+            if (i + (uint32_t)NS < n_steps) attend_issue<NS, META>(sm, stage, sm.steps[i + NS], base_k, base_v, p, lane);
             if (++stage == NS) {
                 stage = 0;
                 parity ^= 1u;
@@ -641,6 +724,8 @@ __global__ void __launch_bounds__(WARPS * 32, 3) attend_kernel(AttendParams p)
 
 // Merges the items of every query head: o = sum_i o_i 2^(m_i - M) / sum_i l_i 2^(m_i - M).
 // One warp per (layer, query head); writes zeros when the first kernel reported a problem.
+// The items' maxima and sums are read one item per lane, so that the loads of an item's
+// accumulators, which need its factor only for the multiplication, all go out at once.
 __global__ void __launch_bounds__(128) attend_merge_kernel(AttendParams p)
 {
     const int lane = threadIdx.x & 31;
@@ -656,18 +741,30 @@ __global__ void __launch_bounds__(128) attend_merge_kernel(AttendParams p)
         const float *base = p.partials + ((uint64_t)lh * p.items_per_head * per_kv + jj) * kPartialFloats;
         const uint64_t stride = (uint64_t)per_kv * kPartialFloats;
         float big = -INFINITY;
-        for (uint32_t i = 0; i < p.items_per_head; ++i) big = fmaxf(big, base[i * stride + kAttendD]);
+        for (uint32_t i = lane; i < p.items_per_head; i += 32) big = fmaxf(big, base[i * stride + kAttendD]);
+#pragma unroll
+        for (int sft = 16; sft > 0; sft >>= 1) big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, sft));
         float denom = 0.0f;
-        for (uint32_t i = 0; i < p.items_per_head; ++i) {
-            const float *part = base + i * stride;
-            const float f = exp2f(part[kAttendD] - big);
-            denom += part[kAttendD + 1] * f;
-            const float4 v = *reinterpret_cast<const float4 *>(part + 4 * lane);
-            o.x += v.x * f;
-            o.y += v.y * f;
-            o.z += v.z * f;
-            o.w += v.w * f;
+        for (uint32_t i0 = 0; i0 < p.items_per_head; i0 += 32) {
+            const uint32_t mine = i0 + (uint32_t)lane;
+            float f = 0.0f;
+            if (mine < p.items_per_head) {
+                f = exp2f(base[mine * stride + kAttendD] - big);
+                denom = fmaf(base[mine * stride + kAttendD + 1], f, denom);
+            }
+            const int n = (int)min(32u, p.items_per_head - i0);
+#pragma unroll 8
+            for (int i = 0; i < n; ++i) {
+                const float fi = __shfl_sync(0xffffffffu, f, i);
+                const float4 v = *reinterpret_cast<const float4 *>(base + (i0 + (uint32_t)i) * stride + 4 * lane);
+                o.x = fmaf(v.x, fi, o.x);
+                o.y = fmaf(v.y, fi, o.y);
+                o.z = fmaf(v.z, fi, o.z);
+                o.w = fmaf(v.w, fi, o.w);
+            }
         }
+#pragma unroll
+        for (int sft = 16; sft > 0; sft >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, sft);
         const float r = 1.0f / denom;
         o.x *= r;
         o.y *= r;

@@ -803,7 +803,13 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
                                const void *q_dev, float softmax_scale, float *out_dev, void *scratch_dev,
                                size_t scratch_bytes, void *stream)
 {
-    constexpr int kAttendStages = 2, kAttendWarps = 4;
+#ifndef QKVS_ATTEND_STAGES
+#define QKVS_ATTEND_STAGES 2
+#endif
+#ifndef QKVS_ATTEND_WARPS
+#define QKVS_ATTEND_WARPS 4
+#endif
+    constexpr int kAttendStages = QKVS_ATTEND_STAGES, kAttendWarps = QKVS_ATTEND_WARPS;
     AttendParams p;
     const qkvs_status_t st = attend_shape(layout, n_q_heads, &p);
     if (st != QKVS_OK) return st;
