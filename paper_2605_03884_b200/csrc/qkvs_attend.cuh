@@ -153,8 +153,9 @@ __device__ __forceinline__ uint32_t make_step(uint32_t idx, const uint32_t (&e)[
 
 // Starts the copies of one step's K and V records into `stage`, packed in list order: one copy
 // per stream when the tokens are neighbours in the card (the offsets grow with the token index,
-// so first and last record a step's length apart leave no room for others in between), else one
-// per record.  All lanes call it.
+// so first and last record a step's length apart leave no room for others in between), else
+// gathered in 16-byte pieces.  Either way the stage's barrier completes when the bytes are there.
+// All lanes call it.
 template <int NS, int META>
 __device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, uint32_t d, uint64_t base_k, uint64_t base_v,
                                              const AttendParams &p, int lane)
@@ -169,13 +170,19 @@ __device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, 
             bulk_load(sm.v[stage], p.card + base_v + first, (uint32_t)n * rec, &sm.full[stage]);
         }
     } else {
-        if (lane == 0) mbar_arrive_expect_tx(&sm.full[stage], 2u * (uint32_t)n * rec);
-        __syncwarp();
-        if (lane < n) {
-            const uint32_t mine = sm.list[step_first(d) + lane];
-            bulk_load(sm.k[stage] + lane * rec, p.card + base_k + mine, rec, &sm.full[stage]);
-            bulk_load(sm.v[stage] + lane * rec, p.card + base_v + mine, rec, &sm.full[stage]);
+        // scattered records of 48 to 256 bytes: 16-byte pieces, one per lane and round, which the
+        // load unit merges into whole sectors; a bulk copy per record costs far more than it moves
+        const uint32_t pieces = rec >> 4, total = (uint32_t)n * pieces;  // at most 160
+        const uint32_t inv = 65536u / pieces + 1u;                      // i / pieces == (i * inv) >> 16 for i < 4096
+        for (uint32_t i = (uint32_t)lane; i < total; i += 32u) {
+            const uint32_t r = (i * inv) >> 16;
+            const uint32_t src = sm.list[step_first(d) + r] + ((i - r * pieces) << 4);
+            async_copy_16(sm.k[stage] + (i << 4), p.card + base_k + src);
+            async_copy_16(sm.v[stage] + (i << 4), p.card + base_v + src);
         }
+        async_copies_arrive_on(&sm.full[stage]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.full[stage]);
     }
 }
 
@@ -456,7 +463,7 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
 }
 
 #ifndef QKVS_ATTEND_CTAS
-#define QKVS_ATTEND_CTAS 4
+#define QKVS_ATTEND_CTAS 2
 #endif
 
 template <int NS, int WARPS, int META>

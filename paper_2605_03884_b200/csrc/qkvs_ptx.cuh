@@ -34,6 +34,21 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 
+// 16 bytes global -> shared, asynchronously, by the calling thread (both addresses 16-byte aligned).
+__device__ __forceinline__ void async_copy_16(void *dst_smem, const void *src_gmem)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src_gmem) : "memory");
+}
+
+// Ties the calling thread's async_copy_16 copies issued so far to `bar`: the barrier's count of
+// pending arrivals goes up by one now and comes down again once those copies have landed (at once
+// if there are none), so the current phase cannot complete before they have.  The thread that
+// makes the phase's own arrival must do so after every thread has executed this.
+__device__ __forceinline__ void async_copies_arrive_on(uint64_t *bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.shared::cta.b64 [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");

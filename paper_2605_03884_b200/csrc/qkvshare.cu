@@ -807,7 +807,7 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
 #define QKVS_ATTEND_STAGES 2
 #endif
 #ifndef QKVS_ATTEND_WARPS
-#define QKVS_ATTEND_WARPS 4
+#define QKVS_ATTEND_WARPS 8  // two CTAs of eight warps per SM: neighbouring items, i.e. neighbouring spans of a stream, start together
 #endif
     constexpr int kAttendStages = QKVS_ATTEND_STAGES, kAttendWarps = QKVS_ATTEND_WARPS;
     AttendParams p;
