@@ -88,14 +88,16 @@ __device__ __forceinline__ int rows_at(const Pos &c, const PathParams &p)
     return c.tt + 1u == p.subs_per_stream ? (int)p.last_rows : R;
 }
 
-// Work distribution.  The sub-tiles of a launch are handed out in chunks of kChunk consecutive
-// ones.  Every warp of the grid starts with the chunk of its own index; further chunks come from
+// Work distribution.  The sub-tiles of a launch are handed out in chunks of p.chunk consecutive
+// ones (eight; four when the launch is so small that chunks of eight would leave most warps with
+// one chunk and a few with two).  Every warp of the grid starts with the chunk of its own index; further chunks come from
 // a counter in device memory -- first come, first served, which evens out SMs that run at
 // different speeds -- or, when the caller gave no scratch block, at a fixed stride.
 // A warp walks its sequence of sub-tiles with two cursors, one ahead of the other: the leading
 // one takes the chunks and leaves their indices in a small ring in shared memory, the trailing
 // one reads them there.  The index n_chunks marks the end of the sequence.
-constexpr uint32_t kChunk = 8;
+constexpr uint32_t kChunk = 8;       // sub-tiles per chunk
+constexpr uint32_t kChunkSmall = 4;  // ... of a launch with fewer than two chunks of eight per warp
 
 struct WorkSource {
     uint32_t *ring;       // shared memory, 4 entries: chunk indices in the order the warp took them
@@ -113,9 +115,9 @@ struct Cursor {
 
 __device__ __forceinline__ void enter_chunk(Cursor &cu, uint32_t chunk, const PathParams &p)
 {
-    const uint32_t first = chunk * kChunk;
+    const uint32_t first = chunk * p.chunk;
     cu.c = position_of(p, first);
-    cu.left = min(kChunk, (uint32_t)p.n_subs - first) - 1u;
+    cu.left = min(p.chunk, (uint32_t)p.n_subs - first) - 1u;
 }
 
 // Moves a cursor to the warp's next sub-tile.  Returns false when that is simply the following
@@ -260,7 +262,7 @@ struct CreateWarpSmem {
     alignas(128) uint8_t in[NS][C::STAGE_BYTES];
     alignas(8) uint64_t full[NS];
     uint32_t ring[4];
-    static_assert(NS >= 2 && NS <= (int)kChunk, "pipeline depth");
+    static_assert(NS >= 2 && NS <= (int)kChunkSmall, "pipeline depth");
 };
 
 // One group: lane l owns group l % G of row l / G of the R rows at `rows_in`, i.e. the 64 input
@@ -460,7 +462,7 @@ struct InjectWarpSmem {
     uint32_t uniform_bits[NS];         // bit-width shared by all ROWS rows, else 0
     int32_t rows[NS];                  // 0 when the sub-tile's table entries did not check out
     uint32_t ring[4];
-    static_assert(NS >= 2 && NS < (int)kChunk, "pipeline depth");
+    static_assert(NS >= 2 && NS < (int)kChunkSmall, "pipeline depth");
 };
 
 // One chunk (8 values) of a record.  B is the bit-width known at compile time, or 0 when it is

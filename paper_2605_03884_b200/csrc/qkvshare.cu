@@ -449,11 +449,15 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
     if (n_subs == 0) return cudaSuccess;
     if (n_subs > 0x7fffffffull) return cudaErrorInvalidValue;
     p.n_subs = (uint32_t)n_subs;
-    p.n_chunks = (p.n_subs + kChunk - 1) / kChunk;
     p.last_rows = (uint32_t)(p.n_tokens - (int64_t)(p.subs_per_stream - 1) * C::ROWS);
     unsigned grid = 0;
-    cudaError_t e = persistent_grid<TAG>(kernel, WARPS * 32, smem, (int64_t)((p.n_chunks + WARPS - 1) / WARPS), &grid);
+    cudaError_t e = persistent_grid<TAG>(kernel, WARPS * 32, smem, (int64_t)((n_subs + kChunkSmall * WARPS - 1) / (kChunkSmall * WARPS)), &grid);
     if (e != cudaSuccess) return e;
+    // with fewer than two chunks of eight per warp the second round of chunks would keep only part
+    // of the grid busy for as long as the first: halve the chunks then
+    p.chunk = (p.n_subs + kChunk - 1) / kChunk < 2u * grid * WARPS ? kChunkSmall : kChunk;
+    p.n_chunks = (p.n_subs + p.chunk - 1) / p.chunk;
+    grid = std::min<unsigned>(grid, (p.n_chunks + WARPS - 1) / WARPS);
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(grid);
