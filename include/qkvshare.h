@@ -176,7 +176,12 @@ QKVS_API qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_
  * Problems only the device can see -- a bit-width outside {2,4,8,16}, or a payload that does
  * not fit card_capacity -- are recorded in the card header's `status` (BAD_BITS,
  * BUFFER_TOO_SMALL); the payload is then not written and nothing outside the buffer is touched.
- * Read the outcome with qkvs_card_info.  The card's bytes are fully determined by the inputs. */
+ * Read the outcome with qkvs_card_info.  The card's bytes are fully determined by the inputs.
+ * A card of part of a cache -- say, only the tokens a hop appended since its last card -- is made
+ * by passing pointers to the first row to encode (base + first * token_stride elements, which
+ * keeps the alignment) with n_tokens rows to take and the strides unchanged; records do not
+ * depend on where a token sits, so such a card's streams equal the matching slices of the whole
+ * cache's card, and qkvs_card_inject places it with dst_token_offset. */
 QKVS_API qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K_layers,
                                const void *const *V_layers, const uint8_t *bits_dev,
                                const qkvs_card_meta_t *meta, void *card_dev,

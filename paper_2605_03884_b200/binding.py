@@ -186,12 +186,19 @@ def _workspace_ptr(workspace):
 
 def card_create(layout: Layout, K_layers: Sequence, V_layers: Sequence, bits_dev, card_dev,
                 meta: Optional[CardMeta] = None, card_capacity: Optional[int] = None,
-                workspace=None, stream=None, check: bool = True) -> int:
+                workspace=None, stream=None, check: bool = True, src_token_offset: int = 0) -> int:
     """qkvs_card_create.  K_layers / V_layers: per-layer CUDA tensors (FP16); bits_dev: CUDA uint8
     tensor; card_dev: CUDA uint8 tensor that receives the card; workspace: CUDA tensor of
-    WORKSPACE_BYTES bytes (see new_workspace) or None.  Returns the status."""
+    WORKSPACE_BYTES bytes (see new_workspace) or None.  src_token_offset: the cache row that
+    becomes token 0 of the card (the library is handed pointers to that row; layout.n_tokens rows
+    from there are encoded) -- a card of only the tokens appended since the last one.  Returns
+    the status."""
     lib = load_library()
     kp, vp = _ptr_array(K_layers), _ptr_array(V_layers)
+    if src_token_offset:
+        step = int(src_token_offset) * int(layout.token_stride) * 2  # FP16 elements
+        kp = (C.c_void_p * len(K_layers))(*[int(t.data_ptr()) + step for t in K_layers])
+        vp = (C.c_void_p * len(V_layers))(*[int(t.data_ptr()) + step for t in V_layers])
     cap = int(card_dev.numel() * card_dev.element_size()) if card_capacity is None else int(card_capacity)
     st = lib.qkvs_card_create(C.byref(layout), kp, vp, int(bits_dev.data_ptr()) if bits_dev is not None else None,
                               C.byref(meta) if meta is not None else None, int(card_dev.data_ptr()), cap,

@@ -213,6 +213,38 @@ def test_card_survives_a_copy_to_another_address():
     assert np.array_equal(Vd[0].cpu().numpy().view(np.uint16), Vw[0].view(np.uint16))
 
 
+def test_card_of_appended_tokens_only():
+    """A hop that appended tokens hands on only those: the card is made from row t0 of the cache
+    on (pointers to that row, n_tokens = what was appended) and injected at t0.  Bit-exact against
+    the oracle given the same rows; the destination's earlier rows stay untouched."""
+    import torch
+    L, H, d, T, t0 = 2, 3, 128, 333, 200
+    Ks, Vs, strides = padded_cache(L, H, T, d, seed=55, t_cap=400, token_stride=136)
+    bits = wl.iid_bits(T, (0.3, 0.3, 0.2, 0.2), seed=56)
+    n = T - t0
+    olay, glay = _olay(L, H, d, n, **strides), _glay(L, H, d, n, **strides)
+    st_o, want = oracle.card_create(olay, [k[:, t0:] for k in Ks], [v[:, t0:] for v in Vs], bits[t0:])
+    assert st_o == oracle.OK
+    Kd, Vd = to_cuda(Ks), to_cuda(Vs)
+    buf = torch.full((want.size + PAD,), POISON, dtype=torch.uint8, device="cuda")
+    q.card_create(glay, Kd, Vd, torch.from_numpy(bits[t0:]).cuda(), buf, card_capacity=want.size,
+                  workspace=q.new_workspace(), src_token_offset=t0)
+    st, hdr = q.card_info(buf)
+    got = buf.cpu().numpy()
+    assert st == 0 and hdr.n_tokens == n
+    assert np.array_equal(got[:want.size], want) and np.all(got[want.size:] == POISON)
+    Ko = [np.full_like(k, -3.0) for k in Ks]
+    Vo = [np.full_like(v, -5.0) for v in Vs]
+    Kw, Vw = [a.copy() for a in Ko], [a.copy() for a in Vo]
+    assert oracle.card_inject(want, olay, Kw, Vw, t0) == oracle.OK
+    stat, Kg, Vg = gpu_inject(q, want, glay, Ko, Vo, dst_token_offset=t0)
+    assert stat == 0
+    for l in range(L):
+        assert np.array_equal(Kg[l].view(np.uint16), Kw[l].view(np.uint16))
+        assert np.array_equal(Vg[l].view(np.uint16), Vw[l].view(np.uint16))
+        assert np.all(Kg[l][:, :t0] == -3.0) and np.all(Vg[l][:, :t0] == -5.0)
+
+
 def test_empty_card():
     L, H, d, T = 1, 2, 64, 0
     Ks = [np.zeros((H, 1, d), np.float16)]

@@ -565,3 +565,35 @@ def test_tiny_config_card():
     assert oracle.card_inject(card, lay, [Ko], [Vo]) == oracle.OK
     err = np.abs(Ko.astype(np.float32) - K.astype(np.float32)).max()
     assert 0 < err < 0.5
+
+
+def test_card_of_appended_tokens_equals_slices_of_the_whole_card():
+    """Records do not depend on a token's position: a card made from rows [t0, t0 + n) of a cache
+    holds, stream by stream, bytes [off[t0], off[t0 + n)) of the whole cache's card, and injecting
+    it at t0 rebuilds the same rows (incremental handoff: only what a hop appended)."""
+    L, H, T, d, t0 = 2, 2, 90, 64, 53
+    Ks, Vs, lay = _cache(L, H, T, d, 91)
+    bits = np.random.default_rng(92).choice(np.array([2, 4, 8, 16], np.uint8), size=T)
+    st, whole = oracle.card_create(lay, Ks, Vs, bits)
+    assert st == oracle.OK
+    n = T - t0
+    part_lay = oracle.make_layout(L, H, d, n, head_stride=lay.head_stride, token_stride=lay.token_stride)
+    st, part = oracle.card_create(part_lay, [k[:, t0:] for k in Ks], [v[:, t0:] for v in Vs], bits[t0:])
+    assert st == oracle.OK
+    hw, hp = oracle.parse_header(whole), oracle.parse_header(part)
+    _, off, _ = oracle.scan_offsets(d, bits)
+    assert hp["n_tokens"] == n and hp["stream_bytes"] == int(off[T] - off[t0])
+    for s in range(2 * L * H):
+        a = hw["payload_off"] + s * hw["stream_bytes"]
+        b = hp["payload_off"] + s * hp["stream_bytes"]
+        assert np.array_equal(part[b:b + hp["stream_bytes"]], whole[a + int(off[t0]):a + int(off[T])])
+    Kw = [np.zeros((H, T, d), np.float16) for _ in range(L)]
+    Vw = [np.zeros((H, T, d), np.float16) for _ in range(L)]
+    assert oracle.card_inject(whole, lay, Kw, Vw) == oracle.OK
+    Kp = [np.full((H, T, d), 9.0, np.float16) for _ in range(L)]
+    Vp = [np.full((H, T, d), 9.0, np.float16) for _ in range(L)]
+    assert oracle.card_inject(part, part_lay, Kp, Vp, dst_token_offset=t0) == oracle.OK
+    for l in range(L):
+        assert np.array_equal(Kp[l][:, t0:].view(np.uint16), Kw[l][:, t0:].view(np.uint16))
+        assert np.array_equal(Vp[l][:, t0:].view(np.uint16), Vw[l][:, t0:].view(np.uint16))
+        assert np.all(Kp[l][:, :t0] == 9.0) and np.all(Vp[l][:, :t0] == 9.0)
