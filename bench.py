@@ -402,6 +402,27 @@ def run_ours(args):
         attend = {"what": "decode-step attention straight from the card, all layers, 4 query heads per KV head",
                   "ms": a_ms, "card_payload_bytes": payload, "card_gbs": payload / (a_ms * 1e-3) / 1e9}
 
+    # what the handoff costs in accuracy: every hop's injected cache against the original FP16 cache
+    # (reporting only, outside every timed region; plain torch reductions)
+    hop_errors = []
+    if rank == 0:
+        def error_of(out, ref):
+            mx, se, sr = 0.0, 0.0, 0.0
+            for o, r in zip(out, ref):
+                dlt = o.float() - r.float()
+                mx = max(mx, float(dlt.abs().max()))
+                se += float(dlt.double().pow(2).sum())
+                sr += float(r.double().pow(2).sum())
+            n = sum(r.numel() for r in ref)
+            return {"max_abs": mx, "rmse": (se / n) ** 0.5, "rel_frobenius": (se / sr) ** 0.5 if sr else 0.0}
+        src_k, src_v = Kd, Vd
+        for h in range(hops):
+            q.card_create(lay, src_k, src_v, bits_d[h], card, card_capacity=sizes[h], workspace=ws, stream=stream)
+            q.card_inject(card, lay, Ko, Vo, card_bytes=sizes[h], workspace=ws, stream=stream)
+            torch.cuda.synchronize()
+            hop_errors.append({"K": error_of(Ko, Kd), "V": error_of(Vo, Vd)})
+            src_k, src_v = Ko, Vo
+
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device="cuda")
 
     if rank != 0:
@@ -420,10 +441,11 @@ def run_ours(args):
         c, i = med(create_ms[h]), med(inject_ms[h])
         per_hop.append({
             "hop": h, "card_bytes": sizes[h], "avg_code_bits": float(bits_per_hop[h].astype(np.float64).mean()),
-            "create_ms": c, "inject_ms": i,
+            "create_ms": c, "inject_ms": i, "create_ms_min": min(create_ms[h]), "inject_ms_min": min(inject_ms[h]),
             "create_kv_gbs": kv_bytes / (c * 1e-3) / 1e9, "inject_kv_gbs": kv_bytes / (i * 1e-3) / 1e9,
             "create_hbm_frac": (kv_bytes + payload) / (c * 1e-3) / 1e9 / peak,
             "inject_hbm_frac": (kv_bytes + payload) / (i * 1e-3) / 1e9 / peak,
+            "error_vs_original": hop_errors[h],
         })
     # dominant kernel: the slower of the two halves on hop 0
     payload0 = sizes[0] - prefix
