@@ -459,7 +459,8 @@ def run_ours(args):
     traffic = captured_traffic(dom_key, L) if w.number == 3 and args.meta_bytes == 8 and args.bits_mode == 0 else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src, "traffic": traffic,
-                "algorithmic_bytes_per_launch": kv_bytes + payload0, "avg_launch_ms": dom_ms}
+                "algorithmic_bytes_per_launch": kv_bytes + payload0, "avg_launch_ms": dom_ms,
+                "datasheet_peak": 8000.0, "frac_of_datasheet": achieved / 8000.0}
 
     # per hop: the offset scan (plus its second stage with per-head bit-widths), then one create
     # and one inject launch per block of 64 layers
