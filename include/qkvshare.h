@@ -163,6 +163,19 @@ QKVS_API qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_
                                     int32_t n_tokens, int32_t n_fp16, int32_t n_8bit,
                                     int32_t n_4bit, uint8_t *bits_dev, void *stream);
 
+/* The combined importance score of Section 3.3, S(t) = alpha * I(t) + (1 - alpha) * T(t): local
+ * importance I and transferability T weighed by alpha in [0, 1], the quantity the bit-widths are
+ * assigned from.  How I and T are obtained (attention statistics, agent topology) is outside this
+ * library; this is the combination itself, elementwise, feeding qkvs_bits_from_scores.
+ * Arithmetic: binary32, each step rounded to nearest, nothing fused:
+ *     S = fl( fl(alpha * I) + fl( fl(1 - alpha) * T ) ).
+ *   importance_dev, transfer_dev   device float32 [n]
+ *   scores_dev                     device float32 [n]; may be one of the inputs
+ * Asynchronous on `stream`.  Errors: INVALID_ARG (null or misaligned pointer, negative n, alpha
+ * outside [0, 1] or not a number), CUDA. */
+QKVS_API qkvs_status_t qkvs_combine_scores(const float *importance_dev, const float *transfer_dev,
+                                  float alpha, int64_t n, float *scores_dev, void *stream);
+
 /* Card creation (Section 4.2.1): offset scan over the bit-widths, then fused
  * min/max -> scale/zero -> quantise -> bit-pack of every (layer, K|V, head) stream.
  *   K_layers, V_layers  HOST arrays of n_layers DEVICE pointers to FP16 blocks (16-byte aligned)

@@ -85,6 +85,8 @@ def lib():
         l.orc_card_inject.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_void_p, C.c_void_p, C.c_int64]
         l.orc_bits_from_scores.restype = C.c_int
         l.orc_bits_from_scores.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]
+        l.orc_combine_scores.restype = C.c_int
+        l.orc_combine_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int64, C.c_void_p]
         l.orc_card_attend.restype = C.c_int
         l.orc_card_attend.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_int, C.c_void_p, C.c_double, C.c_void_p]
         l.orc_num_threads.restype = C.c_int
@@ -272,6 +274,16 @@ def bits_from_scores(scores: np.ndarray, n_fp16: int, n_8bit: int, n_4bit: int) 
     bits = np.zeros(scores.size, dtype=np.uint8)
     st = lib().orc_bits_from_scores(_ptr(scores), scores.size, n_fp16, n_8bit, n_4bit, _ptr(bits))
     return st, bits
+
+
+def combine_scores(importance: np.ndarray, transfer: np.ndarray, alpha: float) -> Tuple[int, np.ndarray]:
+    """S = alpha * I + (1 - alpha) * T in float32 (see orc_combine_scores)."""
+    imp = np.ascontiguousarray(importance, dtype=np.float32)
+    tra = np.ascontiguousarray(transfer, dtype=np.float32)
+    assert imp.shape == tra.shape
+    out = np.zeros(imp.shape, dtype=np.float32)
+    st = lib().orc_combine_scores(_ptr(imp), _ptr(tra), C.c_float(alpha), imp.size, _ptr(out))
+    return st, out
 
 
 def num_threads() -> int:

@@ -767,6 +767,20 @@ int orc_bits_from_scores(const float *scores, int64_t n_tokens, int64_t n_fp16, 
     return ORC_OK;
 }
 
+/* Combined importance score (Section 3.3): S(t) = alpha * I(t) + (1 - alpha) * T(t), in binary32,
+ * every operation rounded on its own (the file is compiled without contraction). */
+int orc_combine_scores(const float *importance, const float *transfer, float alpha, int64_t n, float *scores)
+{
+    if (n < 0 || !(alpha >= 0.0f && alpha <= 1.0f)) return ORC_INVALID_ARG;
+    const float beta = 1.0f - alpha;
+    for (int64_t i = 0; i < n; ++i) {
+        const float a = alpha * importance[i];
+        const float b = beta * transfer[i];
+        scores[i] = a + b;
+    }
+    return ORC_OK;
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP

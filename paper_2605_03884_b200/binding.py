@@ -52,7 +52,7 @@ assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
            "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_attend_scratch_size", "qkvs_card_attend",
-           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_selftest_division", "qkvs_status_string",
+           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_combine_scores", "qkvs_selftest_division", "qkvs_status_string",
            "qkvs_version")
 
 _lib = None
@@ -88,6 +88,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_attend.argtypes = [vp, C.c_size_t, C.POINTER(Layout), C.c_int32, vp, C.c_float, vp, vp, C.c_size_t, vp]
     lib.qkvs_bits_from_scores.restype = C.c_int
     lib.qkvs_bits_from_scores.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp]
+    lib.qkvs_combine_scores.restype = C.c_int
+    lib.qkvs_combine_scores.argtypes = [vp, vp, C.c_float, C.c_int64, vp, vp]
     lib.qkvs_card_info.restype = C.c_int
     lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
     lib.qkvs_selftest_division.restype = C.c_int
@@ -278,6 +280,17 @@ def bits_from_scores(scores_dev, n_fp16: int, n_8bit: int, n_4bit: int, bits_dev
                                               int(n_4bit), int(bits_dev.data_ptr()), _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_bits_from_scores")
+    return st
+
+
+def combine_scores(importance_dev, transfer_dev, alpha: float, scores_dev, stream=None, check: bool = True) -> int:
+    """qkvs_combine_scores: scores = alpha * importance + (1 - alpha) * transfer, CUDA float32 tensors
+    of equal size."""
+    n = int(importance_dev.numel())
+    st = load_library().qkvs_combine_scores(int(importance_dev.data_ptr()), int(transfer_dev.data_ptr()), C.c_float(alpha),
+                                            n, int(scores_dev.data_ptr()), _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_combine_scores")
     return st
 
 

@@ -255,6 +255,16 @@ __global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
 }
 
 // ---------------------------------------------------------------------------------------------
+// S = alpha * I + (1 - alpha) * T, elementwise; every step one rounded binary32 operation.
+__global__ void __launch_bounds__(256) combine_scores_kernel(const float *__restrict__ imp, const float *__restrict__ tra,
+                                                             float alpha, float beta, int64_t n, float *out)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+        out[i] = __fadd_rn(__fmul_rn(alpha, imp[i]), __fmul_rn(beta, tra[i]));
+}
+
+// ---------------------------------------------------------------------------------------------
 // Bit-widths from importance scores by rank (the step in front of the offset scan).
 // rank(t) = #{s : score_s > score_t} + #{s < t : score_s == score_t}; the first n16 ranks keep
 // FP16, the next n8 get 8 bits, the next n4 get 4 bits, the rest 2 bits.  Exact and order-free:
@@ -859,6 +869,20 @@ qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_segments,
     const dim3 grid((unsigned)((n_tokens + kRankThreads / kRankSplit - 1) / (kRankThreads / kRankSplit)), (unsigned)n_segments);
     bits_from_scores_kernel<<<grid, kRankThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
         scores_dev, n_tokens, (uint32_t)n_fp16, (uint32_t)n_8bit, (uint32_t)n_4bit, bits_dev);
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+}
+
+qkvs_status_t qkvs_combine_scores(const float *importance_dev, const float *transfer_dev, float alpha, int64_t n,
+                                  float *scores_dev, void *stream)
+{
+    if (n < 0 || !(alpha >= 0.0f && alpha <= 1.0f)) return QKVS_ERR_INVALID_ARG;
+    if (n == 0) return QKVS_OK;
+    if (!importance_dev || !transfer_dev || !scores_dev) return QKVS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(importance_dev) | reinterpret_cast<uintptr_t>(transfer_dev) | reinterpret_cast<uintptr_t>(scores_dev)) & 3u)
+        return QKVS_ERR_INVALID_ARG;
+    const float beta = 1.0f - alpha;  // one rounded subtraction on the host, as in the definition
+    const unsigned grid = (unsigned)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    combine_scores_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(importance_dev, transfer_dev, alpha, beta, n, scores_dev);
     return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 

@@ -93,3 +93,29 @@ def test_scores_to_card_end_to_end():
     bits_g = _gpu_bits(scores, n16, n8, n4)
     st_g, hdr, whole, cap = gpu_create(q, q.make_layout(L, H, d, T), Ks, Vs, bits_g)
     assert st_g == 0 and np.array_equal(whole[:want.size], want)
+
+
+def test_combined_score_bit_exact_and_feeds_the_rank_rule():
+    import torch
+    rng = np.random.default_rng(83)
+    n = 8192 + 37
+    imp = rng.lognormal(0, 1, n).astype(np.float32)
+    tra = (rng.standard_normal(n) * 2).astype(np.float32)
+    for alpha in (0.0, 0.3, 0.6180339887, 1.0):
+        st, want = oracle.combine_scores(imp, tra, alpha)
+        assert st == oracle.OK
+        out = torch.full((n,), -7.0, dtype=torch.float32, device="cuda")
+        q.combine_scores(torch.from_numpy(imp).cuda(), torch.from_numpy(tra).cuda(), alpha, out)
+        got = out.cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # in place, then straight into the rank rule
+    st, want = oracle.combine_scores(imp, tra, 0.4)
+    stb, bits_want = oracle.bits_from_scores(want, 400, 1200, 3300)
+    buf = torch.from_numpy(imp).cuda()
+    q.combine_scores(buf, torch.from_numpy(tra).cuda(), 0.4, buf)
+    bits = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    q.bits_from_scores(buf, 400, 1200, 3300, bits)
+    assert stb == oracle.OK and np.array_equal(bits.cpu().numpy(), bits_want)
+    with pytest.raises(q.QkvsError) as e:
+        q.combine_scores(buf, buf, 1.5, buf)
+    assert e.value.status == q.binding.ERR_INVALID_ARG

@@ -68,3 +68,46 @@ def test_matches_the_library_sort_of_the_workload_generator():
 def test_bad_counts_are_rejected():
     st, _ = oracle.bits_from_scores(np.zeros(4, np.float32), 3, 2, 0)
     assert st == oracle.INVALID_ARG
+
+
+# ----------------------------------------------------------------------------- combined score
+
+def test_combined_score_special_cases():
+    """Section 3.3's S = alpha I + (1 - alpha) T: alpha = 1 gives I, alpha = 0 gives T, equal inputs
+    come back unchanged when alpha is a power of two, small integers combine exactly."""
+    rng = np.random.default_rng(81)
+    imp = rng.lognormal(0, 1, 500).astype(np.float32)
+    tra = rng.lognormal(0, 1, 500).astype(np.float32)
+    st, s1 = oracle.combine_scores(imp, tra, 1.0)
+    assert st == oracle.OK and np.array_equal(s1, imp)
+    st, s0 = oracle.combine_scores(imp, tra, 0.0)
+    assert st == oracle.OK and np.array_equal(s0, tra)
+    for alpha in (0.5, 0.25, 0.75):
+        st, s = oracle.combine_scores(imp, imp, alpha)
+        assert st == oracle.OK and np.array_equal(s, imp)
+    a = rng.integers(0, 1000, 300).astype(np.float32)
+    b = rng.integers(0, 1000, 300).astype(np.float32)
+    st, s = oracle.combine_scores(a, b, 0.25)
+    assert st == oracle.OK and np.array_equal(s.astype(np.float64), 0.25 * a.astype(np.float64) + 0.75 * b.astype(np.float64))
+    for bad in (-0.1, 1.5, float("nan")):
+        assert oracle.combine_scores(a, b, bad)[0] == oracle.INVALID_ARG
+
+
+def test_combined_score_matches_numpy_float32_step_by_step():
+    """The same three roundings with numpy's float32 scalars and arrays (each numpy operation
+    rounds once); catches a fused multiply-add or double-precision intermediates in the C build."""
+    rng = np.random.default_rng(82)
+    imp = (rng.standard_normal(4000) * 3).astype(np.float32)
+    tra = rng.lognormal(0, 2, 4000).astype(np.float32)
+    for alpha in (0.3, 0.6180339887, 0.9):
+        al = np.float32(alpha)
+        want = al * imp + (np.float32(1.0) - al) * tra
+        assert want.dtype == np.float32
+        st, got = oracle.combine_scores(imp, tra, alpha)
+        assert st == oracle.OK and np.array_equal(got.view(np.uint32), want.view(np.uint32))
+        # and against the real-number expression: three roundings on the larger of the two terms
+        # plus the rounding of 1 - alpha carried by T
+        ta, tb = float(al) * imp.astype(np.float64), (1.0 - float(al)) * tra.astype(np.float64)
+        big = np.maximum(np.maximum(np.abs(ta), np.abs(tb)), np.abs(ta + tb)).astype(np.float32)
+        bound = 2 * np.spacing(big).astype(np.float64) + np.abs(tra).astype(np.float64) * 2.0 ** -24
+        assert np.all(np.abs(got.astype(np.float64) - (ta + tb)) <= bound)
