@@ -101,17 +101,10 @@ __device__ __forceinline__ float exp2_approx(float x)
     return y;
 }
 
-__device__ __forceinline__ uint32_t word_of(const uint4 &v, int i)
-{
-    return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
-}
-
 // The order of tokens does not matter to attention, so a warp regroups the (up to) 256 tokens of
-// its item by bit-width and walks them one width at a time: every step then deals with a single
-// width and runs the body compiled for it, however the widths are mixed in the card.
-
-// Bit-width classes in the order they are walked: 2, 4, 8, 16 bits.
-__device__ __forceinline__ uint32_t class_width(int c) { return c == 0 ? 2u : (c == 1 ? 4u : (c == 2 ? 8u : 16u)); }
+// its item by bit-width (classes 0..3 = 2, 4, 8, 16 bits) and walks them one width at a time:
+// every step then deals with a single width and runs the body compiled for it, however the widths
+// are mixed in the card.
 
 // The item's steps are laid out once per item, one descriptor per step, by the lanes in parallel:
 // the tokens of class c occupy [begin_c, end_c) of the list and are walked 16 at a time (16-bit
@@ -119,6 +112,7 @@ __device__ __forceinline__ uint32_t class_width(int c) { return c == 0 ? 2u : (c
 //   bits 0..8  first list position   9..13  tokens in the step   14..15  class
 //   bit 16     the step's records are neighbours in the card (one copy per stream will do)
 constexpr int kAttendMaxSteps = kAttendRows * kAttendSteps / 8 + 3;  // all 16-bit but three tokens, one per other class
+static_assert(kAttendMaxSteps <= 64, "two descriptors per lane");
 
 __device__ __forceinline__ uint32_t step_first(uint32_t d) { return d & 511u; }
 __device__ __forceinline__ int step_rows(uint32_t d) { return (int)((d >> 9) & 31u); }

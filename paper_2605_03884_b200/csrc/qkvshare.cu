@@ -114,17 +114,32 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
     uint32_t carry = 0;
     uint64_t sum_bits = 0;
     bool bad = false;
+    // A thread's eight tokens are eight bytes in, eight bytes and 32 bytes out: moved as whole words
+    // where the pointers allow (a warp then writes 1 KB of offsets contiguously instead of 32
+    // four-byte pieces 32 bytes apart), one by one at a ragged end or on unaligned tables.
+    static_assert(kScanItems == 8, "word-wise path");
+    const bool words_in = (reinterpret_cast<uintptr_t>(bits) & 7u) == 0u;
+    const bool words_bits = (reinterpret_cast<uintptr_t>(bits_out) & 7u) == 0u;
+    const bool words_off = (reinterpret_cast<uintptr_t>(off_out) & 15u) == 0u;
     for (int64_t tile = 0; tile < T; tile += (int64_t)kScanThreads * kScanItems) {
         const int64_t t0 = tile + (int64_t)threadIdx.x * kScanItems;
+        const bool whole = t0 + kScanItems <= T;
         uint32_t rec[kScanItems];
         uint8_t bv[kScanItems];
         uint32_t mine = 0;
+        uint2 packed = make_uint2(0u, 0u);
+        if (whole && words_in) {
+            packed = *reinterpret_cast<const uint2 *>(bits + t0);
+#pragma unroll
+            for (int i = 0; i < kScanItems; ++i) bv[i] = (uint8_t)((i < 4 ? packed.x : packed.y) >> (8 * (i & 3)));
+        } else {
+#pragma unroll
+            for (int i = 0; i < kScanItems; ++i) bv[i] = t0 + i < T ? bits[t0 + i] : (uint8_t)0;
+        }
 #pragma unroll
         for (int i = 0; i < kScanItems; ++i) {
             rec[i] = 0;
-            bv[i] = 0;
             if (t0 + i < T) {
-                bv[i] = bits[t0 + i];
                 rec[i] = record_bytes(d, bv[i], p.meta_bytes);
                 bad |= rec[i] == 0u;
                 sum_bits += bv[i];
@@ -133,13 +148,26 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
         }
         uint32_t total;
         uint32_t run = carry + block_exclusive_scan(mine, warp_sums, total);
+        uint32_t off[kScanItems];
 #pragma unroll
         for (int i = 0; i < kScanItems; ++i) {
-            if (t0 + i < T) {
-                off_out[t0 + i] = run;
-                bits_out[t0 + i] = bv[i];
-                run += rec[i];
-            }
+            off[i] = run;
+            run += rec[i];
+        }
+        if (whole && words_off) {
+            *reinterpret_cast<uint4 *>(off_out + t0) = make_uint4(off[0], off[1], off[2], off[3]);
+            *reinterpret_cast<uint4 *>(off_out + t0 + 4) = make_uint4(off[4], off[5], off[6], off[7]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < kScanItems; ++i)
+                if (t0 + i < T) off_out[t0 + i] = off[i];
+        }
+        if (whole && words_in && words_bits) {
+            *reinterpret_cast<uint2 *>(bits_out + t0) = packed;
+        } else {
+#pragma unroll
+            for (int i = 0; i < kScanItems; ++i)
+                if (t0 + i < T) bits_out[t0 + i] = bv[i];
         }
         carry += total;
     }
@@ -406,9 +434,6 @@ static uint32_t *work_counter(void *workspace_dev, int launch)
 #endif
 #ifndef QKVS_STAGES_INJECT
 #define QKVS_STAGES_INJECT 2
-#endif
-#ifndef QKVS_INTERLEAVED
-#define QKVS_INTERLEAVED 1
 #endif
 constexpr int kStagesCreate = QKVS_STAGES_CREATE;
 constexpr int kStagesInject = QKVS_STAGES_INJECT;
