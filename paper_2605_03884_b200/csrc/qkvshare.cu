@@ -110,7 +110,8 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
     const int d = p.head_dim;
 
     if (threadIdx.x == 0) s_bad = 0;
-    if (p.workspace && seg == 0 && threadIdx.x < QKVS_WORKSPACE_BYTES / 4) p.workspace[threadIdx.x] = 0u;
+    if (p.workspace && seg == 0)
+        for (int i = threadIdx.x; i < QKVS_WORKSPACE_BYTES / 4; i += blockDim.x) p.workspace[i] = 0u;
     uint32_t carry = 0;
     uint64_t sum_bits = 0;
     bool bad = false;
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
     const bool words_in = (reinterpret_cast<uintptr_t>(bits) & 7u) == 0u;
     const bool words_bits = (reinterpret_cast<uintptr_t>(bits_out) & 7u) == 0u;
     const bool words_off = (reinterpret_cast<uintptr_t>(off_out) & 15u) == 0u;
-    for (int64_t tile = 0; tile < T; tile += (int64_t)kScanThreads * kScanItems) {
+    for (int64_t tile = 0; tile < T; tile += (int64_t)blockDim.x * kScanItems) {
         const int64_t t0 = tile + (int64_t)threadIdx.x * kScanItems;
         const bool whole = t0 + kScanItems <= T;
         uint32_t rec[kScanItems];
@@ -662,7 +663,10 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
     sp.workspace = static_cast<uint32_t *>(workspace_dev);
     const int nseg = layout->bits_mode == 0 ? 1 : layout->n_layers * layout->n_kv_heads;
     if (layout->bits_mode == 1 && cudaMemsetAsync(card_dev, 0, kHeaderBytes, cs) != cudaSuccess) return QKVS_ERR_CUDA;
-    scan_offsets_kernel<<<nseg, kScanThreads, 0, cs>>>(sp);
+    // no more threads than there are groups of eight tokens: a short context then pays for the
+    // block-wide steps of four warps, not of thirty-two
+    const int scan_threads = (int)std::min<int64_t>(kScanThreads, std::max<int64_t>(32, (((int64_t)layout->n_tokens + kScanItems - 1) / kScanItems + 31) / 32 * 32));
+    scan_offsets_kernel<<<nseg, scan_threads, 0, cs>>>(sp);
     if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
     if (layout->bits_mode == 1) {
         finalize_kernel<<<1, kScanThreads, 0, cs>>>(sp);
