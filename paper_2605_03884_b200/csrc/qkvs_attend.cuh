@@ -36,8 +36,13 @@ constexpr int kAttendRows = 16;          // tokens per step
 constexpr int kAttendRecMax = 160;       // largest record of which a step takes 16 (8 bits, fp32 pairs)
 constexpr int kAttendStageBytes = kAttendRows * kAttendRecMax;  // per stream; 16-bit rows go 8 per step
 static_assert(kAttendStageBytes >= 8 * 2 * kAttendD && kAttendStageBytes % 128 == 0, "stage size");
-constexpr int kAttendSteps = 16;         // steps per work item
+#ifndef QKVS_ATTEND_STEPS
+#define QKVS_ATTEND_STEPS 16
+#endif
+constexpr int kAttendSteps = QKVS_ATTEND_STEPS;  // steps of 16 tokens per work item
 constexpr int kAttendPerLane = kAttendRows * kAttendSteps / 32;  // tokens of an item per lane when they are sorted
+constexpr int kAttendMaxSteps = kAttendRows * kAttendSteps / 8 + 3;  // all 16-bit but three tokens, one per other class
+constexpr int kAttendStepSlots = (kAttendMaxSteps + 31) / 32 * 32;   // whole rounds of one descriptor per lane
 constexpr int kAttendMaxPerKv = 8;       // query heads per KV head
 constexpr int kPartialFloats = kAttendD + 4;  // o[128], running maximum (base-2 exponent), running sum, padding
 
@@ -63,7 +68,7 @@ struct AttendWarpSmem {
     alignas(128) uint8_t k[NS][kAttendStageBytes];  // the step's records, packed one after another
     alignas(128) uint8_t v[NS][kAttendStageBytes];
     uint32_t list[kAttendRows * kAttendSteps];  // record offsets of the item's tokens, grouped by bit-width
-    uint32_t steps[64];                         // the item's step descriptors
+    uint32_t steps[kAttendStepSlots];           // the item's step descriptors
     alignas(8) uint64_t full[NS];
 };
 
@@ -109,14 +114,13 @@ __device__ __forceinline__ float exp2_approx(float x)
 // The item's steps are laid out once per item, one descriptor per step, by the lanes in parallel:
 // the tokens of class c occupy [begin_c, end_c) of the list and are walked 16 at a time (16-bit
 // rows, 256 bytes each, 8 at a time: a stage holds eight of them).
-//   bits 0..8  first list position   9..13  tokens in the step   14..15  class
-//   bit 16     the step's records are neighbours in the card (one copy per stream will do)
-constexpr int kAttendMaxSteps = kAttendRows * kAttendSteps / 8 + 3;  // all 16-bit but three tokens, one per other class
-static_assert(kAttendMaxSteps <= 64, "two descriptors per lane");
+//   bits 0..9  first list position   10..14  tokens in the step   15..16  class
+//   bit 17     the step's records are neighbours in the card (one copy per stream will do)
+static_assert(kAttendRows * kAttendSteps <= 512 && kAttendMaxSteps <= kAttendStepSlots, "descriptor fields");
 
-__device__ __forceinline__ uint32_t step_first(uint32_t d) { return d & 511u; }
-__device__ __forceinline__ int step_rows(uint32_t d) { return (int)((d >> 9) & 31u); }
-__device__ __forceinline__ int step_class(uint32_t d) { return (int)((d >> 14) & 3u); }
+__device__ __forceinline__ uint32_t step_first(uint32_t d) { return d & 1023u; }
+__device__ __forceinline__ int step_rows(uint32_t d) { return (int)((d >> 10) & 31u); }
+__device__ __forceinline__ int step_class(uint32_t d) { return (int)((d >> 15) & 3u); }
 
 template <int META>
 __device__ __forceinline__ uint32_t class_record_bytes(int c)
@@ -137,7 +141,7 @@ __device__ __forceinline__ uint32_t make_step(uint32_t idx, const uint32_t (&e)[
             const uint32_t s0 = begin + (idx - first_step) * per;
             const uint32_t rows = min(per, e[c] - s0);
             const bool neighbours = list[s0 + rows - 1] - list[s0] == (rows - 1) * class_record_bytes<META>(c);
-            return s0 | (rows << 9) | ((uint32_t)c << 14) | (neighbours ? 1u << 16 : 0u);
+            return s0 | (rows << 10) | ((uint32_t)c << 15) | (neighbours ? 1u << 17 : 0u);
         }
         first_step += n_steps;
         begin = e[c];
@@ -156,7 +160,7 @@ __device__ __forceinline__ void attend_issue(AttendWarpSmem<NS> &sm, int stage, 
 {
     const int n = step_rows(d);
     const uint32_t rec = class_record_bytes<META>(step_class(d));
-    if (d & (1u << 16)) {
+    if (d & (1u << 17)) {
         if (lane == 0) {
             const uint32_t first = sm.list[step_first(d)];
             mbar_arrive_expect_tx(&sm.full[stage], 2u * (uint32_t)n * rec);
@@ -590,12 +594,14 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
                     if (my_cls[r] == c) sm.list[pos[c]++] = my_off[r];
             }
             __syncwarp();
-            // the steps, two descriptors per lane
-            const uint32_t d_lo = make_step<META>((uint32_t)lane, ends, sm.list);
-            const uint32_t d_hi = make_step<META>((uint32_t)lane + 32u, ends, sm.list);
-            sm.steps[lane] = d_lo;
-            sm.steps[lane + 32] = d_hi;
-            n_steps = __popc(__ballot_sync(0xffffffffu, d_lo != 0u)) + __popc(__ballot_sync(0xffffffffu, d_hi != 0u));
+            // the steps, one descriptor per lane and round
+            n_steps = 0;
+#pragma unroll
+            for (int r = 0; r < kAttendStepSlots / 32; ++r) {
+                const uint32_t d = make_step<META>((uint32_t)(lane + 32 * r), ends, sm.list);
+                sm.steps[lane + 32 * r] = d;
+                n_steps += __popc(__ballot_sync(0xffffffffu, d != 0u));
+            }
             __syncwarp();
         }
 
