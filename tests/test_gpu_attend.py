@@ -155,3 +155,16 @@ def test_full_size_llama_8k(number):
         Vs.append(v)
     worst = _check(Ks, Vs, wl.bits_for(w), w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens, 32, seed=number)
     assert worst <= 2.0 ** -9
+
+
+@pytest.mark.parametrize("T", [2048, 1000])
+def test_mid_sized_caches_all_layers(T):
+    """All 32 layers x 8 heads at shorter contexts: fewer work items than warps, a ragged last item
+    in the second case."""
+    w = wl.WORKLOADS[4].scaled(n_tokens=T)
+    Ks, Vs = [], []
+    for _, k, v in wl.kv_layers(w):
+        Ks.append(k)
+        Vs.append(v)
+    worst = _check(Ks, Vs, wl.bits_for(w), w.n_layers, w.n_kv_heads, w.head_dim, T, 32, seed=T)
+    assert worst <= 2.0 ** -9
