@@ -401,6 +401,21 @@ def run_ours(args):
         payload = sizes[-1] - prefix
         attend = {"what": "decode-step attention straight from the card, all layers, 4 query heads per KV head",
                   "ms": a_ms, "card_payload_bytes": payload, "card_gbs": payload / (a_ms * 1e-3) / 1e9}
+        # eight query rows per KV head fill the products' columns: two new tokens of a 4:1 grouped-query
+        # model (their heads laid out as eight heads per KV head) in one pass over the card
+        n_q2 = 8 * H
+        qd2 = torch.randn((L, n_q2, d), device="cuda").half()
+        od2 = torch.zeros((L, n_q2, d), dtype=torch.float32, device="cuda")
+        scratch2 = torch.zeros(q.attend_scratch_size(lay, n_q2), dtype=torch.uint8, device="cuda")
+        ev = []
+        for _ in range(25):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            q.card_attend(card, lay, qd2, od2, scratch2, card_bytes=sizes[-1], stream=stream)
+            b.record(stream)
+            ev.append((a, b))
+        torch.cuda.synchronize()
+        attend["ms_8_rows_per_kv_head"] = statistics.median(x.elapsed_time(y) for x, y in ev[5:])
 
     # what the handoff costs in accuracy: every hop's injected cache against the original FP16 cache
     # (reporting only, outside every timed region; plain torch reductions)

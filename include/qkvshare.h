@@ -257,7 +257,10 @@ QKVS_API qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t car
  * applied outside the products.
  *   layout        n_layers, n_kv_heads, head_dim, n_tokens and meta_bytes of the card (checked
  *                 against its header on the device); head_dim must be 128; strides are not looked at
- *   n_q_heads     multiple of n_kv_heads, at most 8 query heads per KV head
+ *   n_q_heads     multiple of n_kv_heads, at most 8 query heads per KV head.  The products have
+ *                 eight columns per KV head whatever is used of them, so a model with four query
+ *                 heads per KV head can pass the queries of two new tokens as eight heads per KV
+ *                 head (row kv * 8 + token * 4 + head) and have both attended in the time of one
  *   q_dev         FP16 [n_layers][n_q_heads][head_dim], 16-byte aligned
  *   out_dev       FP32 [n_layers][n_q_heads][head_dim], 16-byte aligned; all zeros if n_tokens is
  *                 0 or the card does not check out
