@@ -36,10 +36,7 @@ constexpr int kAttendRows = 16;          // tokens per step
 constexpr int kAttendRecMax = 160;       // largest record of which a step takes 16 (8 bits, fp32 pairs)
 constexpr int kAttendStageBytes = kAttendRows * kAttendRecMax;  // per stream; 16-bit rows go 8 per step
 static_assert(kAttendStageBytes >= 8 * 2 * kAttendD && kAttendStageBytes % 128 == 0, "stage size");
-#ifndef QKVS_ATTEND_STEPS
-#define QKVS_ATTEND_STEPS 16
-#endif
-constexpr int kAttendSteps = QKVS_ATTEND_STEPS;  // steps of 16 tokens per work item
+constexpr int kAttendSteps = 16;         // steps of 16 tokens per work item
 constexpr int kAttendPerLane = kAttendRows * kAttendSteps / 32;  // tokens of an item per lane when they are sorted
 constexpr int kAttendMaxSteps = kAttendRows * kAttendSteps / 8 + 3;  // all 16-bit but three tokens, one per other class
 constexpr int kAttendStepSlots = (kAttendMaxSteps + 31) / 32 * 32;   // whole rounds of one descriptor per lane
@@ -515,6 +512,7 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
     int stage = 0;
     uint32_t parity = 0;
     bool ok = true;
+    bool try_one_width = true;
     uint32_t item = blockIdx.x * WARPS + (uint32_t)warp;
     while (item < p.n_items && ok) {
         const uint32_t lh = item / p.items_per_head, ck = item - lh * p.items_per_head;
@@ -537,37 +535,65 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
         // ---- the item's tokens, a run of kAttendPerLane per lane: check the table entries, sort by width into the list
         const uint32_t tok0 = sub0 * kAttendRows;
         const int n_tok = (int)min((uint64_t)(kAttendRows * kAttendSteps), T - tok0);
-        uint32_t my_off[kAttendPerLane];
-        int my_cls[kAttendPerLane];
-        uint32_t counts = 0, counts_hi = 0;  // tokens of this lane per class: 16-bit fields (2 | 4 bits), (8 | 16 bits)
-        {
-            const bool base_ok = base_k >= sec.payload_off && base_v >= sec.payload_off && ((base_k | base_v) & 15u) == 0u;
-            bool bad = false;
-            uint32_t o_next = kAttendPerLane * lane <= n_tok ? __ldg(offs_tab + kAttendPerLane * lane) : 0u;
+        uint32_t ends[4];  // where each class ends in the list
+        const bool base_ok = base_k >= sec.payload_off && base_v >= sec.payload_off && ((base_k | base_v) & 15u) == 0u;
+        // A whole item of one width (every item of a uniform card): eight bit-widths per lane in one
+        // word, all equal, and the two offsets at the item's ends a whole item's records apart.  The
+        // records are then neighbours from the first to the last -- the offsets cannot but grow by
+        // the record size in between -- and the list is an arithmetic sequence.  Tried as long as
+        // the warp's previous item was of that kind, so that a mixed card pays for the attempt once.
+        static_assert(kAttendPerLane == 8, "one word of bit-widths per lane");
+        bool one_width = false;
+        if (try_one_width && n_tok == kAttendRows * kAttendSteps && (reinterpret_cast<uintptr_t>(bits_tab) & 7u) == 0u) {
+            const uint2 w8 = __ldg(reinterpret_cast<const uint2 *>(bits_tab) + lane);
+            const uint32_t o_first = __ldg(offs_tab), o_last = __ldg(offs_tab + n_tok);
+            const uint32_t b0 = __shfl_sync(0xffffffffu, w8.x, 0) & 0xffu;
+            const bool same = w8.x == b0 * 0x01010101u && w8.y == w8.x;
+            const uint32_t rec = record_bytes(kAttendD, (int)b0, META);
+            one_width = __all_sync(0xffffffffu, same) && base_ok && rec != 0u && (o_first & 15u) == 0u && o_last >= o_first &&
+                        o_last - o_first == (uint32_t)n_tok * rec && base_k + (uint64_t)o_last <= total_bytes &&
+                        base_v + (uint64_t)o_last <= total_bytes;
+            try_one_width = one_width;
+            if (one_width) {
+                const int cls = b0 == 2u ? 0 : (b0 == 4u ? 1 : (b0 == 8u ? 2 : 3));
 #pragma unroll
-            for (int r = 0; r < kAttendPerLane; ++r) {
-                const int j = kAttendPerLane * lane + r;
-                const uint32_t o = o_next;
-                o_next = j + 1 <= n_tok ? __ldg(offs_tab + j + 1) : 0u;
-                my_off[r] = o;
-                my_cls[r] = 4;
-                if (j < n_tok) {
-                    const uint32_t b = __ldg(bits_tab + j);
-                    const uint32_t rec = record_bytes(kAttendD, (int)b, META);
-                    const bool fine = base_ok && rec != 0u && o_next >= o && o_next - o == rec && (o & 15u) == 0u &&
-                                      base_k + (uint64_t)o_next <= total_bytes && base_v + (uint64_t)o_next <= total_bytes;
-                    bad |= !fine;
-                    if (fine) {
-                        my_cls[r] = b == 2u ? 0 : (b == 4u ? 1 : (b == 8u ? 2 : 3));
-                        if (my_cls[r] < 2) counts += 1u << (16 * my_cls[r]);
-                        else counts_hi += 1u << (16 * (my_cls[r] - 2));
-                    }
-                }
+                for (int c = 0; c < 4; ++c) ends[c] = c < cls ? 0u : (uint32_t)n_tok;
+                __syncwarp();  // the previous item's list is no longer read
+#pragma unroll
+                for (int r = 0; r < kAttendPerLane; ++r) sm.list[kAttendPerLane * lane + r] = o_first + (uint32_t)(kAttendPerLane * lane + r) * rec;
+                __syncwarp();
             }
-            if (__any_sync(0xffffffffu, bad) && lane == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
         }
         uint32_t n_steps;
-        {
+        if (!one_width) {
+            uint32_t my_off[kAttendPerLane];
+            int my_cls[kAttendPerLane];
+            uint32_t counts = 0, counts_hi = 0;  // tokens of this lane per class: 16-bit fields (2 | 4 bits), (8 | 16 bits)
+            {
+                bool bad = false;
+                uint32_t o_next = kAttendPerLane * lane <= n_tok ? __ldg(offs_tab + kAttendPerLane * lane) : 0u;
+#pragma unroll
+                for (int r = 0; r < kAttendPerLane; ++r) {
+                    const int j = kAttendPerLane * lane + r;
+                    const uint32_t o = o_next;
+                    o_next = j + 1 <= n_tok ? __ldg(offs_tab + j + 1) : 0u;
+                    my_off[r] = o;
+                    my_cls[r] = 4;
+                    if (j < n_tok) {
+                        const uint32_t b = __ldg(bits_tab + j);
+                        const uint32_t rec = record_bytes(kAttendD, (int)b, META);
+                        const bool fine = base_ok && rec != 0u && o_next >= o && o_next - o == rec && (o & 15u) == 0u &&
+                                          base_k + (uint64_t)o_next <= total_bytes && base_v + (uint64_t)o_next <= total_bytes;
+                        bad |= !fine;
+                        if (fine) {
+                            my_cls[r] = b == 2u ? 0 : (b == 4u ? 1 : (b == 8u ? 2 : 3));
+                            if (my_cls[r] < 2) counts += 1u << (16 * my_cls[r]);
+                            else counts_hi += 1u << (16 * (my_cls[r] - 2));
+                        }
+                    }
+                }
+                if (__any_sync(0xffffffffu, bad) && lane == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
+            }
             // positions: class-major, then lane, then the lane's own order
             uint32_t inc = counts, inc_hi = counts_hi;
 #pragma unroll
@@ -579,7 +605,6 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
                 }
             }
             const uint32_t tot = __shfl_sync(0xffffffffu, inc, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
-            uint32_t ends[4];  // where each class ends in the list
             ends[0] = tot & 0xffffu;
             ends[1] = ends[0] + (tot >> 16);
             ends[2] = ends[1] + (tot_hi & 0xffffu);
@@ -594,6 +619,8 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
                     if (my_cls[r] == c) sm.list[pos[c]++] = my_off[r];
             }
             __syncwarp();
+        }
+        {
             // the steps, one descriptor per lane and round
             n_steps = 0;
 #pragma unroll
