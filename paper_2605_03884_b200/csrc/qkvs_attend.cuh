@@ -66,6 +66,7 @@ struct AttendWarpSmem {
     alignas(128) uint8_t v[NS][kAttendStageBytes];
     uint32_t list[kAttendRows * kAttendSteps];  // record offsets of the item's tokens, grouped by bit-width
     uint32_t steps[kAttendStepSlots];           // the item's step descriptors
+    alignas(16) float qsum[4][8];               // per tig: sums over group g of the queries of heads 2tig + h, at [2g + h]
     alignas(8) uint64_t full[NS];
 };
 
@@ -317,14 +318,14 @@ __device__ __forceinline__ void group_params_of(const uint8_t *rec, bool valid, 
 // maximum and sum of a head, the factors that rescale its accumulators and the accumulators
 // themselves sit in the same lane.  FULL: all 16 tokens are there.
 //   qb[g][k]     query fragments (B operand): head gid, channels 32g + 8tig + k and + k + 4
-//   qsum[g][h]   sum of head 2tig + h's query over group g
+//   sm.qsum      sums over a group of the queries of the lane's two heads (read here, once per step)
 //   m_run[h], l_run[h]   running maximum of head 2tig + h (the same in all lanes of a tig) and this
 //                lane's share of its running sum (tokens gid, gid + 8 of every step)
 //   zacc[g][h]   this lane's share of sum_t p_t zero_tg for head 2tig + h
 //   acc[g][j][.] channels 32g + 4gid + 2j (+1) x heads 2tig, 2tig + 1, without the zero-point part
 template <int NS, int B, bool FULL, int META>
 __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int stage, int rows, int gid, int tig, float scale_log2,
-                                            const uint32_t (&qb)[4][4], const float (&qsum)[4][2], float (&m_run)[2],
+                                            const uint32_t (&qb)[4][4], float (&m_run)[2],
                                             float (&l_run)[2], float (&zacc)[4][2], float (&acc)[4][2][4])
 {
     constexpr int REC = B == 16 ? 2 * kAttendD : kAttendD * B / 8 + 4 * META;
@@ -336,6 +337,8 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
     float x[2][2];  // logits (base 2): [token gid + 8k][head 2tig + h]
     {
         float sacc[4][4];
+        const float4 qs_lo = *reinterpret_cast<const float4 *>(&sm.qsum[tig][0]), qs_hi = *reinterpret_cast<const float4 *>(&sm.qsum[tig][4]);
+        const float qsum[4][2] = {{qs_lo.x, qs_lo.y}, {qs_lo.z, qs_lo.w}, {qs_hi.x, qs_hi.y}, {qs_hi.z, qs_hi.w}};
         // 4-bit rows: a (token, group) is 16 bytes of codes, a matrix row; two loads hand every
         // lane its words of all four groups of its two tokens
         uint32_t ka[4], kb[4];
@@ -636,7 +639,7 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
         // 32g + 8tig + k paired with + k + 4 (the pairing of key_pairs); and the sums over a group of
         // the queries of the lane's own two heads
         uint32_t qa[4][4];
-        float qsum[4][2];
+        __syncwarp();  // the previous item's steps no longer read the query sums
         {
             const __half *qrow = p.q + ((uint64_t)layer * p.n_q_heads + (uint64_t)head * per_kv + gid) * kAttendD + 8 * tig;
 #pragma unroll
@@ -652,10 +655,14 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
                 float sum = ((f0.x + f0.y) + (f1.x + f1.y)) + ((f2.x + f2.y) + (f3.x + f3.y));
                 sum += __shfl_xor_sync(0xffffffffu, sum, 1);
                 sum += __shfl_xor_sync(0xffffffffu, sum, 2);  // head gid's, in all four lanes of the gid
-                qsum[g][0] = __shfl_sync(0xffffffffu, sum, 8 * tig);
-                qsum[g][1] = __shfl_sync(0xffffffffu, sum, 8 * tig + 4);
+                const float s0 = __shfl_sync(0xffffffffu, sum, 8 * tig), s1 = __shfl_sync(0xffffffffu, sum, 8 * tig + 4);
+                if (gid == 0) {
+                    sm.qsum[tig][2 * g] = s0;
+                    sm.qsum[tig][2 * g + 1] = s1;
+                }
             }
         }
+        __syncwarp();  // the query sums are in place
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
         float zacc[4][2] = {{0.0f, 0.0f}, {0.0f, 0.0f}, {0.0f, 0.0f}, {0.0f, 0.0f}};
         float acc[4][2][4];
@@ -678,16 +685,16 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
             const int rows = step_rows(d), cls = step_class(d);
             if (rows == kAttendRows) {  // 16-bit rows come at most eight per step
                 switch (cls) {
-                    case 0: attend_step<NS, 2, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 1: attend_step<NS, 4, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    default: attend_step<NS, 8, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 0: attend_step<NS, 2, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, m_run, l_run, zacc, acc); break;
+                    case 1: attend_step<NS, 4, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, m_run, l_run, zacc, acc); break;
+                    default: attend_step<NS, 8, true, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, m_run, l_run, zacc, acc); break;
                 }
             } else {
                 switch (cls) {
-                    case 0: attend_step<NS, 2, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 1: attend_step<NS, 4, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    case 2: attend_step<NS, 8, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
-                    default: attend_step<NS, 16, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, qsum, m_run, l_run, zacc, acc); break;
+                    case 0: attend_step<NS, 2, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, m_run, l_run, zacc, acc); break;
+                    case 1: attend_step<NS, 4, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, m_run, l_run, zacc, acc); break;
+                    case 2: attend_step<NS, 8, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, m_run, l_run, zacc, acc); break;
+                    default: attend_step<NS, 16, false, META>(sm, stage, rows, gid, tig, p.scale_log2, qa, m_run, l_run, zacc, acc); break;
                 }
             }
             __syncwarp();  // every lane has read the stage: it can be re-armed
