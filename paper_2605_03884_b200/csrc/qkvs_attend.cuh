@@ -209,6 +209,21 @@ __device__ __forceinline__ void nibble_pairs(uint32_t w, uint32_t (&e)[4])
     e[3] = as_u32(__hfma2(as_half2(f3), sixteenth, minus64));
 }
 
+// The four 2-bit codes in the low byte of each half of a word as four FP16 pairs e[k] = (code k
+// of the low half, code k of the high half), without shifts: code k is picked up where it sits,
+// as 1024 + 4^k n, and brought down by an exact fused multiply-add.
+__device__ __forceinline__ void crumb_pairs(uint32_t y, uint32_t (&e)[4])
+{
+    uint32_t f1, f2, f3;
+    e[0] = int_pair(y, 0x00030003u);
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(f1) : "r"(y), "r"(0x000c000cu), "r"(kHalfMagic));
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(f2) : "r"(y), "r"(0x00300030u), "r"(kHalfMagic));
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(f3) : "r"(y), "r"(0x00c000c0u), "r"(kHalfMagic));
+    e[1] = as_u32(__hfma2(as_half2(f1), __floats2half2_rn(0.25f, 0.25f), __floats2half2_rn(-256.0f, -256.0f)));
+    e[2] = as_u32(__hfma2(as_half2(f2), __floats2half2_rn(0.0625f, 0.0625f), __floats2half2_rn(-64.0f, -64.0f)));
+    e[3] = as_u32(__hfma2(as_half2(f3), __floats2half2_rn(0.015625f, 0.015625f), __floats2half2_rn(-16.0f, -16.0f)));
+}
+
 // Four 8 x 8 matrices of 16-bit elements from shared memory, rows of 16 bytes: lane l gives the
 // address of row l % 8 of matrix l / 8; lane (gid, tig) receives from each matrix the word tig of
 // row gid -- or, transposed, the element gid of the rows 2tig (low half) and 2tig + 1 (high half).
@@ -251,9 +266,7 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, ui
         for (int k = 0; k < 4; ++k) e[k] = int_pair(__byte_perm(w.x, w.y, 0x0011u * k + 0x1100u * (4 + k)), 0x00ff00ffu);
     } else if constexpr (B == 2) {
         const uint32_t w = *reinterpret_cast<const uint16_t *>(codes);
-        const uint32_t y = __byte_perm(w, 0u, 0x4140);  // codes 0..3 in byte 0, codes 4..7 in byte 2
-#pragma unroll
-        for (int k = 0; k < 4; ++k) e[k] = int_pair(y >> (2 * k), 0x00030003u);
+        crumb_pairs(__byte_perm(w, 0u, 0x4140), e);  // codes 0..3 in byte 0, codes 4..7 in byte 2
     }
 }
 
@@ -281,8 +294,7 @@ __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t 
         for (int k = 0; k < 4; ++k) e[k] = int_pair(__byte_perm(wa, wb, 0x0011u * k + 0x1100u * (4 + k)), 0x00ff00ffu);
     } else {
         const uint32_t x = (uint32_t)*(rec_a + CODES + 8 * g + gid) | ((uint32_t)*(rec_b + CODES + 8 * g + gid) << 16);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) e[k] = int_pair(x >> (2 * k), 0x00030003u);
+        crumb_pairs(x, e);
     }
 }
 
