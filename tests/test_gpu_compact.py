@@ -270,3 +270,40 @@ def test_llama_8k_adaptive_full_size():
     for l in range(L):
         worst = max(worst, max_ulp(Ko[l].cpu().numpy(), Kw[l]), max_ulp(Vo[l].cpu().numpy(), Vw[l]))
     assert worst == 0
+
+
+def test_per_head_bits_attention_and_injection_without_a_scratch_block():
+    """The remaining combinations of the compact format: per-(layer, head) bit-widths under
+    attention, and the entry point that keeps its work counters in the library's own memory."""
+    import torch
+    L, H, d, T, nq = 2, 2, 128, 300, 8
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=910)
+    bits = np.stack([wl.iid_bits(T, (0.25, 0.25, 0.25, 0.25), 920 + i) for i in range(L * H)]).reshape(-1)
+    olay, glay = _olay(L, H, d, T, mode=1), _glay(L, H, d, T, mode=1)
+    st, card = oracle.card_create(olay, Ks, Vs, bits)
+    assert st == oracle.OK
+    qh = wl.random_fp16((L, nq, d), 930)
+    st, want = oracle.card_attend(card, olay, qh)
+    assert st == oracle.OK
+    card_d = torch.from_numpy(card).cuda()
+    out = torch.full(qh.shape, 7.0, dtype=torch.float32, device="cuda")
+    scratch = torch.full((q.attend_scratch_size(glay, nq),), 0x5A, dtype=torch.uint8, device="cuda")
+    q.card_attend(card_d, glay, torch.from_numpy(qh).cuda(), out, scratch)
+    torch.cuda.synchronize()
+    assert int(scratch[:4].view(torch.int32).item()) == 0
+    Kr, Vr = [np.zeros_like(k) for k in Ks], [np.zeros_like(v) for v in Vs]
+    assert oracle.card_inject(card, olay, Kr, Vr) == oracle.OK
+    got = out.cpu().numpy()
+    for l in range(L):
+        for j in range(nq):
+            vmax = float(np.abs(Vr[l][j // (nq // H)].astype(np.float64)).max())
+            assert float(np.abs(got[l, j] - want[l, j]).max()) <= 2.0 ** -9 * vmax + 1e-6
+    # injection through the entry point without a scratch block: the oracle's values
+    Ko = [torch.full((H, T, d), -3.0, dtype=torch.float16, device="cuda") for _ in range(L)]
+    Vo = [torch.full((H, T, d), -5.0, dtype=torch.float16, device="cuda") for _ in range(L)]
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    assert q.card_inject_noalloc(card_d, glay, Ko, Vo, status_dev=status) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for l in range(L):
+        assert max_ulp(Ko[l].cpu().numpy(), Kr[l]) == 0 and max_ulp(Vo[l].cpu().numpy(), Vr[l]) == 0
