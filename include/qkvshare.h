@@ -41,8 +41,19 @@
  *
  * All entry points return a qkvs_status_t.  Unless stated otherwise a pointer named *_dev is a
  * device pointer, anything else is a host pointer.  The library allocates no device memory and
- * keeps no state between calls; every buffer belongs to the caller.  Launches are asynchronous
- * on the given CUDA stream (a cudaStream_t passed as void*; NULL is the default stream).
+ * every buffer belongs to the caller.  What it keeps between calls is small and per device: how
+ * many CTAs of each kernel the device holds at once (looked up at a kernel's first launch), and,
+ * for qkvs_card_inject_noalloc, the device address of its built-in counter array together with
+ * that array's content (see there).  Both are remembered for the life of the process; a
+ * cudaDeviceReset() invalidates the remembered address, so do not reset a device between calls.
+ * Launches are asynchronous on the given CUDA stream (a cudaStream_t passed as void*; NULL is the
+ * default stream).
+ *
+ * Non-finite input.  The quantiser is defined for finite values.  A NaN or an infinity inside a
+ * token that is quantised (b < 16) gives unspecified scale, zero and codes for its group -- the
+ * codes of one group may then spill into each other inside the group's own code bytes -- but
+ * every access stays inside the record, the card and the cache: memory-safe, not meaningful.
+ * Tokens kept at 16 bits carry any bit pattern through unchanged.
  *
  * Scratch block.  qkvs_card_create and qkvs_card_inject take an optional `workspace_dev`: a
  * device buffer of QKVS_WORKSPACE_BYTES bytes, 16-byte aligned, owned by the caller.  Its content
@@ -244,6 +255,29 @@ QKVS_API qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t car
                                        void *const *V_layers_out, int64_t dst_token_offset,
                                        int32_t *status_dev, void *stream);
 
+/* Hands a card to another GPU (Section 3.2: agents are the nodes of a graph and a handoff travels
+ * along an edge; Section 4.2.1: the prototype hands the card over in memory, inside one runtime,
+ * and fixes no wire format).  A card is one position-independent blob -- every offset in it is
+ * relative to its first byte -- so the handoff is a plain copy of card_bytes bytes into a buffer
+ * on the receiver's GPU, over NVLink when the two devices can reach each other; the receiver then
+ * calls qkvs_card_inject (or qkvs_card_attend) on its own copy, on its own device.  No kernel of
+ * this library ever reads another GPU's memory.
+ *   card_dev, card_bytes   the card on the sender's GPU (device src_device); card_bytes is the
+ *                          header's total_bytes (qkvs_card_info) or any size that covers it
+ *   dst_dev, dst_capacity  buffer on device dst_device, 16-byte aligned, at least card_bytes
+ *   stream                 a stream of the CURRENT device, which must be src_device or dst_device;
+ *                          the copy is ordered after the work already in it (the create that made
+ *                          the card) and the receiver orders its injection after the copy, e.g.
+ *                          with an event recorded in this stream
+ * src_device == dst_device makes an ordinary device-to-device copy.  With two devices the call
+ * first turns on peer access from the current device to the other one if the hardware allows it
+ * and it is not on yet (a per-process switch that stays on); without it the runtime stages the
+ * copy through host memory, slower but equally correct.
+ * Errors: INVALID_ARG (null or misaligned pointer, negative or unknown device), BAD_CARD
+ * (card_bytes below a header), BUFFER_TOO_SMALL, CUDA.  Asynchronous on `stream`. */
+QKVS_API qkvs_status_t qkvs_card_send(const void *card_dev, size_t card_bytes, int32_t src_device,
+                                      void *dst_dev, size_t dst_capacity, int32_t dst_device, void *stream);
+
 /* Decode-step attention straight from a card (Section 4.3 names consuming the quantised cache
  * inside attention as the goal; the FP16 cache of Section 4.2.2 is never rebuilt).  One query
  * token per layer attends to all n_tokens of the card, with grouped queries: query head j reads
@@ -290,6 +324,19 @@ QKVS_API qkvs_status_t qkvs_card_info(const void *card_dev, void *stream, qkvs_c
  *                   [0] counts mismatches of qmax/range, [1] of range/qmax.  Both must read 0.
  * Asynchronous on `stream`; about 10^9 divisions, a few milliseconds. */
 QKVS_API qkvs_status_t qkvs_selftest_division(uint64_t *mismatches_dev, void *stream);
+
+/* Self-test of the bounded waits.  Inside the kernels a warp only ever waits for its own
+ * asynchronous copies, and every such wait gives up after a time limit (two seconds): the warp then
+ * raises QKVS_ERR_TIMEOUT in the status word, gives the copies it still has in flight the same
+ * bounded time to land, and returns, so that a wedged copy engine costs a call, not the GPU.  This
+ * entry point runs that wait on a barrier nothing will ever complete (one warp, no copy issued,
+ * nothing in flight) with a limit of `limit_us` microseconds (1 .. 1 000 000) and checks that it
+ * comes back.  (The paper has no counterpart.)
+ *   status_dev     device int32 (4-byte aligned), cleared by the call; reads QKVS_ERR_TIMEOUT afterwards
+ *   waited_ns_dev  optional device uint64 (8-byte aligned): how long the warp waited, in nanoseconds
+ * Asynchronous on `stream`; the context stays usable. */
+QKVS_API qkvs_status_t qkvs_selftest_bounded_wait(uint32_t limit_us, int32_t *status_dev,
+                                                  uint64_t *waited_ns_dev, void *stream);
 
 QKVS_API const char *qkvs_status_string(qkvs_status_t status);
 

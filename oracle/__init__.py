@@ -89,6 +89,8 @@ def lib():
         l.orc_combine_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int64, C.c_void_p]
         l.orc_card_attend.restype = C.c_int
         l.orc_card_attend.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_int, C.c_void_p, C.c_double, C.c_void_p]
+        l.orc_card_attend_injected.restype = C.c_int
+        l.orc_card_attend_injected.argtypes = l.orc_card_attend.argtypes
         l.orc_num_threads.restype = C.c_int
         l.orc_set_num_threads.argtypes = [C.c_int]
         _lib = l
@@ -247,6 +249,17 @@ def card_create(layout: Layout, K_layers: List[np.ndarray], V_layers: List[np.nd
     return st, card
 
 
+def card_create_into(layout: Layout, K_layers: List[np.ndarray], V_layers: List[np.ndarray],
+                     bits: np.ndarray, card: np.ndarray, model_id=0, sender_id=0, position_offset=0) -> int:
+    """The same call writing into a caller's buffer (uint8, at least card_size bytes): nothing is
+    allocated, so a stopwatch around it times the oracle's own work."""
+    assert card.dtype == np.uint8 and card.flags["C_CONTIGUOUS"] and bits.dtype == np.uint8
+    S = 2 * layout.n_layers * layout.n_kv_heads
+    kp, vp = _ptr_array(K_layers), _ptr_array(V_layers)
+    return lib().orc_card_create_range(C.byref(layout), kp, vp, _ptr(bits), model_id, sender_id,
+                                       position_offset, _ptr(card), card.size, 0, S)
+
+
 def card_inject(card: np.ndarray, dst: Layout, K_out: List[np.ndarray], V_out: List[np.ndarray],
                 dst_token_offset: int = 0, card_bytes: Optional[int] = None) -> int:
     card = np.ascontiguousarray(card, dtype=np.uint8)
@@ -255,16 +268,18 @@ def card_inject(card: np.ndarray, dst: Layout, K_out: List[np.ndarray], V_out: L
                                  C.byref(dst), kp, vp, dst_token_offset)
 
 
-def card_attend(card: np.ndarray, layout: Layout, q: np.ndarray, softmax_scale: Optional[float] = None
-                ) -> Tuple[int, np.ndarray]:
+def card_attend(card: np.ndarray, layout: Layout, q: np.ndarray, softmax_scale: Optional[float] = None,
+                injected: bool = False) -> Tuple[int, np.ndarray]:
     """Decode-step attention from the card.  q: FP16 [n_layers, n_q_heads, head_dim]; returns
-    (status, float64 [n_layers, n_q_heads, head_dim])."""
+    (status, float64 [n_layers, n_q_heads, head_dim]).  injected=False attends to the values the
+    records stand for (unrounded); injected=True to the FP16 cache injection would rebuild."""
     card = np.ascontiguousarray(card, dtype=np.uint8)
     q = np.ascontiguousarray(q, dtype=np.float16)
     assert q.ndim == 3 and q.shape[0] == layout.n_layers and q.shape[2] == layout.head_dim
     scale = 1.0 / float(np.sqrt(layout.head_dim)) if softmax_scale is None else float(softmax_scale)
     out = np.zeros(q.shape, dtype=np.float64)
-    st = lib().orc_card_attend(_ptr(card), card.size, C.byref(layout), q.shape[1], _ptr(q), scale, _ptr(out))
+    fn = lib().orc_card_attend_injected if injected else lib().orc_card_attend
+    st = fn(_ptr(card), card.size, C.byref(layout), q.shape[1], _ptr(q), scale, _ptr(out))
     return st, out
 
 

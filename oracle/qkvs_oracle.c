@@ -539,6 +539,25 @@ static uint64_t stream_base(const uint8_t *card, const orc_layout *L, int64_t s)
     return po + get_u64(card + get_u64(card + 120) + 8u * (uint64_t)s);
 }
 
+/* A card that is read back is untrusted: stream s must start on a 16-byte boundary inside the
+ * payload and its last record must end inside the card.  Compared without forming base + length,
+ * which a damaged stream-base entry close to 2^64 would wrap around. */
+static int stream_in_bounds(const uint8_t *card, const orc_layout *L, int64_t s, uint64_t stream_len)
+{
+    uint64_t po = get_u64(card + 96), total = get_u64(card + 112);
+    if (po > total) return 0;
+    uint64_t rel;
+    if (L->bits_mode == 0) {
+        uint64_t sb = get_u64(card + 104);
+        if (sb != 0 && (uint64_t)s > (total - po) / sb) return 0;
+        rel = (uint64_t)s * sb;
+    } else {
+        rel = get_u64(card + get_u64(card + 120) + 8u * (uint64_t)s);
+    }
+    if (rel % 16u != 0 || rel > total - po) return 0;
+    return stream_len <= total - po - rel;
+}
+
 /* FP16 cache + bit-widths -> card.  K_layers[l], V_layers[l] point at [H, *, d] FP16 blocks
  * addressed with the layout's strides.  Streams in [s_begin, s_end) are encoded (use 0 and
  * 2*L*H for the whole card); the prefix is always written. */
@@ -602,6 +621,11 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
         return ORC_INVALID_ARG;
     uint64_t bo = get_u64(card + 80), oo = get_u64(card + 88);
     int64_t T = C.n_tokens, S = 2 * (int64_t)C.n_layers * C.n_kv_heads;
+    for (int64_t s = 0; s < S; ++s) {
+        int64_t seg = segment_of(&C, (int)(s / (2 * C.n_kv_heads)), (int)(s % C.n_kv_heads));
+        if (!stream_in_bounds(card, &C, s, get_u32(card + oo + 4u * ((uint64_t)seg * (uint64_t)(T + 1) + (uint64_t)T))))
+            return ORC_BAD_CARD;
+    }
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 1)
 #endif
@@ -639,23 +663,40 @@ static void reconstruct_record(const uint8_t *rec, int d, int b, int meta, doubl
     }
 }
 
-/* Decode-step attention straight from a card, without rebuilding the FP16 cache
- * (Section 4.3: consuming a foreign quantised cache directly inside attention is the paper's
- * stated goal; Section 3.1 for K, V per layer and head).  One new token per layer attends to all
- * n_tokens of the card.  Query head j of a layer reads KV head j / (n_q_heads / n_kv_heads)
- * (grouped-query attention; the paper's model, Llama-3.1-8B, has 32 query and 8 KV heads):
+/* The values injection hands to the receiving framework: the record decoded exactly as
+ * orc_card_inject does (fp16_rne(fl32(fl32(q) * scale) + zero), Section 4.2.2), widened. */
+static void injected_record(const uint8_t *rec, int d, int b, int meta, double *row)
+{
+    uint16_t h[256];
+    decode_record(rec, d, b, meta, h);
+    for (int i = 0; i < d; ++i) row[i] = (double)orc_half_to_float(h[i]);
+}
+
+/* Decode-step attention over the tokens of a card (Section 4.3: consuming a foreign quantised
+ * cache directly inside attention is the paper's stated goal; Section 3.1 for K, V per layer and
+ * head).  One new token per layer attends to all n_tokens of the card.  Query head j of a layer
+ * reads KV head j / (n_q_heads / n_kv_heads) (grouped-query attention; the paper's model,
+ * Llama-3.1-8B, has 32 query and 8 KV heads):
  *     s_t  = softmax_scale * sum_c q[j][c] * K~[t][c]
  *     p_t  = exp(s_t - max_t s_t) / sum_t exp(s_t - max_t s_t)
  *     o[c] = sum_t p_t * V~[t][c]
- * where K~, V~ are the values the records stand for (reconstruct_record).  The paper gives no
- * formula for this step; this is the textbook definition, evaluated in double precision.
+ * The paper gives no formula for this step; this is the textbook definition, evaluated in double
+ * precision.  Two readings of K~, V~ are provided:
+ *   fp16_rounded = 0   the values the records stand for, code * scale + zero unrounded
+ *                      (reconstruct_record): attention that reads the card itself forms no FP16
+ *                      copy.  This is what orc_card_attend computes and what the CUDA path is
+ *                      held to.
+ *   fp16_rounded = 1   the FP16 cache that injection would have produced (injected_record):
+ *                      "inject, then attend".  orc_card_attend_injected; reported beside the
+ *                      other so that the distance between the two readings is a number.
  *   q    [n_layers][n_q_heads][head_dim] FP16 bit patterns
  *   out  [n_layers][n_q_heads][head_dim] double */
-int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *L, int n_q_heads,
-                    const uint16_t *q, double softmax_scale, double *out)
+static int attend_over_card(const uint8_t *card, uint64_t card_bytes, const orc_layout *L, int n_q_heads,
+                            const uint16_t *q, double softmax_scale, double *out, int fp16_rounded)
 {
     int st = layout_ok(L);
     if (st) return st;
+    if (fp16_rounded && L->head_dim > 256) return ORC_UNSUPPORTED_SHAPE; /* injected_record's row buffer */
     if (n_q_heads < L->n_kv_heads || n_q_heads % L->n_kv_heads != 0) return ORC_INVALID_ARG;
     if (card_bytes < 256) return ORC_BAD_CARD;
     if (get_u32(card + 0) != 0x53564B51u || get_u32(card + 4) != 1u || get_u32(card + 8) != 0u) return ORC_BAD_CARD;
@@ -671,6 +712,11 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
     if (T == 0) {
         memset(out, 0, sizeof(double) * (size_t)C.n_layers * (size_t)n_q_heads * (size_t)d);
         return ORC_OK;
+    }
+    for (int64_t s = 0; s < 2 * (int64_t)C.n_layers * H; ++s) {
+        int64_t seg = segment_of(&C, (int)(s / (2 * H)), (int)(s % H));
+        if (!stream_in_bounds(card, &C, s, get_u32(card + oo + 4u * ((uint64_t)seg * (uint64_t)(T + 1) + (uint64_t)T))))
+            return ORC_BAD_CARD;
     }
     int failed = 0;
 #ifdef _OPENMP
@@ -694,8 +740,13 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
         const uint8_t *ks = card + stream_base(card, &C, stream_index(&C, l, 0, h));
         const uint8_t *vs = card + stream_base(card, &C, stream_index(&C, l, 1, h));
         for (int64_t t = 0; t < T; ++t) {
-            reconstruct_record(ks + off[t], d, bits[t], meta_of(&C), kx + t * d);
-            reconstruct_record(vs + off[t], d, bits[t], meta_of(&C), vx + t * d);
+            if (fp16_rounded) {
+                injected_record(ks + off[t], d, bits[t], meta_of(&C), kx + t * d);
+                injected_record(vs + off[t], d, bits[t], meta_of(&C), vx + t * d);
+            } else {
+                reconstruct_record(ks + off[t], d, bits[t], meta_of(&C), kx + t * d);
+                reconstruct_record(vs + off[t], d, bits[t], meta_of(&C), vx + t * d);
+            }
         }
         for (int jj = 0; jj < per_kv; ++jj) {
             const int j = h * per_kv + jj;
@@ -725,6 +776,20 @@ int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *
         free(s);
     }
     return failed ? ORC_INVALID_ARG : ORC_OK;
+}
+
+/* Attention straight from the card: the records' own values, no FP16 rounding. */
+int orc_card_attend(const uint8_t *card, uint64_t card_bytes, const orc_layout *L, int n_q_heads,
+                    const uint16_t *q, double softmax_scale, double *out)
+{
+    return attend_over_card(card, card_bytes, L, n_q_heads, q, softmax_scale, out, 0);
+}
+
+/* Inject, then attend: the same attention over the FP16 cache orc_card_inject rebuilds. */
+int orc_card_attend_injected(const uint8_t *card, uint64_t card_bytes, const orc_layout *L, int n_q_heads,
+                             const uint16_t *q, double softmax_scale, double *out)
+{
+    return attend_over_card(card, card_bytes, L, n_q_heads, q, softmax_scale, out, 1);
 }
 
 /* Bit-width assignment from per-token importance scores, the step in front of card creation

@@ -51,8 +51,9 @@ class CardHeader(C.Structure):
 assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
-           "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_attend_scratch_size", "qkvs_card_attend",
-           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_combine_scores", "qkvs_selftest_division", "qkvs_status_string",
+           "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_card_send", "qkvs_attend_scratch_size", "qkvs_card_attend",
+           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_combine_scores", "qkvs_selftest_division",
+           "qkvs_selftest_bounded_wait", "qkvs_status_string",
            "qkvs_version")
 
 _lib = None
@@ -82,6 +83,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_inject.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
     lib.qkvs_card_inject_noalloc.restype = C.c_int
     lib.qkvs_card_inject_noalloc.argtypes = [vp, C.c_size_t, C.POINTER(Layout), vp, vp, C.c_int64, vp, vp]
+    lib.qkvs_card_send.restype = C.c_int
+    lib.qkvs_card_send.argtypes = [vp, C.c_size_t, C.c_int32, vp, C.c_size_t, C.c_int32, vp]
     lib.qkvs_attend_scratch_size.restype = C.c_int
     lib.qkvs_attend_scratch_size.argtypes = [C.POINTER(Layout), C.c_int32, C.POINTER(C.c_size_t)]
     lib.qkvs_card_attend.restype = C.c_int
@@ -94,6 +97,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
     lib.qkvs_selftest_division.restype = C.c_int
     lib.qkvs_selftest_division.argtypes = [vp, vp]
+    lib.qkvs_selftest_bounded_wait.restype = C.c_int
+    lib.qkvs_selftest_bounded_wait.argtypes = [C.c_uint32, vp, vp, vp]
     lib.qkvs_status_string.restype = C.c_char_p
     lib.qkvs_status_string.argtypes = [C.c_int]
     lib.qkvs_version.restype = C.c_int32
@@ -247,6 +252,18 @@ def card_inject_noalloc(card_dev, dst_layout: Layout, K_out: Sequence, V_out: Se
     return st
 
 
+def card_send(card_dev, dst_dev, card_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """qkvs_card_send: copies a card (CUDA uint8 tensor) into `dst_dev`, a CUDA uint8 tensor on the
+    same or on another GPU; the devices are taken from the tensors."""
+    nbytes = int(card_dev.numel() * card_dev.element_size()) if card_bytes is None else int(card_bytes)
+    st = load_library().qkvs_card_send(int(card_dev.data_ptr()), nbytes, int(card_dev.device.index),
+                                       int(dst_dev.data_ptr()), int(dst_dev.numel() * dst_dev.element_size()),
+                                       int(dst_dev.device.index), _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_card_send")
+    return st
+
+
 def attend_scratch_size(layout: Layout, n_q_heads: int) -> int:
     out = C.c_size_t(0)
     st = load_library().qkvs_attend_scratch_size(C.byref(layout), int(n_q_heads), C.byref(out))
@@ -306,6 +323,17 @@ def selftest_division(mismatches_dev, stream=None) -> int:
     st = load_library().qkvs_selftest_division(int(mismatches_dev.data_ptr()), _stream_handle(stream))
     if st != OK:
         raise QkvsError(st, "qkvs_selftest_division")
+    return st
+
+
+def selftest_bounded_wait(limit_us: int, status_dev, waited_ns_dev=None, stream=None, check: bool = True) -> int:
+    """qkvs_selftest_bounded_wait.  status_dev: CUDA int32 tensor of one element; waited_ns_dev:
+    optional CUDA int64 tensor of one element."""
+    st = load_library().qkvs_selftest_bounded_wait(int(limit_us), int(status_dev.data_ptr()),
+                                                   int(waited_ns_dev.data_ptr()) if waited_ns_dev is not None else None,
+                                                   _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_selftest_bounded_wait")
     return st
 
 

@@ -544,14 +544,18 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
             base_v = sec.payload_off + stream_v * stream_bytes;
         } else {
             const uint64_t *sbase = reinterpret_cast<const uint64_t *>(p.card + sec.sbase_off);
-            base_k = sec.payload_off + __ldg(sbase + stream_k);
-            base_v = sec.payload_off + __ldg(sbase + stream_v);
+            // entries beyond the card (a damaged table) must not wrap the sums around
+            const uint64_t sk = __ldg(sbase + stream_k), sv = __ldg(sbase + stream_v);
+            base_k = sk > total_bytes ? ~uint64_t(0) : sec.payload_off + sk;
+            base_v = sv > total_bytes ? ~uint64_t(0) : sec.payload_off + sv;
         }
         // ---- the item's tokens, a run of kAttendPerLane per lane: check the table entries, sort by width into the list
         const uint32_t tok0 = sub0 * kAttendRows;
         const int n_tok = (int)min((uint64_t)(kAttendRows * kAttendSteps), T - tok0);
         uint32_t ends[4];  // where each class ends in the list
-        const bool base_ok = base_k >= sec.payload_off && base_v >= sec.payload_off && ((base_k | base_v) & 15u) == 0u;
+        const bool base_ok = base_k >= sec.payload_off && base_v >= sec.payload_off && ((base_k | base_v) & 15u) == 0u &&
+                             base_k <= total_bytes && base_v <= total_bytes;
+        const uint64_t room_k = base_ok ? total_bytes - base_k : 0u, room_v = base_ok ? total_bytes - base_v : 0u;
         // A whole item of one width (every item of a uniform card): eight bit-widths per lane in one
         // word, all equal, and the two offsets at the item's ends a whole item's records apart.  The
         // records are then neighbours from the first to the last -- the offsets cannot but grow by
@@ -566,8 +570,7 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
             const bool same = w8.x == b0 * 0x01010101u && w8.y == w8.x;
             const uint32_t rec = record_bytes(kAttendD, (int)b0, META);
             one_width = __all_sync(0xffffffffu, same) && base_ok && rec != 0u && (o_first & 15u) == 0u && o_last >= o_first &&
-                        o_last - o_first == (uint32_t)n_tok * rec && base_k + (uint64_t)o_last <= total_bytes &&
-                        base_v + (uint64_t)o_last <= total_bytes;
+                        o_last - o_first == (uint32_t)n_tok * rec && (uint64_t)o_last <= room_k && (uint64_t)o_last <= room_v;
             try_one_width = one_width;
             if (one_width) {
                 const int cls = b0 == 2u ? 0 : (b0 == 4u ? 1 : (b0 == 8u ? 2 : 3));
@@ -598,7 +601,7 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
                         const uint32_t b = __ldg(bits_tab + j);
                         const uint32_t rec = record_bytes(kAttendD, (int)b, META);
                         const bool fine = base_ok && rec != 0u && o_next >= o && o_next - o == rec && (o & 15u) == 0u &&
-                                          base_k + (uint64_t)o_next <= total_bytes && base_v + (uint64_t)o_next <= total_bytes;
+                                          (uint64_t)o_next <= room_k && (uint64_t)o_next <= room_v;
                         bad |= !fine;
                         if (fine) {
                             my_cls[r] = b == 2u ? 0 : (b == 4u ? 1 : (b == 8u ? 2 : 3));

@@ -201,8 +201,13 @@ struct TableWalk {
         const uint64_t t0 = (uint64_t)c.tt * R;
         bits = p.card + sec.bits_off + seg * T + t0;
         offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off) + seg * (T + 1u) + t0;
-        if (bits_mode == 0) base = sec.payload_off + stream * stream_bytes;
-        else base = sec.payload_off + __ldg(reinterpret_cast<const uint64_t *>(p.card + sec.sbase_off) + stream);
+        if (bits_mode == 0) {
+            base = sec.payload_off + stream * stream_bytes;
+        } else {
+            // a table entry beyond the buffer (a damaged card) must not wrap the sum around
+            const uint64_t sb = __ldg(reinterpret_cast<const uint64_t *>(p.card + sec.sbase_off) + stream);
+            base = sb > p.card_bytes ? ~uint64_t(0) : sec.payload_off + sb;
+        }
     }
     __device__ __forceinline__ void next(WorkSource &ws, const PathParams &p, const Sections &sec, int bits_mode,
                                          uint64_t stream_bytes, int lane)
@@ -566,7 +571,9 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
     bad = __any_sync(0xffffffffu, bad);
     // with consistent records the span is rows * (at most 2*D) bytes, so it fits the stage
     const uint32_t span = off_end - off0;
-    bad |= (off0 & 15u) != 0u || t.base < sec.payload_off || (t.base & 15u) != 0u || t.base + (uint64_t)off_end > total_bytes;
+    // compared without forming base + off_end, which a crafted stream base could wrap around
+    bad |= (off0 & 15u) != 0u || t.base < sec.payload_off || (t.base & 15u) != 0u || t.base > total_bytes ||
+           (uint64_t)off_end > total_bytes - t.base;
     if (lane == 0) {
         sm.rows[stage] = bad ? 0 : rows;
         sm.uniform_bits[stage] = uniform ? b0 : 0u;

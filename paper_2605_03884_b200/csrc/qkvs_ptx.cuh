@@ -78,14 +78,14 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 }
 
 // Waits for the phase with the given parity.  Returns false if the phase did not complete within
-// kWaitLimitNs; the caller then records an error status and winds down.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+// limit_ns; the caller then records an error status and winds down.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long start = global_timer_ns();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - start > kWaitLimitNs) return false;
+        if (global_timer_ns() - start > limit_ns) return false;
     }
 }
 

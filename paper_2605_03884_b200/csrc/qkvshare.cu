@@ -389,6 +389,30 @@ __global__ void selftest_division_kernel(unsigned long long *mismatches)
 }
 
 // ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: a warp arms a barrier with a transaction count that no copy will
+// ever deliver, waits on it with the given limit, and reports the give-up exactly as the
+// pipelines do.  Nothing is in flight, so the kernel simply returns afterwards.
+__global__ void selftest_wait_kernel(unsigned long long limit_ns, int32_t *status, unsigned long long *waited_ns)
+{
+    __shared__ alignas(8) uint64_t bar;
+    const int lane = threadIdx.x & 31;
+    if (lane == 0) {
+        mbar_init(&bar, 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive_expect_tx(&bar, 16u);  // the phase now needs 16 bytes that never come
+    __syncwarp();
+    const unsigned long long t0 = global_timer_ns();
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(&bar, 0, limit_ns));
+    const unsigned long long t1 = global_timer_ns();
+    if (lane == 0) {
+        if (!ok) atomicMax(status, (int)QKVS_ERR_TIMEOUT);
+        if (waited_ns) *waited_ns = t1 - t0;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Host side
 
 static qkvs_status_t check_shape(const qkvs_layout_t *l)
@@ -414,6 +438,14 @@ static qkvs_status_t check_strides(const qkvs_layout_t *l, int64_t first_row)
     if (l->token_stride < l->head_dim || (l->token_stride & 7) || (l->head_stride & 7) || l->head_stride < 0)
         return QKVS_ERR_INVALID_ARG;
     if (first_row < 0) return QKVS_ERR_INVALID_ARG;
+    // the element offsets the kernels form (head * head_stride + row * token_stride + channel) must
+    // stay far inside 64 bits whatever the caller passes
+    constexpr int64_t kMaxElements = int64_t(1) << 48;
+    if (first_row > kMaxElements || l->token_stride > kMaxElements || l->head_stride > kMaxElements) return QKVS_ERR_INVALID_ARG;
+    long long last = 0, span = 0;
+    if (__builtin_mul_overflow((long long)(first_row + l->n_tokens), (long long)l->token_stride, &last) || last > kMaxElements ||
+        __builtin_mul_overflow((long long)l->n_kv_heads, (long long)l->head_stride, &span) || span > kMaxElements)
+        return QKVS_ERR_INVALID_ARG;
     if (l->n_tokens > 0 && (first_row + l->n_tokens - 1) * l->token_stride + l->head_dim > l->head_stride &&
         l->n_kv_heads > 1)
         return QKVS_ERR_INVALID_ARG;
@@ -803,6 +835,32 @@ qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t card_bytes, 
     return QKVS_OK;
 }
 
+qkvs_status_t qkvs_card_send(const void *card_dev, size_t card_bytes, int32_t src_device, void *dst_dev,
+                             size_t dst_capacity, int32_t dst_device, void *stream)
+{
+    if (!card_dev || !dst_dev || !aligned16(card_dev) || !aligned16(dst_dev)) return QKVS_ERR_INVALID_ARG;
+    if (src_device < 0 || dst_device < 0) return QKVS_ERR_INVALID_ARG;
+    if (card_bytes < (size_t)kHeaderBytes) return QKVS_ERR_BAD_CARD;
+    if (dst_capacity < card_bytes) return QKVS_ERR_BUFFER_TOO_SMALL;
+    int n_devices = 0, current = -1;
+    if (cudaGetDeviceCount(&n_devices) != cudaSuccess || cudaGetDevice(&current) != cudaSuccess) return QKVS_ERR_CUDA;
+    if (src_device >= n_devices || dst_device >= n_devices) return QKVS_ERR_INVALID_ARG;
+    if (current != src_device && current != dst_device) return QKVS_ERR_INVALID_ARG;
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    if (src_device == dst_device)
+        return cudaMemcpyAsync(dst_dev, card_dev, card_bytes, cudaMemcpyDeviceToDevice, cs) == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+    // a direct copy over NVLink needs peer access from the device that runs the copy to the other
+    const int other = current == src_device ? dst_device : src_device;
+    int can = 0;
+    if (cudaDeviceCanAccessPeer(&can, current, other) != cudaSuccess) return QKVS_ERR_CUDA;
+    if (can) {
+        const cudaError_t e = cudaDeviceEnablePeerAccess(other, 0);
+        if (e == cudaErrorPeerAccessAlreadyEnabled) (void)cudaGetLastError();  // on already: not an error
+        else if (e != cudaSuccess) return QKVS_ERR_CUDA;
+    }
+    return cudaMemcpyPeerAsync(dst_dev, dst_device, card_dev, src_device, card_bytes, cs) == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+}
+
 // Shape of the attention work: steps of 16 tokens, items of 16 steps, per (layer, KV head).
 static qkvs_status_t attend_shape(const qkvs_layout_t *layout, int32_t n_q_heads, AttendParams *p)
 {
@@ -932,6 +990,18 @@ qkvs_status_t qkvs_selftest_division(uint64_t *mismatches_dev, void *stream)
     cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(mismatches_dev, 0, 2 * sizeof(uint64_t), cs) != cudaSuccess) return QKVS_ERR_CUDA;
     selftest_division_kernel<<<148 * 8, 256, 0, cs>>>(reinterpret_cast<unsigned long long *>(mismatches_dev));
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+}
+
+qkvs_status_t qkvs_selftest_bounded_wait(uint32_t limit_us, int32_t *status_dev, uint64_t *waited_ns_dev, void *stream)
+{
+    if (!status_dev || (reinterpret_cast<uintptr_t>(status_dev) & 3u) || (reinterpret_cast<uintptr_t>(waited_ns_dev) & 7u))
+        return QKVS_ERR_INVALID_ARG;
+    if (limit_us == 0 || limit_us > 1000000u) return QKVS_ERR_INVALID_ARG;  // at most a second
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(status_dev, 0, sizeof(int32_t), cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    selftest_wait_kernel<<<1, 32, 0, cs>>>((unsigned long long)limit_us * 1000ull, status_dev,
+                                           reinterpret_cast<unsigned long long *>(waited_ns_dev));
     return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 

@@ -1,8 +1,9 @@
 """Seeded synthetic inputs for the CacheCard create / inject path.
 
 This module holds *only* input generation: FP16 KV caches with the shapes and value
-distributions of the benchmark configurations, and per-token bit-width vectors.  It contains
-none of the method's arithmetic (no quantisation, packing, offsets or sizes), so both the
+distributions of the benchmark configurations, per-token bit-width vectors drawn at random, and
+importance scores.  It contains none of the method's arithmetic (no quantisation, packing,
+offsets, sizes or rank rule), so both the
 CUDA path and the CPU oracle can be fed from it without sharing any code of the method.
 
 The synthetic caches stand in for real Llama-3.1-8B-Instruct KV caches (Section 5.1 of the
@@ -23,7 +24,7 @@ Seeds (fixed so every run sees the same bytes):
 from __future__ import annotations
 
 from dataclasses import dataclass, replace
-from typing import Iterator, Optional, Tuple
+from typing import Callable, Iterator, Optional, Tuple
 
 import numpy as np
 
@@ -113,30 +114,33 @@ def iid_bits(n_tokens: int, probs, seed: int) -> np.ndarray:
     return BIT_CHOICES[idx]
 
 
-def quantile_bits(n_tokens: int, seed: int) -> np.ndarray:
-    """Bit-widths from a synthetic per-token importance score (config 4).
-
-    score ~ LogNormal(0,1); tokens ranked by score descending (ties: lower index first);
-    top 5 % -> FP16, next 15 % -> 8 bit, next 40 % -> 4 bit, the rest -> 2 bit, with the cut
-    ranks rounded half-up from 0.05 T, 0.20 T and 0.60 T.
-    """
+def importance_scores(n_tokens: int, seed: int) -> np.ndarray:
+    """Synthetic per-token importance (config 4): LogNormal(0, 1), float32."""
     rng = np.random.default_rng(seed)
-    score = rng.lognormal(0.0, 1.0, size=n_tokens)
-    order = np.lexsort((np.arange(n_tokens), -score))
+    return rng.lognormal(0.0, 1.0, size=n_tokens).astype(np.float32)
+
+
+def quantile_counts(n_tokens: int) -> Tuple[int, int, int]:
+    """How many tokens the adaptive recipe keeps in FP16, at 8 bits and at 4 bits (the rest get
+    2 bits): top 5 %, next 15 %, next 40 %, with the cut ranks rounded half-up from 0.05 T, 0.20 T
+    and 0.60 T (410 / 1228 / 3277 of 8192)."""
     c16 = int(np.floor(0.05 * n_tokens + 0.5))
     c8 = int(np.floor(0.20 * n_tokens + 0.5))
     c4 = int(np.floor(0.60 * n_tokens + 0.5))
-    bits = np.empty(n_tokens, dtype=np.uint8)
-    bits[order[:c16]] = 16
-    bits[order[c16:c8]] = 8
-    bits[order[c8:c4]] = 4
-    bits[order[c4:]] = 2
-    return bits
+    return c16, c8 - c16, c4 - c8
 
 
-def bits_for(w: Workload, hop: int = 0, segment: int = 0) -> np.ndarray:
+RankRule = Callable[[np.ndarray, int, int, int], np.ndarray]
+
+
+def bits_for(w: Workload, hop: int = 0, segment: int = 0, rank_rule: Optional[RankRule] = None) -> np.ndarray:
     """Per-token bit-width vector (uint8, values in {2,4,8,16}; 16 means raw FP16).  `segment`
-    varies the draw for the per-(layer, head) mode; segment 0 is the whole-model vector."""
+    varies the draw for the per-(layer, head) mode; segment 0 is the whole-model vector.
+
+    The adaptive recipe ("quantile") only draws the importance scores here; turning scores into
+    bit-widths by rank is a step of the method, so the caller supplies it as
+    `rank_rule(scores, n_fp16, n_8bit, n_4bit) -> bits`: the library's entry point, the oracle's
+    function, or a test's own statement of the rule."""
     t = w.n_tokens
     shift = 7919 * segment
     if w.bits_recipe == "uniform4":
@@ -144,16 +148,20 @@ def bits_for(w: Workload, hop: int = 0, segment: int = 0) -> np.ndarray:
     if w.bits_recipe == "iid":
         return iid_bits(t, w.iid_probs, w.value_seed + 2 + shift)
     if w.bits_recipe == "quantile":
-        return quantile_bits(t, w.value_seed + 3 + shift)
+        if rank_rule is None:
+            raise ValueError("the adaptive recipe needs a rank_rule (scores, n_fp16, n_8bit, n_4bit) -> bits")
+        bits = np.asarray(rank_rule(importance_scores(t, w.value_seed + 3 + shift), *quantile_counts(t)), dtype=np.uint8)
+        assert bits.shape == (t,)
+        return bits
     if w.bits_recipe == "chain":
         return iid_bits(t, w.iid_probs, 1000 + w.number + 10 + hop + shift)
     raise ValueError(w.bits_recipe)
 
 
-def bits_per_head(w: Workload, hop: int = 0) -> np.ndarray:
+def bits_per_head(w: Workload, hop: int = 0, rank_rule: Optional[RankRule] = None) -> np.ndarray:
     """bits[n_layers * n_kv_heads][n_tokens], flattened: every (layer, head) segment draws the
     workload's recipe on its own (as a controller that scores tokens per head would)."""
-    return np.concatenate([bits_for(w, hop, seg) for seg in range(w.n_layers * w.n_kv_heads)])
+    return np.concatenate([bits_for(w, hop, seg, rank_rule) for seg in range(w.n_layers * w.n_kv_heads)])
 
 
 def random_fp16(shape, seed: int, scale: float = 1.0) -> np.ndarray:

@@ -1,5 +1,11 @@
 """Attention straight from the card: CUDA path against the oracle, through the C-ABI, on a B200.
 
+Two readings of "attention over a card" exist in the oracle: over the values the records stand
+for (code * scale + zero, unrounded -- the one the CUDA path is held to, asserted here) and over
+the FP16 cache injection would rebuild ("inject, then attend").  Every case prints the CUDA
+path's distance to both, in units of 2^-9 * max|V^| of the head, and the last test prints the
+largest of each; the distance to the second reading is reported, not asserted.
+
 Tolerance.  Both sides attend to the values the records stand for (code * scale + zero, not
 rounded to FP16).  The CUDA path rounds the softmax weights, times the scale, to FP16 (relative
 2^-11) before the tensor-core product with the codes, accumulates
@@ -16,6 +22,7 @@ import paper_2605_03884_b200 as q
 from paper_2605_03884_b200 import build as qbuild
 from paper_2605_03884_b200 import workloads as wl
 from gpu_utils import padded_cache
+from rank_rule import by_library_sort
 
 pytestmark = pytest.mark.gpu
 
@@ -39,12 +46,17 @@ def _gpu_attend(card_np, L, H, d, T, qh, scale=None, card_bytes=None):
     return status, out.cpu().numpy()
 
 
-def _check(Ks, Vs, bits, L, H, d, T, nq, mode=0, scale=None, qscale=1.0, seed=0):
+DISTANCES = {}   # case label -> (to the records' own values, to the injected FP16 cache), units of 2^-9 max|V^|
+
+
+def _check(Ks, Vs, bits, L, H, d, T, nq, mode=0, scale=None, qscale=1.0, seed=0, label=None):
     olay = oracle.make_layout(L, H, d, T, bits_mode=mode)
     st, card = oracle.card_create(olay, Ks, Vs, bits)
     assert st == oracle.OK
     qh = wl.random_fp16((L, nq, d), 900 + seed, scale=qscale)
     st, want = oracle.card_attend(card, olay, qh, softmax_scale=scale)
+    assert st == oracle.OK
+    st, want_injected = oracle.card_attend(card, olay, qh, softmax_scale=scale, injected=True)
     assert st == oracle.OK
     status, got = _gpu_attend(card, L, H, d, T, qh, scale)
     assert status == 0
@@ -52,13 +64,18 @@ def _check(Ks, Vs, bits, L, H, d, T, nq, mode=0, scale=None, qscale=1.0, seed=0)
     Kr, Vr = [np.zeros_like(k) for k in Ks], [np.zeros_like(v) for v in Vs]
     assert oracle.card_inject(card, olay, Kr, Vr) == oracle.OK
     per_kv = nq // H
-    worst = 0.0
+    worst = worst_injected = 0.0
     for l in range(L):
         for j in range(nq):
             vmax = float(np.abs(Vr[l][j // per_kv][:T, :d].astype(np.float64)).max()) if T else 0.0
             err = float(np.abs(got[l, j] - want[l, j]).max())
             assert err <= 2.0 ** -9 * vmax + 1e-6, (l, j, err, vmax)
             worst = max(worst, err / (vmax + 1e-30))
+            worst_injected = max(worst_injected, float(np.abs(got[l, j] - want_injected[l, j]).max()) / (vmax + 1e-30))
+    label = label or f"L{L} H{H} T{T} nq{nq} mode{mode} scale{scale} qscale{qscale} seed{seed}"
+    DISTANCES[label] = (worst * 2.0 ** 9, worst_injected * 2.0 ** 9)
+    print(f"attend distance [{label}]: to the records' values {worst * 2.0 ** 9:.3f}, "
+          f"to the injected FP16 cache {worst_injected * 2.0 ** 9:.3f} (units of 2^-9 max|V^|)")
     return worst
 
 
@@ -89,7 +106,7 @@ def test_sharp_and_flat_softmax():
     L, H, d, T, nq = 1, 2, 128, 900, 8
     Ks, Vs, _ = padded_cache(L, H, T, d, seed=330)
     bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), seed=331)
-    _check(Ks, Vs, bits, L, H, d, T, nq, scale=1.0, qscale=2.0, seed=1)    # a few tokens take all the weight
+    _check(Ks, Vs, bits, L, H, d, T, nq, scale=1.0, qscale=2.0, seed=1, label="sharp softmax")    # a few tokens take all the weight
     _check(Ks, Vs, bits, L, H, d, T, nq, scale=1e-4, seed=2)                # nearly the mean of the values
     _check(Ks, Vs, bits, L, H, d, T, nq, scale=0.0, seed=3)                 # exactly the mean
 
@@ -145,6 +162,34 @@ def test_damaged_cards_give_zeros_and_a_status():
     assert status == q.binding.ERR_BAD_CARD and np.all(got == 0.0)
 
 
+def test_damaged_stream_bases_give_zeros_and_a_status():
+    """Per-head mode with a stream-base entry that is misaligned, beyond the card or close to 2^64
+    (base + length would wrap around); the card lies inside a larger device tensor."""
+    import torch
+    L, H, d, T, nq = 1, 2, 128, 300, 4
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=360)
+    bits = np.concatenate([wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 361 + s) for s in range(L * H)])
+    olay = oracle.make_layout(L, H, d, T, bits_mode=1)
+    _, card = oracle.card_create(olay, Ks, Vs, bits)
+    hd = oracle.parse_header(card)
+    qh = wl.random_fp16((L, nq, d), 362)
+    lay = q.make_layout(L, H, d, T)
+    margin = 1 << 20
+    for victim in (1, 2):                       # a K stream, a V stream
+        for value in (8, card.size + 4096, 2 ** 64 - 16 - hd["payload_off"], 2 ** 64 - 4096):
+            bad = card.copy()
+            bad[hd["sbase_off"] + 8 * victim:hd["sbase_off"] + 8 * (victim + 1)] = np.frombuffer(int(value).to_bytes(8, "little"), np.uint8)
+            assert oracle.card_attend(bad, olay, qh)[0] == oracle.BAD_CARD
+            big = torch.full((2 * margin + card.size,), 0xA5, dtype=torch.uint8, device="cuda")
+            big[margin:margin + card.size] = torch.from_numpy(bad).cuda()
+            out = torch.full(qh.shape, 7.0, dtype=torch.float32, device="cuda")
+            scratch = torch.full((q.attend_scratch_size(lay, nq),), 0x5A, dtype=torch.uint8, device="cuda")
+            q.card_attend(big[margin:margin + card.size], lay, torch.from_numpy(qh).cuda(), out, scratch, card_bytes=card.size)
+            torch.cuda.synchronize()
+            assert int(scratch[:4].view(torch.int32).item()) == q.binding.ERR_BAD_CARD
+            assert bool((out == 0).all())
+
+
 @pytest.mark.parametrize("number", [3, 4])
 def test_full_size_llama_8k(number):
     """The benchmark's size and launch configuration: 32 layers, 8 KV heads, 32 query heads, 8192 tokens."""
@@ -153,7 +198,8 @@ def test_full_size_llama_8k(number):
     for _, k, v in wl.kv_layers(w):
         Ks.append(k)
         Vs.append(v)
-    worst = _check(Ks, Vs, wl.bits_for(w), w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens, 32, seed=number)
+    worst = _check(Ks, Vs, wl.bits_for(w, rank_rule=by_library_sort), w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens, 32, seed=number,
+                   label=f"full size config {number}")
     assert worst <= 2.0 ** -9
 
 
@@ -166,5 +212,20 @@ def test_mid_sized_caches_all_layers(T):
     for _, k, v in wl.kv_layers(w):
         Ks.append(k)
         Vs.append(v)
-    worst = _check(Ks, Vs, wl.bits_for(w), w.n_layers, w.n_kv_heads, w.head_dim, T, 32, seed=T)
+    worst = _check(Ks, Vs, wl.bits_for(w, rank_rule=by_library_sort), w.n_layers, w.n_kv_heads, w.head_dim, T, 32, seed=T)
     assert worst <= 2.0 ** -9
+
+
+def test_zz_report_distances_to_both_readings():
+    """Prints the largest distance of the CUDA path to each of the oracle's two readings over the
+    cases that ran before it (run with -s or -rP to see the per-case lines)."""
+    if not DISTANCES:
+        pytest.skip("no attention case ran before this one")
+    own = max(v[0] for v in DISTANCES.values())
+    inj_label, inj = max(((k, v[1]) for k, v in DISTANCES.items()), key=lambda kv: kv[1])
+    print(f"attend distances over {len(DISTANCES)} cases: to the records' values at most {own:.3f}, "
+          f"to the injected FP16 cache at most {inj:.3f} ({inj_label}); units of 2^-9 max|V^|")
+    for k in ("sharp softmax", "full size config 3", "full size config 4"):
+        if k in DISTANCES:
+            print(f"  {k}: {DISTANCES[k][0]:.3f} / {DISTANCES[k][1]:.3f}")
+    assert own <= 1.0 + 1e-3

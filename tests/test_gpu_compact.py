@@ -14,6 +14,7 @@ import paper_2605_03884_b200 as q
 from paper_2605_03884_b200 import build as qbuild
 from paper_2605_03884_b200 import workloads as wl
 from golden_io import read_fixture
+from rank_rule import by_library_sort
 from gpu_utils import PAD, POISON, gpu_create, gpu_inject, max_ulp, padded_cache, to_cuda
 
 pytestmark = pytest.mark.gpu
@@ -242,7 +243,7 @@ def test_llama_8k_adaptive_full_size():
     for _, k, v in wl.kv_layers(w):
         Ks.append(k)
         Vs.append(v)
-    bits = wl.bits_for(w)
+    bits = wl.bits_for(w, rank_rule=by_library_sort)
     L, H, d, T = w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens
     st_o, want = oracle.card_create(_olay(L, H, d, T), Ks, Vs, bits)
     assert st_o == oracle.OK

@@ -12,6 +12,7 @@ import paper_2605_03884_b200 as q
 from paper_2605_03884_b200 import build as qbuild
 from paper_2605_03884_b200 import workloads as wl
 from gpu_utils import PAD, POISON, gpu_create, gpu_inject, max_ulp, padded_cache, to_cuda
+from rank_rule import by_library_sort
 
 pytestmark = pytest.mark.gpu
 
@@ -318,6 +319,109 @@ def test_inject_refuses_damaged_cards_without_writing():
     assert st == q.binding.ERR_BAD_CARD and np.all(Kg[0] == -3.0)
 
 
+def test_inject_refuses_damaged_stream_bases():
+    """Per-head mode: a stream-base entry that is misaligned, beyond the card, or so close to 2^64
+    that base + length would wrap around.  The card sits in the interior of a larger device tensor,
+    so every address a wrong sum could form still lies in mapped memory.  The damaged stream's rows
+    stay untouched, the others are injected, and the status word says BAD_CARD."""
+    import torch
+    L, H, d, T = 1, 2, 128, 100
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=163)
+    bits = np.concatenate([wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 164 + s) for s in range(L * H)])
+    _, card = oracle.card_create(_olay(L, H, d, T, mode=1), Ks, Vs, bits)
+    hd = oracle.parse_header(card)
+    Kw, Vw = [np.zeros((H, T, d), np.float16)], [np.zeros((H, T, d), np.float16)]
+    assert oracle.card_inject(card, _olay(L, H, d, T), Kw, Vw) == oracle.OK
+    margin = 1 << 20
+    victim = 2                                  # stream (layer 0, V, head 0)
+    for value in (8, card.size, card.size + 4096, 2 ** 64 - 16 - hd["payload_off"], 2 ** 64 - 4096, 2 ** 63):
+        bad = card.copy()
+        bad[hd["sbase_off"] + 8 * victim:hd["sbase_off"] + 8 * (victim + 1)] = np.frombuffer(int(value).to_bytes(8, "little"), np.uint8)
+        assert oracle.card_inject(bad, _olay(L, H, d, T), [k.copy() for k in Kw], [v.copy() for v in Vw]) == oracle.BAD_CARD
+        big = torch.full((2 * margin + card.size,), POISON, dtype=torch.uint8, device="cuda")
+        big[margin:margin + card.size] = torch.from_numpy(bad).cuda()
+        inner = big[margin:margin + card.size]
+        Kd = to_cuda([np.full((H, T, d), -3.0, np.float16)])
+        Vd = to_cuda([np.full((H, T, d), -5.0, np.float16)])
+        ws = q.new_workspace()
+        q.card_inject(inner, _glay(L, H, d, T), Kd, Vd, card_bytes=card.size, workspace=ws)
+        torch.cuda.synchronize()
+        assert int(ws[0].item()) == q.binding.ERR_BAD_CARD
+        Kg, Vg = Kd[0].cpu().numpy(), Vd[0].cpu().numpy()
+        assert np.all(Vg[0] == -5.0), "rows of the damaged stream were written"
+        assert np.array_equal(Kg.view(np.uint16), Kw[0].view(np.uint16))
+        assert np.array_equal(Vg[1].view(np.uint16), Vw[0][1].view(np.uint16))
+
+
+def test_worked_examples_on_the_gpu():
+    """The stored hand-worked groups (exact ties at 4, 2 and 8 bits; the group with an inexact
+    scale at all three widths) as one-token cards: scale, zero and packed codes as stored."""
+    from golden_io import read_fixture
+    cases = []
+    for name in ("worked_example_a_4bit.txt", "worked_example_b_2bit.txt", "worked_example_c_8bit.txt"):
+        fx = read_fixture(name)
+        x = np.array([float(v) for v in fx["x"][0]], dtype=np.float16)
+        cases.append((int(fx["bits"][0][0]), x, int(fx["scale_bits"][0][0], 16), int(fx["zero_bits"][0][0], 16),
+                      [int(v, 16) for v in fx["packed_hex"][0]], [float(v) for v in fx["dequant"][0]]))
+    fx = read_fixture("worked_example_f_inexact.txt")
+    xf = np.array([int(v) for v in fx["x_bits"][0]], dtype=np.uint16).view(np.float16)
+    for (b, scale_hex, _), packed in zip(fx["case"], fx["packed_hex"]):
+        cases.append((int(b), xf, int(scale_hex, 16), int(fx["zero_bits"][0][0], 16), [int(v, 16) for v in packed], None))
+    for b, x, scale_bits, zero_bits, packed, dequant in cases:
+        K = np.tile(x, 4).reshape(1, 1, 128)
+        st, hdr, whole, _ = gpu_create(q, _glay(1, 1, 128, 1), [K], [K.copy()], np.array([b], np.uint8))
+        assert st == q.binding.OK
+        rec = whole[hdr.payload_off:hdr.payload_off + q.record_bytes(128, b)]
+        assert rec[:32].view("<u4").tolist() == [scale_bits, zero_bits] * 4
+        assert rec[32:].tolist() == packed * 4
+        stat, Kg, _ = gpu_inject(q, whole[:hdr.total_bytes], _glay(1, 1, 128, 1), [np.zeros_like(K)], [np.zeros_like(K)])
+        assert stat == 0
+        if dequant is not None:
+            assert Kg[0].astype(np.float64).reshape(-1).tolist() == dequant * 4
+
+
+def test_card_sent_to_a_buffer_of_its_own_injects_identically():
+    """qkvs_card_send on the one GPU at hand: the copy holds the same bytes, and injecting from it
+    (a different address, other bytes around it) rebuilds the same cache as the oracle.  Unknown
+    devices and a device that is neither end of the copy are refused."""
+    import torch
+    L, H, d, T = 2, 2, 128, 333
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=81)
+    bits = wl.iid_bits(T, (0.3, 0.3, 0.2, 0.2), 82)
+    want = _check_card(Ks, Vs, bits, L, H, d, T)
+    src = torch.from_numpy(want).cuda()
+    dst = torch.full((want.size + 4096,), POISON, dtype=torch.uint8, device="cuda")
+    q.card_send(src, dst[2048:], card_bytes=want.size)
+    torch.cuda.synchronize()
+    got = dst.cpu().numpy()
+    assert np.array_equal(got[2048:2048 + want.size], want)
+    assert np.all(got[:2048] == POISON) and np.all(got[2048 + want.size:] == POISON)
+    assert _check_inject(got[2048:2048 + want.size], L, H, d, T) == 0
+    n = torch.cuda.device_count()
+    lib = q.load_library()
+    st = lib.qkvs_card_send(src.data_ptr(), want.size, 0, dst.data_ptr(), dst.numel(), n, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = q.card_send(src, dst[:want.size - 16], card_bytes=want.size, check=False)
+    assert st == q.binding.ERR_BUFFER_TOO_SMALL
+
+
+def test_a_wait_that_nothing_completes_gives_up_and_reports_it():
+    """The kernels' only waits are bounded; this runs one on a barrier that never completes, with a
+    limit of five milliseconds: the kernel returns, the status word says TIMEOUT, the wait lasted
+    about as long as asked, and the path works afterwards."""
+    import torch
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    q.selftest_bounded_wait(5000, status, waited)
+    torch.cuda.synchronize()
+    assert int(status.item()) == q.binding.ERR_TIMEOUT
+    assert 5_000_000 <= int(waited.item()) < 500_000_000
+    L, H, d, T = 1, 2, 128, 50
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=71)
+    card = _check_card(Ks, Vs, np.full(T, 4, np.uint8), L, H, d, T)
+    assert _check_inject(card, L, H, d, T) == 0
+
+
 # ----------------------------------------------------------------------------- full-size configs
 
 def _full_config(number):
@@ -381,7 +485,7 @@ def test_config3_llama_8k_uniform4_full():
 
 def test_config4_llama_8k_adaptive_full():
     w, Ks, Vs = _full_config(4)
-    bits = wl.bits_for(w)
+    bits = wl.bits_for(w, rank_rule=by_library_sort)
     assert abs(float(bits.astype(np.float64).mean()) - 4.4) < 0.01
     worst, _, _ = _full_parity(w, Ks, Vs, bits)
     assert worst == 0

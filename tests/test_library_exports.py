@@ -109,3 +109,24 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     st = lib.qkvs_card_create(C.byref(lay), ptrs, ptrs, C.c_void_p(256), None, C.c_void_p(256), 1 << 20,
                               C.c_void_p(264), None)
     assert st == q.binding.ERR_INVALID_ARG
+    # row and stride arithmetic that would not fit 64 bits is refused, not wrapped
+    st = lib.qkvs_card_inject(C.c_void_p(256), 4096, C.byref(lay), ptrs, ptrs, 2 ** 62, None, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    huge = q.make_layout(1, 4, 64, 4, head_stride=2 ** 61, token_stride=64)
+    st = lib.qkvs_card_inject(C.c_void_p(256), 4096, C.byref(huge), ptrs, ptrs, 0, None, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = lib.qkvs_selftest_bounded_wait(0, C.c_void_p(256), None, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = lib.qkvs_selftest_bounded_wait(2_000_000, C.c_void_p(256), None, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    # handing a card to another GPU: everything knowable without a device is checked first
+    st = lib.qkvs_card_send(None, 4096, 0, C.c_void_p(256), 4096, 0, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = lib.qkvs_card_send(C.c_void_p(256), 4096, 0, C.c_void_p(264), 4096, 0, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = lib.qkvs_card_send(C.c_void_p(256), 4096, -1, C.c_void_p(512), 4096, 0, None)
+    assert st == q.binding.ERR_INVALID_ARG
+    st = lib.qkvs_card_send(C.c_void_p(256), 100, 0, C.c_void_p(512), 4096, 0, None)
+    assert st == q.binding.ERR_BAD_CARD
+    st = lib.qkvs_card_send(C.c_void_p(256), 4096, 0, C.c_void_p(512), 4095, 0, None)
+    assert st == q.binding.ERR_BUFFER_TOO_SMALL

@@ -139,6 +139,43 @@ def test_quantised_card_is_within_fp16_rounding_of_library_attention_on_the_inje
     assert np.abs(o - ref).max() > 0          # and it is not the rounded cache that is attended to
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_injected_reading_is_library_attention_on_the_injected_cache(mode):
+    """The second reading -- inject, then attend -- equals numpy softmax attention over exactly
+    the FP16 arrays orc_card_inject writes, to double-precision rounding."""
+    L, H, d, T, nq = 2, 3, 64, 150, 6
+    Ks, Vs = _cache(L, H, T, d, 10)
+    if mode == 0:
+        bits = wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 11)
+    else:
+        bits = np.concatenate([wl.iid_bits(T, (0.4, 0.4, 0.15, 0.05), 20 + s) for s in range(L * H)])
+    lay, card = _card(Ks, Vs, bits, L, H, d, T, mode)
+    Kr, Vr = [np.zeros_like(k) for k in Ks], [np.zeros_like(v) for v in Vs]
+    assert oracle.card_inject(card, lay, Kr, Vr) == oracle.OK
+    q = wl.random_fp16((L, nq, d), 12)
+    for scale in (0.3, 1.0 / np.sqrt(d), 2.0):
+        st, o = oracle.card_attend(card, lay, q, softmax_scale=scale, injected=True)
+        assert st == oracle.OK
+        np.testing.assert_allclose(o, _reference_attention(Kr, Vr, q, nq // H, scale), rtol=1e-12, atol=1e-14)
+
+
+def test_the_two_readings_coincide_on_fp16_tokens_and_differ_on_quantised_ones():
+    L, H, d, T, nq = 1, 2, 128, 90, 4
+    Ks, Vs = _cache(L, H, T, d, 15)
+    q = wl.random_fp16((L, nq, d), 16)
+    lay, card = _card(Ks, Vs, np.full(T, 16, np.uint8), L, H, d, T)
+    a = oracle.card_attend(card, lay, q)[1]
+    b = oracle.card_attend(card, lay, q, injected=True)[1]
+    assert np.array_equal(a, b)
+    lay, card = _card(Ks, Vs, np.full(T, 4, np.uint8), L, H, d, T)
+    a = oracle.card_attend(card, lay, q)[1]
+    b = oracle.card_attend(card, lay, q, injected=True)[1]
+    Kr, Vr = [np.zeros_like(k) for k in Ks], [np.zeros_like(v) for v in Vs]
+    assert oracle.card_inject(card, lay, Kr, Vr) == oracle.OK
+    gap = np.abs(a - b).max(axis=2)
+    assert gap.max() > 0 and np.all(gap <= _rounding_bound(Kr, Vr, q, nq // H, 1.0 / np.sqrt(d)))
+
+
 def test_one_dominant_key_selects_its_value_row():
     """K rows are +-e_0 * 8 except token 17 = +e_0 * 64: with q = 32 e_0 the softmax weight of
     every other token is below exp(-64*32*... ) ~ 0, so the output is V[17] to double precision."""

@@ -6,6 +6,7 @@ import pytest
 
 import oracle
 from golden_io import read_fixture
+from rank_rule import by_library_sort
 from paper_2605_03884_b200 import workloads as wl
 
 
@@ -53,16 +54,20 @@ def test_equal_scores_favour_the_lower_index():
     assert st == oracle.OK and bits.tolist() == [16, 16, 8, 8, 8, 4, 2, 2, 2, 2]
 
 
-def test_matches_the_library_sort_of_the_workload_generator():
-    """Same rule as workloads.quantile_bits (numpy lexsort), on scores that are exact in float32."""
+def test_matches_the_library_sort():
+    """The same rule stated with numpy's lexsort (score descending, index ascending), on random
+    scores, on scores with many ties, and on the adaptive workload's own scores."""
     T = 4096
-    scores = np.random.default_rng(77).lognormal(0.0, 1.0, size=T).astype(np.float32)
-    order = np.lexsort((np.arange(T), -scores.astype(np.float64)))
     n16, n8, n4 = _cuts(T)
-    want = np.empty(T, np.uint8)
-    want[order[:n16]] = 16; want[order[n16:n16 + n8]] = 8; want[order[n16 + n8:n16 + n8 + n4]] = 4; want[order[n16 + n8 + n4:]] = 2
-    st, bits = oracle.bits_from_scores(scores, n16, n8, n4)
-    assert st == oracle.OK and np.array_equal(bits, want)
+    for scores in (np.random.default_rng(77).lognormal(0.0, 1.0, size=T).astype(np.float32),
+                   np.random.default_rng(78).integers(0, 9, size=T).astype(np.float32),
+                   wl.importance_scores(T, 1007)):
+        st, bits = oracle.bits_from_scores(scores, n16, n8, n4)
+        assert st == oracle.OK and np.array_equal(bits, by_library_sort(scores, n16, n8, n4))
+    w = wl.WORKLOADS[4]
+    assert wl.quantile_counts(w.n_tokens) == (410, 1228, 3277)
+    from_oracle = wl.bits_for(w, rank_rule=lambda s, a, b, c: oracle.bits_from_scores(s, a, b, c)[1])
+    assert np.array_equal(from_oracle, wl.bits_for(w, rank_rule=by_library_sort))
 
 
 def test_bad_counts_are_rejected():

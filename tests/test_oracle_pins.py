@@ -11,6 +11,7 @@ import pytest
 
 import oracle
 from golden_io import read_fixture
+from rank_rule import by_library_sort
 from paper_2605_03884_b200 import workloads as wl
 
 
@@ -96,7 +97,7 @@ def test_card_size_closed_form_fixture():
 
 def test_quantile_bits_counts_match_fixture():
     """The 8K adaptive recipe gives the 410 / 1228 / 3277 / 3277 split the size fixture assumes."""
-    bits = wl.bits_for(wl.WORKLOADS[4])
+    bits = wl.bits_for(wl.WORKLOADS[4], rank_rule=by_library_sort)
     assert [int((bits == b).sum()) for b in (16, 8, 4, 2)] == [410, 1228, 3277, 3277]
 
 
@@ -168,6 +169,36 @@ def test_worked_examples(name):
     meta = rec[:16].view("<u4")
     assert meta.tolist() == [int(fx["scale_bits"][0][0], 16), int(fx["zero_bits"][0][0], 16)] * 2
     assert rec[16:].tolist() == [int(v, 16) for v in fx["packed_hex"][0]] * 2
+
+
+def test_worked_example_with_an_inexact_scale():
+    """A group whose range / qmax is not a binary32 value, at 4, 2 and 8 bits: the stored figures
+    (worked in rationals, see the fixture's header) against the oracle, and against a fresh
+    recomputation in exact rational arithmetic here, so that the fixture itself is checked."""
+    fx = read_fixture("worked_example_f_inexact.txt")
+    x = np.array([int(v) for v in fx["x_bits"][0]], dtype=np.uint16)
+    xf = [_frac16(v) for v in x.view(np.float16)]
+    mn, mx = min(xf), max(xf)
+    assert mx - mn == Fraction(4097, 1024) and xf.index(mn) == 20 and xf.index(mx) == 7
+    for (b, scale_hex, inv_hex), codes, packed in zip(fx["case"], fx["codes"], fx["packed_hex"]):
+        b, qmax = int(b), (1 << int(b)) - 1
+        want_codes = [int(v) for v in codes]
+        sc, inv = _rn32((mx - mn) / qmax), _rn32(Fraction(qmax) / (mx - mn))
+        assert _f32_bits(np.float32(float(sc))) == int(scale_hex, 16)
+        assert _f32_bits(np.float32(float(inv))) == int(inv_hex, 16)
+        for v, c in zip(xf, want_codes):
+            u = _rn32(_rn32(v - mn) * inv)
+            fl = u.numerator // u.denominator
+            rem = u - fl
+            assert c == min(fl + (1 if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2) else 0), qmax)
+        bitstring = sum(c << (i * b) for i, c in enumerate(want_codes))
+        assert list(bitstring.to_bytes(4 * b, "little")) == [int(v, 16) for v in packed]
+        scale, zero, q = oracle.quantize_group(x, b)
+        assert _f32_bits(scale) == int(scale_hex, 16) and _f32_bits(zero) == int(fx["zero_bits"][0][0], 16)
+        assert q.tolist() == want_codes
+        assert oracle.pack_codes(q, b).tolist() == [int(v, 16) for v in packed]
+        deq = oracle.dequantize_group(q, scale, zero).astype(np.float64)
+        assert np.abs(deq - np.array([float(v) for v in xf])).max() <= float(sc) / 2 + 2.0 ** -11 * 2.5
 
 
 def test_pack_order_matches_little_endian_bitstream():
@@ -490,6 +521,26 @@ def test_inject_rejects_damaged_cards():
         assert oracle.card_inject(bad, dl, Ko, Vo) == oracle.BAD_CARD
     assert oracle.card_inject(card, dl, Ko, Vo, card_bytes=card.size - 1) == oracle.BAD_CARD
     assert oracle.card_inject(card, oracle.make_layout(L, H + 1, d, T), Ko, Vo) == oracle.BAD_CARD
+
+
+def test_inject_rejects_damaged_stream_bases():
+    """Per-head mode: a stream-base entry that is misaligned, points beyond the card, or sits so
+    close to 2^64 that base + length wraps around to a small number, is refused."""
+    L, H, T, d = 1, 2, 16, 64
+    Ks, Vs, _ = _cache(L, H, T, d, 168)
+    lay = oracle.make_layout(L, H, d, T, bits_mode=1)
+    bits = np.concatenate([wl.iid_bits(T, (0.25, 0.25, 0.25, 0.25), 169 + s) for s in range(L * H)])
+    st, card = oracle.card_create(lay, Ks, Vs, bits)
+    assert st == oracle.OK
+    hd = oracle.parse_header(card)
+    Ko, Vo, _ = _cache(L, H, T, d, 170)
+    dl = oracle.make_layout(L, H, d, T)
+    assert oracle.card_inject(card, dl, Ko, Vo) == oracle.OK
+    for value in (8, card.size, 2 ** 64 - 16 - hd["payload_off"], 2 ** 64 - 256, 2 ** 63):
+        bad = card.copy()
+        bad[hd["sbase_off"] + 8 * 2:hd["sbase_off"] + 8 * 3] = np.frombuffer(int(value).to_bytes(8, "little"), np.uint8)
+        assert oracle.card_inject(bad, dl, Ko, Vo) == oracle.BAD_CARD
+        assert oracle.card_attend(bad, oracle.make_layout(L, H, d, T), np.zeros((L, H, d), np.float16))[0] == oracle.BAD_CARD
 
 
 def test_create_reports_bad_bits_and_short_buffer():

@@ -73,6 +73,16 @@ def test_calls_in_a_row_match_the_ordinary_entry_point():
     assert _inject_both_ways(lay, card, L, H, d, T) <= MAX_ULP
 
 
+def test_a_call_of_several_launches_uses_the_higher_counters():
+    """More than 64 layers make more than one kernel launch per call, each with a counter of its
+    own further up the array; run after a large call, so that those words start out non-zero
+    only if a launch left them so, and twice, so that the second run meets the first one's counts."""
+    L, H, d, T = 130, 1, 64, 300
+    lay, card = _make_card(L, H, d, T, seed=503)
+    assert _inject_both_ways(lay, card, L, H, d, T) <= MAX_ULP
+    assert _inject_both_ways(lay, card, L, H, d, T) <= MAX_ULP
+
+
 def test_more_layers_than_the_array_has_counters_for_is_refused():
     import torch
     L = q.binding.NOALLOC_MAX_LAYERS + 1
