@@ -169,10 +169,42 @@ QKVS_API qkvs_status_t qkvs_card_prefix_size(const qkvs_layout_t *layout, size_t
  *   scores_dev   device float32 [n_segments][n_tokens], finite values
  *   bits_dev     device uint8  [n_segments][n_tokens]: ready to be passed to qkvs_card_create
  *                (n_segments = 1 for bits_mode 0, n_layers * n_kv_heads for bits_mode 1)
- * The result is exact (integer ranks).  n_tokens up to 2^20.  Asynchronous on `stream`. */
+ * The result is exact (integer ranks).  n_tokens up to 2^20.  Asynchronous on `stream`.  One CTA per
+ * segment finds the scores at the three cuts by selection (a byte of the key per pass), equal
+ * scores are told apart by a prefix count in index order; nothing is sorted. */
 QKVS_API qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_segments,
                                     int32_t n_tokens, int32_t n_fp16, int32_t n_8bit,
                                     int32_t n_4bit, uint8_t *bits_dev, void *stream);
+
+/* Bit-widths under a byte budget (Section 3.3: minimise sum_t eps(t, b(t)) * S(t) subject to
+ * sum_t b(t) * d <= M).  The paper prints the objective and no solver; this is the greedy solution
+ * of that knapsack by worth per byte, stated so that the result is unique:
+ *   - every token starts at 2 bits; raising a token one rung up the ladder 2 -> 4 -> 8 -> 16 is an
+ *     upgrade i = 0, 1, 2 whose cost is the difference of the two record sizes (metadata included)
+ *     and whose worth per byte is  key = fl32(S(t) * upgrade_weight[i]);
+ *   - all 3 * n_tokens upgrades are ordered by key, larger first, equal keys by lower rung, then by
+ *     lower token index (with non-negative scores and non-increasing weights a token's own upgrades
+ *     come in rung order);
+ *   - upgrades are granted in that order while their cost fits into what the budget leaves after
+ *     2 bits for everybody; the first one that does not fit ends the procedure.
+ *   scores_dev      device float32 [n_segments][n_tokens], finite and non-negative
+ *   head_dim, meta_bytes   fix the record sizes (as in qkvs_record_bytes)
+ *   budget_bytes    bound on the bytes of ONE stream: sum_t record(b(t)) <= budget_bytes
+ *   upgrade_weight  host array of three positive, non-increasing floats, or NULL for 2^-9, 2^-14,
+ *                   2^-23 -- the powers of two next to what a quantisation-noise model
+ *                   eps(b) = 4^-b gives per byte at head_dim 128
+ *   bits_dev        device uint8 [n_segments][n_tokens]
+ *   offsets_dev     optional device uint32 [n_segments][n_tokens + 1]: the exclusive prefix sum of
+ *                   the record sizes the bit-widths imply, i.e. the offset table of a card, from
+ *                   the same launch
+ *   status_dev      optional device int32, cleared by the call; raised to INVALID_ARG by a negative
+ *                   or non-finite score (every token of that segment then gets 2 bits)
+ * Errors on the host: INVALID_ARG, UNSUPPORTED_SHAPE, BUFFER_TOO_SMALL (the budget does not hold
+ * 2 bits per token), CUDA.  Exact; n_tokens up to 2^20; asynchronous on `stream`. */
+QKVS_API qkvs_status_t qkvs_bits_from_scores_budget(const float *scores_dev, int32_t n_segments, int32_t n_tokens,
+                                                    int32_t head_dim, int32_t meta_bytes, uint64_t budget_bytes,
+                                                    const float *upgrade_weight, uint8_t *bits_dev,
+                                                    uint32_t *offsets_dev, int32_t *status_dev, void *stream);
 
 /* The combined importance score of Section 3.3, S(t) = alpha * I(t) + (1 - alpha) * T(t): local
  * importance I and transferability T weighed by alpha in [0, 1], the quantity the bit-widths are

@@ -85,6 +85,8 @@ def lib():
         l.orc_card_inject.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_void_p, C.c_void_p, C.c_int64]
         l.orc_bits_from_scores.restype = C.c_int
         l.orc_bits_from_scores.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]
+        l.orc_bits_from_scores_budget.restype = C.c_int
+        l.orc_bits_from_scores_budget.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_uint64, C.c_void_p, C.c_void_p]
         l.orc_combine_scores.restype = C.c_int
         l.orc_combine_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int64, C.c_void_p]
         l.orc_card_attend.restype = C.c_int
@@ -288,6 +290,21 @@ def bits_from_scores(scores: np.ndarray, n_fp16: int, n_8bit: int, n_4bit: int) 
     scores = np.ascontiguousarray(scores, dtype=np.float32)
     bits = np.zeros(scores.size, dtype=np.uint8)
     st = lib().orc_bits_from_scores(_ptr(scores), scores.size, n_fp16, n_8bit, n_4bit, _ptr(bits))
+    return st, bits
+
+
+DEFAULT_UPGRADE_WEIGHTS = (2.0 ** -9, 2.0 ** -14, 2.0 ** -23)
+
+
+def bits_from_scores_budget(scores: np.ndarray, head_dim: int, budget_bytes: int, weights=DEFAULT_UPGRADE_WEIGHTS,
+                            meta_bytes: int = 8) -> Tuple[int, np.ndarray]:
+    """Per-token bit-widths from float32 scores [T] under a byte budget per stream (see
+    orc_bits_from_scores_budget)."""
+    scores = np.ascontiguousarray(scores, dtype=np.float32)
+    w = np.ascontiguousarray(weights, dtype=np.float32)
+    assert w.size == 3
+    bits = np.zeros(scores.size, dtype=np.uint8)
+    st = lib().orc_bits_from_scores_budget(_ptr(scores), scores.size, head_dim, meta_bytes, int(budget_bytes), _ptr(w), _ptr(bits))
     return st, bits
 
 

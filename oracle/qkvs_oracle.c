@@ -832,6 +832,69 @@ int orc_bits_from_scores(const float *scores, int64_t n_tokens, int64_t n_fp16, 
     return ORC_OK;
 }
 
+/* Bit-widths under a byte budget (Section 3.3: minimise sum_t eps(t, b(t)) * S(t) subject to
+ * sum_t b(t) * d <= M; the paper prints the objective and no solver).  The reading taken here is
+ * the greedy solution of that knapsack by worth per byte, stated so that the result is unique:
+ *   - every token starts at 2 bits; raising a token one rung up the ladder 2 -> 4 -> 8 -> 16 is an
+ *     *upgrade* i = 0, 1, 2 with a cost in bytes, cost_i = rec(next rung) - rec(rung) (record sizes,
+ *     metadata included), and a worth per byte  key = fl32(S(t) * weight_i), where weight_i > 0 says
+ *     how much error an upgrade of that rung removes per byte (weight_0 >= weight_1 >= weight_2:
+ *     the first bits buy the most);
+ *   - all 3 T upgrades are put in one order: larger key first, equal keys by lower rung, then by
+ *     lower token index; with non-negative scores a token's own upgrades appear in rung order;
+ *   - upgrades are granted in that order while their cost still fits into what the budget leaves
+ *     after 2 bits for everybody; the first one that does not fit ends the procedure.
+ * budget_bytes bounds the bytes of one stream: sum_t rec(b(t)) <= budget_bytes.  Scores must be
+ * finite and non-negative (a zero of either sign counts as zero).  Returns ORC_BUFFER_TOO_SMALL if
+ * the budget does not even hold 2 bits per token. */
+typedef struct { float key; int32_t rung; int64_t index; } orc_upgrade;
+
+static int upgrade_before(const void *a, const void *b)
+{
+    const orc_upgrade *x = (const orc_upgrade *)a, *y = (const orc_upgrade *)b;
+    if (x->key > y->key) return -1;
+    if (x->key < y->key) return 1;
+    if (x->rung != y->rung) return x->rung < y->rung ? -1 : 1;
+    return x->index < y->index ? -1 : (x->index > y->index ? 1 : 0);
+}
+
+int orc_bits_from_scores_budget(const float *scores, int64_t n_tokens, int head_dim, int meta,
+                                uint64_t budget_bytes, const float *weight, uint8_t *bits)
+{
+    static const int ladder[4] = {2, 4, 8, 16};
+    if (n_tokens < 0 || !weight) return ORC_INVALID_ARG;
+    if (!(weight[0] > 0.0f && weight[1] > 0.0f && weight[2] > 0.0f && weight[0] >= weight[1] && weight[1] >= weight[2]))
+        return ORC_INVALID_ARG;
+    int64_t rec[4];
+    for (int i = 0; i < 4; ++i) {
+        rec[i] = orc_record_bytes(head_dim, ladder[i], meta);
+        if (rec[i] < 0) return ORC_INVALID_ARG;
+    }
+    for (int64_t t = 0; t < n_tokens; ++t)
+        if (!(scores[t] >= 0.0f) || isinf(scores[t])) return ORC_INVALID_ARG;
+    if ((uint64_t)n_tokens * (uint64_t)rec[0] > budget_bytes) return ORC_BUFFER_TOO_SMALL;
+    uint64_t left = budget_bytes - (uint64_t)n_tokens * (uint64_t)rec[0];
+    orc_upgrade *u = (orc_upgrade *)malloc(sizeof(orc_upgrade) * (size_t)(3 * n_tokens > 0 ? 3 * n_tokens : 1));
+    if (!u) return ORC_INVALID_ARG;
+    for (int64_t t = 0; t < n_tokens; ++t)
+        for (int i = 0; i < 3; ++i) {
+            float s = scores[t] == 0.0f ? 0.0f : scores[t];
+            u[3 * t + i].key = s * weight[i];
+            u[3 * t + i].rung = i;
+            u[3 * t + i].index = t;
+        }
+    qsort(u, (size_t)(3 * n_tokens), sizeof(orc_upgrade), upgrade_before);
+    for (int64_t t = 0; t < n_tokens; ++t) bits[t] = 2;
+    for (int64_t j = 0; j < 3 * n_tokens; ++j) {
+        uint64_t cost = (uint64_t)(rec[u[j].rung + 1] - rec[u[j].rung]);
+        if (cost > left) break;
+        left -= cost;
+        bits[u[j].index] = (uint8_t)ladder[u[j].rung + 1];
+    }
+    free(u);
+    return ORC_OK;
+}
+
 /* Combined importance score (Section 3.3): S(t) = alpha * I(t) + (1 - alpha) * T(t), in binary32,
  * every operation rounded on its own (the file is compiled without contraction). */
 int orc_combine_scores(const float *importance, const float *transfer, float alpha, int64_t n, float *scores)

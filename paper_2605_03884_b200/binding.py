@@ -52,7 +52,7 @@ assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
            "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_card_send", "qkvs_attend_scratch_size", "qkvs_card_attend",
-           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_combine_scores", "qkvs_selftest_division",
+           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_bits_from_scores_budget", "qkvs_combine_scores", "qkvs_selftest_division",
            "qkvs_selftest_bounded_wait", "qkvs_status_string",
            "qkvs_version")
 
@@ -91,6 +91,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_card_attend.argtypes = [vp, C.c_size_t, C.POINTER(Layout), C.c_int32, vp, C.c_float, vp, vp, C.c_size_t, vp]
     lib.qkvs_bits_from_scores.restype = C.c_int
     lib.qkvs_bits_from_scores.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp]
+    lib.qkvs_bits_from_scores_budget.restype = C.c_int
+    lib.qkvs_bits_from_scores_budget.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, vp, vp, vp, vp, vp]
     lib.qkvs_combine_scores.restype = C.c_int
     lib.qkvs_combine_scores.argtypes = [vp, vp, C.c_float, C.c_int64, vp, vp]
     lib.qkvs_card_info.restype = C.c_int
@@ -297,6 +299,23 @@ def bits_from_scores(scores_dev, n_fp16: int, n_8bit: int, n_4bit: int, bits_dev
                                               int(n_4bit), int(bits_dev.data_ptr()), _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_bits_from_scores")
+    return st
+
+
+def bits_from_scores_budget(scores_dev, head_dim: int, budget_bytes: int, bits_dev, weights=None, meta_bytes: int = 8,
+                            offsets_dev=None, status_dev=None, stream=None, check: bool = True) -> int:
+    """qkvs_bits_from_scores_budget.  scores_dev: CUDA float32 [T] or [n_segments, T]; bits_dev: CUDA
+    uint8 of the same shape; weights: three floats or None; offsets_dev: optional CUDA int32/uint32
+    [n_segments, T + 1]; status_dev: optional CUDA int32 of one element."""
+    n_seg = 1 if scores_dev.dim() == 1 else int(scores_dev.shape[0])
+    n_tok = int(scores_dev.shape[-1])
+    w = (C.c_float * 3)(*[float(x) for x in weights]) if weights is not None else None
+    st = load_library().qkvs_bits_from_scores_budget(
+        int(scores_dev.data_ptr()), n_seg, n_tok, int(head_dim), int(meta_bytes), int(budget_bytes), w,
+        int(bits_dev.data_ptr()), int(offsets_dev.data_ptr()) if offsets_dev is not None else None,
+        int(status_dev.data_ptr()) if status_dev is not None else None, _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_bits_from_scores_budget")
     return st
 
 

@@ -70,6 +70,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return done != 0;
 }
 
+// The same poll without a suspend hint: the hardware's own (short) limit applies.  For barriers
+// that other threads of the CTA complete by arriving, where the waiter wants to go on at once.
+__device__ __forceinline__ bool mbar_try_wait_short(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
 __device__ __forceinline__ unsigned long long global_timer_ns()
 {
     unsigned long long t;
@@ -85,6 +100,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, unsign
     const unsigned long long start = global_timer_ns();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() - start > limit_ns) return false;
+    }
+}
+
+// The same wait built on the short poll.
+__device__ __forceinline__ bool mbar_wait_short(uint64_t *bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs)
+{
+    if (mbar_try_wait_short(bar, parity)) return true;
+    const unsigned long long start = global_timer_ns();
+    for (;;) {
+        if (mbar_try_wait_short(bar, parity)) return true;
         if (global_timer_ns() - start > limit_ns) return false;
     }
 }

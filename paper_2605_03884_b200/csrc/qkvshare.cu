@@ -12,12 +12,15 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
 #include "qkvs_common.cuh"
 #include "qkvs_pipeline.cuh"
 #include "qkvs_attend.cuh"
+#include "qkvs_attend_tc.cuh"
+#include "qkvs_select.cuh"
 
 namespace qkvs {
 
@@ -291,70 +294,6 @@ __global__ void __launch_bounds__(256) combine_scores_kernel(const float *__rest
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
         out[i] = __fadd_rn(__fmul_rn(alpha, imp[i]), __fmul_rn(beta, tra[i]));
-}
-
-// ---------------------------------------------------------------------------------------------
-// Bit-widths from importance scores by rank (the step in front of the offset scan).
-// rank(t) = #{s : score_s > score_t} + #{s < t : score_s == score_t}; the first n16 ranks keep
-// FP16, the next n8 get 8 bits, the next n4 get 4 bits, the rest 2 bits.  Exact and order-free:
-// every token counts for itself.  A CTA ranks 32 tokens, eight threads per token, each thread
-// against an eighth of every tile of up to 8192 scores staged in shared memory.
-
-constexpr int kRankThreads = 256;
-constexpr int kRankSplit = 8;       // threads per token
-constexpr int kRankTile = 8192;     // scores per tile (32 KB of shared memory)
-constexpr int kRankBlock = 256;     // scores per block inside a tile
-
-__global__ void __launch_bounds__(kRankThreads) bits_from_scores_kernel(const float *scores, int64_t T, uint32_t n16,
-                                                                        uint32_t n8, uint32_t n4, uint8_t *bits)
-{
-    __shared__ __align__(16) float tile[kRankTile];
-    scores += (int64_t)blockIdx.y * T;
-    bits += (int64_t)blockIdx.y * T;
-    const int part = threadIdx.x % kRankSplit;
-    const int64_t t = (int64_t)blockIdx.x * (kRankThreads / kRankSplit) + threadIdx.x / kRankSplit;
-    const float mine = t < T ? scores[t] : 0.0f;
-    uint32_t rank = 0;
-    for (int64_t base = 0; base < T; base += kRankTile) {
-        const int n = (int)min((int64_t)kRankTile, T - base);
-        const int n_pad = (n + kRankBlock - 1) / kRankBlock * kRankBlock;
-        __syncthreads();
-        for (int i = threadIdx.x; i < n_pad; i += kRankThreads) tile[i] = i < n ? scores[base + i] : -INFINITY;
-        __syncthreads();
-        // padding is -inf and sits behind every real index, so it never counts.  The eight threads
-        // of a token read neighbouring 16-byte pieces (no bank conflicts); a block of 256 scores
-        // that lies wholly in front of the token, or wholly behind it, needs one comparison per score.
-        const float4 *tile4 = reinterpret_cast<const float4 *>(tile);
-        for (int blk = 0; blk < n_pad / kRankBlock; ++blk) {
-            const int64_t first = base + (int64_t)blk * kRankBlock;
-            const float4 *piece = tile4 + blk * (kRankBlock / 4) + part;
-            if (first + kRankBlock <= t) {
-#pragma unroll
-                for (int i = 0; i < kRankBlock / 4 / kRankSplit; ++i) {
-                    const float4 s = piece[i * kRankSplit];
-                    rank += (s.x >= mine) + (s.y >= mine) + (s.z >= mine) + (s.w >= mine);
-                }
-            } else if (first > t) {
-#pragma unroll
-                for (int i = 0; i < kRankBlock / 4 / kRankSplit; ++i) {
-                    const float4 s = piece[i * kRankSplit];
-                    rank += (s.x > mine) + (s.y > mine) + (s.z > mine) + (s.w > mine);
-                }
-            } else {
-                for (int i = 0; i < kRankBlock / 4 / kRankSplit; ++i) {
-                    const float4 s = piece[i * kRankSplit];
-                    const int64_t idx = first + 4 * (i * kRankSplit + part);
-                    rank += (s.x > mine) || (s.x == mine && idx < t);
-                    rank += (s.y > mine) || (s.y == mine && idx + 1 < t);
-                    rank += (s.z > mine) || (s.z == mine && idx + 2 < t);
-                    rank += (s.w > mine) || (s.w == mine && idx + 3 < t);
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int s = 1; s < kRankSplit; s <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, s);
-    if (part == 0 && t < T) bits[t] = rank < n16 ? 16 : (rank < n16 + n8 ? 8 : (rank < n16 + n8 + n4 ? 4 : 2));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -861,7 +800,19 @@ qkvs_status_t qkvs_card_send(const void *card_dev, size_t card_bytes, int32_t sr
     return cudaMemcpyPeerAsync(dst_dev, dst_device, card_dev, src_device, card_bytes, cs) == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 
-// Shape of the attention work: steps of 16 tokens, items of 16 steps, per (layer, KV head).
+// Which attention kernel runs: the mma.sync one unless the environment asks for the tcgen05 one
+// (QKVS_ATTEND_KERNEL=tcgen05), which is correct but, as measured, not yet the faster of the two.
+static bool attend_on_tcgen05()
+{
+    static const bool v = [] {
+        const char *e = getenv("QKVS_ATTEND_KERNEL");
+        return e && strcmp(e, "tcgen05") == 0;
+    }();
+    return v;
+}
+
+// Shape of the attention work per (layer, KV head): items of 512 tokens for the tcgen05 kernel;
+// steps of 16 tokens and items of 16 steps for the mma.sync kernel.
 static qkvs_status_t attend_shape(const qkvs_layout_t *layout, int32_t n_q_heads, AttendParams *p)
 {
     const qkvs_status_t st = check_shape(layout);
@@ -876,7 +827,8 @@ static qkvs_status_t attend_shape(const qkvs_layout_t *layout, int32_t n_q_heads
     p->n_q_heads = n_q_heads;
     p->meta_bytes = meta_bytes_of(layout->meta_bytes);
     p->subs_per_head = (uint32_t)(((int64_t)layout->n_tokens + kAttendRows - 1) / kAttendRows);
-    p->items_per_head = (p->subs_per_head + kAttendSteps - 1) / kAttendSteps;
+    p->items_per_head = attend_on_tcgen05() ? (uint32_t)(((int64_t)layout->n_tokens + kTcItemTokens - 1) / kTcItemTokens)
+                                            : (p->subs_per_head + kAttendSteps - 1) / kAttendSteps;
     const uint64_t n_items = (uint64_t)layout->n_layers * (uint64_t)layout->n_kv_heads * p->items_per_head;
     if (n_items > 0x7fffffffull) return QKVS_ERR_UNSUPPORTED_SHAPE;
     p->n_items = (uint32_t)n_items;
@@ -928,7 +880,19 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
     p.status_dev = static_cast<int32_t *>(scratch_dev);
     p.work_counter = static_cast<uint32_t *>(scratch_dev) + 1;
     p.partials = reinterpret_cast<float *>(static_cast<uint8_t *>(scratch_dev) + QKVS_WORKSPACE_BYTES);
-    if (p.n_items > 0) {
+    if (p.n_items > 0 && attend_on_tcgen05()) {
+        const bool compact = p.meta_bytes == kMetaFp16, wide = n_q_heads / layout->n_kv_heads > 4;
+        auto kernel = compact ? (wide ? attend_tc_kernel<8, kMetaFp16> : attend_tc_kernel<4, kMetaFp16>)
+                              : (wide ? attend_tc_kernel<8, kMetaFp32> : attend_tc_kernel<4, kMetaFp32>);
+        const size_t smem = kTcPipes * sizeof(TcPipeSmem);
+        const int64_t want = (int64_t)((p.n_items + kTcPipes - 1) / kTcPipes);
+        unsigned grid = 0;
+        cudaError_t e = compact ? (wide ? persistent_grid<1013>(kernel, kTcThreads, smem, want, &grid) : persistent_grid<1012>(kernel, kTcThreads, smem, want, &grid))
+                                : (wide ? persistent_grid<1011>(kernel, kTcThreads, smem, want, &grid) : persistent_grid<1010>(kernel, kTcThreads, smem, want, &grid));
+        if (e != cudaSuccess) return QKVS_ERR_CUDA;
+        kernel<<<grid, kTcThreads, smem, cs>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
+    } else if (p.n_items > 0) {
         const bool compact = p.meta_bytes == kMetaFp16;
         auto kernel = compact ? attend_kernel<kAttendStages, kAttendWarps, kMetaFp16> : attend_kernel<kAttendStages, kAttendWarps, kMetaFp32>;
         const size_t smem = kAttendWarps * sizeof(AttendWarpSmem<kAttendStages>);
@@ -950,12 +914,51 @@ qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_segments,
 {
     if (n_segments < 1 || n_tokens < 0 || n_fp16 < 0 || n_8bit < 0 || n_4bit < 0) return QKVS_ERR_INVALID_ARG;
     if ((int64_t)n_fp16 + n_8bit + n_4bit > n_tokens) return QKVS_ERR_INVALID_ARG;
-    if (n_tokens > (1 << 20) || n_segments > 65535) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (n_tokens > (1 << 20) || n_segments > (1 << 24)) return QKVS_ERR_UNSUPPORTED_SHAPE;
     if (n_tokens == 0) return QKVS_OK;
     if (!scores_dev || !bits_dev || (reinterpret_cast<uintptr_t>(scores_dev) & 3u)) return QKVS_ERR_INVALID_ARG;
-    const dim3 grid((unsigned)((n_tokens + kRankThreads / kRankSplit - 1) / (kRankThreads / kRankSplit)), (unsigned)n_segments);
-    bits_from_scores_kernel<<<grid, kRankThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-        scores_dev, n_tokens, (uint32_t)n_fp16, (uint32_t)n_8bit, (uint32_t)n_4bit, bits_dev);
+    bits_by_rank_kernel<<<(unsigned)n_segments, kSelThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        scores_dev, n_tokens, (uint32_t)n_fp16, (uint32_t)n_8bit, (uint32_t)n_4bit, bits_dev, nullptr, 128, kMetaFp32);
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+}
+
+qkvs_status_t qkvs_bits_from_scores_budget(const float *scores_dev, int32_t n_segments, int32_t n_tokens, int32_t head_dim,
+                                           int32_t meta_bytes, uint64_t budget_bytes, const float *upgrade_weight,
+                                           uint8_t *bits_dev, uint32_t *offsets_dev, int32_t *status_dev, void *stream)
+{
+    static const float kDefaultWeight[3] = {0x1p-9f, 0x1p-14f, 0x1p-23f};
+    if (n_segments < 1 || n_tokens < 0) return QKVS_ERR_INVALID_ARG;
+    if (n_tokens > (1 << 20) || n_segments > (1 << 24)) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    const int meta = meta_bytes_of(meta_bytes);
+    if (meta == 0) return QKVS_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128 && head_dim != 192 && head_dim != 256) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (meta == kMetaFp16 && head_dim % 128 != 0) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    const float *w = upgrade_weight ? upgrade_weight : kDefaultWeight;
+    if (!(w[0] > 0.0f && w[1] > 0.0f && w[2] > 0.0f && w[0] >= w[1] && w[1] >= w[2])) return QKVS_ERR_INVALID_ARG;
+    BudgetParams bp;
+    memset(&bp, 0, sizeof(bp));
+    bp.rec2 = record_bytes(head_dim, 2, meta);
+    const uint32_t ladder[4] = {bp.rec2, record_bytes(head_dim, 4, meta), record_bytes(head_dim, 8, meta), record_bytes(head_dim, 16, meta)};
+    if ((uint64_t)n_tokens * bp.rec2 > budget_bytes) return QKVS_ERR_BUFFER_TOO_SMALL;
+    if (n_tokens == 0) return QKVS_OK;
+    if (!scores_dev || !bits_dev || (reinterpret_cast<uintptr_t>(scores_dev) & 3u) || (reinterpret_cast<uintptr_t>(offsets_dev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(status_dev) & 3u))
+        return QKVS_ERR_INVALID_ARG;
+    cudaStream_t cs = reinterpret_cast<cudaStream_t>(stream);
+    if (status_dev && cudaMemsetAsync(status_dev, 0, sizeof(int32_t), cs) != cudaSuccess) return QKVS_ERR_CUDA;
+    bp.scores = scores_dev;
+    bp.T = n_tokens;
+    bp.budget = budget_bytes;
+    for (int i = 0; i < 3; ++i) {
+        bp.weight[i] = w[i];
+        bp.cost[i] = ladder[i + 1] - ladder[i];
+    }
+    bp.bits = bits_dev;
+    bp.offsets = offsets_dev;
+    bp.status = status_dev;
+    bp.head_dim = head_dim;
+    bp.meta = meta;
+    bits_by_budget_kernel<<<(unsigned)n_segments, kSelThreads, 0, cs>>>(bp);
     return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 

@@ -116,3 +116,114 @@ def test_combined_score_matches_numpy_float32_step_by_step():
         big = np.maximum(np.maximum(np.abs(ta), np.abs(tb)), np.abs(ta + tb)).astype(np.float32)
         bound = 2 * np.spacing(big).astype(np.float64) + np.abs(tra).astype(np.float64) * 2.0 ** -24
         assert np.all(np.abs(got.astype(np.float64) - (ta + tb)) <= bound)
+
+
+# ----------------------------------------------------------------------------- byte budget
+
+def _rec(d, meta=8):
+    return [oracle.record_bytes(d, b, meta) for b in (2, 4, 8, 16)]
+
+
+def _stream_bytes(bits, d, meta=8):
+    r = dict(zip((2, 4, 8, 16), _rec(d, meta)))
+    return sum(r[int(b)] for b in bits)
+
+
+def test_budget_rule_special_cases_with_known_answers():
+    """Budget for 2 bits only -> all 2; for FP16 everywhere -> all 16; equal scores and exactly the
+    bytes of 4 bits everywhere -> all 4 (a lower rung always comes first among equal scores); one
+    token so far above the rest that its third upgrade outweighs anybody's first -> it alone climbs."""
+    d, T = 128, 50
+    r2, r4, r8, r16 = _rec(d)
+    s = np.random.default_rng(1).lognormal(0, 1, T).astype(np.float32)
+    st, bits = oracle.bits_from_scores_budget(s, d, T * r2)
+    assert st == oracle.OK and np.all(bits == 2)
+    st, bits = oracle.bits_from_scores_budget(s, d, T * r16)
+    assert st == oracle.OK and np.all(bits == 16)
+    st, bits = oracle.bits_from_scores_budget(s, d, T * r16 + 12345)
+    assert st == oracle.OK and np.all(bits == 16)
+    st, bits = oracle.bits_from_scores_budget(np.ones(T, np.float32), d, T * r4)
+    assert st == oracle.OK and np.all(bits == 4)
+    st, bits = oracle.bits_from_scores_budget(np.ones(T, np.float32), d, T * r4 + 3 * (r8 - r4) + 5)
+    assert st == oracle.OK and bits.tolist() == [8] * 3 + [4] * (T - 3)           # equal keys: lower index first
+    s = np.ones(T, np.float32)
+    s[17] = 2.0 ** 20                                                             # 2^20 * 2^-23 > 1 * 2^-9 ?  no: 2^-3 > 2^-9, yes
+    st, bits = oracle.bits_from_scores_budget(s, d, T * r2 + (r16 - r2))
+    assert st == oracle.OK and bits[17] == 16 and np.all(np.delete(bits, 17) == 2)
+    assert oracle.bits_from_scores_budget(s, d, T * r2 - 1)[0] == oracle.BUFFER_TOO_SMALL
+    bad = s.copy()
+    bad[3] = -1.0
+    assert oracle.bits_from_scores_budget(bad, d, T * r16)[0] == oracle.INVALID_ARG
+    assert oracle.bits_from_scores_budget(s, d, T * r16, weights=(1.0, 2.0, 0.5))[0] == oracle.INVALID_ARG
+
+
+@pytest.mark.parametrize("d,meta", [(128, 8), (64, 8), (128, 4)])
+def test_budget_is_respected_and_the_next_upgrade_would_not_fit(d, meta):
+    """Over a sweep of budgets: the stream never exceeds the budget; with power-of-two weights the
+    keys are exact, so more important tokens never get fewer bits; and what is left of the budget
+    is less than the cost of the upgrade that comes next in the order (recomputed here with
+    Python's sort on (-key, rung, index))."""
+    T = 200
+    rec = _rec(d, meta)
+    s = np.random.default_rng(2).lognormal(0, 1.5, T).astype(np.float32)
+    w = oracle.DEFAULT_UPGRADE_WEIGHTS
+    order = sorted(((-(np.float32(s[t]) * np.float32(w[i])), i, t) for t in range(T) for i in range(3)))
+    for budget in range(T * rec[0], T * rec[3] + 1, 997):
+        st, bits = oracle.bits_from_scores_budget(s, d, budget, meta_bytes=meta)
+        assert st == oracle.OK
+        used = _stream_bytes(bits, d, meta)
+        assert used <= budget
+        by_score = np.argsort(-s, kind="stable")
+        assert np.all(np.diff(bits[by_score].astype(int)) <= 0)
+        level = {2: 0, 4: 1, 8: 2, 16: 3}
+        granted = sum(level[int(b)] for b in bits)
+        if granted < 3 * T:
+            _, rung, t = order[granted]
+            assert level[int(bits[t])] == rung                       # the next upgrade in the order is this token's next rung
+            assert rec[rung + 1] - rec[rung] > budget - used         # and it does not fit
+        for j in range(granted):                                     # everything before it was granted
+            _, rung, t = order[j]
+            assert level[int(bits[t])] > rung
+
+
+def test_budget_rule_is_the_best_use_of_the_bytes_it_spends():
+    """Brute force on tiny inputs: among ALL assignments of {2,4,8,16} to T tokens that cost no more
+    than what the rule spent, none removes more weighted error (sum of key * cost over granted
+    upgrades) -- the rule takes upgrades in order of worth per byte, so at its own spending it is the
+    optimum of the knapsack in Section 3.3's objective under the additive error model."""
+    import itertools
+    d, T = 128, 6
+    rec = _rec(d)
+    cost = [rec[i + 1] - rec[i] for i in range(3)]
+    w = [float(np.float32(x)) for x in oracle.DEFAULT_UPGRADE_WEIGHTS]
+    rng = np.random.default_rng(3)
+    for trial in range(4):
+        s = rng.lognormal(0, 2.0, T).astype(np.float32)
+        for budget in (T * rec[0] + 100, T * rec[0] + 700, T * rec[1] + 333, T * rec[2] + 50):
+            st, bits = oracle.bits_from_scores_budget(s, d, budget)
+            assert st == oracle.OK
+            level = [{2: 0, 4: 1, 8: 2, 16: 3}[int(b)] for b in bits]
+            spent = sum(sum(cost[:l]) for l in level)
+            worth = sum(float(s[t]) * w[i] * cost[i] for t in range(T) for i in range(level[t]))
+            best = 0.0
+            for assign in itertools.product(range(4), repeat=T):
+                c = sum(sum(cost[:l]) for l in assign)
+                if c <= spent:
+                    best = max(best, sum(float(s[t]) * w[i] * cost[i] for t in range(T) for i in range(assign[t])))
+            assert worth >= best * (1 - 1e-12)
+
+
+def test_budget_rule_is_a_rank_rule_with_the_counts_it_arrives_at():
+    """Distinct scores and power-of-two weights: the outcome equals the rank rule run with the
+    class counts the budget rule produced (ties the two functions to each other)."""
+    d, T = 128, 3000
+    rec = _rec(d)
+    s = np.unique(np.random.default_rng(4).lognormal(0, 1, 2 * T).astype(np.float32))[:T].copy()
+    np.random.default_rng(5).shuffle(s)
+    for budget in (T * rec[0] + 5000, T * 80, T * 120, T * 200):
+        st, bits = oracle.bits_from_scores_budget(s, d, budget)
+        assert st == oracle.OK
+        n16, n8, n4 = int((bits == 16).sum()), int((bits == 8).sum()), int((bits == 4).sum())
+        st, ranked = oracle.bits_from_scores(s, n16, n8, n4)
+        assert st == oracle.OK and np.array_equal(bits, ranked)
+        assert np.array_equal(bits, by_library_sort(s, n16, n8, n4))
