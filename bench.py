@@ -265,9 +265,9 @@ def run_reference(args):
 class Case:
     """One workload resident on the device: inputs, outputs, card buffer, scratch block."""
 
-    def __init__(self, q, torch, number, meta_bytes=8, bits_mode=0, n_layers=0, pinned=False, host=None):
+    def __init__(self, q, torch, number, meta_bytes=8, bits_mode=0, n_layers=0, pinned=False, host=None, group_size=32):
         self.q, self.torch = q, torch
-        self.number, self.meta_bytes, self.bits_mode = number, meta_bytes, bits_mode
+        self.number, self.meta_bytes, self.bits_mode, self.group_size = number, meta_bytes, bits_mode, group_size
         w, Ks, Vs = host if host is not None else load_workload(number, n_layers=n_layers)
         self.w, self.Ks, self.Vs = w, Ks, Vs
         self.L, self.H, self.d, self.T = w.n_layers, w.n_kv_heads, w.head_dim, w.n_tokens
@@ -285,7 +285,7 @@ class Case:
             self.bits_per_hop = [wl.bits_per_head(w, h, gpu_rank_rule) for h in range(self.hops)]
         else:
             self.bits_per_hop = [wl.bits_for(w, h, rank_rule=gpu_rank_rule) for h in range(self.hops)]
-        self.lay = q.make_layout(self.L, self.H, self.d, self.T, bits_mode=bits_mode, meta_bytes=meta_bytes)
+        self.lay = q.make_layout(self.L, self.H, self.d, self.T, bits_mode=bits_mode, meta_bytes=meta_bytes, group_size=group_size)
         self.sizes = [q.card_size(self.lay, b) for b in self.bits_per_hop]
         self.prefix = q.card_prefix_size(self.lay)
         self.kv_bytes = w.kv_bytes
@@ -444,7 +444,7 @@ def run_ours(args):
     if rank == 0:
         sampler.start()  # runs through set-up and both timed legs; summarised over the timed window
 
-    case = Case(q, torch, args.config, args.meta_bytes, args.bits_mode, args.layers, pinned=not args.skip_e2e)
+    case = Case(q, torch, args.config, args.meta_bytes, args.bits_mode, args.layers, pinned=not args.skip_e2e, group_size=args.group_size)
     w, L, H, d, T, hops = case.w, case.L, case.H, case.d, case.T, case.hops
     kv_bytes, sizes, prefix = case.kv_bytes, case.sizes, case.prefix
     Kd, Vd, Ko, Vo, Kh, Vh, bits_d, bits_h = case.Kd, case.Vd, case.Ko, case.Vo, case.Kh, case.Vh, case.bits_d, case.bits_h
@@ -537,7 +537,7 @@ def run_ours(args):
     # attention straight from the card (the row after the hot path): one decode step, 32 query
     # heads, over the card the last create left behind; reported beside the main metric
     attend = None
-    if d == 128 and not args.skip_attend:
+    if d == 128 and args.group_size == 32 and not args.skip_attend:
         a_ms = case.attend(stream, 4)
         payload = sizes[-1] - prefix
         attend = {"what": "decode-step attention straight from the card, all layers, 4 query heads per KV head",
@@ -600,25 +600,30 @@ def run_ours(args):
         torch.cuda.synchronize()
         rank_us = a.elapsed_time(b) * 1e3 / 50
 
-    # the other benchmark workloads, a few steps each, after the headline timing and outside it:
-    # the 1K mixed cache, the 8K adaptive cache, the four-hop chain, and the headline cache with
-    # FP16 scale/zero pairs
+    # the other benchmark workloads and card formats, a few steps each, after the headline timing
+    # and outside it: the 1K mixed cache, the 8K adaptive cache, the four-hop chain; then the 8K
+    # uniform and adaptive caches with FP16 scale/zero pairs and with groups of 64 and 128 channels
+    # (these with the reconstruction error of the injected cache against the original)
     per_config = None
-    if args.per_config and w.number == 3 and not args.layers and args.meta_bytes == 8 and args.bits_mode == 0:
+    if args.per_config and w.number == 3 and not args.layers and args.meta_bytes == 8 and args.bits_mode == 0 and args.group_size == 32:
         per_config = []
-        host3 = (case.w, case.Ks, case.Vs)
+        hosts = {3: (case.w, case.Ks, case.Vs)}
         del case, Kd, Vd, Ko, Vo, Kh, Vh, bits_d, bits_h
         torch.cuda.empty_cache()
-        for number, meta, host in ((2, 8, None), (4, 8, None), (5, 8, "headline"), (3, 4, "headline")):
-            if host == "headline":   # the chain starts from the headline cache; same bytes
-                hw = (wl.WORKLOADS[number], host3[1], host3[2])
-            else:
-                hw = None
-            c = Case(q, torch, number, meta, 0, 0, pinned=False, host=hw)
+        runs = ((2, 8, 32), (4, 8, 32), (5, 8, 32), (3, 4, 32), (4, 4, 32), (3, 8, 64), (4, 8, 64), (3, 4, 128), (4, 4, 128))
+        for number, meta, group in runs:
+            src = 3 if number == 5 else number      # the chain starts from the headline cache; same bytes
+            if src not in hosts and src != 2:
+                hosts[src] = load_workload(src)
+            hw = (wl.WORKLOADS[number], hosts[src][1], hosts[src][2]) if src in hosts else None
+            c = Case(q, torch, number, meta, 0, 0, pinned=False, host=hw, group_size=group)
             _, cm, im = c.timed(stream, args.per_config_steps, 3)
-            entry = {"workload": c.w.name, "meta_bytes_per_group": meta, "steps": args.per_config_steps,
-                     "fp16_kv_bytes": c.kv_bytes, "per_hop": c.hop_stats(cm, im, peak)}
-            if c.d == 128 and not args.skip_attend:
+            errs = c.errors(stream) if (meta, group) != (8, 32) else None
+            entry = {"workload": c.w.name, "meta_bytes_per_group": meta, "group_size": group, "steps": args.per_config_steps,
+                     "fp16_kv_bytes": c.kv_bytes,
+                     "bits_per_element": 8.0 * (c.sizes[0] - c.prefix) / (c.kv_bytes / 2),
+                     "per_hop": c.hop_stats(cm, im, peak, errs)}
+            if c.d == 128 and group == 32 and not args.skip_attend:
                 a_ms = c.attend(stream, 4, reps=15)
                 payload = c.sizes[-1] - c.prefix
                 entry["attend_from_card"] = {"ms": a_ms, "card_payload_bytes": payload,
@@ -633,7 +638,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "n_layers": L, "n_kv_heads": H, "head_dim": d, "n_tokens": T,
                    "hops": hops, "fp16_kv_bytes": kv_bytes, "replicas": world,
-                   "meta_bytes_per_group": args.meta_bytes, "bits_mode": args.bits_mode,
+                   "meta_bytes_per_group": args.meta_bytes, "group_size": args.group_size, "bits_mode": args.bits_mode,
                    "reduced_for_profiling": bool(args.layers),
                    "l2": "inputs (1 GiB FP16 KV per pass) exceed the 126 MB L2; no flush"
                    if kv_bytes > 4 * 126e6 else "working set comparable to L2; L2 helps"},
@@ -674,6 +679,8 @@ def main():
     ap.add_argument("--meta-bytes", type=int, default=8, choices=[8, 4],
                     help="bytes of scale and zero per group in the card: 8 = two fp32 (the headline format), "
                          "4 = two FP16 (compact variant)")
+    ap.add_argument("--group-size", type=int, default=32, choices=[32, 64, 128],
+                    help="channels per quantisation group (32 is the headline format)")
     ap.add_argument("--bits-mode", type=int, default=0, choices=[0, 1],
                     help="0: one bit-width vector for the whole model (the paper's); 1: one per (layer, KV head)")
     ap.add_argument("--layers", type=int, default=0,

@@ -38,6 +38,15 @@
  *                   little-endian bit string.  record, b = 16: the d FP16 values verbatim.
  *   record size:    d*b/8 + meta_bytes*(d/32) bytes for b in {2,4,8};  2*d bytes for b = 16;
  *                   always a multiple of 16.
+ * Wider groups (qkvs_layout_t.group_size = 64 or 128, head_dim 128 or 256).  A group of 64 or 128
+ * channels shares one {scale, zero} pair, computed exactly as above over the wider group; a record
+ * then carries d/group pairs followed by zero bytes up to the next multiple of 16, then the codes:
+ *                   d*b/8 + round_up_16(meta_bytes*(d/group)) bytes.
+ * At head_dim 128 that is 80 bytes at 4 bits for every wide combination (5 bits per element, the
+ * same as FP16 pairs on groups of 32, because of the padding); at head_dim 256, one FP16 or fp32
+ * pair per 128 channels gives 144 bytes (4.5 bits per element).  The wider the group, the larger
+ * the range one scale has to cover: channel-wise key outliers then cost every channel of the
+ * group precision.  Card creation and injection support it; attention from the card does not.
  *
  * All entry points return a qkvs_status_t.  Unless stated otherwise a pointer named *_dev is a
  * device pointer, anything else is a host pointer.  The library allocates no device memory and
@@ -84,8 +93,9 @@ extern "C" {
 typedef enum {
     QKVS_OK = 0,
     QKVS_ERR_INVALID_ARG = 1,      /* null pointer, negative size, misaligned pointer or stride */
-    QKVS_ERR_UNSUPPORTED_SHAPE = 2,/* head_dim not in {64,128,192,256}, group_size != 32, compact
-                                      metadata with a head_dim that is not a multiple of 128 */
+    QKVS_ERR_UNSUPPORTED_SHAPE = 2,/* head_dim not in {64,128,192,256}, group_size not in {32,64,128}
+                                      (64 and 128 need head_dim 128 or 256), compact metadata on
+                                      groups of 32 with a head_dim that is not a multiple of 128 */
     QKVS_ERR_BAD_BITS = 3,         /* a bit-width outside {2,4,8,16} */
     QKVS_ERR_BUFFER_TOO_SMALL = 4, /* card capacity below what the bit-widths need */
     QKVS_ERR_BAD_CARD = 5,         /* header magic/version/shape/status/size does not check out */
@@ -101,7 +111,7 @@ typedef struct {
     int32_t n_kv_heads;
     int32_t head_dim;     /* 64, 128, 192 or 256 */
     int32_t n_tokens;     /* tokens in the card (sequence length, Section 4.2.1) */
-    int32_t group_size;   /* must be 32 */
+    int32_t group_size;   /* channels per quantisation group: 32, or 64 / 128 (see above) */
     int32_t bits_mode;    /* 0: one bits[n_tokens] for the whole model (the paper's token-level
                              vector); 1: bits[n_layers*n_kv_heads][n_tokens] */
     int64_t head_stride;  /* elements between heads; multiple of 8 */
@@ -143,7 +153,7 @@ typedef struct {
 } qkvs_card_header_t;
 
 /* Record size in bytes of one token row of `head_dim` channels at bit-width b with meta_bytes
- * (8, 0 for 8, or 4) of scale and zero per group; 0 if b is not one of {2,4,8,16} or the
+ * (8, 0 for 8, or 4) of scale and zero per group of 32 channels; 0 if b is not one of {2,4,8,16} or the
  * combination of head_dim and meta_bytes is not supported.  Host only.  (Closed form above;
  * Section 3.1 for the code bytes.) */
 QKVS_API size_t qkvs_record_bytes(int32_t head_dim, int32_t b, int32_t meta_bytes);

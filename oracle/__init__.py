@@ -56,6 +56,20 @@ def lib():
         l.orc_float_to_half.argtypes = [C.c_float]
         l.orc_record_bytes.restype = C.c_int64
         l.orc_record_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+        l.orc_record_bytes_g.restype = C.c_int64
+        l.orc_record_bytes_g.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
+        l.orc_scan_offsets_g.restype = C.c_int
+        l.orc_scan_offsets_g.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(C.c_uint64)]
+        l.orc_quantize_span.restype = None
+        l.orc_quantize_span.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_void_p]
+        l.orc_quantize_span_compact.restype = None
+        l.orc_quantize_span_compact.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_uint16), C.POINTER(C.c_uint16), C.c_void_p]
+        l.orc_dequantize_span.restype = None
+        l.orc_dequantize_span.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_float, C.c_void_p]
+        l.orc_encode_stream_g.restype = None
+        l.orc_encode_stream_g.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.orc_decode_stream_g.restype = None
+        l.orc_decode_stream_g.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int64]
         l.orc_scan_offsets.restype = C.c_int
         l.orc_scan_offsets.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.POINTER(C.c_uint64)]
         l.orc_card_size.restype = C.c_int
@@ -104,10 +118,10 @@ def _ptr(a: np.ndarray) -> int:
 
 
 def make_layout(n_layers, n_kv_heads, head_dim, n_tokens, bits_mode=0, head_stride=None,
-                token_stride=None, meta_bytes=8) -> Layout:
+                token_stride=None, meta_bytes=8, group_size=32) -> Layout:
     ts = head_dim if token_stride is None else token_stride
     hs = n_tokens * ts if head_stride is None else head_stride
-    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, 32, bits_mode, hs, ts, meta_bytes, 0)
+    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, group_size, bits_mode, hs, ts, meta_bytes, 0)
 
 
 def half_to_float(h: int) -> float:
@@ -118,16 +132,40 @@ def float_to_half(f: float) -> int:
     return int(lib().orc_float_to_half(C.c_float(f)))
 
 
-def record_bytes(head_dim: int, b: int, meta_bytes: int = 8) -> int:
-    return int(lib().orc_record_bytes(head_dim, b, meta_bytes))
+def record_bytes(head_dim: int, b: int, meta_bytes: int = 8, group_size: int = 32) -> int:
+    return int(lib().orc_record_bytes_g(head_dim, b, meta_bytes, group_size))
 
 
-def scan_offsets(head_dim: int, bits: np.ndarray, meta_bytes: int = 8) -> Tuple[int, np.ndarray, int]:
+def scan_offsets(head_dim: int, bits: np.ndarray, meta_bytes: int = 8, group_size: int = 32) -> Tuple[int, np.ndarray, int]:
     bits = np.ascontiguousarray(bits, dtype=np.uint8)
     off = np.zeros(bits.size + 1, dtype=np.uint32)
     sb = C.c_uint64(0)
-    st = lib().orc_scan_offsets(head_dim, meta_bytes, _ptr(bits), bits.size, _ptr(off), C.byref(sb))
+    st = lib().orc_scan_offsets_g(head_dim, meta_bytes, group_size, _ptr(bits), bits.size, _ptr(off), C.byref(sb))
     return st, off, int(sb.value)
+
+
+def quantize_span(x: np.ndarray, b: int, compact: bool = False):
+    """One group of n = x.size (32, 64 or 128) FP16 values -> (scale, zero, codes[n]); with
+    compact=True scale and zero come back as FP16 values."""
+    x = np.ascontiguousarray(x).view(np.uint16)
+    n = x.size
+    assert n in (32, 64, 128)
+    q = np.zeros(n, dtype=np.uint8)
+    if compact:
+        s, z = C.c_uint16(0), C.c_uint16(0)
+        lib().orc_quantize_span_compact(_ptr(x), n, b, C.byref(s), C.byref(z), _ptr(q))
+        return (np.array([s.value], dtype=np.uint16).view(np.float16)[0],
+                np.array([z.value], dtype=np.uint16).view(np.float16)[0], q)
+    s, z = C.c_float(0), C.c_float(0)
+    lib().orc_quantize_span(_ptr(x), n, b, C.byref(s), C.byref(z), _ptr(q))
+    return np.float32(s.value), np.float32(z.value), q
+
+
+def dequantize_span(q: np.ndarray, scale, zero) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    out = np.zeros(q.size, dtype=np.uint16)
+    lib().orc_dequantize_span(_ptr(q), q.size, C.c_float(scale), C.c_float(zero), _ptr(out))
+    return out.view(np.float16)
 
 
 def card_size(layout: Layout, bits: Optional[np.ndarray]) -> Tuple[int, int]:
@@ -184,28 +222,28 @@ def unpack_codes(packed: np.ndarray, n: int, b: int) -> np.ndarray:
     return q
 
 
-def encode_stream(x: np.ndarray, bits: np.ndarray, meta_bytes: int = 8) -> np.ndarray:
+def encode_stream(x: np.ndarray, bits: np.ndarray, meta_bytes: int = 8, group_size: int = 32) -> np.ndarray:
     """One [T, d] FP16 matrix + bits[T] -> the stream's payload bytes."""
     x = np.ascontiguousarray(x).view(np.uint16)
     t, d = x.shape
-    st, off, _ = scan_offsets(d, bits, meta_bytes)
+    st, off, _ = scan_offsets(d, bits, meta_bytes, group_size)
     if st:
         raise ValueError(f"bad bits (status {st})")
     bits = np.ascontiguousarray(bits, dtype=np.uint8)
     out = np.zeros(int(off[-1]), dtype=np.uint8)
-    lib().orc_encode_stream(_ptr(x), d, t, d, meta_bytes, _ptr(bits), _ptr(off), _ptr(out))
+    lib().orc_encode_stream_g(_ptr(x), d, t, d, meta_bytes, group_size, _ptr(bits), _ptr(off), _ptr(out))
     return out
 
 
-def decode_stream(payload: np.ndarray, bits: np.ndarray, d: int, meta_bytes: int = 8) -> np.ndarray:
+def decode_stream(payload: np.ndarray, bits: np.ndarray, d: int, meta_bytes: int = 8, group_size: int = 32) -> np.ndarray:
     payload = np.ascontiguousarray(payload, dtype=np.uint8)
     bits = np.ascontiguousarray(bits, dtype=np.uint8)
-    st, off, _ = scan_offsets(d, bits, meta_bytes)
+    st, off, _ = scan_offsets(d, bits, meta_bytes, group_size)
     if st:
         raise ValueError(f"bad bits (status {st})")
     assert payload.size == int(off[-1])
     x = np.zeros((bits.size, d), dtype=np.uint16)
-    lib().orc_decode_stream(_ptr(payload), _ptr(bits), _ptr(off), bits.size, d, meta_bytes, _ptr(x), d)
+    lib().orc_decode_stream_g(_ptr(payload), _ptr(bits), _ptr(off), bits.size, d, meta_bytes, group_size, _ptr(x), d)
     return x.view(np.float16)
 
 

@@ -51,7 +51,7 @@ enum { ORC_OK = 0, ORC_INVALID_ARG = 1, ORC_UNSUPPORTED_SHAPE = 2, ORC_BAD_BITS 
 
 typedef struct {
     int32_t n_layers, n_kv_heads, head_dim, n_tokens;
-    int32_t group_size; /* 32 */
+    int32_t group_size; /* 32, or 64 / 128 (wider-group variant) */
     int32_t bits_mode;  /* 0: one bits[T] for the whole model; 1: bits[L*H][T] */
     int64_t head_stride;  /* elements between heads  */
     int64_t token_stride; /* elements between tokens */
@@ -60,6 +60,7 @@ typedef struct {
 } orc_layout;
 
 static int meta_of(const orc_layout *L) { return L->meta_bytes == 0 ? 8 : L->meta_bytes; }
+static int group_of(const orc_layout *L) { return L->group_size; }
 
 /* ------------------------------------------------------------------ FP16 <-> FP32 */
 
@@ -108,27 +109,43 @@ uint16_t orc_float_to_half(float f)
 
 static uint64_t round_up_256(uint64_t x) { return (x + 255u) / 256u * 256u; }
 
-/* Bytes of one token row inside one stream: G (scale, zero) pairs of `meta` bytes each (8: two
- * fp32; 4: two FP16) then the packed codes; an FP16 token is the row itself.  Code bytes alone
- * are d*b/8 (Section 3.1's bytes-per-element law). */
-int64_t orc_record_bytes(int head_dim, int b, int meta)
+/* Bytes of one token row inside one stream: d/group (scale, zero) pairs of `meta` bytes each (8: two
+ * fp32; 4: two FP16), then the packed codes; an FP16 token is the row itself.  Code bytes alone
+ * are d*b/8 (Section 3.1's bytes-per-element law).  With groups of 32 channels the pairs take
+ * meta*d/32 bytes, which the supported shapes keep a multiple of 16; with the wider groups of 64
+ * or 128 channels (fewer pairs: Section 3.1's 0.5 bytes per element is approached as the metadata
+ * shrinks) the pairs are followed by zero bytes up to the next multiple of 16, so that the codes
+ * start, and every record ends, on a 16-byte boundary as before. */
+int64_t orc_record_bytes_g(int head_dim, int b, int meta, int group)
 {
     if (meta != 8 && meta != 4) return -1;
+    if (group != 32 && group != 64 && group != 128) return -1;
+    if (head_dim % group != 0) return -1;
     if (b == 16) return 2 * (int64_t)head_dim;
-    if (b == 2 || b == 4 || b == 8) return (int64_t)head_dim * b / 8 + meta * (int64_t)(head_dim / 32);
+    if (b == 2 || b == 4 || b == 8) {
+        int64_t pairs = (int64_t)meta * (head_dim / group);
+        if (group != 32) pairs = (pairs + 15) / 16 * 16;
+        return (int64_t)head_dim * b / 8 + pairs;
+    }
     return -1;
 }
+
+int64_t orc_record_bytes(int head_dim, int b, int meta) { return orc_record_bytes_g(head_dim, b, meta, 32); }
+
+/* where the code bytes begin inside a record */
+static int64_t codes_at(int head_dim, int meta, int group) { return orc_record_bytes_g(head_dim, 4, meta, group) - head_dim / 2; }
 
 static int layout_ok(const orc_layout *L)
 {
     if (!L) return ORC_INVALID_ARG;
     if (L->n_layers < 1 || L->n_kv_heads < 1 || L->n_tokens < 0) return ORC_INVALID_ARG;
     if (L->bits_mode != 0 && L->bits_mode != 1) return ORC_INVALID_ARG;
-    if (L->group_size != 32) return ORC_UNSUPPORTED_SHAPE;
+    if (L->group_size != 32 && L->group_size != 64 && L->group_size != 128) return ORC_UNSUPPORTED_SHAPE;
+    if (L->head_dim % L->group_size != 0) return ORC_UNSUPPORTED_SHAPE;
     if (L->head_dim < 64 || L->head_dim % 64 != 0) return ORC_UNSUPPORTED_SHAPE;
     if (meta_of(L) != 8 && meta_of(L) != 4) return ORC_INVALID_ARG;
     /* records stay multiples of 16 bytes: FP16 pairs need head_dim to be a multiple of 128 */
-    if (meta_of(L) == 4 && L->head_dim % 128 != 0) return ORC_UNSUPPORTED_SHAPE;
+    if (meta_of(L) == 4 && L->group_size == 32 && L->head_dim % 128 != 0) return ORC_UNSUPPORTED_SHAPE;
     return ORC_OK;
 }
 
@@ -150,14 +167,14 @@ static int64_t segment_of(const orc_layout *L, int l, int h)
 
 /* Exclusive prefix sum of record sizes over one segment: off[0] = 0,
  * off[t+1] = off[t] + rec(b_t).  Returns ORC_BAD_BITS on a value outside {2,4,8,16}. */
-int orc_scan_offsets(int head_dim, int meta, const uint8_t *bits, int64_t n_tokens, uint32_t *off,
-                     uint64_t *sum_bits)
+int orc_scan_offsets_g(int head_dim, int meta, int group, const uint8_t *bits, int64_t n_tokens, uint32_t *off,
+                       uint64_t *sum_bits)
 {
-    if (meta != 8 && meta != 4) return ORC_INVALID_ARG;
+    if (orc_record_bytes_g(head_dim, 16, meta, group) < 0) return ORC_INVALID_ARG;
     uint64_t run = 0, sb = 0;
     off[0] = 0;
     for (int64_t t = 0; t < n_tokens; ++t) {
-        int64_t r = orc_record_bytes(head_dim, bits[t], meta);
+        int64_t r = orc_record_bytes_g(head_dim, bits[t], meta, group);
         if (r < 0) return ORC_BAD_BITS;
         run += (uint64_t)r;
         sb += bits[t];
@@ -165,6 +182,11 @@ int orc_scan_offsets(int head_dim, int meta, const uint8_t *bits, int64_t n_toke
     }
     if (sum_bits) *sum_bits = sb;
     return ORC_OK;
+}
+
+int orc_scan_offsets(int head_dim, int meta, const uint8_t *bits, int64_t n_tokens, uint32_t *off, uint64_t *sum_bits)
+{
+    return orc_scan_offsets_g(head_dim, meta, 32, bits, n_tokens, off, sum_bits);
 }
 
 /* Section sizes.  Card = header (256) | bits | offsets | [stream bases, mode 1] | payload. */
@@ -198,7 +220,7 @@ int orc_card_size(const orc_layout *L, const uint8_t *bits, uint64_t *out_bytes)
     for (int64_t seg = 0; seg < nseg; ++seg) {
         uint64_t seg_bytes = 0;
         for (int64_t t = 0; t < L->n_tokens; ++t) {
-            int64_t r = orc_record_bytes(L->head_dim, bits ? bits[seg * L->n_tokens + t] : 16, meta_of(L));
+            int64_t r = orc_record_bytes_g(L->head_dim, bits ? bits[seg * L->n_tokens + t] : 16, meta_of(L), group_of(L));
             if (r < 0) return ORC_BAD_BITS;
             seg_bytes += (uint64_t)r;
         }
@@ -253,13 +275,13 @@ static uint16_t get_u16(const uint8_t *p) { return (uint16_t)(p[0] | (p[1] << 8)
 
 /* ------------------------------------------------------------------ one group of 32 */
 
-/* Quantise 32 FP16 values at b in {2,4,8} bits. */
-void orc_quantize_group(const uint16_t *x, int b, float *scale_out, float *zero_out, uint8_t *q)
+/* Quantise one group of n FP16 values (n = 32, 64 or 128) at b in {2,4,8} bits. */
+void orc_quantize_span(const uint16_t *x, int n, int b, float *scale_out, float *zero_out, uint8_t *q)
 {
-    float xf[32];
-    for (int i = 0; i < 32; ++i) xf[i] = orc_half_to_float(x[i]);
+    float xf[128] = {0};
+    for (int i = 0; i < n; ++i) xf[i] = orc_half_to_float(x[i]);
     float mn = xf[0], mx = xf[0];
-    for (int i = 1; i < 32; ++i) {
+    for (int i = 1; i < n; ++i) {
         if (xf[i] < mn) mn = xf[i];
         if (xf[i] > mx) mx = xf[i];
     }
@@ -275,7 +297,7 @@ void orc_quantize_group(const uint16_t *x, int b, float *scale_out, float *zero_
         scale = range / qmaxf;
         inv = qmaxf / range;
     }
-    for (int i = 0; i < 32; ++i) {
+    for (int i = 0; i < n; ++i) {
         float t = xf[i] - mn;
         float u = t * inv;
         float r = nearbyintf(u); /* ties to even (default rounding mode) */
@@ -287,6 +309,11 @@ void orc_quantize_group(const uint16_t *x, int b, float *scale_out, float *zero_
     }
     *scale_out = scale;
     *zero_out = mn;
+}
+
+void orc_quantize_group(const uint16_t *x, int b, float *scale_out, float *zero_out, uint8_t *q)
+{
+    orc_quantize_span(x, 32, b, scale_out, zero_out, q);
 }
 
 /* Smallest FP16 value that is >= f, for finite f >= 0 not above the largest FP16 value:
@@ -308,14 +335,14 @@ uint16_t orc_float_to_half_up(float f)
  * The largest possible scale, (65504+65504)/3, is below the largest FP16 value, so the rounding
  * up never overflows; the smallest, 2^-24/255, rounds up to the smallest FP16 subnormal 2^-24.
  * Reconstruction is orc_dequantize_group() with the two FP16 values widened to binary32. */
-void orc_quantize_group_compact(const uint16_t *x, int b, uint16_t *scale_out, uint16_t *zero_out,
-                                uint8_t *q)
+void orc_quantize_span_compact(const uint16_t *x, int n, int b, uint16_t *scale_out, uint16_t *zero_out,
+                               uint8_t *q)
 {
-    float xf[32];
-    for (int i = 0; i < 32; ++i) xf[i] = orc_half_to_float(x[i]);
+    float xf[128] = {0};
+    for (int i = 0; i < n; ++i) xf[i] = orc_half_to_float(x[i]);
     float mn = xf[0], mx = xf[0];
     uint16_t mn_bits = x[0];
-    for (int i = 1; i < 32; ++i) {
+    for (int i = 1; i < n; ++i) {
         if (xf[i] < mn) { mn = xf[i]; mn_bits = x[i]; }
         if (xf[i] > mx) mx = xf[i];
     }
@@ -332,7 +359,7 @@ void orc_quantize_group_compact(const uint16_t *x, int b, uint16_t *scale_out, u
         scale16 = orc_float_to_half_up(range / qmaxf);
         inv = 1.0f / orc_half_to_float(scale16);
     }
-    for (int i = 0; i < 32; ++i) {
+    for (int i = 0; i < n; ++i) {
         float t = xf[i] - mn;
         float u = t * inv;
         float r = nearbyintf(u); /* ties to even (default rounding mode) */
@@ -346,15 +373,22 @@ void orc_quantize_group_compact(const uint16_t *x, int b, uint16_t *scale_out, u
     *zero_out = mn_bits;
 }
 
-/* Reconstruct 32 FP16 values: multiply, then add, each rounded to binary32, then to FP16. */
-void orc_dequantize_group(const uint8_t *q, float scale, float zero, uint16_t *out)
+void orc_quantize_group_compact(const uint16_t *x, int b, uint16_t *scale_out, uint16_t *zero_out, uint8_t *q)
 {
-    for (int i = 0; i < 32; ++i) {
+    orc_quantize_span_compact(x, 32, b, scale_out, zero_out, q);
+}
+
+/* Reconstruct 32 FP16 values: multiply, then add, each rounded to binary32, then to FP16. */
+void orc_dequantize_span(const uint8_t *q, int n, float scale, float zero, uint16_t *out)
+{
+    for (int i = 0; i < n; ++i) {
         float p = (float)q[i] * scale;
         float r = p + zero;
         out[i] = orc_float_to_half(r);
     }
 }
+
+void orc_dequantize_group(const uint8_t *q, float scale, float zero, uint16_t *out) { orc_dequantize_span(q, 32, scale, zero, out); }
 
 /* Codes as a little-endian bit string: code i occupies bits [i*b, i*b+b). */
 void orc_pack_codes(const uint8_t *q, int n, int b, uint8_t *out)
@@ -379,7 +413,7 @@ void orc_unpack_codes(const uint8_t *in, int n, int b, uint8_t *q)
 /* Record of a b<16 token: G pairs {scale_g, zero_g} (little-endian; two fp32 when meta == 8,
  * two FP16 when meta == 4), group g covering channels 32g..32g+31, then the d*b/8 code bytes of
  * the whole row.  b == 16: the row's FP16 bit patterns verbatim. */
-static void encode_record(const uint16_t *row, int d, int b, int meta, uint8_t *rec)
+static void encode_record(const uint16_t *row, int d, int b, int meta, int group, uint8_t *rec)
 {
     if (b == 16) {
         for (int i = 0; i < d; ++i) {
@@ -388,21 +422,23 @@ static void encode_record(const uint16_t *row, int d, int b, int meta, uint8_t *
         }
         return;
     }
-    int G = d / 32;
-    uint8_t q[32];
+    int G = d / group;
+    int64_t codes = codes_at(d, meta, group);
+    uint8_t q[128];
+    memset(rec, 0, (size_t)codes); /* the pairs, and the zero bytes that follow them with wide groups */
     for (int g = 0; g < G; ++g) {
         if (meta == 8) {
             float scale, zero;
-            orc_quantize_group(row + 32 * g, b, &scale, &zero, q);
+            orc_quantize_span(row + group * g, group, b, &scale, &zero, q);
             put_f32(rec + 8 * g, scale);
             put_f32(rec + 8 * g + 4, zero);
         } else {
             uint16_t scale16, zero16;
-            orc_quantize_group_compact(row + 32 * g, b, &scale16, &zero16, q);
+            orc_quantize_span_compact(row + group * g, group, b, &scale16, &zero16, q);
             put_u16(rec + 4 * g, scale16);
             put_u16(rec + 4 * g + 2, zero16);
         }
-        orc_pack_codes(q, 32, b, rec + meta * G + (size_t)g * 32 * b / 8);
+        orc_pack_codes(q, group, b, rec + codes + (size_t)g * group * b / 8);
     }
 }
 
@@ -418,35 +454,48 @@ static void group_meta(const uint8_t *rec, int g, int meta, float *scale, float 
     }
 }
 
-static void decode_record(const uint8_t *rec, int d, int b, int meta, uint16_t *row)
+static void decode_record(const uint8_t *rec, int d, int b, int meta, int group, uint16_t *row)
 {
     if (b == 16) {
         for (int i = 0; i < d; ++i) row[i] = (uint16_t)(rec[2 * i] | (rec[2 * i + 1] << 8));
         return;
     }
-    int G = d / 32;
-    uint8_t q[32];
+    int G = d / group;
+    int64_t codes = codes_at(d, meta, group);
+    uint8_t q[128];
     for (int g = 0; g < G; ++g) {
         float scale, zero;
         group_meta(rec, g, meta, &scale, &zero);
-        orc_unpack_codes(rec + meta * G + (size_t)g * 32 * b / 8, 32, b, q);
-        orc_dequantize_group(q, scale, zero, row + 32 * g);
+        orc_unpack_codes(rec + codes + (size_t)g * group * b / 8, group, b, q);
+        orc_dequantize_span(q, group, scale, zero, row + group * g);
     }
 }
 
 /* One stream (a [T, d] matrix with a row stride) -> its payload bytes. */
+void orc_encode_stream_g(const uint16_t *x, int64_t token_stride, int64_t n_tokens, int d, int meta, int group,
+                         const uint8_t *bits, const uint32_t *off, uint8_t *out)
+{
+    for (int64_t t = 0; t < n_tokens; ++t)
+        encode_record(x + t * token_stride, d, bits[t], meta, group, out + off[t]);
+}
+
+void orc_decode_stream_g(const uint8_t *in, const uint8_t *bits, const uint32_t *off,
+                         int64_t n_tokens, int d, int meta, int group, uint16_t *x, int64_t token_stride)
+{
+    for (int64_t t = 0; t < n_tokens; ++t)
+        decode_record(in + off[t], d, bits[t], meta, group, x + t * token_stride);
+}
+
 void orc_encode_stream(const uint16_t *x, int64_t token_stride, int64_t n_tokens, int d, int meta,
                        const uint8_t *bits, const uint32_t *off, uint8_t *out)
 {
-    for (int64_t t = 0; t < n_tokens; ++t)
-        encode_record(x + t * token_stride, d, bits[t], meta, out + off[t]);
+    orc_encode_stream_g(x, token_stride, n_tokens, d, meta, 32, bits, off, out);
 }
 
 void orc_decode_stream(const uint8_t *in, const uint8_t *bits, const uint32_t *off,
                        int64_t n_tokens, int d, int meta, uint16_t *x, int64_t token_stride)
 {
-    for (int64_t t = 0; t < n_tokens; ++t)
-        decode_record(in + off[t], d, bits[t], meta, x + t * token_stride);
+    orc_decode_stream_g(in, bits, off, n_tokens, d, meta, 32, x, token_stride);
 }
 
 /* ------------------------------------------------------------------ whole card */
@@ -481,7 +530,7 @@ int orc_write_prefix(const orc_layout *L, const uint8_t *bits, uint64_t model_id
         uint32_t *off_tmp = (uint32_t *)(void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1));
         /* the host is little-endian, so writing uint32_t in place equals put_u32 */
         uint64_t sb = 0;
-        status = orc_scan_offsets(L->head_dim, meta_of(L), bits + seg * T, T, off_tmp, &sb);
+        status = orc_scan_offsets_g(L->head_dim, meta_of(L), group_of(L), bits + seg * T, T, off_tmp, &sb);
         sum_bits += sb;
         memcpy(card + bo + (uint64_t)seg * (uint64_t)T, bits + seg * T, (size_t)T);
     }
@@ -579,7 +628,7 @@ int orc_card_create_range(const orc_layout *L, const uint16_t *const *K_layers,
         int l = (int)(s / (2 * L->n_kv_heads));
         int64_t seg = segment_of(L, l, h);
         const uint16_t *x = (kv == 0 ? K_layers[l] : V_layers[l]) + (int64_t)h * L->head_stride;
-        orc_encode_stream(x, L->token_stride, T, L->head_dim, meta_of(L), card + bo + (uint64_t)seg * (uint64_t)T,
+        orc_encode_stream_g(x, L->token_stride, T, L->head_dim, meta_of(L), group_of(L), card + bo + (uint64_t)seg * (uint64_t)T,
                           (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1)),
                           card + stream_base(card, L, s));
     }
@@ -610,7 +659,7 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
     C.bits_mode = (int32_t)get_u32(card + 12);
     C.n_tokens = (int32_t)get_u32(card + 28);
     if ((int32_t)get_u32(card + 16) != dst->n_layers || (int32_t)get_u32(card + 20) != dst->n_kv_heads ||
-        (int32_t)get_u32(card + 24) != dst->head_dim || get_u32(card + 32) != 32u ||
+        (int32_t)get_u32(card + 24) != dst->head_dim || get_u32(card + 32) != (uint32_t)group_of(dst) ||
         get_u32(card + 36) != (uint32_t)meta_of(dst) || (C.bits_mode != 0 && C.bits_mode != 1) ||
         C.n_tokens != dst->n_tokens)
         return ORC_BAD_CARD;
@@ -636,9 +685,9 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
         int64_t seg = segment_of(&C, l, h);
         uint16_t *x = (kv == 0 ? K_out[l] : V_out[l]) + (int64_t)h * dst->head_stride +
                       dst_token_offset * dst->token_stride;
-        orc_decode_stream(card + stream_base(card, &C, s), card + bo + (uint64_t)seg * (uint64_t)T,
+        orc_decode_stream_g(card + stream_base(card, &C, s), card + bo + (uint64_t)seg * (uint64_t)T,
                           (const uint32_t *)(const void *)(card + oo + 4u * (uint64_t)seg * (uint64_t)(T + 1)),
-                          T, C.head_dim, meta_of(&C), x, dst->token_stride);
+                          T, C.head_dim, meta_of(&C), group_of(&C), x, dst->token_stride);
     }
     return ORC_OK;
 }
@@ -647,28 +696,29 @@ int orc_card_inject(const uint8_t *card, uint64_t card_bytes, const orc_layout *
  * the FP16 values themselves for a 16-bit row.  No rounding to FP16: that rounding belongs to
  * injection, which has to hand an FP16 cache to the receiving framework (Section 4.2.2); attention
  * that reads the card itself (Section 4.3) has no FP16 copy to round into. */
-static void reconstruct_record(const uint8_t *rec, int d, int b, int meta, double *row)
+static void reconstruct_record(const uint8_t *rec, int d, int b, int meta, int group, double *row)
 {
     if (b == 16) {
         for (int i = 0; i < d; ++i) row[i] = (double)orc_half_to_float((uint16_t)(rec[2 * i] | (rec[2 * i + 1] << 8)));
         return;
     }
-    int G = d / 32;
-    uint8_t q[32];
+    int G = d / group;
+    int64_t codes = codes_at(d, meta, group);
+    uint8_t q[128];
     for (int g = 0; g < G; ++g) {
         float scale, zero;
         group_meta(rec, g, meta, &scale, &zero);
-        orc_unpack_codes(rec + meta * G + (size_t)g * 32 * b / 8, 32, b, q);
-        for (int i = 0; i < 32; ++i) row[32 * g + i] = (double)q[i] * (double)scale + (double)zero;
+        orc_unpack_codes(rec + codes + (size_t)g * group * b / 8, group, b, q);
+        for (int i = 0; i < group; ++i) row[group * g + i] = (double)q[i] * (double)scale + (double)zero;
     }
 }
 
 /* The values injection hands to the receiving framework: the record decoded exactly as
  * orc_card_inject does (fp16_rne(fl32(fl32(q) * scale) + zero), Section 4.2.2), widened. */
-static void injected_record(const uint8_t *rec, int d, int b, int meta, double *row)
+static void injected_record(const uint8_t *rec, int d, int b, int meta, int group, double *row)
 {
     uint16_t h[256];
-    decode_record(rec, d, b, meta, h);
+    decode_record(rec, d, b, meta, group, h);
     for (int i = 0; i < d; ++i) row[i] = (double)orc_half_to_float(h[i]);
 }
 
@@ -704,7 +754,8 @@ static int attend_over_card(const uint8_t *card, uint64_t card_bytes, const orc_
     C.bits_mode = (int32_t)get_u32(card + 12);
     if ((int32_t)get_u32(card + 16) != L->n_layers || (int32_t)get_u32(card + 20) != L->n_kv_heads ||
         (int32_t)get_u32(card + 24) != L->head_dim || (int32_t)get_u32(card + 28) != L->n_tokens ||
-        get_u32(card + 36) != (uint32_t)meta_of(L) || (C.bits_mode != 0 && C.bits_mode != 1) || get_u64(card + 112) > card_bytes)
+        get_u32(card + 36) != (uint32_t)meta_of(L) || get_u32(card + 32) != (uint32_t)group_of(L) ||
+        (C.bits_mode != 0 && C.bits_mode != 1) || get_u64(card + 112) > card_bytes)
         return ORC_BAD_CARD;
     const int d = C.head_dim, H = C.n_kv_heads, per_kv = n_q_heads / H;
     const int64_t T = C.n_tokens;
@@ -741,11 +792,11 @@ static int attend_over_card(const uint8_t *card, uint64_t card_bytes, const orc_
         const uint8_t *vs = card + stream_base(card, &C, stream_index(&C, l, 1, h));
         for (int64_t t = 0; t < T; ++t) {
             if (fp16_rounded) {
-                injected_record(ks + off[t], d, bits[t], meta_of(&C), kx + t * d);
-                injected_record(vs + off[t], d, bits[t], meta_of(&C), vx + t * d);
+                injected_record(ks + off[t], d, bits[t], meta_of(&C), group_of(&C), kx + t * d);
+                injected_record(vs + off[t], d, bits[t], meta_of(&C), group_of(&C), vx + t * d);
             } else {
-                reconstruct_record(ks + off[t], d, bits[t], meta_of(&C), kx + t * d);
-                reconstruct_record(vs + off[t], d, bits[t], meta_of(&C), vx + t * d);
+                reconstruct_record(ks + off[t], d, bits[t], meta_of(&C), group_of(&C), kx + t * d);
+                reconstruct_record(vs + off[t], d, bits[t], meta_of(&C), group_of(&C), vx + t * d);
             }
         }
         for (int jj = 0; jj < per_kv; ++jj) {

@@ -115,10 +115,10 @@ def status_string(status: int) -> str:
 
 def make_layout(n_layers: int, n_kv_heads: int, head_dim: int, n_tokens: int, bits_mode: int = 0,
                 head_stride: Optional[int] = None, token_stride: Optional[int] = None,
-                meta_bytes: int = 8) -> Layout:
+                meta_bytes: int = 8, group_size: int = 32) -> Layout:
     ts = head_dim if token_stride is None else token_stride
     hs = n_tokens * ts if head_stride is None else head_stride
-    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, 32, bits_mode, hs, ts, meta_bytes, 0)
+    return Layout(n_layers, n_kv_heads, head_dim, n_tokens, group_size, bits_mode, hs, ts, meta_bytes, 0)
 
 
 def layout_of(tensors: Sequence, n_tokens: Optional[int] = None, bits_mode: int = 0,

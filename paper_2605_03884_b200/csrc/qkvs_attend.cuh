@@ -496,6 +496,7 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
         hp.head_dim = kAttendD;
         hp.n_tokens = p.n_tokens;
         hp.meta_bytes = META;
+        hp.group_size = kGroup;
         const uint32_t mode = hdr->bits_mode;
         int ok = 0;
         if (mode <= 1u) {

@@ -51,6 +51,7 @@ namespace qkvs {
 constexpr int kTcItemTokens = 512;
 constexpr int kTcSlotTokens = 32;                   // tokens per slot; FP16 rows take half a slot
 constexpr int kTcMaxSlots = 36;                     // 509 FP16 rows and one of each other width: 32 + 3, rounded up to tiles
+constexpr int kTcMaxTiles = kTcMaxSlots / 4;
 constexpr int kTcRawBytes = kTcSlotTokens * kAttendRecMax;  // 5120: 32 eight-bit records, or 16 FP16 rows
 constexpr int kTcRing = 3;
 constexpr int kTcPipes = 2;
@@ -66,7 +67,9 @@ struct TcItem {
     uint32_t item;       // index of the item, or n_items when there is none
     uint32_t n_slots;
     uint64_t base_k, base_v;          // byte offsets inside the card of the item's first record in the two streams
-    uint32_t slots[kTcMaxSlots];      // per slot: first list position | tokens << 10 | class << 16 | neighbours << 18
+    uint32_t slots[kTcMaxSlots];      // per slot: first list position | tokens << 10 | class << 16 | neighbours << 18 |
+                                      // (where the slot's records start in the tile's buffer, in 16-byte units) << 20
+    uint32_t tiles[kTcMaxTiles];      // per tile: (bytes of its records >> 4) << 1 | the whole tile is one run of neighbours
     uint16_t list[kTcItemTokens];     // the item's tokens grouped by bit-width: record offsets from the item's first, in 16-byte units
     float qsum[4][8];                 // sums of the item's queries over a group of channels, per head
     float sums[8 + 4 * 8];            // what the token threads add up: l[h], then zero-point sums [group][head]
@@ -74,11 +77,11 @@ struct TcItem {
 };
 
 struct TcPipeSmem {
-    alignas(128) uint8_t raw[4][kTcRing][kTcRawBytes];  // per token warp: records of a slot, packed in list order
+    alignas(128) uint8_t raw[kTcRing][4 * kTcRawBytes]; // records of a tile: its slots one after another, each packed in list order
     alignas(128) uint8_t a2[128 * kAttendD * 2];        // V codes as FP16, [token][channel], MN-major core matrices
     alignas(128) uint8_t w[128 * 32 * 2];               // weights, [token][(group, head)], MN-major core matrices
     TcItem items[2];
-    alignas(8) uint64_t full[4][kTcRing];               // a ring buffer's bytes have landed
+    alignas(8) uint64_t full[kTcRing];                  // a ring buffer's bytes have landed
     uint64_t a_ready, w_ready;                          // the token warps have stored A / W (and a2) of a tile
     uint64_t s_full, o_done;                            // the tensor cores have finished the scores / the outputs of a tile
     uint64_t item_ready[2], item_done[2];
@@ -109,6 +112,7 @@ __device__ __forceinline__ bool tokens_any(int pipe, bool pred)
 __device__ __forceinline__ uint32_t tc_slot_first(uint32_t d) { return d & 1023u; }
 __device__ __forceinline__ int tc_slot_count(uint32_t d) { return (int)((d >> 10) & 63u); }
 __device__ __forceinline__ int tc_slot_class(uint32_t d) { return (int)((d >> 16) & 3u); }
+__device__ __forceinline__ uint32_t tc_slot_raw(uint32_t d) { return (d >> 20) << 4; }
 
 // The 32 channels of group g of one token as 16 FP16 pairs: e[4 j + k] = (channel 8 j + k,
 // channel 8 j + k + 4) inside the group -- codes for a quantised row, the values themselves for a
@@ -194,34 +198,49 @@ __device__ __forceinline__ void store_value_row(const uint8_t *rec, uint8_t *row
     }
 }
 
-// Starts one load of a token warp's ring: the K or V records of a slot, packed in list order into
-// `dst`; `bar` completes when the bytes are there (at once for an empty slot).  Called by all
-// lanes of the driver warp.
+// Starts the copy of one tile's K or V records into a ring buffer: its slots one after another,
+// each packed in list order.  One bulk copy when the whole tile is a run of neighbours in the
+// card, else one per slot of neighbours and 16-byte asynchronous pieces for the scattered ones;
+// `bar` completes when all bytes are there.  Called by all lanes of the driver warp.
 template <int META>
-__device__ __forceinline__ void tc_issue(uint8_t *dst, uint64_t *bar, uint32_t d, const uint16_t *list, uint64_t base,
-                                         const AttendParams &p, int lane)
+__device__ __forceinline__ void tc_issue_tile(uint8_t *dst, uint64_t *bar, const TcItem &it, uint32_t tile, uint64_t base,
+                                              const AttendParams &p, int lane)
 {
-    const int n = tc_slot_count(d);
-    if (n == 0) {
-        if (lane == 0) mbar_arrive(bar);
+    const uint32_t info = it.tiles[tile];
+    if (info & 1u) {
+        if (lane == 0) {
+            const uint32_t bytes = (info >> 1) << 4;
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_load(dst, p.card + base + ((uint32_t)it.list[tc_slot_first(it.slots[4u * tile])] << 4), bytes, bar);
+        }
         return;
     }
-    const uint32_t rec = class_record_bytes<META>(tc_slot_class(d));
-    if (d & (1u << 18)) {
-        if (lane == 0) {
-            mbar_arrive_expect_tx(bar, (uint32_t)n * rec);
-            bulk_load(dst, p.card + base + ((uint32_t)list[tc_slot_first(d)] << 4), (uint32_t)n * rec, bar);
+    uint32_t bulk_bytes = 0;
+    for (uint32_t w = 0; w < 4; ++w) {
+        const uint32_t slot = 4u * tile + w;
+        const uint32_t d = slot < it.n_slots ? it.slots[slot] : 0u;
+        const int n = tc_slot_count(d);
+        if (n == 0) continue;
+        const uint32_t rec = class_record_bytes<META>(tc_slot_class(d));
+        uint8_t *to = dst + tc_slot_raw(d);
+        if (d & (1u << 18)) {
+            if (lane == 0) bulk_load(to, p.card + base + ((uint32_t)it.list[tc_slot_first(d)] << 4), (uint32_t)n * rec, bar);
+            bulk_bytes += (uint32_t)n * rec;
+        } else {
+            const uint32_t pieces = rec >> 4, total = (uint32_t)n * pieces;  // at most 320
+            const uint32_t inv = 65536u / pieces + 1u;                       // i / pieces == (i * inv) >> 16 for i < 4096
+            for (uint32_t i = (uint32_t)lane; i < total; i += 32u) {
+                const uint32_t r = (i * inv) >> 16;
+                async_copy_16(to + (i << 4), p.card + base + (((uint32_t)it.list[tc_slot_first(d) + r] + (i - r * pieces)) << 4));
+            }
         }
-    } else {
-        const uint32_t pieces = rec >> 4, total = (uint32_t)n * pieces;  // at most 320
-        const uint32_t inv = 65536u / pieces + 1u;                       // i / pieces == (i * inv) >> 16 for i < 4096
-        for (uint32_t i = (uint32_t)lane; i < total; i += 32u) {
-            const uint32_t r = (i * inv) >> 16;
-            async_copy_16(dst + (i << 4), p.card + base + (((uint32_t)list[tc_slot_first(d) + r] + (i - r * pieces)) << 4));
-        }
-        async_copies_arrive_on(bar);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar);
+    }
+    // the barrier's one arrival comes last: bytes that land before it cannot complete the phase
+    async_copies_arrive_on(bar);
+    __syncwarp();
+    if (lane == 0) {
+        if (bulk_bytes) mbar_arrive_expect_tx(bar, bulk_bytes);
+        else mbar_arrive(bar);
     }
 }
 
@@ -232,13 +251,73 @@ struct TcCard {
     uint64_t stream_bytes, total_bytes;
 };
 
-// Driver warp: reads, checks and sorts the tables of `item` into buffer `it`, lays out its slots,
-// writes its queries as the B operand of the score product and their sums.  32 lanes, 16
-// consecutive tokens each.
-template <int META>
-__device__ __forceinline__ void tc_prepare(TcItem &it, uint32_t item, const AttendParams &p, const TcCard &cd, int lane)
+// Driver warp, preparing an item in two steps so that the memory latency falls between them.
+// tc_fetch starts the reads (the item's table entries, 16 consecutive tokens per lane, and its
+// queries) and keeps the results in registers; tc_finish, called a tile's worth of work later,
+// checks and sorts the entries into buffer `it`, lays out its slots and tiles, and writes the
+// queries as the B operand of the score product, and their sums.
+struct TcFetch {
+    static constexpr int PER = kTcItemTokens / 32;
+    uint32_t item;           // n_items when there is none
+    uint32_t layer, head;
+    int n_tok;
+    uint64_t base_k, base_v;
+    uint32_t o_first;
+    uint32_t offs[PER + 1];
+    uint32_t bits[PER];
+    uint4 q[4];
+};
+
+__device__ __forceinline__ void tc_fetch(TcFetch &f, uint32_t item, const AttendParams &p, const TcCard &cd, int lane)
 {
-    if (item >= p.n_items) {
+    f.item = min(item, p.n_items);
+    if (item >= p.n_items) return;
+    const uint32_t H = (uint32_t)p.n_kv_heads;
+    const int per_kv = p.n_q_heads / p.n_kv_heads;
+    const uint64_t T = (uint64_t)p.n_tokens;
+    const uint32_t lh = item / p.items_per_head, ck = item - lh * p.items_per_head;
+    f.layer = lh / H;
+    f.head = lh - f.layer * H;
+    const uint64_t tok0 = (uint64_t)ck * kTcItemTokens;
+    f.n_tok = (int)min((uint64_t)kTcItemTokens, T - tok0);
+    const uint64_t seg = cd.mode == 0 ? 0u : lh;
+    const uint8_t *bits_tab = p.card + cd.sec.bits_off + seg * T + tok0;
+    const uint32_t *offs_tab = reinterpret_cast<const uint32_t *>(p.card + cd.sec.offs_off) + seg * (T + 1u) + tok0;
+    const uint64_t stream_k = ((uint64_t)f.layer * 2u) * H + f.head, stream_v = stream_k + H;
+    if (cd.mode == 0) {
+        f.base_k = cd.sec.payload_off + stream_k * cd.stream_bytes;
+        f.base_v = cd.sec.payload_off + stream_v * cd.stream_bytes;
+    } else {
+        // entries beyond the card (a damaged table) must not wrap the sums around
+        const uint64_t *sbase = reinterpret_cast<const uint64_t *>(p.card + cd.sec.sbase_off);
+        const uint64_t sk = __ldg(sbase + stream_k), sv = __ldg(sbase + stream_v);
+        f.base_k = sk > cd.total_bytes ? ~uint64_t(0) : cd.sec.payload_off + sk;
+        f.base_v = sv > cd.total_bytes ? ~uint64_t(0) : cd.sec.payload_off + sv;
+    }
+    f.o_first = __ldg(offs_tab);
+#pragma unroll
+    for (int r = 0; r <= TcFetch::PER; ++r) {
+        const int j = TcFetch::PER * lane + r;
+        f.offs[r] = j <= f.n_tok ? __ldg(offs_tab + j) : 0u;
+    }
+#pragma unroll
+    for (int r = 0; r < TcFetch::PER; ++r) {
+        const int j = TcFetch::PER * lane + r;
+        f.bits[r] = j < f.n_tok ? (uint32_t)__ldg(bits_tab + j) : 0u;
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int h = lane / 16 + 2 * r;
+        f.q[r] = make_uint4(0u, 0u, 0u, 0u);
+        if (h < per_kv)
+            f.q[r] = __ldg(reinterpret_cast<const uint4 *>(p.q + ((uint64_t)f.layer * p.n_q_heads + (uint64_t)f.head * per_kv + h) * kAttendD) + lane % 16);
+    }
+}
+
+template <int META>
+__device__ __forceinline__ void tc_finish(TcItem &it, const TcFetch &f, const AttendParams &p, const TcCard &cd, int lane)
+{
+    if (f.item >= p.n_items) {
         if (lane == 0) {
             it.item = p.n_items;
             it.n_slots = 0;
@@ -246,28 +325,9 @@ __device__ __forceinline__ void tc_prepare(TcItem &it, uint32_t item, const Atte
         __syncwarp();
         return;
     }
-    const uint32_t H = (uint32_t)p.n_kv_heads;
-    const int per_kv = p.n_q_heads / p.n_kv_heads;
-    const uint64_t T = (uint64_t)p.n_tokens;
-    const uint32_t lh = item / p.items_per_head, ck = item - lh * p.items_per_head;
-    const uint32_t layer = lh / H, head = lh - layer * H;
-    const uint64_t tok0 = (uint64_t)ck * kTcItemTokens;
-    const int n_tok = (int)min((uint64_t)kTcItemTokens, T - tok0);
-    const uint64_t seg = cd.mode == 0 ? 0u : lh;
-    const uint8_t *bits_tab = p.card + cd.sec.bits_off + seg * T + tok0;
-    const uint32_t *offs_tab = reinterpret_cast<const uint32_t *>(p.card + cd.sec.offs_off) + seg * (T + 1u) + tok0;
-    const uint64_t stream_k = ((uint64_t)layer * 2u) * H + head, stream_v = stream_k + H;
-    uint64_t base_k, base_v;
-    if (cd.mode == 0) {
-        base_k = cd.sec.payload_off + stream_k * cd.stream_bytes;
-        base_v = cd.sec.payload_off + stream_v * cd.stream_bytes;
-    } else {
-        // entries beyond the card (a damaged table) must not wrap the sums around
-        const uint64_t *sbase = reinterpret_cast<const uint64_t *>(p.card + cd.sec.sbase_off);
-        const uint64_t sk = __ldg(sbase + stream_k), sv = __ldg(sbase + stream_v);
-        base_k = sk > cd.total_bytes ? ~uint64_t(0) : cd.sec.payload_off + sk;
-        base_v = sv > cd.total_bytes ? ~uint64_t(0) : cd.sec.payload_off + sv;
-    }
+    const uint32_t item = f.item;
+    const int n_tok = f.n_tok;
+    const uint64_t base_k = f.base_k, base_v = f.base_v;
     const bool base_ok = base_k >= cd.sec.payload_off && base_v >= cd.sec.payload_off && ((base_k | base_v) & 15u) == 0u &&
                          base_k <= cd.total_bytes && base_v <= cd.total_bytes;
     const uint64_t room_k = base_ok ? cd.total_bytes - base_k : 0u, room_v = base_ok ? cd.total_bytes - base_v : 0u;
@@ -279,9 +339,7 @@ __device__ __forceinline__ void tc_prepare(TcItem &it, uint32_t item, const Atte
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const int h = lane / 16 + 2 * r;
-            uint4 qv = make_uint4(0u, 0u, 0u, 0u);
-            if (h < per_kv)
-                qv = __ldg(reinterpret_cast<const uint4 *>(p.q + ((uint64_t)layer * p.n_q_heads + (uint64_t)head * per_kv + h) * kAttendD) + ch);
+            const uint4 qv = f.q[r];
             *reinterpret_cast<uint4 *>(it.qb + ch * 256 + (h % 8) * 16) =
                 make_uint4(__byte_perm(qv.x, qv.z, 0x5410), __byte_perm(qv.x, qv.z, 0x7632), __byte_perm(qv.y, qv.w, 0x5410),
                            __byte_perm(qv.y, qv.w, 0x7632));
@@ -296,22 +354,20 @@ __device__ __forceinline__ void tc_prepare(TcItem &it, uint32_t item, const Atte
     }
 
     // ---- the tables: 16 consecutive tokens per lane
-    constexpr int PER = kTcItemTokens / 32;
+    constexpr int PER = TcFetch::PER;
     uint32_t my_off[PER];
     uint8_t my_cls[PER];
     uint32_t counts = 0, counts_hi = 0;  // 16-bit fields: (2 | 4 bits), (8 | 16 bits)
     bool bad = false;
-    const uint32_t o_first = __ldg(offs_tab);
-    uint32_t o_next = PER * lane <= n_tok ? __ldg(offs_tab + PER * lane) : 0u;
+    const uint32_t o_first = f.o_first;
 #pragma unroll
     for (int r = 0; r < PER; ++r) {
         const int j = PER * lane + r;
-        const uint32_t o = o_next;
-        o_next = j + 1 <= n_tok ? __ldg(offs_tab + j + 1) : 0u;
+        const uint32_t o = f.offs[r], o_next = f.offs[r + 1];
         my_off[r] = o;
         my_cls[r] = 4;
         if (j < n_tok) {
-            const uint32_t bw = __ldg(bits_tab + j);
+            const uint32_t bw = f.bits[r];
             const uint32_t rec = record_bytes(kAttendD, (int)bw, META);
             // also: inside the span an item's records can take from its first one, which is what a list entry can express
             const bool fine = base_ok && rec != 0u && o_next >= o && o_next - o == rec && (o & 15u) == 0u && o >= o_first &&
@@ -365,6 +421,25 @@ __device__ __forceinline__ void tc_prepare(TcItem &it, uint32_t item, const Atte
         begin = ends[c];
     }
     for (uint32_t s = n_slots + (uint32_t)lane; s < (uint32_t)kTcMaxSlots; s += 32u) it.slots[s] = 0u;
+    __syncwarp();
+    // ---- tiles: where each slot's records go in the tile's buffer, and whether the tile is one run
+    if (lane < kTcMaxTiles) {
+        uint32_t at = 0;          // bytes of the tile so far
+        bool run = true;
+        uint32_t follow = 0;      // list value the next slot's first record must have to continue the run
+        for (uint32_t w = 0; w < 4; ++w) {
+            const uint32_t slot = 4u * (uint32_t)lane + w;
+            if (slot >= n_slots) break;
+            const uint32_t d = it.slots[slot];
+            const uint32_t bytes = (uint32_t)tc_slot_count(d) * class_record_bytes<META>(tc_slot_class(d));
+            const uint32_t first = it.list[tc_slot_first(d)];
+            run = run && (d & (1u << 18)) != 0u && (w == 0 || first == follow);
+            follow = first + (bytes >> 4);
+            it.slots[slot] = d | ((at >> 4) << 20);
+            at += bytes;
+        }
+        it.tiles[lane] = ((at >> 4) << 1) | (run && at > 0u ? 1u : 0u);
+    }
     if (lane == 0) {
         it.item = item;
         it.n_slots = n_slots;
@@ -399,6 +474,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
         hp.head_dim = kAttendD;
         hp.n_tokens = p.n_tokens;
         hp.meta_bytes = META;
+        hp.group_size = kGroup;
         const uint32_t mode = hdr->bits_mode;
         int ok = 0;
         if (mode <= 1u) {
@@ -411,8 +487,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
         s_total_bytes = hdr->total_bytes;
     }
     if (is_driver && lane == 0) {
-        for (int w = 0; w < 4; ++w)
-            for (int s = 0; s < kTcRing; ++s) mbar_init(&sm.full[w][s], 1);
+        for (int s = 0; s < kTcRing; ++s) mbar_init(&sm.full[s], 1);
         mbar_init(&sm.a_ready, 4);
         mbar_init(&sm.w_ready, 4);
         mbar_init(&sm.s_full, 1);
@@ -460,28 +535,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
         bool ok = true;
 
         auto issue = [&](const TcItem &it, uint32_t tile, uint32_t kv, uint32_t flat) {
-            const uint32_t j = 2u * flat + kv, ring = j % kTcRing;   // the same load number in all four rings
-            for (uint32_t w = 0; w < 4; ++w) {
-                const uint32_t slot = 4u * tile + w;
-                const uint32_t d = slot < it.n_slots ? it.slots[slot] : 0u;
-                tc_issue<META>(sm.raw[w][ring], &sm.full[w][ring], d, it.list, kv ? it.base_v : it.base_k, p, lane);
-            }
+            const uint32_t ring = (2u * flat + kv) % kTcRing;   // loads are numbered K, V, K, V, ... over the pipeline's tiles
+            tc_issue_tile<META>(sm.raw[ring], &sm.full[ring], it, tile, kv ? it.base_v : it.base_k, p, lane);
         };
-        auto draw = [&]() -> uint32_t {
-            uint32_t v = 0;
-            if (lane == 0) v = atomicAdd(p.work_counter, 1u);
-            v = __shfl_sync(0xffffffffu, v, 0);
+        // The work counter is read one item ahead of its use: lane 0 keeps the raw result of the
+        // atomic in a register and nobody looks at it before the next item is finished.
+        uint32_t drawn_raw = 0;
+        auto draw_start = [&]() {
+            if (lane == 0) drawn_raw = atomicAdd(p.work_counter, 1u);
+        };
+        auto draw_result = [&]() -> uint32_t {
+            const uint32_t v = __shfl_sync(0xffffffffu, drawn_raw, 0);
             return v < p.n_items ? min(n_pipes + v, p.n_items) : p.n_items;
         };
 
-        // items 0 and 1 of this pipeline; from then on the item after the next is drawn while the
-        // next one is prepared, so that the counter's latency is never waited for
-        uint32_t idx_next = (uint32_t)(blockIdx.x * kTcPipes + pipe);
-        idx_next = min(idx_next, p.n_items);
-        tc_prepare<META>(sm.items[0], idx_next, p, cd, lane);
+        // item 0 of this pipeline is its own index; the following ones come from the counter
+        TcFetch fetch;
+        tc_fetch(fetch, (uint32_t)(blockIdx.x * kTcPipes + pipe), p, cd, lane);
+        draw_start();
+        tc_finish<META>(sm.items[0], fetch, p, cd, lane);
         if (lane == 0) mbar_arrive(&sm.item_ready[0]);
-        idx_next = draw();
-        uint32_t idx_after = p.n_items;
+        uint32_t idx_next = draw_result();   // index of item k + 1, known at the top of item k
 
         for (uint32_t k = 0; ok; ++k) {
             const uint32_t b = k & 1u;
@@ -489,15 +563,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
             if (it.item >= p.n_items) break;
             const uint32_t nt = (it.n_slots + 3u) / 4u;
             bool next_prepared = false;
+            // the reads for the next item start now and are used a tile later; so does the draw of
+            // the item after it
+            tc_fetch(fetch, idx_next, p, cd, lane);
+            if (idx_next < p.n_items) draw_start();
             auto prepare_next = [&]() {
                 // buffer b ^ 1 held item k - 1: the token warps must be done with it
                 if (k >= 1) ok = ok && mbar_wait_short(&sm.item_done[b ^ 1u], ((k - 1u) >> 1) & 1u);
                 ok = __all_sync(0xffffffffu, ok);
                 if (ok) {
-                    if (k >= 1) idx_next = idx_after;
-                    tc_prepare<META>(sm.items[b ^ 1u], idx_next, p, cd, lane);
+                    tc_finish<META>(sm.items[b ^ 1u], fetch, p, cd, lane);
                     if (lane == 0) mbar_arrive(&sm.item_ready[b ^ 1u]);
-                    idx_after = idx_next < p.n_items ? draw() : p.n_items;
+                    idx_next = idx_next < p.n_items ? draw_result() : p.n_items;
                 }
                 next_prepared = true;
             };
@@ -538,16 +615,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
                     tc_commit(&sm.s_full);
                 }
                 __syncwarp();
-                // the K buffers of this tile are free: the V records of the following tile go there
-                if (t == 0 && !next_prepared) {
-                    prepare_next();
-                    if (!ok) break;
-                    if (t + 1 >= nt && sm.items[b ^ 1u].item < p.n_items && sm.items[b ^ 1u].n_slots > 0) nx = &sm.items[b ^ 1u];
-                }
-                if (nx && k_issued == n + 1) {
-                    issue(*nx, nx_tile, 0u, n + 1);
-                    ++k_issued;
-                }
+                // the K buffer of this tile is free: the V records of the following tile go there
                 if (nx && v_issued == n + 1 && k_issued == n + 2) {
                     issue(*nx, nx_tile, 1u, n + 1);
                     ++v_issued;
@@ -565,6 +633,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
                 }
                 __syncwarp();
                 ++n;
+                // the next item's tables have had a tile's time to arrive
+                if (t == 0) {
+                    prepare_next();
+                    if (!ok) break;
+                }
             }
         }
         if (!ok) {
@@ -576,7 +649,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
         {
             const int last = max(2 * (int)k_issued - 2, 2 * (int)v_issued - 1);
             for (int j = last; j > last - kTcRing && j >= 0; --j)
-                for (uint32_t w = 0; w < 4; ++w) mbar_wait(&sm.full[w][(uint32_t)j % kTcRing], ((uint32_t)j / kTcRing) & 1u);
+                mbar_wait(&sm.full[(uint32_t)j % kTcRing], ((uint32_t)j / kTcRing) & 1u);
         }
     } else {
         // =====================================================================================
@@ -613,8 +686,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
                 // ---- K: codes -> this token's row of the A operand in tensor memory
                 {
                     const uint32_t j = 2u * n, ring = j % kTcRing;
-                    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[warp][ring], (j / kTcRing) & 1u));
-                    const uint8_t *rec = sm.raw[warp][ring] + (present ? lane : 0) * class_record_bytes<META>(cls);
+                    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[ring], (j / kTcRing) & 1u));
+                    const uint8_t *rec = sm.raw[ring] + tc_slot_raw(d) + (present ? lane : 0) * class_record_bytes<META>(cls);
                     if (ok && cnt > 0) {
                         switch (cls) {
                             case 0: store_key_row<2, META>(rec, tm_row + kTcColA, ksc, kze); break;
@@ -635,8 +708,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
                 {
                     if (ok && n > 0) ok = __all_sync(0xffffffffu, mbar_wait_short(&sm.o_done, (n - 1u) & 1u));  // the last product has read a2 and w
                     const uint32_t j = 2u * n + 1u, ring = j % kTcRing;
-                    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[warp][ring], (j / kTcRing) & 1u));
-                    const uint8_t *rec = sm.raw[warp][ring] + (present ? lane : 0) * class_record_bytes<META>(cls);
+                    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sm.full[ring], (j / kTcRing) & 1u));
+                    const uint8_t *rec = sm.raw[ring] + tc_slot_raw(d) + (present ? lane : 0) * class_record_bytes<META>(cls);
                     uint8_t *row = sm.a2 + (ptid >> 3) * 2048 + (ptid & 7) * 16;
                     if (ok && present) {
                         switch (cls) {

@@ -276,10 +276,13 @@ struct CreateWarpSmem {
 // 16-byte bank columns; the packed codes are put back in channel order before they are stored.
 // `rec` is the row's record in the card.  B is the warp-uniform bit-width, or 0 when rows
 // differ (then `b`); META the bytes of {scale, zero} per group.
-template <int D, int B, int META>
-__device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *rec, int lane, int g, int b)
+// GS: log2 of (channels per quantisation group / 32).  With wider groups the lanes that share a group
+// (2 or 4 neighbours of one row) combine their minima and maxima and all arrive at the same scale
+// and zero; `peers` names the lanes that run the quantiser (the shuffle's mask).
+template <int D, int B, int META, int GS>
+__device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *rec, int lane, int g, int b, unsigned peers)
 {
-    constexpr int G = D / kGroup;
+    constexpr int PAIRS = (int)pairs_bytes(D, META, kGroup << GS);
     const uint8_t *src = rows_in + lane * 64;
     const int rot = (lane >> 1) & 3;
     uint4 v[4];
@@ -293,11 +296,23 @@ __device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *re
     }
     float mn, mx;
     group_min_max(v, mn, mx);
+#pragma unroll
+    for (int s = 1; s < (1 << GS); s <<= 1) {
+        mn = fminf(mn, __shfl_xor_sync(peers, mn, s));
+        mx = fmaxf(mx, __shfl_xor_sync(peers, mx, s));
+    }
     const GroupParams gp = group_params<META>(mn, mx, bb);
-    if (META == kMetaFp16)  // both are FP16 values: the conversion is exact
-        __stcs(reinterpret_cast<uint32_t *>(rec + g * META), as_u32(__floats2half2_rn(gp.scale, gp.zero)));
-    else
-        __stcs(reinterpret_cast<float2 *>(rec + g * META), make_float2(gp.scale, gp.zero));
+    if ((g & ((1 << GS) - 1)) == 0) {  // one lane per group stores the pair
+        if (META == kMetaFp16)  // both are FP16 values: the conversion is exact
+            __stcs(reinterpret_cast<uint32_t *>(rec + (g >> GS) * META), as_u32(__floats2half2_rn(gp.scale, gp.zero)));
+        else
+            __stcs(reinterpret_cast<float2 *>(rec + (g >> GS) * META), make_float2(gp.scale, gp.zero));
+    }
+    if (GS > 0 && g == 0) {  // the zero bytes between the pairs and the codes
+        constexpr int USED = (D >> (5 + GS)) * META;
+#pragma unroll
+        for (int o = USED; o < PAIRS; o += 4) __stcs(reinterpret_cast<uint32_t *>(rec + o), 0u);
+    }
     const uint64_t inv2 = pack_f32x2(gp.inv, gp.inv);
     uint32_t lo[4], hi[4];
 #pragma unroll
@@ -307,7 +322,7 @@ __device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *re
         pack_chunk<B>(f, bb, lo[c], hi[c]);
     }
     unrotate4(lo, rot);
-    uint8_t *codes = rec + G * META + g * (4 * bb);  // 32 codes of b bits = 4b bytes
+    uint8_t *codes = rec + PAIRS + g * (4 * bb);  // 32 codes of b bits = 4b bytes
     if (bb == 8) {
         unrotate4(hi, rot);
         __stcs(reinterpret_cast<uint4 *>(codes), make_uint4(lo[0], hi[0], lo[1], hi[1]));
@@ -320,7 +335,7 @@ __device__ __forceinline__ void encode_group(const uint8_t *rows_in, uint8_t *re
 }
 
 // All U passes of a sub-tile.  Every lane of the warp calls this (it shuffles).
-template <int D, int B, int META>
+template <int D, int B, int META, int GS>
 __device__ __forceinline__ void encode_rows(const uint8_t *in, uint8_t *stream, const Tables &t, int lane)
 {
     using C = WarpCfg<D>;
@@ -330,8 +345,9 @@ __device__ __forceinline__ void encode_rows(const uint8_t *in, uint8_t *stream, 
         const int row = u * C::R + lrow;
         const uint32_t off_row = __shfl_sync(0xffffffffu, t.off, row);
         const int b = B ? B : (int)__shfl_sync(0xffffffffu, t.bits, row);
-        if (lane < C::GROUPS && row < t.rows)
-            encode_group<D, B, META>(in + u * (C::R * C::ROW_BYTES), stream + off_row, lane, g, b);
+        const bool mine = lane < C::GROUPS && row < t.rows;
+        const unsigned peers = GS > 0 ? __ballot_sync(0xffffffffu, mine && b != 16) : 0u;
+        if (mine) encode_group<D, B, META, GS>(in + u * (C::R * C::ROW_BYTES), stream + off_row, lane, g, b, peers);
     }
 }
 
@@ -354,7 +370,7 @@ __device__ __forceinline__ void create_issue(CreateWarpSmem<D, NS> &sm, int stag
     }
 }
 
-template <int D, int NS, int WARPS, int META>
+template <int D, int NS, int WARPS, int META, int GS>
 __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) create_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
@@ -422,13 +438,13 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) create_kernel(Pa
         uint8_t *stream = p.card + cur.base;
         if (uniform) {
             switch (b0) {
-                case 4: encode_rows<D, 4, META>(in, stream, cur, lane); break;
-                case 2: encode_rows<D, 2, META>(in, stream, cur, lane); break;
-                case 8: encode_rows<D, 8, META>(in, stream, cur, lane); break;
-                default: encode_rows<D, 16, META>(in, stream, cur, lane); break;
+                case 4: encode_rows<D, 4, META, GS>(in, stream, cur, lane); break;
+                case 2: encode_rows<D, 2, META, GS>(in, stream, cur, lane); break;
+                case 8: encode_rows<D, 8, META, GS>(in, stream, cur, lane); break;
+                default: encode_rows<D, 16, META, GS>(in, stream, cur, lane); break;
             }
         } else {
-            encode_rows<D, 0, META>(in, stream, cur, lane);
+            encode_rows<D, 0, META, GS>(in, stream, cur, lane);
         }
         __syncwarp();  // every lane has read the stage: it can be re-armed
         if (!ahead.cu.done) {
@@ -476,16 +492,16 @@ struct InjectWarpSmem {
 // are applied by selection -- so that lanes of different widths do not serialise; only FP16 rows
 // branch off.  META: bytes of {scale, zero} per group (the code bytes start 16-byte aligned either
 // way, see qkvs_card_create).
-template <int D, int B, int META>
+template <int D, int B, int META, int GS>
 __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos)
 {
-    constexpr int G = D / kGroup;
+    constexpr int PAIRS = (int)pairs_bytes(D, META, kGroup << GS);
     const int bb = B ? B : b;
     if (bb == 16) return *reinterpret_cast<const uint4 *>(rec + pos * 16);
     float2 m;
-    if (META == kMetaFp16) m = __half22float2(*reinterpret_cast<const __half2 *>(rec + (pos >> 2) * META));
-    else m = *reinterpret_cast<const float2 *>(rec + (pos >> 2) * META);
-    const uint8_t *codes = rec + G * META + pos * bb;
+    if (META == kMetaFp16) m = __half22float2(*reinterpret_cast<const __half2 *>(rec + (pos >> (2 + GS)) * META));
+    else m = *reinterpret_cast<const float2 *>(rec + (pos >> (2 + GS)) * META);
+    const uint8_t *codes = rec + PAIRS + pos * bb;
     uint32_t lo, hi;
     if (B == 8) {
         const uint2 w = *reinterpret_cast<const uint2 *>(codes);
@@ -511,7 +527,7 @@ __device__ __forceinline__ uint4 decode_chunk(const uint8_t *rec, int b, int pos
 }
 
 // FULL: the sub-tile has all ROWS rows and every lane has a chunk in every pass.
-template <int D, int NS, int B, bool FULL, int META>
+template <int D, int NS, int B, bool FULL, int META, int GS>
 __device__ __forceinline__ void inject_rows(const InjectWarpSmem<D, NS> &sm, int stage, int lane, int rows, __half *dst0,
                                             int64_t token_stride)
 {
@@ -523,7 +539,7 @@ __device__ __forceinline__ void inject_rows(const InjectWarpSmem<D, NS> &sm, int
         const int row = ci / C::CPR, pos = ci % C::CPR;
         if (FULL || (ci < C::CHUNKS && row < rows)) {
             const uint32_t inf = sm.info[stage][row];
-            const uint4 out = decode_chunk<D, B, META>(in + (inf >> 8), (int)(inf & 0xffu), pos);
+            const uint4 out = decode_chunk<D, B, META, GS>(in + (inf >> 8), (int)(inf & 0xffu), pos);
             __stcs(reinterpret_cast<uint4 *>(dst0 + (int64_t)row * token_stride + pos * 8), out);
         }
     }
@@ -536,7 +552,7 @@ __device__ __forceinline__ bool header_matches(const qkvs_card_header_t *h, cons
 {
     bool ok = h->magic == kMagic && h->version == kVersion && h->status == QKVS_OK;
     ok = ok && h->n_layers == p.n_layers && h->n_kv_heads == p.n_kv_heads && h->head_dim == p.head_dim;
-    ok = ok && h->n_tokens == p.n_tokens && h->group_size == kGroup && h->meta_bytes_per_group == (uint32_t)p.meta_bytes;
+    ok = ok && h->n_tokens == p.n_tokens && h->group_size == p.group_size && h->meta_bytes_per_group == (uint32_t)p.meta_bytes;
     ok = ok && h->bits_off == sec.bits_off && h->offs_off == sec.offs_off && h->payload_off == sec.payload_off;
     ok = ok && h->sbase_off == sec.sbase_off;
     ok = ok && h->total_bytes <= p.card_bytes && h->total_bytes >= sec.payload_off;
@@ -563,7 +579,7 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
     const uint32_t b0 = __shfl_sync(0xffffffffu, t.bits, 0);
     int bad = 0;
     if (lane < rows) {
-        const uint32_t rec = record_bytes(D, (int)t.bits, p.meta_bytes);
+        const uint32_t rec = record_bytes(D, (int)t.bits, p.meta_bytes, p.group_size);
         bad = (rec == 0u) || (off_next < t.off) || (off_next - t.off != rec);
         sm.info[stage][lane] = ((t.off - off0) << 8) | (t.bits & 0xffu);
     }
@@ -588,7 +604,7 @@ __device__ __forceinline__ void inject_issue(InjectWarpSmem<D, NS> &sm, int stag
     __syncwarp();
 }
 
-template <int D, int NS, int WARPS, int META>
+template <int D, int NS, int WARPS, int META, int GS>
 __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) inject_kernel(PathParams p, LayerPtrs ptrs)
 {
     using C = WarpCfg<D>;
@@ -659,14 +675,14 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_CTAS_PER_SM) inject_kernel(Pa
         __half *dst0 = cons.row;
         if (C::CHUNKS % 32 == 0 && rows == C::ROWS) {
             switch (ub) {
-                case 4: inject_rows<D, NS, 4, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                case 2: inject_rows<D, NS, 2, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                case 8: inject_rows<D, NS, 8, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                case 16: inject_rows<D, NS, 16, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
-                default: inject_rows<D, NS, 0, true, META>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 4: inject_rows<D, NS, 4, true, META, GS>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 2: inject_rows<D, NS, 2, true, META, GS>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 8: inject_rows<D, NS, 8, true, META, GS>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                case 16: inject_rows<D, NS, 16, true, META, GS>(sm, stage, lane, rows, dst0, p.token_stride); break;
+                default: inject_rows<D, NS, 0, true, META, GS>(sm, stage, lane, rows, dst0, p.token_stride); break;
             }
         } else {
-            inject_rows<D, NS, 0, false, META>(sm, stage, lane, rows, dst0, p.token_stride);
+            inject_rows<D, NS, 0, false, META, GS>(sm, stage, lane, rows, dst0, p.token_stride);
         }
         __syncwarp();  // every lane has read the stage: it can be re-armed
         if (more) {

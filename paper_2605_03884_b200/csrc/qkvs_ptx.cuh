@@ -70,14 +70,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return done != 0;
 }
 
-// The same poll without a suspend hint: the hardware's own (short) limit applies.  For barriers
-// that other threads of the CTA complete by arriving, where the waiter wants to go on at once.
+// A poll that never suspends the warp: it only tests whether the phase has completed.  For
+// barriers completed a few hundred cycles after the wait begins (by other warps of the CTA or by
+// the tensor cores), where the waiter wants to go on the moment that happens.
 __device__ __forceinline__ bool mbar_try_wait_short(uint64_t *bar, uint32_t parity)
 {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
         : "r"(smem_addr(bar)), "r"(parity)
@@ -104,14 +105,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, unsign
     }
 }
 
-// The same wait built on the short poll.
-__device__ __forceinline__ bool mbar_wait_short(uint64_t *bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs)
+// The same wait built on the short poll.  The limit is counted in SM clock cycles (reading the
+// cycle counter costs a few cycles, reading the nanosecond timer stalls the warp for far longer,
+// which would put that delay between the arrival and the moment the waiter notices it):
+// 4 * 10^9 cycles are at least two seconds at any clock this part runs at.
+constexpr long long kWaitLimitCycles = 4000000000ll;
+
+__device__ __forceinline__ bool mbar_wait_short(uint64_t *bar, uint32_t parity, long long limit_cycles = kWaitLimitCycles)
 {
     if (mbar_try_wait_short(bar, parity)) return true;
-    const unsigned long long start = global_timer_ns();
+    const long long start = clock64();
     for (;;) {
-        if (mbar_try_wait_short(bar, parity)) return true;
-        if (global_timer_ns() - start > limit_ns) return false;
+#pragma unroll 1
+        for (int i = 0; i < 8; ++i)
+            if (mbar_try_wait_short(bar, parity)) return true;
+        if (clock64() - start > limit_cycles) return false;
     }
 }
 

@@ -21,6 +21,7 @@
 namespace qkvs {
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelStaged = 8192;   // segments up to this many tokens are read once and kept in shared memory
 
 // Larger score -> larger key; +0 and -0 get the same key.
 __device__ __forceinline__ uint32_t order_key(float s)
@@ -33,7 +34,7 @@ __device__ __forceinline__ uint32_t order_key(float s)
 // One warp looks for the byte value d with  above(d) < need <= above(d) + h[d],  above(d) being
 // the sum of h over all larger byte values.  Returns d (or -1 when even the total is below need)
 // and above(d) through `above`.  All 32 lanes call it; the result is the same in all.
-__device__ __forceinline__ int pick_byte(const unsigned long long *h, unsigned long long need, unsigned long long &above, int lane)
+__device__ __forceinline__ int pick_byte(const uint32_t *h, unsigned long long need, unsigned long long &above, int lane)
 {
     unsigned long long mine = 0;
 #pragma unroll
@@ -95,9 +96,46 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan64(unsigned lo
     return scratch[warp] + inc - v;
 }
 
+// Adds `weight` to hist[digit] for every lane with `active` set.  When all active lanes of the
+// warp hold the same digit (few distinct scores, or the leading bits of a narrow range) one lane
+// adds for all; otherwise every lane adds for itself, and the digits being spread out keeps the
+// counters from colliding.  All 32 lanes call it together.
+__device__ __forceinline__ void hist_add(uint32_t *hist, uint32_t digit, uint32_t weight, bool active, int lane)
+{
+    const uint32_t who = __ballot_sync(0xffffffffu, active);
+    if (who == 0u) return;
+    const int leader = __ffs(who) - 1;
+    const uint32_t d0 = __shfl_sync(0xffffffffu, digit, leader);
+    if (__all_sync(0xffffffffu, !active || digit == d0)) {
+        if (lane == leader) atomicAdd(&hist[d0], weight * (uint32_t)__popc(who));
+    } else if (active) {
+        atomicAdd(&hist[digit], weight);
+    }
+}
+
+// Smallest and largest of one key per thread over the block (threads without a key pass
+// 0xffffffff / 0); `scratch` holds 64 entries of 32 bits.
+__device__ __forceinline__ void block_min_max(uint32_t &lo, uint32_t &hi, uint32_t *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    __syncthreads();
+    if (lane == 0) {
+        scratch[warp] = lo;
+        scratch[32 + warp] = hi;
+    }
+    __syncthreads();
+    const int n = (int)(blockDim.x >> 5);
+    uint32_t a = lane < n ? scratch[lane] : 0xffffffffu, b = lane < n ? scratch[32 + lane] : 0u;
+    lo = __reduce_min_sync(0xffffffffu, a);
+    hi = __reduce_max_sync(0xffffffffu, b);
+}
+
 struct SelectShared {
-    unsigned long long hist[3][256];
+    uint32_t hist[3][256];
     unsigned long long scratch[33];
+    uint32_t minmax[64];
     uint32_t prefix[3];
     unsigned long long need[3];
     uint32_t ties[3];
@@ -125,10 +163,15 @@ __global__ void __launch_bounds__(kSelThreads) bits_by_rank_kernel(const float *
                                                                     uint8_t *bits, uint32_t *offsets, int head_dim, int meta)
 {
     __shared__ SelectShared sh;
+    __shared__ float stage[kSelStaged];
     scores += (int64_t)blockIdx.x * T;
     bits += (int64_t)blockIdx.x * T;
     if (offsets) offsets += (int64_t)blockIdx.x * (T + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool staged = T <= kSelStaged;
+    if (staged)
+        for (int64_t t = tid; t < T; t += kSelThreads) stage[t] = scores[t];
+    auto score_at = [&](int64_t t) { return staged ? stage[t] : scores[t]; };
     const int64_t per = (T + kSelThreads - 1) / kSelThreads;
     const int64_t first = min(T, (int64_t)tid * per), last = min(T, first + per);
     // the three cuts: a token is in the top `cut` when fewer than `cut` tokens come before it
@@ -140,26 +183,41 @@ __global__ void __launch_bounds__(kSelThreads) bits_by_rank_kernel(const float *
         sh.prefix[tid] = 0u;
         sh.need[tid] = cut[tid];
     }
-    // ---- the key of the token of rank cut - 1, one byte per pass from the top
-    for (int pass = 3; pass >= 0; --pass) {
-        for (int i = tid; i < 3 * 256; i += kSelThreads) (&sh.hist[0][0])[i] = 0ull;
+    // ---- keys are taken relative to the smallest one, and only the bits in which they differ are
+    // walked: scores crowd into a few values of a float's leading byte, but spread evenly over the
+    // leading bits of their own range, so the counters of a pass are not all the same one
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    for (int64_t t = tid; t < T; t += kSelThreads) {
+        const uint32_t key = order_key(score_at(t));
+        kmin = min(kmin, key);
+        kmax = max(kmax, key);
+    }
+    block_min_max(kmin, kmax, sh.minmax);
+    const int nbits = 32 - __clz(kmax - kmin);   // 0 when all keys are equal
+    auto rel_key = [&](int64_t t) { return order_key(score_at(t)) - kmin; };
+    // ---- the key of the token of rank cut - 1, up to eight bits per pass from the top
+    for (int hi = nbits; hi > 0; hi -= 8) {
+        const int lo = max(hi - 8, 0);
+        const uint32_t digit_mask = (1u << (hi - lo)) - 1u;
+        for (int i = tid; i < 3 * 256; i += kSelThreads) (&sh.hist[0][0])[i] = 0u;
         __syncthreads();
-        const uint32_t hi_mask = pass == 3 ? 0u : 0xffffffffu << (8 * (pass + 1));
         uint32_t pf[3];
 #pragma unroll
         for (int j = 0; j < 3; ++j) pf[j] = sh.prefix[j];
-        for (int64_t t = first; t < last; ++t) {
-            const uint32_t key = order_key(scores[t]);
+        // counting does not care about the order: neighbouring threads read neighbouring scores
+        for (int64_t t0 = (int64_t)(tid - lane); t0 < T; t0 += kSelThreads) {
+            const int64_t t = t0 + lane;
+            const uint32_t key = t < T ? rel_key(t) : 0u;
 #pragma unroll
             for (int j = 0; j < 3; ++j)
-                if (active[j] && (key & hi_mask) == pf[j]) atomicAdd(&sh.hist[j][(key >> (8 * pass)) & 255u], 1ull);
+                if (active[j]) hist_add(sh.hist[j], (key >> lo) & digit_mask, 1u, t < T && (hi >= 32 || (key >> hi) == (pf[j] >> hi)), lane);
         }
         __syncthreads();
         if (warp < 3 && active[warp]) {
             unsigned long long above;
             const int dsel = pick_byte(sh.hist[warp], sh.need[warp], above, lane);
             if (lane == 0) {
-                sh.prefix[warp] |= (uint32_t)max(dsel, 0) << (8 * pass);
+                sh.prefix[warp] |= (uint32_t)max(dsel, 0) << lo;
                 sh.need[warp] -= above;
             }
         }
@@ -176,14 +234,14 @@ __global__ void __launch_bounds__(kSelThreads) bits_by_rank_kernel(const float *
     // ---- equal keys by index: how many tokens with the cut's key lie in front of this thread's run
     unsigned long long packed = 0;  // three counts of 21 bits (T <= 2^20)
     for (int64_t t = first; t < last; ++t) {
-        const uint32_t key = order_key(scores[t]);
+        const uint32_t key = rel_key(t);
 #pragma unroll
         for (int j = 0; j < 3; ++j) packed += (unsigned long long)(active[j] && key == tau[j]) << (21 * j);
     }
     unsigned long long total;
     unsigned long long before = block_exclusive_scan64(packed, sh.scratch, total);
     for (int64_t t = first; t < last; ++t) {
-        const uint32_t key = order_key(scores[t]);
+        const uint32_t key = rel_key(t);
         bool top[3];
 #pragma unroll
         for (int j = 0; j < 3; ++j) {
@@ -218,6 +276,7 @@ struct BudgetParams {
 __global__ void __launch_bounds__(kSelThreads) bits_by_budget_kernel(BudgetParams p)
 {
     __shared__ SelectShared sh;
+    __shared__ float stage[kSelStaged];
     __shared__ unsigned long long s_left;
     __shared__ int s_bad;
     const float *scores = p.scores + (int64_t)blockIdx.x * p.T;
@@ -234,36 +293,52 @@ __global__ void __launch_bounds__(kSelThreads) bits_by_budget_kernel(BudgetParam
         s_bad = 0;
         sh.ties[0] = sh.ties[1] = sh.ties[2] = 0u;
     }
-    auto key_of = [&](float s, int i) { return order_key(__fmul_rn(s == 0.0f ? 0.0f : s, p.weight[i])); };
-    // ---- the key at which the budget runs out, one byte per pass from the top (sums of costs)
-    for (int pass = 3; pass >= 0; --pass) {
-        for (int i = tid; i < 256; i += kSelThreads) sh.hist[0][i] = 0ull;
+    const bool staged = T <= kSelStaged;
+    if (staged)
+        for (int64_t t = tid; t < T; t += kSelThreads) stage[t] = scores[t];
+    auto score_at = [&](int64_t t) { return staged ? stage[t] : scores[t]; };
+    __syncthreads();   // the flags above are set before anybody raises one
+    auto abs_key = [&](float s, int i) { return order_key(__fmul_rn(s == 0.0f ? 0.0f : s, p.weight[i])); };
+    // keys relative to the smallest one, walked over the bits in which they differ (see the rank rule)
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+    bool bad = false;
+    for (int64_t t = tid; t < T; t += kSelThreads) {
+        const float s = score_at(t);
+        bad |= !(s >= 0.0f) || s > 3.0e38f;
+        kmin = min(kmin, abs_key(s, 2));    // weights do not increase with the rung
+        kmax = max(kmax, abs_key(s, 0));
+    }
+    if (bad) s_bad = 1;
+    block_min_max(kmin, kmax, sh.minmax);
+    const int nbits = 32 - __clz(kmax - kmin);
+    auto key_of = [&](float s, int i) { return abs_key(s, i) - kmin; };
+    if (tid == 0 && (unsigned long long)T * (p.cost[0] + p.cost[1] + p.cost[2]) <= s_left) sh.take_all = 1;  // everything fits: all tokens keep FP16
+    __syncthreads();
+    // ---- the key at which the budget runs out, up to eight bits per pass from the top (sums of costs)
+    for (int hi = sh.take_all ? 0 : nbits; hi > 0; hi -= 8) {
+        const int lo = max(hi - 8, 0);
+        const uint32_t digit_mask = (1u << (hi - lo)) - 1u;
+        for (int i = tid; i < 256; i += kSelThreads) sh.hist[0][i] = 0u;
         __syncthreads();
-        if (sh.take_all) break;
-        const uint32_t hi_mask = pass == 3 ? 0u : 0xffffffffu << (8 * (pass + 1));
         const uint32_t pf = sh.prefix[0];
-        bool bad = false;
-        for (int64_t t = first; t < last; ++t) {
-            const float s = scores[t];
-            bad |= !(s >= 0.0f) || s > 3.0e38f;
+        // sums of costs per digit (at most 2^20 tokens * 512 bytes: 32 bits hold them); the order
+        // does not matter here, so neighbouring threads read neighbouring scores
+        for (int64_t t0 = (int64_t)(tid - lane); t0 < T; t0 += kSelThreads) {
+            const int64_t t = t0 + lane;
+            const float s = t < T ? score_at(t) : 0.0f;
 #pragma unroll
             for (int i = 0; i < 3; ++i) {
                 const uint32_t key = key_of(s, i);
-                if ((key & hi_mask) == pf) atomicAdd(&sh.hist[0][(key >> (8 * pass)) & 255u], (unsigned long long)p.cost[i]);
+                hist_add(sh.hist[0], (key >> lo) & digit_mask, p.cost[i], t < T && (hi >= 32 || (key >> hi) == (pf >> hi)), lane);
             }
         }
-        if (bad) s_bad = 1;
         __syncthreads();
         if (warp == 0) {
             unsigned long long above;
-            const int dsel = pick_byte(sh.hist[0], s_left + 1ull, above, lane);  // the byte value with which the budget is first exceeded
+            const int dsel = pick_byte(sh.hist[0], s_left + 1ull, above, lane);  // the digit with which the budget is first exceeded
             if (lane == 0) {
-                if (dsel < 0) {
-                    sh.take_all = 1;   // (first pass only) everything fits: all tokens keep FP16
-                } else {
-                    sh.prefix[0] |= (uint32_t)dsel << (8 * pass);
-                    s_left -= above;
-                }
+                sh.prefix[0] |= (uint32_t)max(dsel, 0) << lo;
+                s_left -= above;
             }
         }
         __syncthreads();
@@ -275,7 +350,7 @@ __global__ void __launch_bounds__(kSelThreads) bits_by_budget_kernel(BudgetParam
         uint32_t c[3] = {0u, 0u, 0u};
         for (int64_t t = first; t < last; ++t)
 #pragma unroll
-            for (int i = 0; i < 3; ++i) c[i] += key_of(scores[t], i) == tau;
+            for (int i = 0; i < 3; ++i) c[i] += key_of(score_at(t), i) == tau;
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
 #pragma unroll
@@ -303,7 +378,7 @@ __global__ void __launch_bounds__(kSelThreads) bits_by_budget_kernel(BudgetParam
     }
     unsigned long long mine = 0;
     if (partial < 3)
-        for (int64_t t = first; t < last; ++t) mine += key_of(scores[t], partial) == tau;
+        for (int64_t t = first; t < last; ++t) mine += key_of(score_at(t), partial) == tau;
     unsigned long long total;
     unsigned long long before = block_exclusive_scan64(mine, sh.scratch, total);
     const bool invalid = s_bad != 0;
@@ -314,7 +389,7 @@ __global__ void __launch_bounds__(kSelThreads) bits_by_budget_kernel(BudgetParam
         } else {
 #pragma unroll
             for (int i = 0; i < 3; ++i) {
-                const uint32_t key = key_of(scores[t], i);
+                const uint32_t key = key_of(score_at(t), i);
                 bool take = key > tau;
                 if (key == tau) {
                     take = i < partial || (i == partial && before < granted);

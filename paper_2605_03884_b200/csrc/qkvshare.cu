@@ -36,6 +36,7 @@ struct ScanParams {
     uint64_t capacity;
     int32_t n_layers, n_kv_heads, head_dim, n_tokens, bits_mode;
     int32_t meta_bytes;   // 8 or 4
+    int32_t group_size;   // 32, 64 or 128
     uint64_t model_id, sender_id;
     int64_t position_offset;
     uint32_t *workspace;  // the call's scratch block, cleared here for the kernels that follow; or null
@@ -80,7 +81,7 @@ __device__ __forceinline__ void write_header_static(qkvs_card_header_t *h, const
     h->n_kv_heads = p.n_kv_heads;
     h->head_dim = p.head_dim;
     h->n_tokens = p.n_tokens;
-    h->group_size = kGroup;
+    h->group_size = p.group_size;
     h->meta_bytes_per_group = (uint32_t)p.meta_bytes;
     h->model_id = p.model_id;
     h->sender_id = p.sender_id;
@@ -144,7 +145,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
         for (int i = 0; i < kScanItems; ++i) {
             rec[i] = 0;
             if (t0 + i < T) {
-                rec[i] = record_bytes(d, bv[i], p.meta_bytes);
+                rec[i] = record_bytes(d, bv[i], p.meta_bytes, p.group_size);
                 bad |= rec[i] == 0u;
                 sum_bits += bv[i];
                 mine += rec[i];
@@ -359,9 +360,11 @@ static qkvs_status_t check_shape(const qkvs_layout_t *l)
     if (!l) return QKVS_ERR_INVALID_ARG;
     if (l->n_layers < 1 || l->n_kv_heads < 1 || l->n_tokens < 0) return QKVS_ERR_INVALID_ARG;
     if (l->bits_mode != 0 && l->bits_mode != 1) return QKVS_ERR_INVALID_ARG;
-    if (l->group_size != kGroup) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (l->group_size != kGroup && l->group_size != 64 && l->group_size != 128) return QKVS_ERR_UNSUPPORTED_SHAPE;
     if (l->head_dim != 64 && l->head_dim != 128 && l->head_dim != 192 && l->head_dim != 256)
         return QKVS_ERR_UNSUPPORTED_SHAPE;
+    // the wider groups are built for the head dimensions of 128 and 256 channels
+    if (l->group_size != kGroup && l->head_dim != 128 && l->head_dim != 256) return QKVS_ERR_UNSUPPORTED_SHAPE;
     // offsets inside a stream are 32-bit
     if ((uint64_t)l->n_tokens * 2u * (uint64_t)l->head_dim > 0xffffffffull) return QKVS_ERR_UNSUPPORTED_SHAPE;
     if ((uint64_t)l->n_layers * (uint64_t)l->n_kv_heads > (1u << 24)) return QKVS_ERR_UNSUPPORTED_SHAPE;
@@ -480,24 +483,43 @@ static cudaError_t launch_path(Kernel kernel, size_t smem, const PathParams &pp,
     return cudaLaunchKernelEx(&cfg, kernel, p, ptrs);
 }
 
-template <int D, int META>
+template <int D, int META, int GS = 0>
 static cudaError_t launch_create(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D, QKVS_WARPS_CREATE, D * 4 + META>(create_kernel<D, kStagesCreate, QKVS_WARPS_CREATE, META>,
-                                                          QKVS_WARPS_CREATE * sizeof(CreateWarpSmem<D, kStagesCreate>), p, ptrs, streams, st, true);
+    return launch_path<D, QKVS_WARPS_CREATE, (D * 4 + META) * 8 + 2 * GS>(create_kernel<D, kStagesCreate, QKVS_WARPS_CREATE, META, GS>,
+                                                                         QKVS_WARPS_CREATE * sizeof(CreateWarpSmem<D, kStagesCreate>), p, ptrs, streams, st, true);
 }
 
-template <int D, int META>
+template <int D, int META, int GS = 0>
 static cudaError_t launch_inject(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
-    return launch_path<D, QKVS_WARPS_INJECT, D * 4 + META + 1>(inject_kernel<D, kStagesInject, QKVS_WARPS_INJECT, META>,
-                                                              QKVS_WARPS_INJECT * sizeof(InjectWarpSmem<D, kStagesInject>), p, ptrs, streams, st, false);
+    return launch_path<D, QKVS_WARPS_INJECT, (D * 4 + META) * 8 + 2 * GS + 1>(inject_kernel<D, kStagesInject, QKVS_WARPS_INJECT, META, GS>,
+                                                                             QKVS_WARPS_INJECT * sizeof(InjectWarpSmem<D, kStagesInject>), p, ptrs, streams, st, false);
+}
+
+// The wider-group instances: head_dim 128 or 256, either kind of pair, groups of 64 or 128.
+template <int GS>
+static cudaError_t launch_create_wide(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+{
+    if (p.meta_bytes == kMetaFp16)
+        return p.head_dim == 128 ? launch_create<128, kMetaFp16, GS>(p, ptrs, streams, st) : launch_create<256, kMetaFp16, GS>(p, ptrs, streams, st);
+    return p.head_dim == 128 ? launch_create<128, kMetaFp32, GS>(p, ptrs, streams, st) : launch_create<256, kMetaFp32, GS>(p, ptrs, streams, st);
+}
+
+template <int GS>
+static cudaError_t launch_inject_wide(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
+{
+    if (p.meta_bytes == kMetaFp16)
+        return p.head_dim == 128 ? launch_inject<128, kMetaFp16, GS>(p, ptrs, streams, st) : launch_inject<256, kMetaFp16, GS>(p, ptrs, streams, st);
+    return p.head_dim == 128 ? launch_inject<128, kMetaFp32, GS>(p, ptrs, streams, st) : launch_inject<256, kMetaFp32, GS>(p, ptrs, streams, st);
 }
 
 // The kernel instance for a checked shape: every head_dim with fp32 pairs, 128 and 256 with FP16
 // pairs.
 static cudaError_t launch_create_for(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
+    if (p.group_size == 64) return launch_create_wide<1>(p, ptrs, streams, st);
+    if (p.group_size == 128) return launch_create_wide<2>(p, ptrs, streams, st);
     if (p.meta_bytes == kMetaFp16)
         return p.head_dim == 128 ? launch_create<128, kMetaFp16>(p, ptrs, streams, st)
                                  : launch_create<256, kMetaFp16>(p, ptrs, streams, st);
@@ -511,6 +533,8 @@ static cudaError_t launch_create_for(const PathParams &p, const LayerPtrs &ptrs,
 
 static cudaError_t launch_inject_for(const PathParams &p, const LayerPtrs &ptrs, int64_t streams, cudaStream_t st)
 {
+    if (p.group_size == 64) return launch_inject_wide<1>(p, ptrs, streams, st);
+    if (p.group_size == 128) return launch_inject_wide<2>(p, ptrs, streams, st);
     if (p.meta_bytes == kMetaFp16)
         return p.head_dim == 128 ? launch_inject<128, kMetaFp16>(p, ptrs, streams, st)
                                  : launch_inject<256, kMetaFp16>(p, ptrs, streams, st);
@@ -592,7 +616,7 @@ qkvs_status_t qkvs_card_size(const qkvs_layout_t *layout, const uint8_t *bits_ho
     for (int64_t seg = 0; seg < nseg; ++seg) {
         uint64_t seg_bytes = 0;
         for (int64_t t = 0; t < T; ++t) {
-            const uint32_t r = record_bytes(layout->head_dim, bits_host ? bits_host[seg * T + t] : 16, meta_bytes_of(layout->meta_bytes));
+            const uint32_t r = record_bytes(layout->head_dim, bits_host ? bits_host[seg * T + t] : 16, meta_bytes_of(layout->meta_bytes), layout->group_size);
             if (r == 0) return QKVS_ERR_BAD_BITS;
             seg_bytes += r;
         }
@@ -628,6 +652,7 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
     sp.n_tokens = layout->n_tokens;
     sp.bits_mode = layout->bits_mode;
     sp.meta_bytes = meta_bytes_of(layout->meta_bytes);
+    sp.group_size = layout->group_size;
     sp.model_id = meta ? meta->model_id : 0;
     sp.sender_id = meta ? meta->sender_id : 0;
     sp.position_offset = meta ? meta->position_offset : 0;
@@ -654,6 +679,7 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
     p.n_tokens = layout->n_tokens;
     p.bits_mode = layout->bits_mode;
     p.meta_bytes = meta_bytes_of(layout->meta_bytes);
+    p.group_size = layout->group_size;
     p.head_stride = layout->head_stride;
     p.token_stride = layout->token_stride;
     for (int l0 = 0; l0 < layout->n_layers; l0 += kMaxLayersPerLaunch) {
@@ -700,6 +726,7 @@ qkvs_status_t qkvs_card_inject(const void *card_dev, size_t card_bytes, const qk
     p.n_tokens = dst->n_tokens;
     p.bits_mode = 0;  // taken from the card on the device
     p.meta_bytes = meta_bytes_of(dst->meta_bytes);  // the card's header must say the same
+    p.group_size = dst->group_size;                 // ... and this
     p.head_stride = dst->head_stride;
     p.token_stride = dst->token_stride;
     p.dst_token_offset = dst_token_offset;
@@ -753,6 +780,7 @@ qkvs_status_t qkvs_card_inject_noalloc(const void *card_dev, size_t card_bytes, 
     p.n_tokens = dst->n_tokens;
     p.bits_mode = 0;  // taken from the card on the device
     p.meta_bytes = meta_bytes_of(dst->meta_bytes);  // the card's header must say the same
+    p.group_size = dst->group_size;                 // ... and this
     p.head_stride = dst->head_stride;
     p.token_stride = dst->token_stride;
     p.dst_token_offset = dst_token_offset;
@@ -817,7 +845,7 @@ static qkvs_status_t attend_shape(const qkvs_layout_t *layout, int32_t n_q_heads
 {
     const qkvs_status_t st = check_shape(layout);
     if (st != QKVS_OK) return st;
-    if (layout->head_dim != kAttendD) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (layout->head_dim != kAttendD || layout->group_size != kGroup) return QKVS_ERR_UNSUPPORTED_SHAPE;
     if (n_q_heads < layout->n_kv_heads || n_q_heads % layout->n_kv_heads != 0) return QKVS_ERR_INVALID_ARG;
     if (n_q_heads / layout->n_kv_heads > kAttendMaxPerKv) return QKVS_ERR_UNSUPPORTED_SHAPE;
     memset(p, 0, sizeof(*p));

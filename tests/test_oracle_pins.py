@@ -110,7 +110,7 @@ def test_card_size_worst_case_and_errors():
     assert oracle.card_size(oracle.make_layout(1, 1, 32, 4), None)[0] == oracle.UNSUPPORTED_SHAPE
     assert oracle.card_size(oracle.make_layout(1, 1, 96, 4), None)[0] == oracle.UNSUPPORTED_SHAPE
     bad = oracle.make_layout(1, 1, 64, 4)
-    bad.group_size = 64
+    bad.group_size = 48
     assert oracle.card_size(bad, None)[0] == oracle.UNSUPPORTED_SHAPE
 
 
