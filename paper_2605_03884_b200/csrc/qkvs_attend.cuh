@@ -780,36 +780,40 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
 }
 
 // Merges the items of every query head: o = sum_i o_i 2^(m_i - M) / sum_i l_i 2^(m_i - M).
-// One warp per (layer, query head); writes zeros when the first kernel reported a problem.
-// The items' maxima and sums are read one item per lane, so that the loads of an item's
-// accumulators, which need its factor only for the multiplication, all go out at once.
+// One CTA of four warps per (layer, query head), a quarter of the items per warp, so that the
+// whole merge is two rounds of loads and one exchange through shared memory; writes zeros when
+// the first kernel reported a problem.  Inside a warp the items' maxima and sums are read one
+// item per lane, so that the loads of an item's accumulators, which need its factor only for the
+// multiplication, all go out at once.
 __global__ void __launch_bounds__(128) attend_merge_kernel(AttendParams p)
 {
-    const int lane = threadIdx.x & 31;
-    const uint32_t w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const uint32_t n_rows = (uint32_t)p.n_layers * (uint32_t)p.n_q_heads;
-    if (w >= n_rows) return;
+    __shared__ float s_big[4], s_den[4];
+    __shared__ float4 s_o[4][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t w = blockIdx.x;
     const int per_kv = p.n_q_heads / p.n_kv_heads;
     const uint32_t layer = w / (uint32_t)p.n_q_heads, j = w - layer * (uint32_t)p.n_q_heads;
     const uint32_t lh = layer * (uint32_t)p.n_kv_heads + j / (uint32_t)per_kv, jj = j % (uint32_t)per_kv;
-    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     const bool usable = p.items_per_head > 0 && (!p.status_dev || *p.status_dev == 0);
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    float big = -INFINITY, denom = 0.0f;
     if (usable) {
         const float *base = p.partials + ((uint64_t)lh * p.items_per_head * per_kv + jj) * kPartialFloats;
         const uint64_t stride = (uint64_t)per_kv * kPartialFloats;
-        float big = -INFINITY;
-        for (uint32_t i = lane; i < p.items_per_head; i += 32) big = fmaxf(big, base[i * stride + kAttendD]);
+        // this warp's items: [first, last)
+        const uint32_t share = (p.items_per_head + 3u) / 4u;
+        const uint32_t first = min((uint32_t)warp * share, p.items_per_head), last = min(first + share, p.items_per_head);
+        for (uint32_t i = first + lane; i < last; i += 32) big = fmaxf(big, base[i * stride + kAttendD]);
 #pragma unroll
         for (int sft = 16; sft > 0; sft >>= 1) big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, sft));
-        float denom = 0.0f;
-        for (uint32_t i0 = 0; i0 < p.items_per_head; i0 += 32) {
+        for (uint32_t i0 = first; i0 < last; i0 += 32) {
             const uint32_t mine = i0 + (uint32_t)lane;
             float f = 0.0f;
-            if (mine < p.items_per_head) {
+            if (mine < last) {
                 f = exp2f(base[mine * stride + kAttendD] - big);
                 denom = fmaf(base[mine * stride + kAttendD + 1], f, denom);
             }
-            const int n = (int)min(32u, p.items_per_head - i0);
+            const int n = (int)min(32u, last - i0);
 #pragma unroll 8
             for (int i = 0; i < n; ++i) {
                 const float fi = __shfl_sync(0xffffffffu, f, i);
@@ -822,13 +826,33 @@ __global__ void __launch_bounds__(128) attend_merge_kernel(AttendParams p)
         }
 #pragma unroll
         for (int sft = 16; sft > 0; sft >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, sft);
-        const float r = 1.0f / denom;
-        o.x *= r;
-        o.y *= r;
-        o.z *= r;
-        o.w *= r;
     }
-    *reinterpret_cast<float4 *>(p.out + (uint64_t)w * kAttendD + 4 * lane) = o;
+    s_o[warp][lane] = o;
+    if (lane == 0) {
+        s_big[warp] = big;
+        s_den[warp] = denom;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (usable) {
+            const float top = fmaxf(fmaxf(s_big[0], s_big[1]), fmaxf(s_big[2], s_big[3]));
+            float den = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float f = s_big[k] == -INFINITY ? 0.0f : exp2f(s_big[k] - top);   // a warp without items
+                const float4 v = s_o[k][lane];
+                den = fmaf(s_den[k], f, den);
+                sum.x = fmaf(v.x, f, sum.x);
+                sum.y = fmaf(v.y, f, sum.y);
+                sum.z = fmaf(v.z, f, sum.z);
+                sum.w = fmaf(v.w, f, sum.w);
+            }
+            const float r = 1.0f / den;
+            sum.x *= r, sum.y *= r, sum.z *= r, sum.w *= r;
+        }
+        *reinterpret_cast<float4 *>(p.out + (uint64_t)w * kAttendD + 4 * lane) = sum;
+    }
 }
 
 }  // namespace qkvs

@@ -56,7 +56,7 @@ constexpr int kTcRawBytes = kTcSlotTokens * kAttendRecMax;  // 5120: 32 eight-bi
 constexpr int kTcRing = 3;
 constexpr int kTcPipes = 2;
 constexpr int kTcTokenThreads = 128;                // per pipeline
-constexpr int kTcThreads = kTcPipes * (kTcTokenThreads + 32);
+constexpr int kTcThreads = kTcPipes * (kTcTokenThreads + 64);  // token warps, a driver warp and a planner warp per pipeline
 constexpr uint32_t kTcTmemCols = 512, kTcPipeCols = 256;
 constexpr uint32_t kTcColA = 0, kTcColS = 64, kTcColO = 128;  // inside a pipeline's 256 columns
 constexpr float kTcRefreshAbove = 8.0f;             // base-2 exponent by which a logit may exceed the reference
@@ -69,10 +69,10 @@ struct TcItem {
     uint64_t base_k, base_v;          // byte offsets inside the card of the item's first record in the two streams
     uint32_t slots[kTcMaxSlots];      // per slot: first list position | tokens << 10 | class << 16 | neighbours << 18 |
                                       // (where the slot's records start in the tile's buffer, in 16-byte units) << 20
-    uint32_t tiles[kTcMaxTiles];      // per tile: (bytes of its records >> 4) << 1 | the whole tile is one run of neighbours
+    uint32_t tiles[kTcMaxTiles];      // per tile: the whole tile is one run of neighbours | (bytes of its records >> 4) << 1 |
+                                      // (list value of its first record) << 12
     uint16_t list[kTcItemTokens];     // the item's tokens grouped by bit-width: record offsets from the item's first, in 16-byte units
     float qsum[4][8];                 // sums of the item's queries over a group of channels, per head
-    float sums[8 + 4 * 8];            // what the token threads add up: l[h], then zero-point sums [group][head]
     alignas(128) uint8_t qb[16 * kAttendD * 2];  // the item's queries, [head][channel], K-major core matrices
 };
 
@@ -86,6 +86,7 @@ struct TcPipeSmem {
     uint64_t s_full, o_done;                            // the tensor cores have finished the scores / the outputs of a tile
     uint64_t item_ready[2], item_done[2];
     float red[4][8];                                    // per-warp maxima of a refresh
+    float sums[4][8 + 4 * 8];                           // per-warp sums at the end of an item: l[h], then zero-point sums [group][head]
     int abort;                                          // read by the token threads after their barrier
     int driver_abort;                                   // raised by the driver; token thread 0 carries it over
 };
@@ -209,9 +210,9 @@ __device__ __forceinline__ void tc_issue_tile(uint8_t *dst, uint64_t *bar, const
     const uint32_t info = it.tiles[tile];
     if (info & 1u) {
         if (lane == 0) {
-            const uint32_t bytes = (info >> 1) << 4;
+            const uint32_t bytes = ((info >> 1) & 2047u) << 4;
             mbar_arrive_expect_tx(bar, bytes);
-            bulk_load(dst, p.card + base + ((uint32_t)it.list[tc_slot_first(it.slots[4u * tile])] << 4), bytes, bar);
+            bulk_load(dst, p.card + base + ((uint64_t)(info >> 12) << 4), bytes, bar);
         }
         return;
     }
@@ -251,11 +252,12 @@ struct TcCard {
     uint64_t stream_bytes, total_bytes;
 };
 
-// Driver warp, preparing an item in two steps so that the memory latency falls between them.
-// tc_fetch starts the reads (the item's table entries, 16 consecutive tokens per lane, and its
-// queries) and keeps the results in registers; tc_finish, called a tile's worth of work later,
-// checks and sorts the entries into buffer `it`, lays out its slots and tiles, and writes the
-// queries as the B operand of the score product, and their sums.
+// Planner warp, preparing an item in two steps.  tc_fetch reads the item's table entries (16
+// consecutive tokens per lane) and its queries into registers; tc_finish checks and sorts the
+// entries into buffer `it`, lays out its slots and tiles, and writes the queries as the B operand
+// of the score product, and their sums.  A single warp runs this dependent code at a small
+// fraction of an instruction per cycle (about 9000 cycles per item as measured), which is why it
+// has a warp of its own, one item ahead of the others, instead of sitting in the driver's loop.
 struct TcFetch {
     static constexpr int PER = kTcItemTokens / 32;
     uint32_t item;           // n_items when there is none
@@ -350,7 +352,6 @@ __device__ __forceinline__ void tc_finish(TcItem &it, const TcFetch &f, const At
             sum += __shfl_xor_sync(0xffffffffu, sum, 2);   // the four pieces of a group sit in neighbouring lanes
             if ((ch & 3) == 0) it.qsum[ch >> 2][h] = sum;
         }
-        for (int i = lane; i < 8 + 4 * 8; i += 32) it.sums[i] = 0.0f;
     }
 
     // ---- the tables: 16 consecutive tokens per lane
@@ -427,6 +428,7 @@ __device__ __forceinline__ void tc_finish(TcItem &it, const TcFetch &f, const At
         uint32_t at = 0;          // bytes of the tile so far
         bool run = true;
         uint32_t follow = 0;      // list value the next slot's first record must have to continue the run
+        uint32_t origin = 0;      // list value of the tile's first record
         for (uint32_t w = 0; w < 4; ++w) {
             const uint32_t slot = 4u * (uint32_t)lane + w;
             if (slot >= n_slots) break;
@@ -434,11 +436,12 @@ __device__ __forceinline__ void tc_finish(TcItem &it, const TcFetch &f, const At
             const uint32_t bytes = (uint32_t)tc_slot_count(d) * class_record_bytes<META>(tc_slot_class(d));
             const uint32_t first = it.list[tc_slot_first(d)];
             run = run && (d & (1u << 18)) != 0u && (w == 0 || first == follow);
+            if (w == 0) origin = first;
             follow = first + (bytes >> 4);
             it.slots[slot] = d | ((at >> 4) << 20);
             at += bytes;
         }
-        it.tiles[lane] = ((at >> 4) << 1) | (run && at > 0u ? 1u : 0u);
+        it.tiles[lane] = (origin << 12) | ((at >> 4) << 1) | (run && at > 0u ? 1u : 0u);
     }
     if (lane == 0) {
         it.item = item;
@@ -459,8 +462,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
     __shared__ uint64_t s_stream_bytes, s_total_bytes;
     const int tid = threadIdx.x;
     const int cta_warp = tid >> 5, lane = tid & 31;
-    const bool is_driver = cta_warp >= 4 * kTcPipes;            // warps 0..3, 4..7: token warps; 8, 9: drivers
-    const int pipe = is_driver ? cta_warp - 4 * kTcPipes : cta_warp / 4;
+    // warps 0..3, 4..7: token warps of the two pipelines; 8, 9: their drivers; 10, 11: their planners
+    const bool is_driver = cta_warp >= 4 * kTcPipes && cta_warp < 5 * kTcPipes;
+    const bool is_planner = cta_warp >= 5 * kTcPipes;
+    const int pipe = is_planner ? cta_warp - 5 * kTcPipes : (is_driver ? cta_warp - 4 * kTcPipes : cta_warp / 4);
     const int warp = cta_warp % 4;                              // token warp inside the pipeline = its quarter of the tensor-memory lanes
     const int ptid = 32 * warp + lane;                          // token threads: row of the tile
     TcPipeSmem &sm = reinterpret_cast<TcPipeSmem *>(smem_raw)[pipe];
@@ -494,7 +499,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
         mbar_init(&sm.o_done, 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm.item_ready[b], 1);
-            mbar_init(&sm.item_done[b], 4);
+            mbar_init(&sm.item_done[b], 5);   // four token warps and the driver
         }
         sm.abort = 0;
         sm.driver_abort = 0;
@@ -523,62 +528,52 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
     constexpr uint32_t kWLbo = 16u * N2;                        // bytes between blocks of 8 tokens in W
     const uint32_t tm_pipe = s_tmem_base + (uint32_t)pipe * kTcPipeCols;
 
-    if (is_driver) {
+    if (is_planner) {
         // =====================================================================================
-        // Driver warp: items, copies, matrix multiplies.  Lane 0 issues; all lanes share the
-        // table work and the gathers.
+        // Planner warp: draws the pipeline's items and prepares each one item ahead of its use.
         const uint32_t n_pipes = gridDim.x * kTcPipes;
+        uint32_t idx = (uint32_t)(blockIdx.x * kTcPipes + pipe);   // the first item is the pipeline's own index
+        bool ok = true;
+        TcFetch fetch;
+        for (uint32_t k = 0;; ++k) {
+            const uint32_t b = k & 1u;
+            tc_fetch(fetch, idx, p, cd, lane);
+            uint32_t drawn = 0;
+            if (idx < p.n_items && lane == 0) drawn = atomicAdd(p.work_counter, 1u);
+            // buffer b held item k - 2: the token warps and the driver must be done with it
+            if (k >= 2) ok = __all_sync(0xffffffffu, mbar_wait_short(&sm.item_done[b], ((k - 2u) >> 1) & 1u));
+            if (!ok) break;
+            tc_finish<META>(sm.items[b], fetch, p, cd, lane);
+            if (lane == 0) mbar_arrive(&sm.item_ready[b]);
+            if (idx >= p.n_items) break;
+            drawn = __shfl_sync(0xffffffffu, drawn, 0);
+            idx = drawn < p.n_items ? min(n_pipes + drawn, p.n_items) : p.n_items;
+        }
+        if (!ok) {
+            sm.driver_abort = 1;
+            if (lane == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_TIMEOUT);
+        }
+    } else if (is_driver) {
+        // =====================================================================================
+        // Driver warp: copies and matrix multiplies.  Lane 0 issues; all lanes share the gathers.
         const uint32_t idesc1 = mma_idesc_f16(128, 16, false, false);
         const uint32_t idesc2 = mma_idesc_f16(128, N2, true, true);
         uint32_t n = 0;                           // tiles of this pipeline so far (phase of the per-tile barriers)
-        uint32_t k_issued = 0, v_issued = 0;      // tiles whose K / V loads are on their way (all four warps)
+        uint32_t k_issued = 0, v_issued = 0;      // tiles whose K / V loads are on their way
         bool ok = true;
 
         auto issue = [&](const TcItem &it, uint32_t tile, uint32_t kv, uint32_t flat) {
             const uint32_t ring = (2u * flat + kv) % kTcRing;   // loads are numbered K, V, K, V, ... over the pipeline's tiles
             tc_issue_tile<META>(sm.raw[ring], &sm.full[ring], it, tile, kv ? it.base_v : it.base_k, p, lane);
         };
-        // The work counter is read one item ahead of its use: lane 0 keeps the raw result of the
-        // atomic in a register and nobody looks at it before the next item is finished.
-        uint32_t drawn_raw = 0;
-        auto draw_start = [&]() {
-            if (lane == 0) drawn_raw = atomicAdd(p.work_counter, 1u);
-        };
-        auto draw_result = [&]() -> uint32_t {
-            const uint32_t v = __shfl_sync(0xffffffffu, drawn_raw, 0);
-            return v < p.n_items ? min(n_pipes + v, p.n_items) : p.n_items;
-        };
-
-        // item 0 of this pipeline is its own index; the following ones come from the counter
-        TcFetch fetch;
-        tc_fetch(fetch, (uint32_t)(blockIdx.x * kTcPipes + pipe), p, cd, lane);
-        draw_start();
-        tc_finish<META>(sm.items[0], fetch, p, cd, lane);
-        if (lane == 0) mbar_arrive(&sm.item_ready[0]);
-        uint32_t idx_next = draw_result();   // index of item k + 1, known at the top of item k
 
         for (uint32_t k = 0; ok; ++k) {
             const uint32_t b = k & 1u;
             TcItem &it = sm.items[b];
-            if (it.item >= p.n_items) break;
+            ok = __all_sync(0xffffffffu, mbar_wait_short(&sm.item_ready[b], (k >> 1) & 1u));
+            if (!ok || it.item >= p.n_items) break;
             const uint32_t nt = (it.n_slots + 3u) / 4u;
-            bool next_prepared = false;
-            // the reads for the next item start now and are used a tile later; so does the draw of
-            // the item after it
-            tc_fetch(fetch, idx_next, p, cd, lane);
-            if (idx_next < p.n_items) draw_start();
-            auto prepare_next = [&]() {
-                // buffer b ^ 1 held item k - 1: the token warps must be done with it
-                if (k >= 1) ok = ok && mbar_wait_short(&sm.item_done[b ^ 1u], ((k - 1u) >> 1) & 1u);
-                ok = __all_sync(0xffffffffu, ok);
-                if (ok) {
-                    tc_finish<META>(sm.items[b ^ 1u], fetch, p, cd, lane);
-                    if (lane == 0) mbar_arrive(&sm.item_ready[b ^ 1u]);
-                    idx_next = idx_next < p.n_items ? draw_result() : p.n_items;
-                }
-                next_prepared = true;
-            };
-            if (nt == 0) prepare_next();
+            bool next_seen = false;               // the planner has finished item k + 1
             for (uint32_t t = 0; t < nt && ok; ++t) {
                 if (k_issued == n) {
                     issue(it, t, 0u, n);
@@ -594,8 +589,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
                 if (t + 1 < nt) {
                     nx = &it;
                     nx_tile = t + 1;
-                } else if (next_prepared && sm.items[b ^ 1u].item < p.n_items && sm.items[b ^ 1u].n_slots > 0) {
-                    nx = &sm.items[b ^ 1u];
+                } else {
+                    if (!next_seen) next_seen = __all_sync(0xffffffffu, mbar_try_wait_short(&sm.item_ready[b ^ 1u], ((k + 1u) >> 1) & 1u));
+                    if (next_seen && sm.items[b ^ 1u].item < p.n_items && sm.items[b ^ 1u].n_slots > 0) nx = &sm.items[b ^ 1u];
                 }
                 if (nx && k_issued == n + 1) {
                     issue(*nx, nx_tile, 0u, n + 1);
@@ -633,12 +629,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
                 }
                 __syncwarp();
                 ++n;
-                // the next item's tables have had a tile's time to arrive
-                if (t == 0) {
-                    prepare_next();
-                    if (!ok) break;
-                }
             }
+            // the planner may put the item after the next into this buffer
+            if (lane == 0) mbar_arrive(&sm.item_done[b]);
         }
         if (!ok) {
             sm.driver_abort = 1;
@@ -836,13 +829,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
                 float v = l_run[h];
 #pragma unroll
                 for (int sft = 16; sft > 0; sft >>= 1) v += __shfl_xor_sync(0xffffffffu, v, sft);
-                if (lane == 0) atomicAdd(&it.sums[h], v);
+                if (lane == 0) sm.sums[warp][h] = v;
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     float z = zacc[g][h];
 #pragma unroll
                     for (int sft = 16; sft > 0; sft >>= 1) z += __shfl_xor_sync(0xffffffffu, z, sft);
-                    if (lane == 0) atomicAdd(&it.sums[8 + 8 * g + h], z);
+                    if (lane == 0) sm.sums[warp][8 + 8 * g + h] = z;
                 }
             }
             tokens_sync(pipe);
@@ -861,23 +854,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) attend_tc_kernel(AttendParams p
             float *part = p.partials + (uint64_t)it.item * per_kv * kPartialFloats;
 #pragma unroll
             for (int h = 0; h < PK; ++h)
-                if (h < per_kv) part[h * kPartialFloats + ch] = __uint_as_float(o[h]) + it.sums[8 + 8 * warp + h];
+                if (h < per_kv) {
+                    const int i = 8 + 8 * warp + h;   // the zero-point sum of this thread's group of channels
+                    part[h * kPartialFloats + ch] = __uint_as_float(o[h]) + ((sm.sums[0][i] + sm.sums[1][i]) + (sm.sums[2][i] + sm.sums[3][i]));
+                }
             if (ptid < per_kv) {
                 float m = -INFINITY;
 #pragma unroll
                 for (int h = 0; h < PK; ++h)
                     if (h == ptid) m = mref[h];
                 part[ptid * kPartialFloats + kAttendD] = m;
-                part[ptid * kPartialFloats + kAttendD + 1] = it.sums[ptid];
+                part[ptid * kPartialFloats + kAttendD + 1] = (sm.sums[0][ptid] + sm.sums[1][ptid]) + (sm.sums[2][ptid] + sm.sums[3][ptid]);
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.item_done[b]);   // the driver may put the item after the next into this buffer
+            if (lane == 0) mbar_arrive(&sm.item_done[b]);
         }
     }
 
     // ---- leaving: tensor memory goes back
-    if (!is_driver && ptid == 0 && sm.abort && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_TIMEOUT);
+    if (!is_driver && !is_planner && ptid == 0 && sm.abort && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_TIMEOUT);
     tc_fence_before_sync();
     __syncthreads();
     if (cta_warp == 4 * kTcPipes) tmem_dealloc(s_tmem_base, kTcTmemCols);

@@ -933,7 +933,7 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
         if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
     }
     const unsigned rows = (unsigned)p.n_layers * (unsigned)p.n_q_heads;
-    attend_merge_kernel<<<(rows + 3) / 4, 128, 0, cs>>>(p);
+    attend_merge_kernel<<<rows, 128, 0, cs>>>(p);
     return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 
