@@ -43,6 +43,10 @@ def measured_peaks():
     return 6650.0, "fallback (6.65 TB/s, an earlier measurement of the same copy)"
 
 
+# what create_kernel and inject_kernel are compiled from
+TRAFFIC_SOURCES = ("qkvs_common.cuh", "qkvs_pipeline.cuh", "qkvs_ptx.cuh")
+
+
 def captured_traffic(kernel: str, n_layers: int):
     """DRAM bytes of one launch of `kernel` at `n_layers` layers, from the committed ncu captures
     of the 8- and the 16-layer case of the headline workload: reads and writes are each taken as
@@ -59,7 +63,7 @@ def captured_traffic(kernel: str, n_layers: int):
                 parts = line.split()
                 entries[parts[0]] = parts[1:]
         h = hashlib.sha256()
-        for f in sorted(os.listdir(csrc)):
+        for f in TRAFFIC_SOURCES:
             h.update(open(os.path.join(csrc, f), "rb").read())
         if entries.get("csrc_sha256", [""])[0] != h.hexdigest():
             return None, "kernel sources changed since the counters were taken"
