@@ -541,7 +541,7 @@ def run_ours(args):
     # attention straight from the card (the row after the hot path): one decode step, 32 query
     # heads, over the card the last create left behind; reported beside the main metric
     attend = None
-    if d == 128 and args.group_size == 32 and not args.skip_attend:
+    if d == 128 and not args.skip_attend:
         a_ms = case.attend(stream, 4)
         payload = sizes[-1] - prefix
         attend = {"what": "decode-step attention straight from the card, all layers, 4 query heads per KV head",
@@ -627,7 +627,7 @@ def run_ours(args):
                      "fp16_kv_bytes": c.kv_bytes,
                      "bits_per_element": 8.0 * (c.sizes[0] - c.prefix) / (c.kv_bytes / 2),
                      "per_hop": c.hop_stats(cm, im, peak, errs)}
-            if c.d == 128 and group == 32 and not args.skip_attend:
+            if c.d == 128 and not args.skip_attend:
                 a_ms = c.attend(stream, 4, reps=15)
                 payload = c.sizes[-1] - c.prefix
                 entry["attend_from_card"] = {"ms": a_ms, "card_payload_bytes": payload,

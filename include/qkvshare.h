@@ -46,7 +46,7 @@
  * same as FP16 pairs on groups of 32, because of the padding); at head_dim 256, one FP16 or fp32
  * pair per 128 channels gives 144 bytes (4.5 bits per element).  The wider the group, the larger
  * the range one scale has to cover: channel-wise key outliers then cost every channel of the
- * group precision.  Card creation and injection support it; attention from the card does not.
+ * group precision.  Card creation, injection and attention from the card (head_dim 128) support it.
  *
  * All entry points return a qkvs_status_t.  Unless stated otherwise a pointer named *_dev is a
  * device pointer, anything else is a host pointer.  The library allocates no device memory and
@@ -331,8 +331,9 @@ QKVS_API qkvs_status_t qkvs_card_send(const void *card_dev, size_t card_bytes, i
  * Products run on the tensor cores with FP16 inputs (the integer codes, exact in FP16, and the
  * probabilities times the scales, rounded to FP16) and FP32 accumulation; scale and zero are
  * applied outside the products.
- *   layout        n_layers, n_kv_heads, head_dim, n_tokens and meta_bytes of the card (checked
- *                 against its header on the device); head_dim must be 128; strides are not looked at
+ *   layout        n_layers, n_kv_heads, head_dim, n_tokens, meta_bytes and group_size of the card
+ *                 (checked against its header on the device); head_dim must be 128; strides are
+ *                 not looked at
  *   n_q_heads     multiple of n_kv_heads, at most 8 query heads per KV head.  The products have
  *                 eight columns per KV head whatever is used of them, so a model with four query
  *                 heads per KV head can pass the queries of two new tokens as eight heads per KV

@@ -120,10 +120,21 @@ __device__ __forceinline__ uint32_t step_first(uint32_t d) { return d & 1023u; }
 __device__ __forceinline__ int step_rows(uint32_t d) { return (int)((d >> 10) & 31u); }
 __device__ __forceinline__ int step_class(uint32_t d) { return (int)((d >> 15) & 3u); }
 
+// The record format is a template parameter of everything below, as one number: the bytes of a
+// {scale, zero} pair (8 or 4) plus 16 times log2(channels per group / 32).  Formats with groups of
+// 32 are therefore named by their pair size alone.
+__host__ __device__ constexpr int format_code(int meta, int group_size) { return meta + 16 * (group_size == 128 ? 2 : (group_size == 64 ? 1 : 0)); }
+__host__ __device__ constexpr int format_meta(int fmt) { return fmt & 15; }
+__host__ __device__ constexpr int format_gs(int fmt) { return fmt >> 4; }
+__host__ __device__ constexpr int format_group(int fmt) { return kGroup << format_gs(fmt); }
+// bytes of a record's pairs, i.e. where its code bytes start
+__host__ __device__ constexpr int format_pairs(int fmt) { return (int)pairs_bytes(kAttendD, format_meta(fmt), format_group(fmt)); }
+
 template <int META>
 __device__ __forceinline__ uint32_t class_record_bytes(int c)
 {
-    return c == 0 ? (uint32_t)(kAttendD / 4 + 4 * META) : (c == 1 ? (uint32_t)(kAttendD / 2 + 4 * META) : (c == 2 ? (uint32_t)(kAttendD + 4 * META) : 2u * kAttendD));
+    constexpr int P = format_pairs(META);
+    return c == 0 ? (uint32_t)(kAttendD / 4 + P) : (c == 1 ? (uint32_t)(kAttendD / 2 + P) : (c == 2 ? (uint32_t)(kAttendD + P) : 2u * kAttendD));
 }
 
 // Descriptor of step `idx` given where the classes end in the list (e[c], with e[-1] = 0); 0 past the last step.
@@ -257,7 +268,7 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, ui
         e[3] = __byte_perm(h.y, h.w, 0x7632);
         return;
     }
-    const uint8_t *codes = rec + 4 * META + (4 * g + tig) * bb;  // the lane's 8 codes: b bytes
+    const uint8_t *codes = rec + format_pairs(META) + (4 * g + tig) * bb;  // the lane's 8 codes: b bytes
     if constexpr (B == 4) {
         nibble_pairs(*reinterpret_cast<const uint32_t *>(codes), e);  // nibble k and k + 4 are 16 bits apart
     } else if constexpr (B == 8) {
@@ -275,7 +286,7 @@ __device__ __forceinline__ void key_pairs(const uint8_t *rec, int g, int tig, ui
 template <int B, int META>
 __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t *rec_b, int g, int gid, uint32_t (&e)[4])
 {
-    constexpr int CODES = 4 * META;  // the code bytes follow the four {scale, zero} pairs
+    constexpr int CODES = format_pairs(META);  // the code bytes follow the {scale, zero} pairs
     if (B == 16) {
         const uint2 ha = *reinterpret_cast<const uint2 *>(rec_a + 64 * g + 8 * gid);
         const uint2 hb = *reinterpret_cast<const uint2 *>(rec_b + 64 * g + 8 * gid);
@@ -298,11 +309,28 @@ __device__ __forceinline__ void value_pairs(const uint8_t *rec_a, const uint8_t 
     }
 }
 
-// Scale / zero pairs of a token's four groups; (1, 0) for a 16-bit row, (0, 0) for no token.
+// Scale / zero pairs of a token's four spans of 32 channels; (1, 0) for a 16-bit row, (0, 0) for no
+// token.  With groups of 64 or 128 channels neighbouring spans share a pair.
 template <int B, int META>
 __device__ __forceinline__ void group_params_of(const uint8_t *rec, bool valid, float (&sc)[4], float (&ze)[4])
 {
-    if (B != 16 && valid && META == kMetaFp16) {
+    if (B != 16 && valid && format_gs(META) > 0) {
+        constexpr int GS = format_gs(META);
+        const uint4 m = *reinterpret_cast<const uint4 *>(rec);  // the whole (padded) pairs area
+        const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int pair = g >> GS;
+            if (format_meta(META) == kMetaFp16) {
+                const float2 f = __half22float2(as_half2(w[pair]));
+                sc[g] = f.x;
+                ze[g] = f.y;
+            } else {
+                sc[g] = __uint_as_float(w[2 * pair]);
+                ze[g] = __uint_as_float(w[2 * pair + 1]);
+            }
+        }
+    } else if (B != 16 && valid && META == kMetaFp16) {
         const uint4 m = *reinterpret_cast<const uint4 *>(rec);  // four FP16 pairs
         const uint32_t w[4] = {m.x, m.y, m.z, m.w};
 #pragma unroll
@@ -340,7 +368,7 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
                                             const uint32_t (&qb)[4][4], float (&m_run)[2],
                                             float (&l_run)[2], float (&zacc)[4][2], float (&acc)[4][2][4])
 {
-    constexpr int REC = B == 16 ? 2 * kAttendD : kAttendD * B / 8 + 4 * META;
+    constexpr int REC = B == 16 ? 2 * kAttendD : kAttendD * B / 8 + format_pairs(META);
     const bool have[2] = {FULL || gid < rows, FULL || gid + 8 < rows};
     const uint8_t *krec[2] = {sm.k[stage] + gid * REC, sm.k[stage] + (gid + 8) * REC};
     const uint8_t *vrec[2] = {sm.v[stage] + gid * REC, sm.v[stage] + (gid + 8) * REC};
@@ -356,7 +384,7 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
         uint32_t ka[4], kb[4];
         if (B == 4) {
             const int l = gid * 4 + tig;
-            const uint8_t *row = sm.k[stage] + (l & 7) * REC + 4 * META + 16 * (l >> 3);
+            const uint8_t *row = sm.k[stage] + (l & 7) * REC + format_pairs(META) + 16 * (l >> 3);
             load_matrices(row, ka);
             load_matrices(row + 8 * REC, kb);
         }
@@ -453,7 +481,7 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
     uint32_t va[4], vb[4];
     if (B == 4) {
         const int l = gid * 4 + tig;
-        const uint8_t *row = sm.v[stage] + ((l & 7) + 8 * ((l >> 3) & 1)) * REC + 4 * META + 16 * (l >> 4);
+        const uint8_t *row = sm.v[stage] + ((l & 7) + 8 * ((l >> 3) & 1)) * REC + format_pairs(META) + 16 * (l >> 4);
         load_matrices_transposed(row, va);       // groups 0, 1
         load_matrices_transposed(row + 32, vb);  // groups 2, 3
     }
@@ -495,8 +523,8 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
         hp.n_kv_heads = p.n_kv_heads;
         hp.head_dim = kAttendD;
         hp.n_tokens = p.n_tokens;
-        hp.meta_bytes = META;
-        hp.group_size = kGroup;
+        hp.meta_bytes = format_meta(META);
+        hp.group_size = format_group(META);
         const uint32_t mode = hdr->bits_mode;
         int ok = 0;
         if (mode <= 1u) {
@@ -513,6 +541,9 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
         fence_mbar_init();
     }
     __syncthreads();
+    // the merge kernel may be brought onto the device now: it waits for this grid to complete
+    // before it reads anything
+    allow_dependents();
     if (!s_header_ok) {
         if (threadIdx.x == 0 && p.status_dev) atomicMax(p.status_dev, (int)QKVS_ERR_BAD_CARD);
         return;
@@ -569,7 +600,7 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
             const uint32_t o_first = __ldg(offs_tab), o_last = __ldg(offs_tab + n_tok);
             const uint32_t b0 = __shfl_sync(0xffffffffu, w8.x, 0) & 0xffu;
             const bool same = w8.x == b0 * 0x01010101u && w8.y == w8.x;
-            const uint32_t rec = record_bytes(kAttendD, (int)b0, META);
+            const uint32_t rec = record_bytes(kAttendD, (int)b0, format_meta(META), format_group(META));
             one_width = __all_sync(0xffffffffu, same) && base_ok && rec != 0u && (o_first & 15u) == 0u && o_last >= o_first &&
                         o_last - o_first == (uint32_t)n_tok * rec && (uint64_t)o_last <= room_k && (uint64_t)o_last <= room_v;
             try_one_width = one_width;
@@ -600,7 +631,7 @@ __global__ void __launch_bounds__(WARPS * 32, QKVS_ATTEND_CTAS) attend_kernel(At
                     my_cls[r] = 4;
                     if (j < n_tok) {
                         const uint32_t b = __ldg(bits_tab + j);
-                        const uint32_t rec = record_bytes(kAttendD, (int)b, META);
+                        const uint32_t rec = record_bytes(kAttendD, (int)b, format_meta(META), format_group(META));
                         const bool fine = base_ok && rec != 0u && o_next >= o && o_next - o == rec && (o & 15u) == 0u &&
                                           (uint64_t)o_next <= room_k && (uint64_t)o_next <= room_v;
                         bad |= !fine;
@@ -791,6 +822,7 @@ __global__ void __launch_bounds__(128) attend_merge_kernel(AttendParams p)
     __shared__ float4 s_o[4][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t w = blockIdx.x;
+    grid_dependency_wait();   // launched while the first kernel may still run: its results are complete from here on
     const int per_kv = p.n_q_heads / p.n_kv_heads;
     const uint32_t layer = w / (uint32_t)p.n_q_heads, j = w - layer * (uint32_t)p.n_q_heads;
     const uint32_t lh = layer * (uint32_t)p.n_kv_heads + j / (uint32_t)per_kv, jj = j % (uint32_t)per_kv;

@@ -845,7 +845,8 @@ static qkvs_status_t attend_shape(const qkvs_layout_t *layout, int32_t n_q_heads
 {
     const qkvs_status_t st = check_shape(layout);
     if (st != QKVS_OK) return st;
-    if (layout->head_dim != kAttendD || layout->group_size != kGroup) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (layout->head_dim != kAttendD) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (layout->group_size != kGroup && attend_on_tcgen05()) return QKVS_ERR_UNSUPPORTED_SHAPE;  // that variant reads groups of 32 only
     if (n_q_heads < layout->n_kv_heads || n_q_heads % layout->n_kv_heads != 0) return QKVS_ERR_INVALID_ARG;
     if (n_q_heads / layout->n_kv_heads > kAttendMaxPerKv) return QKVS_ERR_UNSUPPORTED_SHAPE;
     memset(p, 0, sizeof(*p));
@@ -870,6 +871,42 @@ static size_t attend_scratch_bytes(const AttendParams &p)
     return (size_t)QKVS_WORKSPACE_BYTES + (size_t)p.n_items * per_kv * kPartialFloats * sizeof(float);
 }
 
+extern "C++" {
+#ifndef QKVS_ATTEND_STAGES
+#define QKVS_ATTEND_STAGES 2
+#endif
+#ifndef QKVS_ATTEND_WARPS
+#define QKVS_ATTEND_WARPS 8  // two CTAs of eight warps per SM: neighbouring items, i.e. neighbouring spans of a stream, start together
+#endif
+constexpr int kAttendStages = QKVS_ATTEND_STAGES, kAttendWarps = QKVS_ATTEND_WARPS;
+
+// One instance of the mma.sync kernel per record format (pair size x group size).
+template <int FMT>
+static qkvs_status_t launch_attend_format(const AttendParams &p, cudaStream_t cs)
+{
+    auto kernel = attend_kernel<kAttendStages, kAttendWarps, FMT>;
+    const size_t smem = kAttendWarps * sizeof(AttendWarpSmem<kAttendStages>);
+    unsigned grid = 0;
+    if (persistent_grid<1000 + FMT>(kernel, kAttendWarps * 32, smem, (int64_t)((p.n_items + kAttendWarps - 1) / kAttendWarps), &grid) != cudaSuccess)
+        return QKVS_ERR_CUDA;
+    kernel<<<grid, kAttendWarps * 32, smem, cs>>>(p);
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+}
+
+static qkvs_status_t launch_attend(const AttendParams &p, int group_size, cudaStream_t cs)
+{
+    switch (format_code(p.meta_bytes, group_size)) {
+        case format_code(kMetaFp32, 32): return launch_attend_format<format_code(kMetaFp32, 32)>(p, cs);
+        case format_code(kMetaFp16, 32): return launch_attend_format<format_code(kMetaFp16, 32)>(p, cs);
+        case format_code(kMetaFp32, 64): return launch_attend_format<format_code(kMetaFp32, 64)>(p, cs);
+        case format_code(kMetaFp16, 64): return launch_attend_format<format_code(kMetaFp16, 64)>(p, cs);
+        case format_code(kMetaFp32, 128): return launch_attend_format<format_code(kMetaFp32, 128)>(p, cs);
+        case format_code(kMetaFp16, 128): return launch_attend_format<format_code(kMetaFp16, 128)>(p, cs);
+        default: return QKVS_ERR_UNSUPPORTED_SHAPE;
+    }
+}
+}  // extern "C++"
+
 qkvs_status_t qkvs_attend_scratch_size(const qkvs_layout_t *layout, int32_t n_q_heads, size_t *out_bytes)
 {
     AttendParams p;
@@ -884,13 +921,6 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
                                const void *q_dev, float softmax_scale, float *out_dev, void *scratch_dev,
                                size_t scratch_bytes, void *stream)
 {
-#ifndef QKVS_ATTEND_STAGES
-#define QKVS_ATTEND_STAGES 2
-#endif
-#ifndef QKVS_ATTEND_WARPS
-#define QKVS_ATTEND_WARPS 8  // two CTAs of eight warps per SM: neighbouring items, i.e. neighbouring spans of a stream, start together
-#endif
-    constexpr int kAttendStages = QKVS_ATTEND_STAGES, kAttendWarps = QKVS_ATTEND_WARPS;
     AttendParams p;
     const qkvs_status_t st = attend_shape(layout, n_q_heads, &p);
     if (st != QKVS_OK) return st;
@@ -921,20 +951,24 @@ qkvs_status_t qkvs_card_attend(const void *card_dev, size_t card_bytes, const qk
         kernel<<<grid, kTcThreads, smem, cs>>>(p);
         if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
     } else if (p.n_items > 0) {
-        const bool compact = p.meta_bytes == kMetaFp16;
-        auto kernel = compact ? attend_kernel<kAttendStages, kAttendWarps, kMetaFp16> : attend_kernel<kAttendStages, kAttendWarps, kMetaFp32>;
-        const size_t smem = kAttendWarps * sizeof(AttendWarpSmem<kAttendStages>);
-        unsigned grid = 0;
-        if ((compact ? persistent_grid<1001>(kernel, kAttendWarps * 32, smem, (int64_t)((p.n_items + kAttendWarps - 1) / kAttendWarps), &grid)
-                     : persistent_grid<1000>(kernel, kAttendWarps * 32, smem, (int64_t)((p.n_items + kAttendWarps - 1) / kAttendWarps), &grid)) !=
-            cudaSuccess)
-            return QKVS_ERR_CUDA;
-        kernel<<<grid, kAttendWarps * 32, smem, cs>>>(p);
-        if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
+        const qkvs_status_t ls = launch_attend(p, layout->group_size, cs);
+        if (ls != QKVS_OK) return ls;
     }
+    // the merge is launched so that it can come onto the device while the first kernel drains
+    // (it waits for that kernel's completion before its first read)
     const unsigned rows = (unsigned)p.n_layers * (unsigned)p.n_q_heads;
-    attend_merge_kernel<<<rows, 128, 0, cs>>>(p);
-    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(rows);
+    cfg.blockDim = dim3(128);
+    cfg.stream = cs;
+    cudaLaunchAttribute attr;
+    memset(&attr, 0, sizeof(attr));
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, attend_merge_kernel, p) == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 
 qkvs_status_t qkvs_bits_from_scores(const float *scores_dev, int32_t n_segments, int32_t n_tokens, int32_t n_fp16,

@@ -97,10 +97,51 @@ def test_sizes_padding_and_mismatch_are_refused():
         stat, Kg, _ = gpu_inject(q, card, q.make_layout(L, H, d, T, group_size=other), [np.full((H, T, d), -3.0, np.float16)],
                                  [np.full((H, T, d), -5.0, np.float16)])
         assert stat == q.binding.ERR_BAD_CARD and np.all(Kg[0] == -3.0)
-    # attention straight from the card is built for groups of 32
-    with pytest.raises(q.QkvsError) as e:
-        q.attend_scratch_size(q.make_layout(L, H, d, T, group_size=64), 4)
-    assert e.value.status == q.binding.ERR_UNSUPPORTED_SHAPE
+
+
+def _attend(card_np, lay, qh):
+    import torch
+    card = torch.from_numpy(np.ascontiguousarray(card_np)).cuda()
+    out = torch.full(qh.shape, 7.0, dtype=torch.float32, device="cuda")
+    scratch = torch.full((q.attend_scratch_size(lay, qh.shape[1]),), 0x5A, dtype=torch.uint8, device="cuda")
+    q.card_attend(card, lay, torch.from_numpy(qh).cuda(), out, scratch)
+    torch.cuda.synchronize()
+    return int(scratch[:4].view(torch.int32).item()), out.cpu().numpy()
+
+
+@pytest.mark.parametrize("group,meta", [(64, 8), (64, 4), (128, 8), (128, 4)])
+@pytest.mark.parametrize("T,uniform", [(1, 0), (100, 0), (530, 0), (1000, 4), (300, 2), (300, 8)])
+def test_attention_from_a_wide_group_card(group, meta, T, uniform):
+    """Attention straight from the card reads wide groups too (head_dim 128): against the oracle's
+    attention over the values the records stand for, tolerance as for groups of 32
+    (2^-9 of the head's largest reconstructed value: the weights are rounded to FP16)."""
+    L, H, d, nq = 2, 2, 128, 8
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=40 + T)
+    bits = np.full(T, uniform, np.uint8) if uniform else wl.iid_bits(T, (0.3, 0.3, 0.2, 0.2), seed=T)
+    olay = oracle.make_layout(L, H, d, T, meta_bytes=meta, group_size=group)
+    st, card = oracle.card_create(olay, Ks, Vs, bits)
+    assert st == oracle.OK
+    qh = wl.random_fp16((L, nq, d), 77 + T)
+    st, want = oracle.card_attend(card, olay, qh)
+    assert st == oracle.OK
+    status, got = _attend(card, q.make_layout(L, H, d, T, meta_bytes=meta, group_size=group), qh)
+    assert status == 0
+    Kr, Vr = [np.zeros_like(k) for k in Ks], [np.zeros_like(v) for v in Vs]
+    assert oracle.card_inject(card, olay, Kr, Vr) == oracle.OK
+    for l in range(L):
+        for j in range(nq):
+            vmax = float(np.abs(Vr[l][j // (nq // H)][:T, :d].astype(np.float64)).max())
+            assert float(np.abs(got[l, j] - want[l, j]).max()) <= 2.0 ** -9 * vmax + 1e-6, (l, j)
+
+
+def test_attention_refuses_a_card_of_another_group_size():
+    L, H, d, T = 1, 2, 128, 40
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=6)
+    _, card = oracle.card_create(oracle.make_layout(L, H, d, T, group_size=64), Ks, Vs, np.full(T, 4, np.uint8))
+    qh = wl.random_fp16((L, 4, d), 7)
+    for other in (32, 128):
+        status, got = _attend(card, q.make_layout(L, H, d, T, group_size=other), qh)
+        assert status == q.binding.ERR_BAD_CARD and np.all(got == 0.0)
 
 
 def test_full_size_llama_8k_adaptive_groups_of_64():
