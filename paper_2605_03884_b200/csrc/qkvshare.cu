@@ -98,8 +98,80 @@ __device__ __forceinline__ void zero_fill(uint8_t *p, uint64_t begin, uint64_t e
     for (uint64_t i = begin + threadIdx.x; i < end; i += blockDim.x) p[i] = 0;
 }
 
+// bits_mode 1 only: the CTA that finishes last turns the per-segment totals into the stream-base
+// table, pads the tables with zeros and completes the header.  The other CTAs' results are read
+// past the first-level cache.  Works for any block size that is a multiple of 32.
+__device__ void finalize_card(const ScanParams &p, uint64_t *s_carry_ptr, uint64_t *s_warp)
+{
+    uint64_t &s_carry = *s_carry_ptr;
+    const int64_t T = p.n_tokens;
+    const int H = p.n_kv_heads;
+    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
+    const int64_t nseg = (int64_t)p.n_layers * H;
+    const int64_t S = 2 * nseg;
+    qkvs_card_header_t *h = reinterpret_cast<qkvs_card_header_t *>(p.card);
+    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off);
+    uint64_t *sbase = reinterpret_cast<uint64_t *>(p.card + sec.sbase_off);
+    const bool bad = __ldcg(&h->status) != QKVS_OK;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < S; base += blockDim.x) {
+        const int64_t s = base + threadIdx.x;
+        uint64_t v = 0;
+        if (s < S && !bad) {
+            const int64_t l = s / (2 * H), hh = s % H;
+            v = __ldcg(offs + (l * H + hh) * (T + 1) + T);
+        }
+        uint64_t inc = v;
+#pragma unroll
+        for (int k = 1; k < 32; k <<= 1) {
+            const uint64_t n = __shfl_up_sync(0xffffffffu, inc, k);
+            if (lane >= k) inc += n;
+        }
+        if (lane == 31) s_warp[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            const uint64_t w = lane < (int)(blockDim.x >> 5) ? s_warp[lane] : 0u;
+            uint64_t winc = w;
+#pragma unroll
+            for (int k = 1; k < 32; k <<= 1) {
+                const uint64_t n = __shfl_up_sync(0xffffffffu, winc, k);
+                if (lane >= k) winc += n;
+            }
+            s_warp[lane] = winc - w;
+            if (lane == 31) s_warp[32] = winc;
+        }
+        __syncthreads();
+        if (s < S) sbase[s] = bad ? 0 : s_carry + s_warp[warp] + inc - v;
+        __syncthreads();
+        if (threadIdx.x == 0) s_carry += s_warp[32];
+        __syncthreads();
+    }
+    zero_fill(p.card, sec.bits_off + (uint64_t)nseg * (uint64_t)T, sec.offs_off);
+    zero_fill(p.card, sec.offs_off + 4u * (uint64_t)nseg * (uint64_t)(T + 1), sec.sbase_off);
+    zero_fill(p.card, sec.sbase_off + 8u * (uint64_t)(S + 1), sec.payload_off);
+    if (threadIdx.x == 0) {
+        const uint64_t payload = s_carry;
+        sbase[S] = bad ? 0 : payload;
+        uint32_t status = __ldcg(&h->status);
+        const uint64_t total = sec.payload_off + payload;
+        if (status == QKVS_OK && total > p.capacity) status = QKVS_ERR_BUFFER_TOO_SMALL;
+        const uint64_t sb = __ldcg(&h->sum_bits);
+        write_header_static(h, p, sec);
+        h->status = status;
+        const bool ok = status == QKVS_OK;
+        h->sum_bits = ok ? sb : 0;
+        h->avg_code_bits = (ok && nseg * T > 0) ? __fdiv_rn((float)sb, (float)(uint64_t)(nseg * T)) : 0.0f;
+        h->stream_bytes = 0;
+        h->total_bytes = ok ? total : 0;
+        *reinterpret_cast<uint32_t *>(h->reserved_) = 0u;   // the count of finished CTAs
+    }
+}
+
 // One CTA per segment.  bits_mode 0 has a single segment, and its CTA also finishes the
-// header; in bits_mode 1 the per-segment results are combined by finalize_kernel.
+// header; in bits_mode 1 the CTA that finishes last combines the per-segment results (the header,
+// cleared before the launch, counts the finished CTAs in its reserved bytes meanwhile).
 __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p)
 {
     __shared__ uint32_t warp_sums[33];
@@ -209,81 +281,23 @@ __global__ void __launch_bounds__(kScanThreads) scan_offsets_kernel(ScanParams p
             h->stream_bytes = ok ? carry : 0;
             h->total_bytes = ok ? total : 0;
         }
-    } else if (threadIdx.x == 0) {
-        // header was cleared before this launch; combine across segments
-        atomicAdd(reinterpret_cast<unsigned long long *>(&h->sum_bits), s_sum);
-        if (s_bad) atomicMax(&h->status, (uint32_t)QKVS_ERR_BAD_BITS);
-    }
-}
-
-// bits_mode 1 only: one CTA turns the per-segment totals into the stream-base table, pads the
-// tables with zeros and completes the header.
-__global__ void __launch_bounds__(kScanThreads) finalize_kernel(ScanParams p)
-{
-    __shared__ uint64_t s_carry;
-    __shared__ uint64_t s_warp[33];
-    allow_dependents();
-    const int64_t T = p.n_tokens;
-    const int H = p.n_kv_heads;
-    const Sections sec = card_sections(p.n_layers, p.n_kv_heads, p.n_tokens, p.bits_mode);
-    const int64_t nseg = (int64_t)p.n_layers * H;
-    const int64_t S = 2 * nseg;
-    qkvs_card_header_t *h = reinterpret_cast<qkvs_card_header_t *>(p.card);
-    const uint32_t *offs = reinterpret_cast<const uint32_t *>(p.card + sec.offs_off);
-    uint64_t *sbase = reinterpret_cast<uint64_t *>(p.card + sec.sbase_off);
-    const bool bad = h->status != QKVS_OK;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) s_carry = 0;
-    __syncthreads();
-    for (int64_t base = 0; base < S; base += kScanThreads) {
-        const int64_t s = base + threadIdx.x;
-        uint64_t v = 0;
-        if (s < S && !bad) {
-            const int64_t l = s / (2 * H), hh = s % H;
-            v = offs[(l * H + hh) * (T + 1) + T];
+    } else {
+        __shared__ int s_last;
+        __shared__ uint64_t s_carry;
+        __shared__ uint64_t s_warp64[33];
+        if (threadIdx.x == 0) {
+            // header was cleared before this launch; combine across segments
+            atomicAdd(reinterpret_cast<unsigned long long *>(&h->sum_bits), s_sum);
+            if (s_bad) atomicMax(&h->status, (uint32_t)QKVS_ERR_BAD_BITS);
         }
-        uint64_t inc = v;
-#pragma unroll
-        for (int k = 1; k < 32; k <<= 1) {
-            const uint64_t n = __shfl_up_sync(0xffffffffu, inc, k);
-            if (lane >= k) inc += n;
+        __threadfence();   // this CTA's table entries, before it counts as finished
+        __syncthreads();
+        if (threadIdx.x == 0) s_last = atomicAdd(reinterpret_cast<uint32_t *>(h->reserved_), 1u) + 1u == gridDim.x;
+        __syncthreads();
+        if (s_last) {
+            __threadfence();
+            finalize_card(p, &s_carry, s_warp64);
         }
-        if (lane == 31) s_warp[warp] = inc;
-        __syncthreads();
-        if (warp == 0) {
-            const uint64_t w = s_warp[lane];
-            uint64_t winc = w;
-#pragma unroll
-            for (int k = 1; k < 32; k <<= 1) {
-                const uint64_t n = __shfl_up_sync(0xffffffffu, winc, k);
-                if (lane >= k) winc += n;
-            }
-            s_warp[lane] = winc - w;
-            if (lane == 31) s_warp[32] = winc;
-        }
-        __syncthreads();
-        if (s < S) sbase[s] = bad ? 0 : s_carry + s_warp[warp] + inc - v;
-        __syncthreads();
-        if (threadIdx.x == 0) s_carry += s_warp[32];
-        __syncthreads();
-    }
-    zero_fill(p.card, sec.bits_off + (uint64_t)nseg * (uint64_t)T, sec.offs_off);
-    zero_fill(p.card, sec.offs_off + 4u * (uint64_t)nseg * (uint64_t)(T + 1), sec.sbase_off);
-    zero_fill(p.card, sec.sbase_off + 8u * (uint64_t)(S + 1), sec.payload_off);
-    if (threadIdx.x == 0) {
-        const uint64_t payload = s_carry;
-        sbase[S] = bad ? 0 : payload;
-        uint32_t status = h->status;
-        const uint64_t total = sec.payload_off + payload;
-        if (status == QKVS_OK && total > p.capacity) status = QKVS_ERR_BUFFER_TOO_SMALL;
-        write_header_static(h, p, sec);
-        h->status = status;
-        const bool ok = status == QKVS_OK;
-        const uint64_t sb = h->sum_bits;
-        h->sum_bits = ok ? sb : 0;
-        h->avg_code_bits = (ok && nseg * T > 0) ? __fdiv_rn((float)sb, (float)(uint64_t)(nseg * T)) : 0.0f;
-        h->stream_bytes = 0;
-        h->total_bytes = ok ? total : 0;
     }
 }
 
@@ -661,13 +675,12 @@ qkvs_status_t qkvs_card_create(const qkvs_layout_t *layout, const void *const *K
     if (layout->bits_mode == 1 && cudaMemsetAsync(card_dev, 0, kHeaderBytes, cs) != cudaSuccess) return QKVS_ERR_CUDA;
     // no more threads than there are groups of eight tokens: a short context then pays for the
     // block-wide steps of four warps, not of thirty-two
-    const int scan_threads = (int)std::min<int64_t>(kScanThreads, std::max<int64_t>(32, (((int64_t)layout->n_tokens + kScanItems - 1) / kScanItems + 31) / 32 * 32));
+    // ... and with a segment per (layer, head) CTAs of 256 threads, of which every SM holds several:
+    // a thousand threads at the kernel's register count leave one CTA per SM and a second round
+    const int64_t most_threads = nseg > 1 ? 256 : kScanThreads;
+    const int scan_threads = (int)std::min<int64_t>(most_threads, std::max<int64_t>(32, (((int64_t)layout->n_tokens + kScanItems - 1) / kScanItems + 31) / 32 * 32));
     scan_offsets_kernel<<<nseg, scan_threads, 0, cs>>>(sp);
     if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
-    if (layout->bits_mode == 1) {
-        finalize_kernel<<<1, kScanThreads, 0, cs>>>(sp);
-        if (cudaGetLastError() != cudaSuccess) return QKVS_ERR_CUDA;
-    }
 
     PathParams p;
     memset(&p, 0, sizeof(p));
