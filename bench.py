@@ -588,21 +588,36 @@ def run_ours(args):
     if not args.no_cpu_baseline:
         cpu = cpu_oracle_leg(w, case.Ks, case.Vs, case.bits_per_hop[0][:T], L, args.meta_bytes)
 
-    # the step in front of the path: bit-widths from importance scores by rank (config 4's recipe)
+    # the step in front of the path: bit-widths from importance scores (config 4's recipe by rank;
+    # the same under a byte budget of 100 bytes per token, with the offset table from the same
+    # launch), at the workload's length and at 128K tokens
     rank_us = None
+    bits_rules = None
     if not args.skip_attend:
-        sc = torch.randn(T, device="cuda").exp()
-        bd = torch.zeros(T, dtype=torch.uint8, device="cuda")
-        c16, c8, c4 = wl.quantile_counts(T)
-        for _ in range(5):
-            q.bits_from_scores(sc, c16, c8, c4, bd, stream=stream)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(50):  # back to back: one call alone would time the host's launch latency
-            q.bits_from_scores(sc, c16, c8, c4, bd, stream=stream)
-        b.record(stream)
-        torch.cuda.synchronize()
-        rank_us = a.elapsed_time(b) * 1e3 / 50
+        def timed_us(fn, reps):
+            for _ in range(5):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):  # back to back: one call alone would time the host's launch latency
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) * 1e3 / reps
+
+        bits_rules = {}
+        for n_tok, reps in ((T, 50), (131072, 10)):
+            sc = torch.randn(n_tok, device="cuda").exp()
+            bd = torch.zeros(n_tok, dtype=torch.uint8, device="cuda")
+            od = torch.zeros(n_tok + 1, dtype=torch.int32, device="cuda")
+            c16, c8, c4 = wl.quantile_counts(n_tok)
+            by_rank = timed_us(lambda: q.bits_from_scores(sc, c16, c8, c4, bd, stream=stream), reps)
+            by_budget = timed_us(lambda: q.bits_from_scores_budget(sc, d, 100 * n_tok, bd, meta_bytes=args.meta_bytes,
+                                                                   offsets_dev=od, stream=stream), reps)
+            bits_rules[str(n_tok)] = {"by_rank_us": by_rank, "by_budget_with_offsets_us": by_budget}
+            if n_tok == T:
+                rank_us = by_rank
+            del sc, bd, od
 
     # the other benchmark workloads and card formats, a few steps each, after the headline timing
     # and outside it: the 1K mixed cache, the 8K adaptive cache, the four-hop chain; then the 8K
@@ -660,6 +675,7 @@ def run_ours(args):
         "clocks": clocks,
         "attend_from_card": attend,
         "bits_from_scores_us": rank_us,
+        "bits_from_scores": bits_rules,
         "per_config": per_config,
     }
     print(json.dumps(line))

@@ -414,24 +414,26 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
             }
         }
     }
-    // ---- running softmax of heads 2tig and 2tig + 1 (the maximum goes over all 16 tokens: the
-    // eight lanes of a tig)
-    float pr[2][2], alpha[2];
+    // ---- running softmax of heads 2tig and 2tig + 1.  The running maximum only moves when some
+    // token of the step exceeds it, which after the first steps of an item is rare: one vote
+    // decides whether the step goes through the reduction over its 16 tokens (the eight lanes of
+    // a tig), the factor for what has been summed so far and the rescaling of the accumulators.
+    float pr[2][2];
+    const bool above = x[0][0] > m_run[0] || x[1][0] > m_run[0] || x[0][1] > m_run[1] || x[1][1] > m_run[1];
+    if (__any_sync(0xffffffffu, above)) {
+        float alpha[2];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        float m_loc = fmaxf(x[0][h], x[1][h]);
-        m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 4));
-        m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 8));
-        m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 16));
-        const float m_new = fmaxf(m_run[h], m_loc);
-        const float m_ref = m_new == -INFINITY ? 0.0f : m_new;
-        alpha[h] = exp2_approx(m_run[h] - m_ref);  // 0 on the first tokens of the item
-        pr[0][h] = exp2_approx(x[0][h] - m_ref);
-        pr[1][h] = exp2_approx(x[1][h] - m_ref);
-        l_run[h] = fmaf(l_run[h], alpha[h], pr[0][h] + pr[1][h]);
-        m_run[h] = m_new;
-    }
-    if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
+        for (int h = 0; h < 2; ++h) {
+            float m_loc = fmaxf(x[0][h], x[1][h]);
+            m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 4));
+            m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 8));
+            m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 16));
+            const float m_new = fmaxf(m_run[h], m_loc);
+            const float m_ref = m_new == -INFINITY ? 0.0f : m_new;
+            alpha[h] = exp2_approx(m_run[h] - m_ref);  // 0 on the first tokens of the item
+            l_run[h] *= alpha[h];
+            m_run[h] = m_new;
+        }
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
             zacc[g][0] *= alpha[0];
@@ -444,6 +446,13 @@ __device__ __forceinline__ void attend_step(const AttendWarpSmem<NS> &sm, int st
                 acc[g][j][3] *= alpha[1];
             }
         }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const float m_ref = m_run[h] == -INFINITY ? 0.0f : m_run[h];
+        pr[0][h] = exp2_approx(x[0][h] - m_ref);
+        pr[1][h] = exp2_approx(x[1][h] - m_ref);
+        l_run[h] += pr[0][h] + pr[1][h];
     }
     // ---- values.  The weights p_t * scale_tg are formed where the probabilities are (tokens gid,
     // gid + 8 x heads 2tig, 2tig + 1), rounded to FP16 and transposed inside the warp into the B
