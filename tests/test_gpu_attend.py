@@ -87,6 +87,14 @@ def test_mixed_bits_ragged_lengths(T):
     _check(Ks, Vs, bits, L, H, d, T, nq, seed=T)
 
 
+def test_long_context_with_a_ragged_end():
+    """131 109 tokens per head: 513 work items per head, the last one with 37 tokens."""
+    L, H, d, T, nq = 1, 2, 128, 131072 + 37, 8
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=305)
+    bits = wl.iid_bits(T, (0.3, 0.4, 0.2, 0.1), seed=306)
+    _check(Ks, Vs, bits, L, H, d, T, nq, seed=307, label="long context, mixed widths")
+
+
 @pytest.mark.parametrize("b", [2, 4, 8, 16])
 def test_uniform_bits(b):
     L, H, d, T, nq = 1, 2, 128, 700, 8

@@ -188,6 +188,16 @@ def test_per_head_bits_mode():
     assert _check_inject(card, L, H, d, T) == 0
 
 
+def test_long_context_with_a_ragged_end():
+    """131 109 tokens of one (layer, head): far beyond the benchmark's lengths, offsets past 2^24,
+    a last sub-tile of five rows; whole card and whole cache compared."""
+    L, H, d, T = 1, 1, 128, 131072 + 37
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=43)
+    bits = wl.iid_bits(T, (0.3, 0.4, 0.2, 0.1), 44)
+    card = _check_card(Ks, Vs, bits, L, H, d, T)
+    assert _check_inject(card, L, H, d, T) == 0
+
+
 def test_many_layers_span_several_launches():
     """More layers than one launch's pointer block carries."""
     L, H, d, T = 70, 1, 64, 20
