@@ -103,6 +103,8 @@ def lib():
         l.orc_bits_from_scores_budget.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_uint64, C.c_void_p, C.c_void_p]
         l.orc_combine_scores.restype = C.c_int
         l.orc_combine_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int64, C.c_void_p]
+        l.orc_bits_from_features.restype = C.c_int
+        l.orc_bits_from_features.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         l.orc_card_attend.restype = C.c_int
         l.orc_card_attend.argtypes = [C.c_void_p, C.c_uint64, C.POINTER(Layout), C.c_int, C.c_void_p, C.c_double, C.c_void_p]
         l.orc_card_attend_injected.restype = C.c_int
@@ -354,6 +356,18 @@ def combine_scores(importance: np.ndarray, transfer: np.ndarray, alpha: float) -
     out = np.zeros(imp.shape, dtype=np.float32)
     st = lib().orc_combine_scores(_ptr(imp), _ptr(tra), C.c_float(alpha), imp.size, _ptr(out))
     return st, out
+
+
+def bits_from_features(features: np.ndarray, hidden: int, params: np.ndarray) -> Tuple[int, np.ndarray, np.ndarray]:
+    """(status, bits [n], outputs [n, 4]) of the two-layer controller (see orc_bits_from_features).
+    features: [n, 6]; params: W1 [hidden, 6], b1 [hidden], W2 [4, hidden], b2 [4] flattened in this order."""
+    x = np.ascontiguousarray(features, dtype=np.float32).reshape(-1, 6)
+    w = np.ascontiguousarray(params, dtype=np.float32).reshape(-1)
+    assert w.size == 11 * hidden + 4
+    bits = np.zeros(x.shape[0], dtype=np.uint8)
+    outs = np.zeros((x.shape[0], 4), dtype=np.float32)
+    st = lib().orc_bits_from_features(_ptr(x), x.shape[0], int(hidden), _ptr(w), _ptr(bits), _ptr(outs))
+    return st, bits, outs
 
 
 def num_threads() -> int:

@@ -960,6 +960,50 @@ int orc_combine_scores(const float *importance, const float *transfer, float alp
     return ORC_OK;
 }
 
+/* Bit-widths from the controller of Section 4.1.2: a two-layer perceptron over six features per
+ * token (frequency, quality, attention variance, entropy, downstream demand, segment type) whose
+ * four outputs stand for the bit-widths 2, 4, 8, 16; the token gets the one with the largest
+ * output.  The paper gives the shape (6 -> hidden -> 4, "512 parameters") and no formula; the
+ * reading taken here: hidden_j = max(0, b1[j] + sum_i W1[j][i] x[i]), out_k = b2[k] + sum_j
+ * W2[k][j] hidden_j, sums taken in index order starting from the bias, every product and every
+ * sum rounded to binary32 on its own; the largest output wins, equal outputs go to the fewer bits.
+ *   features  [n][6]; params: W1 [hidden][6], b1 [hidden], W2 [4][hidden], b2 [4], one after another
+ *   bits      [n]; outputs (optional) [n][4] */
+int orc_bits_from_features(const float *features, int64_t n, int hidden, const float *params, uint8_t *bits, float *outputs)
+{
+    static const int ladder[4] = {2, 4, 8, 16};
+    if (n < 0 || hidden < 1 || hidden > 128) return ORC_INVALID_ARG;
+    const float *w1 = params, *b1 = w1 + 6 * hidden, *w2 = b1 + hidden, *b2 = w2 + 4 * hidden;
+    for (int64_t t = 0; t < n; ++t) {
+        const float *x = features + 6 * t;
+        float hid[128];
+        for (int j = 0; j < hidden; ++j) {
+            float acc = b1[j];
+            for (int i = 0; i < 6; ++i) {
+                const float prod = w1[6 * j + i] * x[i];
+                acc = acc + prod;
+            }
+            hid[j] = acc > 0.0f ? acc : 0.0f;
+        }
+        int best = 0;
+        float best_out = 0.0f;
+        for (int k = 0; k < 4; ++k) {
+            float acc = b2[k];
+            for (int j = 0; j < hidden; ++j) {
+                const float prod = w2[hidden * k + j] * hid[j];
+                acc = acc + prod;
+            }
+            if (outputs) outputs[4 * t + k] = acc;
+            if (k == 0 || acc > best_out) {
+                best = k;
+                best_out = acc;
+            }
+        }
+        bits[t] = (uint8_t)ladder[best];
+    }
+    return ORC_OK;
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP

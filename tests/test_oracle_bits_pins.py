@@ -227,3 +227,110 @@ def test_budget_rule_is_a_rank_rule_with_the_counts_it_arrives_at():
         st, ranked = oracle.bits_from_scores(s, n16, n8, n4)
         assert st == oracle.OK and np.array_equal(bits, ranked)
         assert np.array_equal(bits, by_library_sort(s, n16, n8, n4))
+
+
+# ---------------------------------------------------------------------------------------------
+# The controller of Section 4.1.2 (two-layer perceptron over six features -> one of four widths)
+
+def _pack(w1, b1, w2, b2):
+    return np.concatenate([np.asarray(w1, np.float32).reshape(-1), np.asarray(b1, np.float32).reshape(-1),
+                           np.asarray(w2, np.float32).reshape(-1), np.asarray(b2, np.float32).reshape(-1)])
+
+
+def test_controller_with_hand_set_weights_follows_the_rule_it_encodes():
+    """hidden_0 = relu(x0 - 1), hidden_1 = relu(x0 - 2), hidden_2 = relu(x0 - 3); outputs
+    (0.5, h0, 2 h1, 4 h2): the winner changes at x0 = 1.5, 2.5, 3.5 -- worked out by hand."""
+    w1 = np.zeros((3, 6)); w1[:, 0] = 1.0
+    b1 = [-1.0, -2.0, -3.0]
+    w2 = np.zeros((4, 3)); w2[1, 0] = 1.0; w2[2, 1] = 2.0; w2[3, 2] = 4.0
+    b2 = [0.5, 0.0, 0.0, 0.0]
+    x = np.zeros((8, 6), np.float32)
+    x[:, 0] = [0.0, 1.25, 1.75, 2.25, 2.75, 3.25, 3.75, 10.0]
+    x[:, 1:] = 7.0   # features the network does not look at
+    st, bits, outs = oracle.bits_from_features(x, 3, _pack(w1, b1, w2, b2))
+    assert st == oracle.OK
+    # x0: outputs -> winner
+    #  0.00: (0.5, 0,    0,   0)  -> 2      1.25: (0.5, 0.25, 0,   0)  -> 2
+    #  1.75: (0.5, 0.75, 0,   0)  -> 4      2.25: (0.5, 1.25, 0.5, 0)  -> 4
+    #  2.75: (0.5, 1.75, 1.5, 0)  -> 4      3.25: (0.5, 2.25, 2.5, 1)  -> 8
+    #  3.75: (0.5, 2.75, 3.5, 3)  -> 8     10.00: (0.5, 9,    16,  28) -> 16
+    assert bits.tolist() == [2, 2, 4, 4, 4, 8, 8, 16]
+    assert outs[5].tolist() == [0.5, 2.25, 2.5, 1.0] and outs[7].tolist() == [0.5, 9.0, 16.0, 28.0]
+
+
+def test_controller_rectifies_the_hidden_layer():
+    """One hidden unit with a negative pre-activation and a negative outgoing weight: without the
+    rectifier class 1 would win (-1 * -3 = 3); with it the unit is silent and the bias decides."""
+    w1 = np.zeros((1, 6)); w1[0, 2] = 1.0
+    w2 = np.zeros((4, 1)); w2[1, 0] = -1.0
+    x = np.zeros((2, 6), np.float32); x[0, 2] = -3.0; x[1, 2] = 3.0
+    st, bits, outs = oracle.bits_from_features(x, 1, _pack(w1, [0.0], w2, [0.0, 0.0, 1.0, 0.0]))
+    assert st == oracle.OK and bits.tolist() == [8, 8]
+    assert outs[0].tolist() == [0.0, 0.0, 1.0, 0.0] and outs[1].tolist() == [0.0, -3.0, 1.0, 0.0]
+
+
+def test_controller_ties_go_to_fewer_bits_and_biases_alone_decide_without_weights():
+    x = np.random.default_rng(3).standard_normal((5, 6)).astype(np.float32)
+    for b2, want in (([1, 1, 1, 1], 2), ([0, 2, 2, 1], 4), ([0, 0, 3, 3], 8), ([0, 0, 0, 1], 16)):
+        st, bits, _ = oracle.bits_from_features(x, 4, _pack(np.zeros((4, 6)), np.zeros(4), np.zeros((4, 4)), b2))
+        assert st == oracle.OK and np.all(bits == want)
+
+
+def test_controller_against_numpy_float32_step_by_step():
+    """The same network with numpy float32 scalars, one rounded operation at a time in the stated
+    order (bias first, then the terms by index)."""
+    rng = np.random.default_rng(11)
+    hidden = 46   # 11 * 46 + 4 = 510 parameters: the size nearest to the paper's 512 for this shape
+    w1 = rng.standard_normal((hidden, 6)).astype(np.float32)
+    b1 = rng.standard_normal(hidden).astype(np.float32)
+    w2 = rng.standard_normal((4, hidden)).astype(np.float32)
+    b2 = rng.standard_normal(4).astype(np.float32)
+    x = rng.standard_normal((300, 6)).astype(np.float32)
+    st, bits, outs = oracle.bits_from_features(x, hidden, _pack(w1, b1, w2, b2))
+    assert st == oracle.OK
+    ladder = [2, 4, 8, 16]
+    for t in range(x.shape[0]):
+        hid = []
+        for j in range(hidden):
+            acc = np.float32(b1[j])
+            for i in range(6):
+                acc = np.float32(acc + np.float32(w1[j, i] * x[t, i]))
+            hid.append(acc if acc > 0 else np.float32(0.0))
+        out = []
+        for k in range(4):
+            acc = np.float32(b2[k])
+            for j in range(hidden):
+                acc = np.float32(acc + np.float32(w2[k, j] * hid[j]))
+            out.append(acc)
+        assert [float(o) for o in out] == outs[t].tolist()
+        assert bits[t] == ladder[int(np.argmax(out))]   # numpy's argmax also takes the first of equals
+    assert len(set(bits.tolist())) == 4                 # every width occurs
+
+
+def test_controller_outputs_are_close_to_the_matrix_form():
+    """Against the library routine: relu(x W1^T + b1) W2^T + b2 in float64 -- equal up to the
+    rounding of float32 sums, and the same widths wherever the two largest outputs are not close."""
+    rng = np.random.default_rng(12)
+    hidden = 46
+    w1, b1 = rng.standard_normal((hidden, 6)), rng.standard_normal(hidden)
+    w2, b2 = rng.standard_normal((4, hidden)), rng.standard_normal(4)
+    x = rng.standard_normal((2000, 6))
+    st, bits, outs = oracle.bits_from_features(x, hidden, _pack(w1, b1, w2, b2))
+    f32 = lambda a: np.asarray(a, np.float32).astype(np.float64)
+    ref = np.maximum(f32(x) @ f32(w1).T + f32(b1), 0.0) @ f32(w2).T + f32(b2)
+    assert np.abs(outs - ref).max() < 1e-4
+    top2 = np.sort(ref, axis=1)[:, -2:]
+    clear = top2[:, 1] - top2[:, 0] > 1e-3
+    assert clear.sum() > 1900
+    assert np.array_equal(bits[clear], np.array([2, 4, 8, 16])[np.argmax(ref, axis=1)][clear])
+
+
+def test_controller_argument_checks():
+    x = np.zeros((1, 6), np.float32)
+    for hidden in (0, 129):
+        import ctypes as C
+        bits = np.zeros(1, np.uint8)
+        p = np.zeros(11 * 129 + 4, np.float32)
+        st = oracle.lib().orc_bits_from_features(x.ctypes.data_as(C.c_void_p), 1, hidden, p.ctypes.data_as(C.c_void_p),
+                                                 bits.ctypes.data_as(C.c_void_p), None)
+        assert st == oracle.INVALID_ARG
