@@ -229,6 +229,25 @@ QKVS_API qkvs_status_t qkvs_bits_from_scores_budget(const float *scores_dev, int
 QKVS_API qkvs_status_t qkvs_combine_scores(const float *importance_dev, const float *transfer_dev,
                                   float alpha, int64_t n, float *scores_dev, void *stream);
 
+/* Bit-widths from the controller of Section 4.1.2: a two-layer perceptron over six features per
+ * token (frequency, quality, attention variance, entropy, downstream demand, segment type) with
+ * one output per bit-width; the paper gives the shape (6 -> hidden -> 4, 512 parameters, trained)
+ * and no formula or weights, so the caller supplies the parameters and the arithmetic is fixed as
+ *     hidden_j = max(0, b1[j] + sum_i W1[j][i] * x[i]),   out_k = b2[k] + sum_j W2[k][j] * hidden_j,
+ * sums starting from the bias and taking the terms in index order, every product and every sum
+ * rounded to binary32 on its own; b(t) = 2, 4, 8, 16 for the largest of out_0..3, equal outputs
+ * going to the fewer bits.  How the features are obtained is outside this library.
+ *   features_dev  device float32 [n_tokens][6]
+ *   hidden        1..128 (46 gives 510 parameters, the size of this shape nearest to 512)
+ *   params_dev    device float32: W1 [hidden][6], b1 [hidden], W2 [4][hidden], b2 [4], in this order
+ *   bits_dev      device uint8 [n_tokens]: ready to be passed to qkvs_card_create
+ *   outputs_dev   optional device float32 [n_tokens][4]: the four outputs per token
+ * Asynchronous on `stream`.  Errors: INVALID_ARG (null or misaligned pointer, negative n_tokens,
+ * hidden < 1), UNSUPPORTED_SHAPE (hidden > 128), CUDA. */
+QKVS_API qkvs_status_t qkvs_bits_from_features(const float *features_dev, int64_t n_tokens, int32_t hidden,
+                                      const float *params_dev, uint8_t *bits_dev, float *outputs_dev,
+                                      void *stream);
+
 /* Card creation (Section 4.2.1): offset scan over the bit-widths, then fused
  * min/max -> scale/zero -> quantise -> bit-pack of every (layer, K|V, head) stream.
  *   K_layers, V_layers  HOST arrays of n_layers DEVICE pointers to FP16 blocks (16-byte aligned)

@@ -963,7 +963,7 @@ int orc_combine_scores(const float *importance, const float *transfer, float alp
 /* Bit-widths from the controller of Section 4.1.2: a two-layer perceptron over six features per
  * token (frequency, quality, attention variance, entropy, downstream demand, segment type) whose
  * four outputs stand for the bit-widths 2, 4, 8, 16; the token gets the one with the largest
- * output.  The paper gives the shape (6 -> hidden -> 4, "512 parameters") and no formula; the
+ * output.  The paper gives the shape (6 -> hidden -> 4, 512 parameters in all) and no formula; the
  * reading taken here: hidden_j = max(0, b1[j] + sum_i W1[j][i] x[i]), out_k = b2[k] + sum_j
  * W2[k][j] hidden_j, sums taken in index order starting from the bias, every product and every
  * sum rounded to binary32 on its own; the largest output wins, equal outputs go to the fewer bits.

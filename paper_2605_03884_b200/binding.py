@@ -52,7 +52,7 @@ assert C.sizeof(CardHeader) == 256
 
 EXPORTS = ("qkvs_record_bytes", "qkvs_card_size", "qkvs_card_prefix_size", "qkvs_card_create",
            "qkvs_card_inject", "qkvs_card_inject_noalloc", "qkvs_card_send", "qkvs_attend_scratch_size", "qkvs_card_attend",
-           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_bits_from_scores_budget", "qkvs_combine_scores", "qkvs_selftest_division",
+           "qkvs_card_info", "qkvs_bits_from_scores", "qkvs_bits_from_scores_budget", "qkvs_combine_scores", "qkvs_bits_from_features", "qkvs_selftest_division",
            "qkvs_selftest_bounded_wait", "qkvs_status_string",
            "qkvs_version")
 
@@ -95,6 +95,8 @@ def load_library(path: Optional[str] = None):
     lib.qkvs_bits_from_scores_budget.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, vp, vp, vp, vp, vp]
     lib.qkvs_combine_scores.restype = C.c_int
     lib.qkvs_combine_scores.argtypes = [vp, vp, C.c_float, C.c_int64, vp, vp]
+    lib.qkvs_bits_from_features.restype = C.c_int
+    lib.qkvs_bits_from_features.argtypes = [vp, C.c_int64, C.c_int32, vp, vp, vp, vp]
     lib.qkvs_card_info.restype = C.c_int
     lib.qkvs_card_info.argtypes = [vp, vp, C.POINTER(CardHeader)]
     lib.qkvs_selftest_division.restype = C.c_int
@@ -327,6 +329,19 @@ def combine_scores(importance_dev, transfer_dev, alpha: float, scores_dev, strea
                                             n, int(scores_dev.data_ptr()), _stream_handle(stream))
     if check and st != OK:
         raise QkvsError(st, "qkvs_combine_scores")
+    return st
+
+
+def bits_from_features(features_dev, hidden: int, params_dev, bits_dev, outputs_dev=None, stream=None, check: bool = True) -> int:
+    """qkvs_bits_from_features.  features_dev: CUDA float32 [n, 6]; params_dev: CUDA float32 of
+    11 * hidden + 4 elements (W1, b1, W2, b2); bits_dev: CUDA uint8 [n]; outputs_dev: optional CUDA
+    float32 [n, 4]."""
+    n = int(features_dev.shape[0])
+    st = load_library().qkvs_bits_from_features(
+        int(features_dev.data_ptr()), n, int(hidden), int(params_dev.data_ptr()), int(bits_dev.data_ptr()),
+        int(outputs_dev.data_ptr()) if outputs_dev is not None else None, _stream_handle(stream))
+    if check and st != OK:
+        raise QkvsError(st, "qkvs_bits_from_features")
     return st
 
 

@@ -312,6 +312,52 @@ __global__ void __launch_bounds__(256) combine_scores_kernel(const float *__rest
 }
 
 // ---------------------------------------------------------------------------------------------
+// The controller of Section 4.1.2 as a two-layer perceptron: six features per token -> hidden
+// units (rectified) -> four outputs, one per bit-width; the largest output wins, equal outputs go
+// to the fewer bits.  One thread per token, the parameters in shared memory; sums start from the
+// bias and take the terms in index order, every product and every sum one rounded binary32
+// operation (nothing fused), so that the outputs are the same bits wherever they are computed.
+constexpr int kControllerMaxHidden = 128;
+
+__global__ void __launch_bounds__(256) controller_kernel(const float *__restrict__ features, int64_t n, int hidden,
+                                                         const float *__restrict__ params, uint8_t *bits, float *outputs)
+{
+    __shared__ float s_params[11 * kControllerMaxHidden + 4];
+    for (int i = threadIdx.x; i < 11 * hidden + 4; i += blockDim.x) s_params[i] = params[i];
+    __syncthreads();
+    const float *w1 = s_params, *b1 = w1 + 6 * hidden, *w2 = b1 + hidden, *b2 = w2 + 4 * hidden;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < n; t += stride) {
+        float x[6];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) x[i] = features[6 * t + i];
+        float out[4] = {b2[0], b2[1], b2[2], b2[3]};
+        for (int j = 0; j < hidden; ++j) {
+            float acc = b1[j];
+#pragma unroll
+            for (int i = 0; i < 6; ++i) acc = __fadd_rn(acc, __fmul_rn(w1[6 * j + i], x[i]));
+            const float h = acc > 0.0f ? acc : 0.0f;
+            // the four output sums advance together: each still takes its terms in the order of j
+#pragma unroll
+            for (int k = 0; k < 4; ++k) out[k] = __fadd_rn(out[k], __fmul_rn(w2[hidden * k + j], h));
+        }
+        int best = 0;
+        float best_out = out[0];
+#pragma unroll
+        for (int k = 1; k < 4; ++k)
+            if (out[k] > best_out) {
+                best = k;
+                best_out = out[k];
+            }
+        bits[t] = (uint8_t)(2 << best);   // 2, 4, 8, 16
+        if (outputs) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) outputs[4 * t + k] = out[k];
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Self-test of the two division shortcuts against the IEEE division, over every range value the
 // path can produce (binary32 values from 2^-24 to 131008) and the three qmax values.
 
@@ -1048,6 +1094,20 @@ qkvs_status_t qkvs_combine_scores(const float *importance_dev, const float *tran
     const float beta = 1.0f - alpha;  // one rounded subtraction on the host, as in the definition
     const unsigned grid = (unsigned)std::min<int64_t>((n + 255) / 256, 148 * 8);
     combine_scores_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(importance_dev, transfer_dev, alpha, beta, n, scores_dev);
+    return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
+}
+
+qkvs_status_t qkvs_bits_from_features(const float *features_dev, int64_t n_tokens, int32_t hidden, const float *params_dev,
+                                      uint8_t *bits_dev, float *outputs_dev, void *stream)
+{
+    if (n_tokens < 0 || hidden < 1) return QKVS_ERR_INVALID_ARG;
+    if (hidden > kControllerMaxHidden) return QKVS_ERR_UNSUPPORTED_SHAPE;
+    if (n_tokens == 0) return QKVS_OK;
+    if (!features_dev || !params_dev || !bits_dev) return QKVS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(features_dev) | reinterpret_cast<uintptr_t>(params_dev) | reinterpret_cast<uintptr_t>(outputs_dev)) & 3u)
+        return QKVS_ERR_INVALID_ARG;
+    const unsigned grid = (unsigned)std::min<int64_t>((n_tokens + 255) / 256, 148 * 8);
+    controller_kernel<<<grid, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(features_dev, n_tokens, hidden, params_dev, bits_dev, outputs_dev);
     return cudaGetLastError() == cudaSuccess ? QKVS_OK : QKVS_ERR_CUDA;
 }
 

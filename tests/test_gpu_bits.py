@@ -228,3 +228,62 @@ def test_budgeted_scores_to_card_end_to_end():
     st_g, hdr, whole, cap = gpu_create(q, q.make_layout(L, H, d, T), Ks, Vs, bits_g)
     assert st_g == 0 and np.array_equal(whole[:want.size], want)
     assert hdr.stream_bytes <= budget and hdr.stream_bytes == int(off[-1])
+
+
+def _controller_params(rng, hidden):
+    return np.concatenate([rng.standard_normal(6 * hidden), rng.standard_normal(hidden),
+                           rng.standard_normal(4 * hidden), rng.standard_normal(4)]).astype(np.float32)
+
+
+@pytest.mark.parametrize("n,hidden", [(1, 1), (37, 46), (8192, 46), (100003, 46), (5000, 128)])
+def test_controller_bit_exact(n, hidden):
+    """The two-layer controller: outputs equal bit for bit, hence the same bit-widths."""
+    import torch
+    rng = np.random.default_rng(1000 + n + hidden)
+    x = rng.standard_normal((n, 6)).astype(np.float32)
+    params = _controller_params(rng, hidden)
+    st, want_bits, want_out = oracle.bits_from_features(x, hidden, params)
+    assert st == oracle.OK
+    bits = torch.full((n,), 99, dtype=torch.uint8, device="cuda")
+    outs = torch.full((n, 4), -7.0, dtype=torch.float32, device="cuda")
+    q.bits_from_features(torch.from_numpy(x).cuda(), hidden, torch.from_numpy(params).cuda(), bits, outs)
+    assert np.array_equal(outs.cpu().numpy().view(np.uint32), want_out.view(np.uint32))
+    assert np.array_equal(bits.cpu().numpy(), want_bits)
+    # without the optional outputs
+    bits2 = torch.full((n,), 99, dtype=torch.uint8, device="cuda")
+    q.bits_from_features(torch.from_numpy(x).cuda(), hidden, torch.from_numpy(params).cuda(), bits2)
+    assert np.array_equal(bits2.cpu().numpy(), want_bits)
+
+
+def test_controller_ties_special_values_and_a_card_from_its_bits():
+    import torch
+    from gpu_utils import gpu_create, padded_cache
+    rng = np.random.default_rng(77)
+    hidden = 8
+    # all weights zero: the biases decide, equal ones go to the fewer bits
+    for b2, want in (([1, 1, 1, 1], 2), ([0, 2, 2, 1], 4), ([0, 0, 0, 1], 16)):
+        params = np.concatenate([np.zeros(11 * hidden), np.asarray(b2, np.float64)]).astype(np.float32)
+        bits = torch.zeros(50, dtype=torch.uint8, device="cuda")
+        q.bits_from_features(torch.from_numpy(rng.standard_normal((50, 6)).astype(np.float32)).cuda(), hidden,
+                             torch.from_numpy(params).cuda(), bits)
+        assert bool((bits == want).all())
+    # infinities and a not-a-number among the features: whatever comes out, both sides agree
+    x = rng.standard_normal((64, 6)).astype(np.float32)
+    x[3, 0] = np.inf
+    x[4, 1] = -np.inf
+    x[5, 2] = np.nan
+    params = _controller_params(rng, hidden)
+    st, want_bits, _ = oracle.bits_from_features(x, hidden, params)
+    bits = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    q.bits_from_features(torch.from_numpy(x).cuda(), hidden, torch.from_numpy(params).cuda(), bits)
+    assert st == oracle.OK and np.array_equal(bits.cpu().numpy(), want_bits)
+    # features -> bits -> card, all on the device, against the oracle's card from the oracle's bits
+    L, H, d, T = 1, 2, 128, 333
+    Ks, Vs, _ = padded_cache(L, H, T, d, seed=78)
+    feats = rng.standard_normal((T, 6)).astype(np.float32)
+    st, obits, _ = oracle.bits_from_features(feats, hidden, params)
+    _, want = oracle.card_create(oracle.make_layout(L, H, d, T), Ks, Vs, obits)
+    gbits = torch.zeros(T, dtype=torch.uint8, device="cuda")
+    q.bits_from_features(torch.from_numpy(feats).cuda(), hidden, torch.from_numpy(params).cuda(), gbits)
+    st, hdr, whole, _ = gpu_create(q, q.make_layout(L, H, d, T), Ks, Vs, gbits.cpu().numpy())
+    assert st == q.binding.OK and np.array_equal(whole[:want.size], want)

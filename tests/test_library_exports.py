@@ -130,3 +130,15 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert st == q.binding.ERR_BAD_CARD
     st = lib.qkvs_card_send(C.c_void_p(256), 4096, 0, C.c_void_p(512), 4095, 0, None)
     assert st == q.binding.ERR_BUFFER_TOO_SMALL
+
+
+def test_controller_argument_checks_need_no_gpu(lib):
+    p = C.c_void_p(256)
+    f = lib.qkvs_bits_from_features
+    assert f(p, -1, 46, p, p, None, None) == q.binding.ERR_INVALID_ARG
+    assert f(p, 10, 0, p, p, None, None) == q.binding.ERR_INVALID_ARG
+    assert f(p, 10, 129, p, p, None, None) == q.binding.ERR_UNSUPPORTED_SHAPE
+    assert f(None, 10, 46, p, p, None, None) == q.binding.ERR_INVALID_ARG
+    assert f(C.c_void_p(258), 10, 46, p, p, None, None) == q.binding.ERR_INVALID_ARG
+    assert f(p, 10, 46, p, p, C.c_void_p(258), None) == q.binding.ERR_INVALID_ARG
+    assert f(None, 0, 46, None, None, None, None) == q.binding.OK   # no tokens: nothing to do
