@@ -835,39 +835,48 @@ __global__ void __launch_bounds__(128) attend_merge_kernel(AttendParams p)
     const int per_kv = p.n_q_heads / p.n_kv_heads;
     const uint32_t layer = w / (uint32_t)p.n_q_heads, j = w - layer * (uint32_t)p.n_q_heads;
     const uint32_t lh = layer * (uint32_t)p.n_kv_heads + j / (uint32_t)per_kv, jj = j % (uint32_t)per_kv;
-    const bool usable = p.items_per_head > 0 && (!p.status_dev || *p.status_dev == 0);
+    // the status word is only needed at the end: its load travels with the others
+    const int32_t status = p.status_dev ? *reinterpret_cast<volatile const int32_t *>(p.status_dev) : 0;
     float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
     float big = -INFINITY, denom = 0.0f;
-    if (usable) {
+    if (p.items_per_head > 0) {
         const float *base = p.partials + ((uint64_t)lh * p.items_per_head * per_kv + jj) * kPartialFloats;
         const uint64_t stride = (uint64_t)per_kv * kPartialFloats;
-        // this warp's items: [first, last)
+        // this warp's items: [first, last), eight at a time: their maxima, sums and accumulators are
+        // requested together, and the running maximum is brought up to date block by block
         const uint32_t share = (p.items_per_head + 3u) / 4u;
         const uint32_t first = min((uint32_t)warp * share, p.items_per_head), last = min(first + share, p.items_per_head);
-        for (uint32_t i = first + lane; i < last; i += 32) big = fmaxf(big, base[i * stride + kAttendD]);
+        constexpr int kBlock = 8;
+        for (uint32_t i0 = first; i0 < last; i0 += kBlock) {
+            float2 ml[kBlock];   // maximum, sum
+            float4 v[kBlock];
 #pragma unroll
-        for (int sft = 16; sft > 0; sft >>= 1) big = fmaxf(big, __shfl_xor_sync(0xffffffffu, big, sft));
-        for (uint32_t i0 = first; i0 < last; i0 += 32) {
-            const uint32_t mine = i0 + (uint32_t)lane;
-            float f = 0.0f;
-            if (mine < last) {
-                f = exp2f(base[mine * stride + kAttendD] - big);
-                denom = fmaf(base[mine * stride + kAttendD + 1], f, denom);
+            for (int i = 0; i < kBlock; ++i) {
+                const bool there = i0 + (uint32_t)i < last;
+                const float *row = base + (there ? i0 + (uint32_t)i : i0) * stride;
+                ml[i] = *reinterpret_cast<const float2 *>(row + kAttendD);
+                v[i] = *reinterpret_cast<const float4 *>(row + 4 * lane);
+                if (!there) ml[i] = make_float2(-INFINITY, 0.0f);
             }
-            const int n = (int)min(32u, last - i0);
-#pragma unroll 8
-            for (int i = 0; i < n; ++i) {
-                const float fi = __shfl_sync(0xffffffffu, f, i);
-                const float4 v = *reinterpret_cast<const float4 *>(base + (i0 + (uint32_t)i) * stride + 4 * lane);
-                o.x = fmaf(v.x, fi, o.x);
-                o.y = fmaf(v.y, fi, o.y);
-                o.z = fmaf(v.z, fi, o.z);
-                o.w = fmaf(v.w, fi, o.w);
+            float top = big;
+#pragma unroll
+            for (int i = 0; i < kBlock; ++i) top = fmaxf(top, ml[i].x);
+            const float keep = top == -INFINITY ? 0.0f : exp2f(big - top);   // 0 the first time round
+            denom *= keep;
+            o.x *= keep, o.y *= keep, o.z *= keep, o.w *= keep;
+#pragma unroll
+            for (int i = 0; i < kBlock; ++i) {
+                const float f = ml[i].x == -INFINITY ? 0.0f : exp2f(ml[i].x - top);
+                denom = fmaf(ml[i].y, f, denom);
+                o.x = fmaf(v[i].x, f, o.x);
+                o.y = fmaf(v[i].y, f, o.y);
+                o.z = fmaf(v[i].z, f, o.z);
+                o.w = fmaf(v[i].w, f, o.w);
             }
+            big = top;
         }
-#pragma unroll
-        for (int sft = 16; sft > 0; sft >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, sft);
     }
+    const bool usable = p.items_per_head > 0 && status == 0;
     s_o[warp][lane] = o;
     if (lane == 0) {
         s_big[warp] = big;
